@@ -1,0 +1,384 @@
+"""CPU pins of the oracle: what the paper and the mathematics fix, independent of the oracle.
+
+Each test compares the C oracle with something that is not the oracle: hand-worked values
+(tests/golden), Python's exact summation, exact rationals, a brute-force sort, the closed
+forms of Appendix A, or an independently written vanilla AMSGrad.
+"""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+import oracle as orc
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def read_golden(name):
+    out = {}
+    with open(os.path.join(GOLD, name)) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            key, *vals = line.split()
+            out[key] = [float(v) for v in vals]
+    return out
+
+
+# ------------------------------------------------------------------ exact l1 sum
+
+def test_l1_exact_matches_fsum_wide_range():
+    rng = np.random.default_rng(1)
+    for trial in range(40):
+        nel = int(rng.integers(1, 5000))
+        # magnitudes spread over ~200 binades, both signs, some exact zeros and subnormals
+        x = (rng.standard_normal(nel) * np.exp2(rng.uniform(-140, 60, nel))).astype(np.float32)
+        x[rng.random(nel) < 0.05] = 0.0
+        x[rng.random(nel) < 0.02] = np.float32(1e-42)
+        want = math.fsum(abs(float(v)) for v in x)
+        assert orc.l1_exact(x) == want
+
+
+def test_l1_exact_matches_rationals_and_rounds_ties_to_even():
+    # 2^60 + 2^7 is a tie between two doubles (spacing 2^8): ties-to-even keeps 2^60
+    x = np.array([2.0 ** 60, 2.0 ** 7], dtype=np.float32)
+    assert orc.l1_exact(x) == float(Fraction(2) ** 60)
+    # 2^60 + 2^8 + 2^7: tie again, the even neighbour is now the upper one
+    x = np.array([2.0 ** 60, 2.0 ** 8, 2.0 ** 7], dtype=np.float32)
+    assert orc.l1_exact(x) == 2.0 ** 60 + 2.0 ** 9
+    # sticky bit breaks the tie upward
+    x = np.array([2.0 ** 60, 2.0 ** 7, 2.0 ** -100], dtype=np.float32)
+    assert orc.l1_exact(x) == 2.0 ** 60 + 2.0 ** 8
+    rng = np.random.default_rng(2)
+    for _ in range(20):
+        x = (rng.standard_normal(37) * np.exp2(rng.integers(-60, 60, 37))).astype(np.float32)
+        exact = sum(Fraction(abs(float(v))) for v in x)
+        got = Fraction(orc.l1_exact(x))
+        # correctly rounded: no double is strictly closer to the exact sum
+        f = orc.l1_exact(x)
+        for nb in (np.nextafter(f, np.inf), np.nextafter(f, -np.inf)):
+            assert abs(got - exact) <= abs(Fraction(float(nb)) - exact)
+
+
+def test_l1_exact_order_independent_and_large():
+    rng = np.random.default_rng(3)
+    x = (rng.standard_normal(300_000) * np.exp2(rng.uniform(-30, 30, 300_000))).astype(np.float32)
+    a = orc.l1_exact(x)
+    assert a == orc.l1_exact(x[::-1].copy()) == orc.l1_exact(np.sort(x))
+    assert a == math.fsum(np.abs(x.astype(np.float64)).tolist())
+
+
+# ------------------------------------------------------------------ scaled sign
+
+def test_sign_closed_form_appendix_a():
+    """||C(x) - x||^2 = ||x||^2 - ||x||_1^2 / d  (Appendix A, scaled sign, an equality)."""
+    rng = np.random.default_rng(4)
+    for d in (1, 2, 31, 32, 33, 1000, 4097):
+        x = rng.standard_normal(d).astype(np.float32)
+        bits, scales, c = orc.compress_sign(x)
+        x64, c64 = x.astype(np.float64), c.astype(np.float64)
+        lhs = np.sum((c64 - x64) ** 2)
+        rhs = np.sum(x64 ** 2) - np.sum(np.abs(x64)) ** 2 / d
+        assert lhs == pytest.approx(rhs, rel=1e-6, abs=1e-9)
+        # payload: exactly d sign bits and one 32-bit scale
+        assert bits.size == (d + 31) // 32 and scales.size == 1
+        unpacked = (bits[np.arange(d) // 32] >> (np.arange(d) % 32)) & 1
+        assert np.array_equal(unpacked.astype(bool), x >= 0)
+        if d % 32:
+            assert bits[-1] >> (d % 32) == 0
+        assert np.array_equal(c, np.where(x >= 0, scales[0], -scales[0]).astype(np.float32))
+        assert scales[0] == np.float32(math.fsum(abs(float(v)) for v in x) / d)
+
+
+def test_sign_gaussian_limits():
+    """Half-normal mean: scale -> sigma sqrt(2/pi); error ratio -> 1 - 2/pi."""
+    rng = np.random.default_rng(5)
+    sigma = 0.37
+    x = (rng.standard_normal(2_000_000) * sigma).astype(np.float32)
+    _, scales, c = orc.compress_sign(x)
+    assert scales[0] == pytest.approx(sigma * math.sqrt(2 / math.pi), rel=3e-3)
+    ratio = np.sum((c.astype(np.float64) - x) ** 2) / np.sum(x.astype(np.float64) ** 2)
+    assert ratio == pytest.approx(1 - 2 / math.pi, rel=5e-3)
+
+
+def test_sign_zero_maps_to_plus_and_zero_vector():
+    bits, scales, c = orc.compress_sign(np.array([0.0, -0.0, -1.0, 2.0], dtype=np.float32))
+    assert bits[0] == 0b1011 and scales[0] == np.float32(0.75)
+    bits, scales, c = orc.compress_sign(np.zeros(40, dtype=np.float32))
+    assert scales[0] == 0 and np.all(c == 0) and bits[0] == 0xFFFFFFFF and bits[1] == 0xFF
+
+
+def test_sign_segments_equal_flat_on_slices():
+    rng = np.random.default_rng(6)
+    d = 1000
+    off = np.array([0, 1, 34, 64, 65, 500, 997, 1000])
+    x = (rng.standard_normal(d) * np.repeat(rng.uniform(1e-3, 10, 7), np.diff(off))).astype(np.float32)
+    bits, scales, c = orc.compress_sign(x, off)
+    fb, _, _ = orc.compress_sign(x)
+    assert np.array_equal(bits, fb)                      # bits do not depend on segments
+    for r in range(7):
+        _, s, cs = orc.compress_sign(x[off[r]:off[r + 1]])
+        assert scales[r] == s[0]
+        assert np.array_equal(c[off[r]:off[r + 1]], cs)
+
+
+# ------------------------------------------------------------------ top-k
+
+def brute_topk(x, k):
+    order = sorted(range(len(x)), key=lambda j: (-abs(float(x[j])), j))
+    return sorted(order[:k])
+
+
+def test_topk_brute_force_small_all_k_with_ties():
+    rng = np.random.default_rng(7)
+    for d in list(range(1, 20)) + [33, 64]:
+        for trial in range(3):
+            # few distinct magnitudes -> many ties
+            x = (rng.integers(-3, 4, d) * 0.5).astype(np.float32)
+            for k in range(1, d + 1):
+                idx, val, c = orc.compress_topk(x, k)
+                want = brute_topk(x, k)
+                assert idx.tolist() == want
+                assert np.array_equal(val, x[want])
+                dense = np.zeros(d, np.float32)
+                dense[want] = x[want]
+                assert np.array_equal(c, dense)
+
+
+def test_topk_inequality_appendix_a():
+    """||C(x) - x||^2 <= (1 - k/d) ||x||^2 (Appendix A, top-k, squared on both sides)."""
+    rng = np.random.default_rng(8)
+    for d, k in ((100, 1), (100, 50), (1000, 10), (1000, 999), (257, 257)):
+        x = rng.standard_normal(d).astype(np.float32)
+        idx, val, c = orc.compress_topk(x, k)
+        assert idx.size == k and np.all(np.diff(idx.astype(np.int64)) > 0) and idx[-1] < d
+        err = np.sum((c.astype(np.float64) - x) ** 2)
+        assert err <= (1 - k / d) * np.sum(x.astype(np.float64) ** 2) + 1e-12
+        # every kept magnitude dominates every dropped one
+        dropped = np.setdiff1d(np.arange(d), idx)
+        if dropped.size:
+            assert np.abs(x[idx]).min() >= np.abs(x[dropped]).max()
+
+
+def test_topk_worked_example_ties():
+    gold = read_golden("worked_example_topk.txt")
+    d, k = int(gold["d"][0]), int(gold["k"][0])
+    g = np.array(gold["g"], dtype=np.float32)
+    o = orc.Oracle(d, 1, orc.TOPK, k=k)
+    for t in (1, 2):
+        o.step(g[None, :])
+        idx, val = o.payload(0)
+        assert idx.tolist() == gold["t%d.idx" % t]
+        assert val.tolist() == gold["t%d.val" % t]
+        assert o.state("ghat_w")[0].tolist() == gold["t%d.ghat" % t]
+
+
+# ------------------------------------------------------------------ whole step
+
+def test_sign_worked_example_two_iterations():
+    gold = read_golden("worked_example_sign.txt")
+    n, d = int(gold["n"][0]), int(gold["d"][0])
+    o = orc.Oracle(d, n, orc.SIGN, beta1=gold["beta1"][0], beta2=gold["beta2"][0],
+                   lr=gold["alpha"][0], eps=gold["nu"][0], x0=gold["x1"])
+    for t in (1, 2):
+        p = "t%d." % t
+        o.step(np.array([gold[p + "g0"], gold[p + "g1"]], dtype=np.float32))
+        for i in range(n):
+            bits, scales = o.payload(i)
+            assert scales[0] == gold[p + "w%d.scale" % i][0]
+            assert bits[0] == gold[p + "w%d.word" % i][0]
+            assert o.state("ghat_w")[i].tolist() == gold[p + "w%d.ghat" % i]
+        bits, scales = o.payload(-1)
+        assert scales[0] == gold[p + "s.scale"][0] and bits[0] == gold[p + "s.word"][0]
+        assert o.state("ghat_s").tolist() == gold[p + "s.ghat"]
+        assert o.state("gtil").tolist() == gold[p + "gtil"]
+        assert o.state("m").tolist() == gold[p + "m"]
+        assert o.state("v").tolist() == gold[p + "v"]
+        assert o.state("vhat").tolist() == gold[p + "vhat"]
+        if t == 1:
+            assert o.state("x").tolist() == gold[p + "x"]
+        else:
+            np.testing.assert_allclose(o.state("x"), gold[p + "x"], rtol=0, atol=1.5e-7)   # fixture has 7 digits
+            # and to full binary32 accuracy from the exact expression
+            want = [0.75 - 0.5 * 1.0 / math.sqrt(223 / 128), 1.25 + 0.5 * 0.125 / 0.75,
+                    0.75 - 0.5 * 1.0 / math.sqrt(223 / 128), 1.25 + 0.5 * 1.0 / math.sqrt(223 / 128)]
+            np.testing.assert_allclose(o.state("x"), want, rtol=2e-7)
+
+
+def vanilla_amsgrad(x0, grads_mean, b1, b2, lr, nu):
+    """Distributed AMSGrad of the paper's Section 3, written independently in numpy fp32."""
+    f = np.float32
+    x = x0.astype(f).copy()
+    m = np.zeros_like(x); v = np.zeros_like(x); vh = np.zeros_like(x)
+    b1, b2, lr, nu = f(b1), f(b2), f(lr), f(nu)
+    for g in grads_mean:
+        g = g.astype(f)
+        m = b1 * m + (f(1) - b1) * g
+        v = b2 * v + (f(1) - b2) * (g * g)
+        vh = np.maximum(vh, v)
+        x = x - (lr * m) / np.sqrt(vh + nu)
+    return x, m, v, vh
+
+
+@pytest.mark.parametrize("mode", [orc.MARKOV, orc.EF])
+def test_identity_compressor_is_vanilla_amsgrad(mode):
+    rng = np.random.default_rng(9)
+    d, n, T = 513, 4, 6
+    x0 = (rng.standard_normal(d) * 0.02).astype(np.float32)
+    G = rng.standard_normal((T, n, d)).astype(np.float32)
+    o = orc.Oracle(d, n, orc.IDENTITY, beta1=0.9, beta2=0.99, lr=1e-2, eps=1e-8, x0=x0, mode=mode)
+    means = []
+    for t in range(T):
+        o.step(G[t])
+        acc = np.zeros(d, np.float32)
+        for i in range(n):
+            acc = acc + G[t, i]
+        means.append(acc / np.float32(n))
+        if t == 0:
+            x, m, v, vh = vanilla_amsgrad(x0, means, 0.9, 0.99, 1e-2, 1e-8)
+            assert np.array_equal(o.state("x"), x) and np.array_equal(o.state("m"), m)
+            assert np.array_equal(o.state("v"), v) and np.array_equal(o.state("vhat"), vh)
+    x, m, v, vh = vanilla_amsgrad(x0, means, 0.9, 0.99, 1e-2, 1e-8)
+    if mode == orc.EF:          # error terms stay exactly zero: bitwise reduction
+        assert np.array_equal(o.state("x"), x) and np.array_equal(o.state("vhat"), vh)
+        assert not o.state("ghat_w").any() and not o.state("gtil").any()
+    else:                       # ghat + fl(g - ghat) is g only to an ulp after step 1
+        np.testing.assert_allclose(o.state("m"), m, rtol=1e-5, atol=1e-7)
+        np.testing.assert_allclose(o.state("vhat"), vh, rtol=1e-5, atol=1e-9)
+        np.testing.assert_allclose(o.state("x"), x, rtol=0, atol=1e-6)
+
+
+def decode_sign(bits, scales, off, d):
+    j = np.arange(d)
+    b = ((bits[j // 32] >> (j % 32)) & 1).astype(bool)
+    s = np.repeat(scales, np.diff(off)).astype(np.float32)
+    return np.where(b, s, -s).astype(np.float32)
+
+
+@pytest.mark.parametrize("comp", [orc.SIGN, orc.TOPK])
+def test_markov_identity_contraction_and_invariants(comp):
+    """ghat_t - ghat_{t-1} = c_t bit-exactly (decoded from the payload), the contraction of
+    the Markov sequence (equality for scaled sign with pi from Appendix A), vhat monotone,
+    |x_{t+1} - x_t| <= alpha |m| / sqrt(nu), and the n = 1 server equals the worker."""
+    rng = np.random.default_rng(10)
+    d, n, k, T = 777, 3, 20, 8
+    off = np.array([0, 100, 131, 777])
+    kw = dict(offsets=off) if comp == orc.SIGN else dict(k=k)
+    x0 = (rng.standard_normal(d) * 0.02).astype(np.float32)
+    o = orc.Oracle(d, n, comp, lr=1e-3, eps=1e-8, x0=x0, **kw)
+    base = rng.standard_normal((n, d)).astype(np.float32)
+    prev = {name: o.state(name).copy() for name in orc.STATE_NAMES}
+    for t in range(T):
+        g = base + 0.3 * rng.standard_normal((n, d)).astype(np.float32)
+        o.step(g)
+        acc = np.zeros(d, np.float32)
+        for i in range(n):
+            u = g[i] - prev["ghat_w"][i]
+            if comp == orc.SIGN:
+                bits, scales = o.payload(i)
+                c = decode_sign(bits, scales, off, d)
+                for r in range(3):      # contraction, equality form, per segment
+                    sl = slice(off[r], off[r + 1])
+                    u64 = u[sl].astype(np.float64)
+                    pi_r = 1 - np.sum(np.abs(u64)) ** 2 / (u64.size * np.sum(u64 ** 2))
+                    err = np.sum((o.state("ghat_w")[i][sl].astype(np.float64) - g[i][sl]) ** 2)
+                    assert err == pytest.approx(pi_r * np.sum(u64 ** 2), rel=1e-4)
+            else:
+                idx, val = o.payload(i)
+                assert np.array_equal(val, u[idx])
+                c = np.zeros(d, np.float32); c[idx] = val
+                err = np.sum((o.state("ghat_w")[i].astype(np.float64) - g[i]) ** 2)
+                assert err <= (1 - k / d) * np.sum(u.astype(np.float64) ** 2) * (1 + 1e-6)
+            assert np.array_equal(o.state("ghat_w")[i], prev["ghat_w"][i] + c)
+            acc = acc + c
+        assert np.array_equal(o.state("ghat_s"), prev["ghat_s"] + acc / np.float32(n))
+        if comp == orc.SIGN:
+            c = decode_sign(*o.payload(-1), off, d)
+        else:
+            idx, val = o.payload(-1)
+            assert np.array_equal(val, (o.state("ghat_s") - prev["gtil"])[idx])
+            c = np.zeros(d, np.float32); c[idx] = val
+        assert np.array_equal(o.state("gtil"), prev["gtil"] + c)
+        assert np.all(o.state("vhat") >= prev["vhat"]) and np.all(o.state("vhat") >= o.state("v"))
+        dx = np.abs(o.state("x").astype(np.float64) - prev["x"])
+        assert np.all(dx <= 1e-3 * np.abs(o.state("m")) / math.sqrt(1e-8) * (1 + 1e-5) + 1e-9)
+        prev = {name: o.state(name).copy() for name in orc.STATE_NAMES}
+
+
+def test_first_step_closed_form_and_single_worker():
+    """Zero initial state: ghat_1^(i) = C(g_1^(i)); with n = 1 the server aggregate equals
+    the worker state bit for bit."""
+    rng = np.random.default_rng(11)
+    d = 300
+    g = rng.standard_normal((1, d)).astype(np.float32)
+    o = orc.Oracle(d, 1, orc.SIGN)
+    o.step(g)
+    _, _, c = orc.compress_sign(g[0])
+    assert np.array_equal(o.state("ghat_w")[0], c)
+    assert np.array_equal(o.state("ghat_s"), o.state("ghat_w")[0])
+    for _ in range(4):
+        o.step(rng.standard_normal((1, d)).astype(np.float32))
+    # n = 1: ghat_s accumulates the same c as ghat_w, in the same order
+    assert np.array_equal(o.state("ghat_s"), o.state("ghat_w")[0])
+    # identical gradients on every worker: average of equal payloads is the payload (n = 4)
+    o4 = orc.Oracle(d, 4, orc.SIGN)
+    o1 = orc.Oracle(d, 1, orc.SIGN)
+    for _ in range(3):
+        g = rng.standard_normal((1, d)).astype(np.float32)
+        o4.step(np.repeat(g, 4, axis=0)); o1.step(g)
+        assert np.array_equal(o4.state("x"), o1.state("x"))
+
+
+def test_topk_constant_gradient_converges_exactly():
+    """With a fixed gradient and top-k, every coordinate is transmitted once: after
+    ceil(d/k) steps ghat = g exactly and all later payload values are zero."""
+    rng = np.random.default_rng(12)
+    d, k = 103, 10
+    g = rng.standard_normal((1, d)).astype(np.float32)
+    o = orc.Oracle(d, 1, orc.TOPK, k=k)
+    for _ in range(-(-d // k)):
+        o.step(g)
+    assert np.array_equal(o.state("ghat_w")[0], g[0])
+    o.step(g)
+    assert not o.payload(0)[1].any()
+
+
+def test_error_feedback_reconstruction():
+    """Classical error feedback: delta_new + C(g + delta) gives back g + delta, exactly
+    for top-k and identity, to rounding for scaled sign."""
+    rng = np.random.default_rng(13)
+    d, n = 200, 2
+    for comp, kw in ((orc.TOPK, dict(k=7)), (orc.SIGN, {}), (orc.IDENTITY, {})):
+        o = orc.Oracle(d, n, comp, mode=orc.EF, **kw)
+        for _ in range(4):
+            delta = o.state("ghat_w").copy()
+            g = rng.standard_normal((n, d)).astype(np.float32)
+            o.step(g)
+            for i in range(n):
+                p = g[i] + delta[i]
+                if comp == orc.TOPK:
+                    idx, val = o.payload(i)
+                    c = np.zeros(d, np.float32); c[idx] = val
+                    assert np.array_equal(o.state("ghat_w")[i] + c, p)
+                elif comp == orc.SIGN:
+                    c = decode_sign(*o.payload(i), np.array([0, d]), d)
+                    np.testing.assert_allclose(o.state("ghat_w")[i] + c, p, rtol=0, atol=1e-6)
+                else:
+                    assert not o.state("ghat_w")[i].any()
+
+
+def test_planted_mistakes_are_caught():
+    """The pins above must be able to fail: perturb inputs the way a plausible slip would
+    (wrong sign convention, transposed workers) and check the worked example notices."""
+    gold = read_golden("worked_example_sign.txt")
+    o = orc.Oracle(4, 2, orc.SIGN, beta1=0.5, beta2=0.5, lr=0.5, eps=0.28125, x0=gold["x1"])
+    o.step(np.array([gold["t1.g1"], gold["t1.g0"]], dtype=np.float32))   # workers swapped
+    assert o.payload(0)[0][0] != gold["t1.w0.word"][0]
+    # server result is symmetric in the workers at step 1, so x agrees: the asymmetry shows
+    # only from step 2 on, which is why the example has two iterations
+    assert o.state("x").tolist() == gold["t1.x"]
+    o.step(np.array([gold["t2.g0"], gold["t2.g1"]], dtype=np.float32))
+    assert o.state("ghat_s").tolist() != gold["t2.s.ghat"]
