@@ -1,0 +1,177 @@
+/*
+ * cdadam.h - C interface of the B200 (sm_100a) CD-Adam library.
+ *
+ * One context simulates, on ONE GPU, the n workers and the server of the paper's
+ * Algorithm 1 (communication-compressed distributed AMSGrad).  The caller owns the n
+ * stochastic gradients of the problem statement (Section 3, Eq. 1); the context owns the
+ * model x, the moments m, v, vhat and all compression state.  One call of cdadam_step is one
+ * iteration t of Algorithm 1:
+ *
+ *   worker i :  c^(i) = C(g^(i) - ghat^(i));  ghat^(i) += c^(i)            (lines 5-6)
+ *   server   :  ghat += (1/n) sum_i c^(i);  c = C(ghat - gtil);  gtil += c  (lines 8-10)
+ *   worker   :  gtil += c (the same vector on every worker, kept once);
+ *               m = b1 m + (1-b1) gtil;  v = b2 v + (1-b2) gtil^2;
+ *               vhat = max(vhat, v);  x -= lr * m / sqrt(vhat + eps)       (lines 12-16)
+ *
+ * C is the scaled-sign compressor (||u||_1 / |segment| * sign(u), one bit per coordinate plus
+ * one float per segment), the top-k compressor (k (index, value) pairs) or the identity
+ * (Appendix A).  eps is the paper's nu: it sits INSIDE the square root and there is no bias
+ * correction.  All vectors are IEEE binary32; every operation above is rounded once, in the
+ * order written, without fused multiply-add.  The l1 norm is accumulated in double-double
+ * arithmetic in a fixed order, rounded to binary64, divided by the segment length in
+ * binary64 and rounded to binary32, so the scale is the correctly rounded value and does
+ * not depend on the launch shape.  The sum over workers runs over i = 0, 1, ..., n-1 in
+ * binary32 and is divided once by (float)n.
+ *
+ * Conventions.  "device" pointers are CUDA global-memory addresses on the context's GPU
+ * (the device current at cdadam_create); "host" pointers are ordinary CPU addresses.  All
+ * functions returning int return CDADAM_OK (0) or a negative CDADAM_ERR_* code and never
+ * abort; cdadam_last_error() gives the message of the calling thread's last failure.
+ * Unless stated, work is queued on the given stream (a cudaStream_t passed as void*, NULL =
+ * the legacy default stream) and the call returns without waiting.  A context must be used
+ * from one host thread at a time and with one stream at a time.  Gradients must be finite;
+ * the result for NaN or infinite input is unspecified (no call hangs or faults on them).
+ */
+#ifndef CDADAM_H
+#define CDADAM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cdadam_ctx cdadam_ctx;
+
+/* compressor C of Algorithm 1 (Appendix A) */
+enum { CDADAM_SIGN = 0, CDADAM_TOPK = 1, CDADAM_IDENTITY = 2 };
+
+/* status codes */
+enum {
+    CDADAM_OK = 0,
+    CDADAM_ERR_ARG = -1,     /* invalid argument; nothing was queued */
+    CDADAM_ERR_ALLOC = -2,   /* device or host allocation failed */
+    CDADAM_ERR_CUDA = -3,    /* a CUDA runtime call failed; see cdadam_last_error */
+    CDADAM_ERR_STATE = -4    /* call not allowed in the context's current state */
+};
+
+/* names of the state vectors for cdadam_get_state / cdadam_set_state */
+enum {
+    CDADAM_STATE_GHAT_W = 0, /* worker Markov states ghat^(i), n x d row-major */
+    CDADAM_STATE_GHAT_S = 1, /* server aggregate ghat, d */
+    CDADAM_STATE_GTIL = 2,   /* second Markov state gtil, d */
+    CDADAM_STATE_M = 3,
+    CDADAM_STATE_V = 4,
+    CDADAM_STATE_VHAT = 5,
+    CDADAM_STATE_X = 6
+};
+
+#define CDADAM_SERVER (-1)   /* "who" argument of cdadam_last_payload */
+
+/*
+ * Create a context (inputs of Algorithm 1: beta1, beta2, nu = eps, step size lr, C).
+ *   d          model dimension, 1 <= d < 2^32
+ *   n          number of simulated workers, 1 <= n <= 65535
+ *   compressor CDADAM_SIGN, CDADAM_TOPK or CDADAM_IDENTITY
+ *   k          entries kept by top-k at the workers and at the server, 1 <= k <= d;
+ *              ignored for the other compressors
+ * All state is allocated here, on the current device, and zero-initialised (Algorithm 1
+ * line 1; x_1 = 0 until cdadam_set_params).  Scaled sign starts with one segment [0, d).
+ * Synchronous.  Returns NULL on failure (see cdadam_last_error).  The caller destroys the
+ * context with cdadam_destroy.
+ */
+cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k,
+                          float beta1, float beta2, float lr, float eps);
+
+/* Free a context and its device memory (waits for the device).  NULL is allowed. */
+void cdadam_destroy(cdadam_ctx *ctx);
+
+/*
+ * One iteration of Algorithm 1 (lines 4-16) on the n gradients g_t^(i).
+ *   grads   device, n x d floats, row i = worker i, row-major, contiguous; borrowed until
+ *           the work queued on `stream` has completed; never written.  A base address
+ *           that is a multiple of 16 bytes together with d % 4 == 0 selects the
+ *           vectorised kernels; any other alignment is accepted and gives the same result.
+ *   stream  cudaStream_t
+ * Allocates nothing.  After the stream has completed, cdadam_params() holds x_{t+1}.
+ */
+int cdadam_step(cdadam_ctx *ctx, const float *grads, void *stream);
+
+/*
+ * The same iteration with the gradients in HOST memory: copies n x d floats host->device
+ * into a staging buffer owned by the context (allocated at the first call), runs the step,
+ * copies x_{t+1} (d floats) into x_out (host; may be NULL to skip) and waits for `stream`.
+ * Pinned host memory makes the copies asynchronous to the host but the call still waits.
+ */
+int cdadam_step_host(cdadam_ctx *ctx, const float *grads_host, float *x_out_host,
+                     void *stream);
+
+/* Device pointer to the model x (d floats), owned by the context, valid until destroy.
+ * Its contents are x_{t+1} once the stream of the last step has completed.  NULL if ctx
+ * is NULL. */
+const float *cdadam_params(cdadam_ctx *ctx);
+
+/* Set the initial point x_1 (Algorithm 1 input) from d device floats. */
+int cdadam_set_params(cdadam_ctx *ctx, const float *x0, void *stream);
+
+/*
+ * Apply the scaled-sign compressor independently to q contiguous segments ("per tensor"):
+ * segment r is [offsets[r], offsets[r+1]), offsets (host, q+1 values) strictly increasing
+ * with offsets[0] = 0 and offsets[q] = d; each segment has its own scale
+ * ||u_segment||_1 / |segment|, at the workers and at the server; sign bits stay in one
+ * d-bit array.  Allowed only before the first step (CDADAM_ERR_STATE afterwards) and only
+ * for CDADAM_SIGN.  Synchronous (re-allocates tables).
+ */
+int cdadam_set_segments(cdadam_ctx *ctx, int q, const int64_t *offsets);
+
+/* Step size alpha_t for the following steps (Algorithm 1 takes a non-increasing sequence;
+ * monotonicity is not enforced). */
+int cdadam_set_lr(cdadam_ctx *ctx, float lr);
+
+/*
+ * Copy a state vector to / from device memory (dst / src: n*d floats for GHAT_W, else d).
+ * get first applies any payload whose application the kernels had deferred, so the values
+ * are those of Algorithm 1 after the last completed iteration.  set replaces the vector;
+ * used to resume from a checkpoint or to start a step from a given state.
+ */
+int cdadam_get_state(cdadam_ctx *ctx, int name, float *dst, void *stream);
+int cdadam_set_state(cdadam_ctx *ctx, int name, const float *src, void *stream);
+
+/*
+ * The message sent in the last iteration by worker `who` (0..n-1) or by the server
+ * (CDADAM_SERVER): device pointers owned by the context, valid until the next step.
+ *   scaled sign: *a = uint32 words, bit (j % 32) of word j / 32 is 1 iff u_j >= 0 (so a
+ *                zero counts as positive), unused high bits of the last word are 0;
+ *                *b = q float scales; *count = d.  The message is d + 32 q bits.
+ *   top-k:       *a = k uint32 coordinates in increasing order, *b = their k float values
+ *                u_j; *count = k.  Among equal |u_j| the lower j is kept.
+ * CDADAM_ERR_STATE before the first step or for the identity compressor.
+ */
+int cdadam_last_payload(cdadam_ctx *ctx, int who, const void **a, const float **b,
+                        int64_t *count);
+
+/* Number of completed calls of cdadam_step on this context. */
+int64_t cdadam_step_count(cdadam_ctx *ctx);
+
+/* Number of kernels one cdadam_step launches in the context's current configuration. */
+int cdadam_launches_per_step(cdadam_ctx *ctx);
+
+/*
+ * Stand-alone compressors of Appendix A on a device vector x of d floats.
+ * Scaled sign: writes ceil(d/32) words to bits and q floats to scales (segments as in
+ * cdadam_set_segments; offsets == NULL means one segment).  Top-k: writes k increasing
+ * coordinates to idx and their values to val.  Scratch memory is taken from and returned
+ * to the stream-ordered allocator of the current device inside the call.
+ */
+int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offsets,
+                         uint32_t *bits, float *scales, void *stream);
+int cdadam_compress_topk(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,
+                         void *stream);
+
+/* Message of the calling thread's most recent failure ("" if none).  Never NULL. */
+const char *cdadam_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CDADAM_H */

@@ -1,0 +1,225 @@
+"""ctypes binding of libcdadam.so: the same entry points as include/cdadam.h.
+
+Argument marshalling only.  PyTorch supplies device memory and streams; every step of the
+method runs in the library's CUDA kernels.  There is no CPU fallback: if the shared library
+is missing, loading raises.
+"""
+import ctypes
+import os
+
+import torch
+
+SIGN, TOPK, IDENTITY = 0, 1, 2
+SERVER = -1
+STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
+OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE = 0, -1, -2, -3, -4
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcdadam.so")
+_lib = None
+
+_c = ctypes
+_SIGNATURES = {
+    "cdadam_create": (_c.c_void_p, [_c.c_int64, _c.c_int, _c.c_int, _c.c_int64,
+                                    _c.c_float, _c.c_float, _c.c_float, _c.c_float]),
+    "cdadam_destroy": (None, [_c.c_void_p]),
+    "cdadam_step": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_step_host": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
+    "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
+    "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
+    "cdadam_get_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
+    "cdadam_set_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
+    "cdadam_last_payload": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_void_p),
+                                       _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_int64)]),
+    "cdadam_step_count": (_c.c_int64, [_c.c_void_p]),
+    "cdadam_launches_per_step": (_c.c_int, [_c.c_void_p]),
+    "cdadam_compress_sign": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int,
+                                        _c.POINTER(_c.c_int64), _c.c_void_p, _c.c_void_p,
+                                        _c.c_void_p]),
+    "cdadam_compress_topk": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int64, _c.c_void_p,
+                                        _c.c_void_p, _c.c_void_p]),
+    "cdadam_last_error": (_c.c_char_p, []),
+}
+
+
+def exported_symbols():
+    """Names of the C entry points this binding expects (those include/cdadam.h declares)."""
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    """Load libcdadam.so (once).  Raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError("libcdadam.so is missing: run `python -m paper_2111_00705_b200.build`"
+                               " (there is no fallback path)")
+        handle = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            f = getattr(handle, name)
+            f.restype, f.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+class CdadamError(RuntimeError):
+    def __init__(self, code, message):
+        super().__init__("cdadam error %d: %s" % (code, message))
+        self.code = code
+
+
+def last_error():
+    return lib().cdadam_last_error().decode()
+
+
+def _check(code):
+    if code != OK:
+        raise CdadamError(code, last_error())
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+def _dev_f32(t, count, what):
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous() and t.numel() == count):
+        raise ValueError("%s must be a contiguous CUDA float32 tensor of %d elements" % (what, count))
+    return ctypes.c_void_p(t.data_ptr())
+
+
+class _DevView:
+    """Zero-copy view of library-owned device memory for torch.as_tensor."""
+
+    def __init__(self, ptr, count, typestr):
+        self.__cuda_array_interface__ = {"shape": (count,), "typestr": typestr,
+                                         "data": (ptr, False), "version": 2}
+
+
+def _view(ptr, count, dtype, device):
+    typestr = {torch.float32: "<f4", torch.int32: "<i4"}[dtype]
+    if count == 0:
+        return torch.empty(0, dtype=dtype, device=device)
+    return torch.as_tensor(_DevView(ptr, count, typestr), device=device)
+
+
+class CDAdam:
+    """One context of the library: n simulated workers and the server on one GPU."""
+
+    def __init__(self, d, n, compressor=SIGN, k=0, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
+                 offsets=None, x0=None, device=None):
+        self._h = None
+        self.device = torch.device("cuda", torch.cuda.current_device()) if device is None \
+            else torch.device(device)
+        self.d, self.n, self.compressor, self.k = int(d), int(n), int(compressor), int(k)
+        self.q = 1
+        with torch.cuda.device(self.device):
+            self._h = lib().cdadam_create(self.d, self.n, self.compressor, self.k,
+                                          beta1, beta2, lr, eps)
+        if not self._h:
+            raise CdadamError(ERR_ARG, last_error())
+        if offsets is not None:
+            self.set_segments(offsets)
+        if x0 is not None:
+            self.set_params(x0)
+
+    def close(self):
+        if self._h:
+            lib().cdadam_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the three calls of the hot path ------------------------------------------------
+    def step(self, grads, stream=None):
+        """One iteration of Algorithm 1 on the n x d device gradients."""
+        _check(lib().cdadam_step(self._h, _dev_f32(grads, self.n * self.d, "grads"), _stream(stream)))
+
+    def step_host(self, grads_host, x_out_host=None, stream=None):
+        """The same with host gradients (pinned or pageable) and x copied back to the host."""
+        if grads_host.is_cuda or grads_host.dtype != torch.float32 or not grads_host.is_contiguous() \
+                or grads_host.numel() != self.n * self.d:
+            raise ValueError("grads_host must be a contiguous CPU float32 tensor of n*d elements")
+        xo = None
+        if x_out_host is not None:
+            if x_out_host.is_cuda or x_out_host.dtype != torch.float32 or x_out_host.numel() != self.d \
+                    or not x_out_host.is_contiguous():
+                raise ValueError("x_out_host must be a contiguous CPU float32 tensor of d elements")
+            xo = ctypes.c_void_p(x_out_host.data_ptr())
+        _check(lib().cdadam_step_host(self._h, ctypes.c_void_p(grads_host.data_ptr()), xo, _stream(stream)))
+
+    def params(self):
+        """The model x as a torch view of the library's memory (no copy)."""
+        return _view(lib().cdadam_params(self._h), self.d, torch.float32, self.device)
+
+    # -- helpers ------------------------------------------------------------------------
+    def set_params(self, x0, stream=None):
+        _check(lib().cdadam_set_params(self._h, _dev_f32(x0, self.d, "x0"), _stream(stream)))
+
+    def set_segments(self, offsets):
+        off = (ctypes.c_int64 * len(offsets))(*[int(v) for v in offsets])
+        _check(lib().cdadam_set_segments(self._h, len(offsets) - 1, off))
+        self.q = len(offsets) - 1
+
+    def set_lr(self, lr):
+        _check(lib().cdadam_set_lr(self._h, lr))
+
+    def get_state(self, name, stream=None):
+        count = self.n * self.d if name == "ghat_w" else self.d
+        out = torch.empty(count, dtype=torch.float32, device=self.device)
+        _check(lib().cdadam_get_state(self._h, STATE_NAMES.index(name), ctypes.c_void_p(out.data_ptr()),
+                                      _stream(stream)))
+        return out.view(self.n, self.d) if name == "ghat_w" else out
+
+    def set_state(self, name, value, stream=None):
+        count = self.n * self.d if name == "ghat_w" else self.d
+        _check(lib().cdadam_set_state(self._h, STATE_NAMES.index(name), _dev_f32(value, count, name),
+                                      _stream(stream)))
+
+    def last_payload(self, who):
+        """(bits int32[ceil(d/32)], scales float32[q]) or (idx int32[k], val float32[k]) as
+        views of library memory, valid until the next step.  Integer words are returned as
+        int32 tensors holding the uint32 bit patterns."""
+        a, b, cnt = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_int64()
+        _check(lib().cdadam_last_payload(self._h, who, ctypes.byref(a), ctypes.byref(b), ctypes.byref(cnt)))
+        if self.compressor == SIGN:
+            return (_view(a.value, (self.d + 31) // 32, torch.int32, self.device),
+                    _view(b.value, self.q, torch.float32, self.device))
+        return (_view(a.value, self.k, torch.int32, self.device),
+                _view(b.value, self.k, torch.float32, self.device))
+
+    def step_count(self):
+        return lib().cdadam_step_count(self._h)
+
+    def launches_per_step(self):
+        return lib().cdadam_launches_per_step(self._h)
+
+
+def compress_sign(x, offsets=None, stream=None):
+    """Stand-alone scaled-sign compressor on a CUDA vector: (bits int32, scales float32)."""
+    d = x.numel()
+    q = 1 if offsets is None else len(offsets) - 1
+    off = None if offsets is None else (ctypes.c_int64 * len(offsets))(*[int(v) for v in offsets])
+    bits = torch.empty((d + 31) // 32, dtype=torch.int32, device=x.device)
+    scales = torch.empty(q, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(lib().cdadam_compress_sign(_dev_f32(x, d, "x"), d, q, off, ctypes.c_void_p(bits.data_ptr()),
+                                          ctypes.c_void_p(scales.data_ptr()), _stream(stream)))
+    return bits, scales
+
+
+def compress_topk(x, k, stream=None):
+    """Stand-alone top-k compressor on a CUDA vector: (idx int32[k] increasing, val float32[k])."""
+    d = x.numel()
+    idx = torch.empty(k, dtype=torch.int32, device=x.device)
+    val = torch.empty(k, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(lib().cdadam_compress_topk(_dev_f32(x, d, "x"), d, k, ctypes.c_void_p(idx.data_ptr()),
+                                          ctypes.c_void_p(val.data_ptr()), _stream(stream)))
+    return idx, val

@@ -1,0 +1,414 @@
+// C interface of the CD-Adam library (see include/cdadam.h): context, state buffers and the
+// per-step launch sequence.  No arithmetic of the method lives here.
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/cdadam.h"
+#include "kernels.h"
+#include "topk.h"
+
+using namespace cdadam;
+
+namespace {
+
+thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define CU_TRY(expr)                                                                       \
+    do {                                                                                   \
+        cudaError_t e_ = (expr);                                                           \
+        if (e_ != cudaSuccess)                                                             \
+            return fail(e_ == cudaErrorMemoryAllocation ? CDADAM_ERR_ALLOC : CDADAM_ERR_CUDA, \
+                        "%s: %s", #expr, cudaGetErrorString(e_));                          \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            cudaSetDevice(dev);
+            switched = true;
+        }
+    }
+    ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
+};
+
+// Tile size: a multiple of kSub; larger vectors use larger tiles so that the number of
+// partial sums per segment stays small.
+int choose_tile(int64_t d)
+{
+    if (d >= (int64_t)1 << 28) return 4 * kSub;
+    if (d >= (int64_t)1 << 24) return 2 * kSub;
+    return kSub;
+}
+
+// Host tables + their device copies.
+struct TableSet {
+    Tables tb{};
+    std::vector<int64_t> off;
+    void *dev = nullptr;        // one allocation holding off, pbase, tile_first, tile_last
+
+    int build(int64_t d, int q, const int64_t *offsets, int tile, cudaStream_t st, bool async)
+    {
+        release(st, async);
+        off.assign(offsets, offsets + q + 1);
+        const int64_t ntiles = (d + tile - 1) / tile;
+        std::vector<int32_t> first(ntiles), last(ntiles);
+        std::vector<int64_t> pbase(ntiles);
+        int r = 0;
+        int64_t np = 0;
+        for (int64_t T = 0; T < ntiles; ++T) {
+            const int64_t lo = T * tile, hi = std::min<int64_t>(d, lo + tile) - 1;
+            while (off[r + 1] <= lo) ++r;
+            first[T] = r;
+            int e = r;
+            while (off[e + 1] <= hi) ++e;
+            last[T] = e;
+            pbase[T] = np;
+            np += e - r + 1;
+        }
+        const size_t b_off = (size_t)(q + 1) * 8, b_pb = (size_t)ntiles * 8, b_t = (size_t)ntiles * 4;
+        const size_t total = b_off + b_pb + 2 * b_t;
+        cudaError_t e = async ? cudaMallocAsync(&dev, total, st) : cudaMalloc(&dev, total);
+        if (e != cudaSuccess) { dev = nullptr; return fail(CDADAM_ERR_ALLOC, "table allocation: %s", cudaGetErrorString(e)); }
+        char *p = (char *)dev;
+        // pageable sources: the runtime stages them before these calls return
+        CU_TRY(cudaMemcpyAsync(p, off.data(), b_off, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(p + b_off, pbase.data(), b_pb, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(p + b_off + b_pb, first.data(), b_t, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(p + b_off + b_pb + b_t, last.data(), b_t, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaStreamSynchronize(st));
+        tb.d = d; tb.q = q; tb.tile = tile; tb.ntiles = ntiles; tb.nparts = np;
+        tb.off = (const int64_t *)p;
+        tb.pbase = (const int64_t *)(p + b_off);
+        tb.tile_first = (const int32_t *)(p + b_off + b_pb);
+        tb.tile_last = (const int32_t *)(p + b_off + b_pb + b_t);
+        return CDADAM_OK;
+    }
+    void release(cudaStream_t st, bool async)
+    {
+        if (dev) { if (async) cudaFreeAsync(dev, st); else cudaFree(dev); }
+        dev = nullptr;
+    }
+};
+
+bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
+
+}  // namespace
+
+struct cdadam_ctx {
+    int64_t d = 0, k = 0, wp = 0, steps = 0;
+    int n = 0, comp = 0, device = 0;
+    Hyper hp{};
+    TableSet ts;
+    float *ghat_w = nullptr, *ghat_s = nullptr, *gtil = nullptr;
+    float *m = nullptr, *v = nullptr, *vhat = nullptr, *x = nullptr;
+    // scaled sign
+    uint32_t *wbits = nullptr, *sbits = nullptr;
+    float *wscale[2] = {nullptr, nullptr}, *sscale = nullptr, *zero_scale = nullptr;
+    dd *wpart = nullptr, *spart = nullptr;
+    int cur = 0;            // wscale[cur] holds the scales of the last worker payloads
+    bool pending = false;   // the last worker payloads are not yet added to ghat_w
+    // top-k
+    TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
+    float *acc = nullptr;   // dense per-coordinate sum of the workers' sparse payloads
+    // host-gradient staging
+    float *stage = nullptr;
+};
+
+namespace {
+
+template <typename T>
+int dev_zalloc(T **p, size_t count)
+{
+    *p = nullptr;
+    const size_t bytes = (count ? count : 1) * sizeof(T);
+    cudaError_t e = cudaMalloc((void **)p, bytes);
+    if (e != cudaSuccess) return fail(CDADAM_ERR_ALLOC, "cudaMalloc(%zu bytes): %s", bytes, cudaGetErrorString(e));
+    CU_TRY(cudaMemset(*p, 0, bytes));
+    return CDADAM_OK;
+}
+
+int alloc_sign_buffers(cdadam_ctx *c)
+{
+    const int q = c->ts.tb.q;
+    cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
+    cudaFree(c->wpart); cudaFree(c->spart);
+    int rc;
+    if ((rc = dev_zalloc(&c->wscale[0], (size_t)c->n * q))) return rc;
+    if ((rc = dev_zalloc(&c->wscale[1], (size_t)c->n * q))) return rc;
+    if ((rc = dev_zalloc(&c->zero_scale, (size_t)c->n * q))) return rc;
+    if ((rc = dev_zalloc(&c->sscale, (size_t)q))) return rc;
+    if ((rc = dev_zalloc(&c->wpart, (size_t)c->n * c->ts.tb.nparts))) return rc;
+    if ((rc = dev_zalloc(&c->spart, (size_t)c->ts.tb.nparts))) return rc;
+    return CDADAM_OK;
+}
+
+float *state_ptr(cdadam_ctx *c, int name)
+{
+    switch (name) {
+    case CDADAM_STATE_GHAT_W: return c->ghat_w;
+    case CDADAM_STATE_GHAT_S: return c->ghat_s;
+    case CDADAM_STATE_GTIL: return c->gtil;
+    case CDADAM_STATE_M: return c->m;
+    case CDADAM_STATE_V: return c->v;
+    case CDADAM_STATE_VHAT: return c->vhat;
+    case CDADAM_STATE_X: return c->x;
+    }
+    return nullptr;
+}
+
+int check_launch(const char *what)
+{
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(CDADAM_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+    return CDADAM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *cdadam_last_error(void) { return g_err; }
+
+cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float beta1, float beta2,
+                          float lr, float eps)
+{
+    if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
+    if (n < 1 || n > 65535) { fail(CDADAM_ERR_ARG, "n must be in [1, 65535]"); return nullptr; }
+    if (compressor < CDADAM_SIGN || compressor > CDADAM_IDENTITY) { fail(CDADAM_ERR_ARG, "unknown compressor %d", compressor); return nullptr; }
+    if (compressor == CDADAM_TOPK && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k needs 1 <= k <= d"); return nullptr; }
+    cdadam_ctx *c = new (std::nothrow) cdadam_ctx;
+    if (!c) { fail(CDADAM_ERR_ALLOC, "out of host memory"); return nullptr; }
+    c->d = d; c->n = n; c->comp = compressor; c->k = compressor == CDADAM_TOPK ? k : 0;
+    c->wp = (d + 31) / 32;
+    c->hp.beta1 = beta1; c->hp.beta2 = beta2; c->hp.lr = lr; c->hp.nu = eps;
+    c->hp.omb1 = 1.0f - beta1; c->hp.omb2 = 1.0f - beta2;
+    if (cudaGetDevice(&c->device) != cudaSuccess) { fail(CDADAM_ERR_CUDA, "no CUDA device"); delete c; return nullptr; }
+    int rc = CDADAM_OK;
+    const int64_t flat[2] = {0, d};
+    do {
+        if ((rc = dev_zalloc(&c->ghat_w, (size_t)n * d))) break;
+        if ((rc = dev_zalloc(&c->ghat_s, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->gtil, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->m, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->v, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->vhat, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->x, (size_t)d))) break;
+        if (compressor == CDADAM_SIGN) {
+            if ((rc = dev_zalloc(&c->wbits, (size_t)n * c->wp))) break;
+            if ((rc = dev_zalloc(&c->sbits, (size_t)c->wp))) break;
+            if ((rc = c->ts.build(d, 1, flat, choose_tile(d), nullptr, false))) break;
+            if ((rc = alloc_sign_buffers(c))) break;
+        } else if (compressor == CDADAM_TOPK) {
+            if ((rc = dev_zalloc(&c->acc, (size_t)d))) break;
+            if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n))) { fail(rc, "top-k workspace allocation failed"); break; }
+            if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1))) { fail(rc, "top-k workspace allocation failed"); break; }
+        }
+    } while (0);
+    if (rc != CDADAM_OK || cudaDeviceSynchronize() != cudaSuccess) { cdadam_destroy(c); return nullptr; }
+    return c;
+}
+
+void cdadam_destroy(cdadam_ctx *c)
+{
+    if (!c) return;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    cudaFree(c->ghat_w); cudaFree(c->ghat_s); cudaFree(c->gtil);
+    cudaFree(c->m); cudaFree(c->v); cudaFree(c->vhat); cudaFree(c->x);
+    cudaFree(c->wbits); cudaFree(c->sbits);
+    cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
+    cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->acc); cudaFree(c->stage);
+    topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
+    c->ts.release(nullptr, false);
+    delete c;
+}
+
+int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
+{
+    if (!c || !grads) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool vec = aligned16(grads) && c->d % 4 == 0;
+    if (c->comp == CDADAM_SIGN) {
+        const Tables &tb = c->ts.tb;
+        const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
+        float *new_scale = c->wscale[c->cur ^ 1];
+        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, st);
+        launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
+        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, c->d % 4 == 0, st);
+        launch_finalize_scales(c->spart, c->sscale, tb, 1, st);
+        launch_update_sign(c->sbits, c->sscale, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, c->d % 4 == 0, st);
+        c->cur ^= 1;
+        c->pending = true;
+    } else if (c->comp == CDADAM_TOPK) {
+        int rc = topk_step(c->tk_w, c->tk_s, grads, c->ghat_w, c->ghat_s, c->gtil, c->acc, c->d, c->n, vec, st);
+        if (rc) return fail(rc, "top-k step failed");
+        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, c->d % 4 == 0, st);
+    } else {
+        launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, st);
+    }
+    int rc = check_launch("cdadam_step");
+    if (rc) return rc;
+    c->steps += 1;
+    return CDADAM_OK;
+}
+
+int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, void *stream)
+{
+    if (!c || !grads_host) return fail(CDADAM_ERR_ARG, "cdadam_step_host: NULL argument");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = (size_t)c->n * c->d * sizeof(float);
+    if (!c->stage) {
+        cudaError_t e = cudaMalloc((void **)&c->stage, bytes);
+        if (e != cudaSuccess) { c->stage = nullptr; return fail(CDADAM_ERR_ALLOC, "staging buffer: %s", cudaGetErrorString(e)); }
+    }
+    CU_TRY(cudaMemcpyAsync(c->stage, grads_host, bytes, cudaMemcpyHostToDevice, st));
+    int rc = cdadam_step(c, c->stage, stream);
+    if (rc) return rc;
+    if (x_out_host)
+        CU_TRY(cudaMemcpyAsync(x_out_host, c->x, (size_t)c->d * sizeof(float), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    return CDADAM_OK;
+}
+
+const float *cdadam_params(cdadam_ctx *c) { return c ? c->x : nullptr; }
+
+int cdadam_set_params(cdadam_ctx *c, const float *x0, void *stream)
+{
+    return cdadam_set_state(c, CDADAM_STATE_X, x0, stream);
+}
+
+int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
+{
+    if (!c || !offsets) return fail(CDADAM_ERR_ARG, "cdadam_set_segments: NULL argument");
+    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "segments apply to the scaled-sign compressor only");
+    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
+    if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
+    if (offsets[0] != 0 || offsets[q] != c->d) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
+    for (int r = 0; r < q; ++r)
+        if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
+    DeviceGuard guard(c->device);
+    CU_TRY(cudaDeviceSynchronize());
+    int rc = c->ts.build(c->d, q, offsets, choose_tile(c->d), nullptr, false);
+    if (rc) return rc;
+    return alloc_sign_buffers(c);
+}
+
+int cdadam_set_lr(cdadam_ctx *c, float lr)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_lr: NULL context");
+    c->hp.lr = lr;
+    return CDADAM_OK;
+}
+
+int cdadam_get_state(cdadam_ctx *c, int name, float *dst, void *stream)
+{
+    if (!c || !dst) return fail(CDADAM_ERR_ARG, "cdadam_get_state: NULL argument");
+    float *src = state_ptr(c, name);
+    if (!src) return fail(CDADAM_ERR_ARG, "unknown state name %d", name);
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (name == CDADAM_STATE_GHAT_W && c->comp == CDADAM_SIGN && c->pending) {
+        launch_apply_sign(c->ghat_w, c->wbits, c->wscale[c->cur], c->ts.tb, c->n, c->wp, st);
+        int rc = check_launch("apply deferred payload");
+        if (rc) return rc;
+        c->pending = false;
+    }
+    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->n * c->d : (size_t)c->d;
+    CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    return CDADAM_OK;
+}
+
+int cdadam_set_state(cdadam_ctx *c, int name, const float *src, void *stream)
+{
+    if (!c || !src) return fail(CDADAM_ERR_ARG, "cdadam_set_state: NULL argument");
+    float *dst = state_ptr(c, name);
+    if (!dst) return fail(CDADAM_ERR_ARG, "unknown state name %d", name);
+    DeviceGuard guard(c->device);
+    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->n * c->d : (size_t)c->d;
+    CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    if (name == CDADAM_STATE_GHAT_W) c->pending = false;   // the given values are final
+    return CDADAM_OK;
+}
+
+int cdadam_last_payload(cdadam_ctx *c, int who, const void **a, const float **b, int64_t *count)
+{
+    if (!c || !a || !b || !count) return fail(CDADAM_ERR_ARG, "cdadam_last_payload: NULL argument");
+    if (who != CDADAM_SERVER && (who < 0 || who >= c->n)) return fail(CDADAM_ERR_ARG, "who out of range");
+    if (c->steps == 0) return fail(CDADAM_ERR_STATE, "no step has run yet");
+    if (c->comp == CDADAM_SIGN) {
+        if (who == CDADAM_SERVER) { *a = c->sbits; *b = c->sscale; }
+        else { *a = c->wbits + (int64_t)who * c->wp; *b = c->wscale[c->cur] + (int64_t)who * c->ts.tb.q; }
+        *count = c->d;
+        return CDADAM_OK;
+    }
+    if (c->comp == CDADAM_TOPK) {
+        TopkWorkspace *w = who == CDADAM_SERVER ? c->tk_s : c->tk_w;
+        topk_payload(w, who == CDADAM_SERVER ? 0 : who, (const uint32_t **)a, b);
+        *count = c->k;
+        return CDADAM_OK;
+    }
+    return fail(CDADAM_ERR_STATE, "the identity compressor sends no payload");
+}
+
+int64_t cdadam_step_count(cdadam_ctx *c) { return c ? c->steps : 0; }
+
+int cdadam_launches_per_step(cdadam_ctx *c)
+{
+    if (!c) return 0;
+    if (c->comp == CDADAM_SIGN) return 5;
+    if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1;
+    return 1;
+}
+
+int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offsets, uint32_t *bits,
+                         float *scales, void *stream)
+{
+    if (!x || !bits || !scales) return fail(CDADAM_ERR_ARG, "cdadam_compress_sign: NULL argument");
+    if (d < 1 || d >= ((int64_t)1 << 32)) return fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)");
+    const int64_t flat[2] = {0, d};
+    if (!offsets) { offsets = flat; q = 1; }
+    if (q < 1 || (int64_t)q > d || offsets[0] != 0 || offsets[q] != d) return fail(CDADAM_ERR_ARG, "bad segment offsets");
+    for (int r = 0; r < q; ++r)
+        if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing");
+    cudaStream_t st = (cudaStream_t)stream;
+    TableSet ts;
+    int rc = ts.build(d, q, offsets, choose_tile(d), st, true);
+    if (rc) return rc;
+    dd *part = nullptr;
+    cudaError_t e = cudaMallocAsync((void **)&part, (size_t)ts.tb.nparts * sizeof(dd), st);
+    if (e != cudaSuccess) { ts.release(st, true); return fail(CDADAM_ERR_ALLOC, "scratch allocation: %s", cudaGetErrorString(e)); }
+    launch_pack_sign(x, bits, part, ts.tb, aligned16(x) && d % 4 == 0, st);
+    launch_finalize_scales(part, scales, ts.tb, 1, st);
+    rc = check_launch("cdadam_compress_sign");
+    cudaFreeAsync(part, st);
+    ts.release(st, true);
+    return rc;
+}
+
+int cdadam_compress_topk(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, void *stream)
+{
+    if (!x || !idx || !val) return fail(CDADAM_ERR_ARG, "cdadam_compress_topk: NULL argument");
+    if (d < 1 || d >= ((int64_t)1 << 32) || k < 1 || k > d) return fail(CDADAM_ERR_ARG, "need 1 <= k <= d < 2^32");
+    int rc = topk_compress(x, d, k, idx, val, (cudaStream_t)stream);
+    if (rc) return fail(rc, "cdadam_compress_topk failed");
+    return check_launch("cdadam_compress_topk");
+}
+
+}  // extern "C"

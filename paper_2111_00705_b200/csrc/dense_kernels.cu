@@ -1,0 +1,82 @@
+// Dense kernels that need no compressor state: the identity-compressor iteration of
+// Algorithm 1 fused into one pass, and the AMSGrad update alone (used after the top-k
+// payload has been scattered into gtil).
+#include "kernels.h"
+
+namespace cdadam {
+
+// C(u) = u: every line of Algorithm 1 for one coordinate, workers in increasing order.
+__global__ void __launch_bounds__(kBlock)
+k_step_identity(const float *__restrict__ grads, float *__restrict__ ghat_w,
+                float *__restrict__ ghat_s, float *__restrict__ gtil, float *__restrict__ m,
+                float *__restrict__ v, float *__restrict__ vhat, float *__restrict__ x,
+                int64_t d, int n, Hyper hp)
+{
+    const float fn = (float)n;
+    for (int64_t j = (int64_t)blockIdx.x * kBlock + threadIdx.x; j < d;
+         j += (int64_t)gridDim.x * kBlock) {
+        float a = 0.0f;
+        for (int i = 0; i < n; ++i) {
+            const int64_t p = (int64_t)i * d + j;
+            const float gh = ghat_w[p];
+            const float u = __fsub_rn(grads[p], gh);      // c^(i) = u
+            ghat_w[p] = __fadd_rn(gh, u);
+            a = __fadd_rn(a, u);
+        }
+        const float hs = __fadd_rn(ghat_s[j], __fdiv_rn(a, fn));
+        ghat_s[j] = hs;
+        const float gt0 = gtil[j];
+        const float gt = __fadd_rn(gt0, __fsub_rn(hs, gt0));   // c = w
+        gtil[j] = gt;
+        float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
+        amsgrad1(gt, mm, vv, vh, xx, hp);
+        m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
+    }
+}
+
+__global__ void __launch_bounds__(kBlock)
+k_amsgrad(const float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
+          float *__restrict__ vhat, float *__restrict__ x, int64_t d, Hyper hp, int vec_ok)
+{
+    const int64_t nvec = vec_ok ? d / 4 : 0;
+    const int64_t stride = (int64_t)gridDim.x * kBlock;
+    const int64_t t0 = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    for (int64_t q = t0; q < nvec; q += stride) {
+        const int64_t j = q * 4;
+        const float4 G = ld_ro4(gtil + j);
+        float4 M = ld_rw4(m + j), V = ld_rw4(v + j), Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
+        amsgrad1(G.x, M.x, V.x, Vh.x, X.x, hp);
+        amsgrad1(G.y, M.y, V.y, Vh.y, X.y, hp);
+        amsgrad1(G.z, M.z, V.z, Vh.z, X.z, hp);
+        amsgrad1(G.w, M.w, V.w, Vh.w, X.w, hp);
+        st_rw4(m + j, M); st_rw4(v + j, V); st_rw4(vhat + j, Vh); st_rw4(x + j, X);
+    }
+    for (int64_t j = nvec * 4 + t0; j < d; j += stride) {
+        float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
+        amsgrad1(gtil[j], mm, vv, vh, xx, hp);
+        m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
+    }
+}
+
+static unsigned grid_for(int64_t items)
+{
+    int64_t blocks = (items + kBlock - 1) / kBlock;
+    const int64_t cap = 148 * 16;
+    return (unsigned)(blocks < 1 ? 1 : (blocks > cap ? cap : blocks));
+}
+
+void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
+                          float *m, float *v, float *vhat, float *x, int64_t d, int n,
+                          Hyper hp, cudaStream_t st)
+{
+    k_step_identity<<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x,
+                                                    d, n, hp);
+}
+
+void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
+                    Hyper hp, bool vec_ok, cudaStream_t st)
+{
+    k_amsgrad<<<grid_for(vec_ok ? d / 4 : d), kBlock, 0, st>>>(gtil, m, v, vhat, x, d, hp, vec_ok);
+}
+
+}  // namespace cdadam

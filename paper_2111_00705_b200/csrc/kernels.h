@@ -1,0 +1,44 @@
+// Host-side launchers of the CD-Adam kernels.  Every launcher queues work on `st` and
+// returns; errors are picked up by the caller with cudaGetLastError().
+#pragma once
+#include "common.cuh"
+
+namespace cdadam {
+
+// ---- scaled sign -------------------------------------------------------------------
+// Worker pass (Algorithm 1 lines 5-6) for all n workers: applies the previous payload
+// (bits in wbits, scales in scale_old) to ghat_w, forms u = g - ghat_w, packs sign(u) into
+// wbits and writes per-tile double-double partial sums of |u| to wpart.
+void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
+                        const float *scale_old, dd *wpart, const Tables &tb, int n,
+                        int64_t wp, bool vec_ok, cudaStream_t st);
+// Correctly rounded scale of every (row, segment) from the partial sums.
+void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
+                            cudaStream_t st);
+// Server pass A (lines 8-9): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
+// sign(w) into sbits and writes partial sums of |w| to spart.
+void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
+                        const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
+                        int n, int64_t wp, bool vec_ok, cudaStream_t st);
+// Server pass B and worker update (lines 10, 12-16): gtil += decode(c); AMSGrad.
+void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil, float *m,
+                        float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
+                        bool vec_ok, cudaStream_t st);
+// ghat_w += decode(bits, scales) for all workers (applies a deferred payload).
+void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
+                       const Tables &tb, int n, int64_t wp, cudaStream_t st);
+// Stand-alone scaled-sign compressor of one vector: bits and partial sums of |x|.
+void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
+                      bool vec_ok, cudaStream_t st);
+
+// ---- identity ----------------------------------------------------------------------
+// The whole iteration with C(u) = u, one fused pass.
+void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
+                          float *m, float *v, float *vhat, float *x, int64_t d, int n,
+                          Hyper hp, cudaStream_t st);
+
+// ---- AMSGrad alone (top-k path: gtil already updated) ---------------------------------
+void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
+                    Hyper hp, bool vec_ok, cudaStream_t st);
+
+}  // namespace cdadam

@@ -1,0 +1,396 @@
+// Scaled-sign path of Algorithm 1 (CD-Adam) for sm_100a: worker pass, server pass A,
+// server pass B + AMSGrad, scale finalisation, deferred-payload application.
+//
+// Every kernel streams its vectors exactly once.  A block owns one tile of the index
+// space.  Tiles that lie inside one segment, inside [0, d) and whose rows are 16-byte
+// aligned take the vector path (128-bit accesses, ballot packing, no bounds checks); all
+// other tiles (segment boundaries, the ragged tail, unaligned rows) take a scalar path with
+// the same arithmetic in the same order, so both paths give identical bits.
+#include "kernels.h"
+
+namespace cdadam {
+
+constexpr uint32_t kFull = 0xffffffffu;
+
+__device__ __forceinline__ float signed_scale(uint32_t bit, float s) { return bit ? s : -s; }
+
+// ------------------------------------------------------------------------------------
+// Worker pass.  grid = (ntiles, n).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
+              uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
+              dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
+{
+    const int i = blockIdx.y;
+    const int64_t T = blockIdx.x;
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    const float *g = grads + (int64_t)i * tb.d;
+    float *gh = ghat_w + (int64_t)i * tb.d;
+    uint32_t *bw = wbits + (int64_t)i * wp;
+    const float *so = scale_old + (int64_t)i * tb.q;
+    dd *part = wpart + (int64_t)i * tb.nparts + tb.pbase[T];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    if (vec_ok && first == last && base + tb.tile <= tb.d) {
+        const float s = so[first];
+        dd acc = {0.0, 0.0};
+        for (int it = 0; it < tb.tile / kSub; ++it) {
+            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+            float4 G[4], H[4];
+            uint32_t ow[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int64_t j = wb + v * 128 + lane * 4;
+                G[v] = ld_ro4(g + j);
+                H[v] = ld_rw4(gh + j);
+                ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
+            }
+            uint32_t B[4][4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const uint32_t nib = ow[v] >> ((lane & 7) * 4);
+                // ghat_{t-1} = ghat_{t-2} + c_{t-1}: the previous payload, applied now
+                H[v].x = __fadd_rn(H[v].x, signed_scale(nib & 1u, s));
+                H[v].y = __fadd_rn(H[v].y, signed_scale(nib & 2u, s));
+                H[v].z = __fadd_rn(H[v].z, signed_scale(nib & 4u, s));
+                H[v].w = __fadd_rn(H[v].w, signed_scale(nib & 8u, s));
+                st_rw4(gh + wb + v * 128 + lane * 4, H[v]);
+                const float ux = __fsub_rn(G[v].x, H[v].x), uy = __fsub_rn(G[v].y, H[v].y);
+                const float uz = __fsub_rn(G[v].z, H[v].z), uw = __fsub_rn(G[v].w, H[v].w);
+                dd_acc(acc, fabsf(ux)); dd_acc(acc, fabsf(uy));
+                dd_acc(acc, fabsf(uz)); dd_acc(acc, fabsf(uw));
+                B[v][0] = __ballot_sync(kFull, ux >= 0.0f);
+                B[v][1] = __ballot_sync(kFull, uy >= 0.0f);
+                B[v][2] = __ballot_sync(kFull, uz >= 0.0f);
+                B[v][3] = __ballot_sync(kFull, uw >= 0.0f);
+            }
+            const uint32_t word = warp_words(B, lane);
+            if (lane < 16) bw[(wb >> 5) + lane] = word;
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[0] = acc;
+        return;
+    }
+
+    // scalar path: lane L of a warp holds coordinate (word start + L), ballot = word
+    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
+    for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+        const bool valid = j < end;
+        float u = -1.0f;
+        if (valid) {
+            const int r = find_segment(tb.off, first, last, j);
+            const uint32_t bit = (bw[j >> 5] >> (j & 31)) & 1u;
+            const float hn = __fadd_rn(gh[j], signed_scale(bit, so[r]));
+            gh[j] = hn;
+            u = __fsub_rn(g[j], hn);
+        }
+        const uint32_t word = __ballot_sync(kFull, valid && u >= 0.0f);
+        if (lane == 0) bw[j >> 5] = word;
+    }
+    __syncthreads();
+    for (int r = first; r <= last; ++r) {
+        const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
+        dd acc = {0.0, 0.0};
+        for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
+            dd_acc(acc, fabsf(__fsub_rn(g[j], gh[j])));
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[r - first] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Scale of (row, segment): partial sums added in a fixed order, rounded to binary64,
+// divided by the segment length in binary64, rounded to binary32.  grid = (q, rows).
+// ------------------------------------------------------------------------------------
+constexpr int kFinBlock = 512;
+
+__global__ void __launch_bounds__(kFinBlock)
+k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Tables tb)
+{
+    const int r = blockIdx.x, row = blockIdx.y;
+    const int64_t lo = tb.off[r], hi = tb.off[r + 1];
+    const int64_t T0 = lo / tb.tile, T1 = (hi - 1) / tb.tile;
+    const dd *p = part + (int64_t)row * tb.nparts;
+    dd acc = {0.0, 0.0};
+    for (int64_t T = T0 + threadIdx.x; T <= T1; T += kFinBlock)
+        acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
+    acc = block_sum<kFinBlock>(acc);
+    if (threadIdx.x == 0) {
+        const double l1 = __dadd_rn(acc.hi, acc.lo);
+        scales[(int64_t)row * tb.q + r] = __double2float_rn(__ddiv_rn(l1, (double)(hi - lo)));
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Server pass A.  grid = (ntiles).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
+              float *__restrict__ ghat_s, const float *__restrict__ gtil,
+              uint32_t *__restrict__ sbits, dd *__restrict__ spart, Tables tb, int n,
+              int64_t wp, int vec_ok)
+{
+    const int64_t T = blockIdx.x;
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    dd *part = spart + tb.pbase[T];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float fn = (float)n;
+
+    if (vec_ok && first == last && base + tb.tile <= tb.d) {
+        dd acc = {0.0, 0.0};
+        for (int it = 0; it < tb.tile / kSub; ++it) {
+            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+            float4 H[4], Gt[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int64_t j = wb + v * 128 + lane * 4;
+                H[v] = ld_rw4(ghat_s + j);
+                Gt[v] = ld_ro4(gtil + j);
+            }
+            float a[4][4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) a[v][0] = a[v][1] = a[v][2] = a[v][3] = 0.0f;
+            const uint32_t *wq = wbits + (wb >> 5) + (lane >> 3);
+            const int sh = (lane & 7) * 4;
+#pragma unroll 4
+            for (int i = 0; i < n; ++i) {            // workers in increasing order
+                const float s = __ldg(wscale + (int64_t)i * tb.q + first);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const uint32_t nib = ld_ro_u32(wq + (int64_t)i * wp + v * 4) >> sh;
+                    a[v][0] = __fadd_rn(a[v][0], signed_scale(nib & 1u, s));
+                    a[v][1] = __fadd_rn(a[v][1], signed_scale(nib & 2u, s));
+                    a[v][2] = __fadd_rn(a[v][2], signed_scale(nib & 4u, s));
+                    a[v][3] = __fadd_rn(a[v][3], signed_scale(nib & 8u, s));
+                }
+            }
+            uint32_t B[4][4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                H[v].x = __fadd_rn(H[v].x, __fdiv_rn(a[v][0], fn));
+                H[v].y = __fadd_rn(H[v].y, __fdiv_rn(a[v][1], fn));
+                H[v].z = __fadd_rn(H[v].z, __fdiv_rn(a[v][2], fn));
+                H[v].w = __fadd_rn(H[v].w, __fdiv_rn(a[v][3], fn));
+                st_rw4(ghat_s + wb + v * 128 + lane * 4, H[v]);
+                const float wx = __fsub_rn(H[v].x, Gt[v].x), wy = __fsub_rn(H[v].y, Gt[v].y);
+                const float wz = __fsub_rn(H[v].z, Gt[v].z), ww = __fsub_rn(H[v].w, Gt[v].w);
+                dd_acc(acc, fabsf(wx)); dd_acc(acc, fabsf(wy));
+                dd_acc(acc, fabsf(wz)); dd_acc(acc, fabsf(ww));
+                B[v][0] = __ballot_sync(kFull, wx >= 0.0f);
+                B[v][1] = __ballot_sync(kFull, wy >= 0.0f);
+                B[v][2] = __ballot_sync(kFull, wz >= 0.0f);
+                B[v][3] = __ballot_sync(kFull, ww >= 0.0f);
+            }
+            const uint32_t word = warp_words(B, lane);
+            if (lane < 16) sbits[(wb >> 5) + lane] = word;
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[0] = acc;
+        return;
+    }
+
+    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
+    for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+        const bool valid = j < end;
+        float w = -1.0f;
+        if (valid) {
+            const int r = find_segment(tb.off, first, last, j);
+            float a = 0.0f;
+            for (int i = 0; i < n; ++i) {
+                const uint32_t bit = (wbits[(int64_t)i * wp + (j >> 5)] >> (j & 31)) & 1u;
+                a = __fadd_rn(a, signed_scale(bit, wscale[(int64_t)i * tb.q + r]));
+            }
+            const float hn = __fadd_rn(ghat_s[j], __fdiv_rn(a, fn));
+            ghat_s[j] = hn;
+            w = __fsub_rn(hn, gtil[j]);
+        }
+        const uint32_t word = __ballot_sync(kFull, valid && w >= 0.0f);
+        if (lane == 0) sbits[j >> 5] = word;
+    }
+    __syncthreads();
+    for (int r = first; r <= last; ++r) {
+        const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
+        dd acc = {0.0, 0.0};
+        for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
+            dd_acc(acc, fabsf(__fsub_rn(ghat_s[j], gtil[j])));
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[r - first] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Server pass B + worker update.  grid = (ntiles).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ sscale,
+              float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
+              float *__restrict__ vhat, float *__restrict__ x, Tables tb, Hyper hp, int vec_ok)
+{
+    const int64_t T = blockIdx.x;
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    if (vec_ok && first == last && base + tb.tile <= tb.d) {
+        const float s = __ldg(sscale + first);
+        for (int it = 0; it < tb.tile / kSub; ++it) {
+            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+#pragma unroll 2
+            for (int v4 = 0; v4 < 4; ++v4) {
+                const int64_t j = wb + v4 * 128 + lane * 4;
+                float4 Gt = ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
+                float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
+                const uint32_t nib = ld_ro_u32(sbits + (wb >> 5) + v4 * 4 + (lane >> 3)) >>
+                                     ((lane & 7) * 4);
+                Gt.x = __fadd_rn(Gt.x, signed_scale(nib & 1u, s));
+                Gt.y = __fadd_rn(Gt.y, signed_scale(nib & 2u, s));
+                Gt.z = __fadd_rn(Gt.z, signed_scale(nib & 4u, s));
+                Gt.w = __fadd_rn(Gt.w, signed_scale(nib & 8u, s));
+                amsgrad1(Gt.x, M.x, V.x, Vh.x, X.x, hp);
+                amsgrad1(Gt.y, M.y, V.y, Vh.y, X.y, hp);
+                amsgrad1(Gt.z, M.z, V.z, Vh.z, X.z, hp);
+                amsgrad1(Gt.w, M.w, V.w, Vh.w, X.w, hp);
+                st_rw4(gtil + j, Gt); st_rw4(m + j, M); st_rw4(v + j, V);
+                st_rw4(vhat + j, Vh); st_rw4(x + j, X);
+            }
+        }
+        return;
+    }
+
+    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
+    for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
+        const int r = find_segment(tb.off, first, last, j);
+        const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
+        const float gt = __fadd_rn(gtil[j], signed_scale(bit, sscale[r]));
+        gtil[j] = gt;
+        float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
+        amsgrad1(gt, mm, vv, vh, xx, hp);
+        m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// ghat_w += decode(bits, scales): applies a payload whose application was deferred.
+// grid = (ntiles, n).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_apply_sign(float *__restrict__ ghat_w, const uint32_t *__restrict__ wbits,
+             const float *__restrict__ scales, Tables tb, int64_t wp)
+{
+    const int i = blockIdx.y;
+    const int64_t T = blockIdx.x;
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile, end = min(base + (int64_t)tb.tile, tb.d);
+    float *gh = ghat_w + (int64_t)i * tb.d;
+    const uint32_t *bw = wbits + (int64_t)i * wp;
+    for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
+        const int r = find_segment(tb.off, first, last, j);
+        const uint32_t bit = (bw[j >> 5] >> (j & 31)) & 1u;
+        gh[j] = __fadd_rn(gh[j], signed_scale(bit, scales[(int64_t)i * tb.q + r]));
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Stand-alone compressor: sign bits of x and partial sums of |x|.  grid = (ntiles).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__restrict__ part_all,
+            Tables tb, int vec_ok)
+{
+    const int64_t T = blockIdx.x;
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    dd *part = part_all + tb.pbase[T];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    if (vec_ok && first == last && base + tb.tile <= tb.d) {
+        dd acc = {0.0, 0.0};
+        for (int it = 0; it < tb.tile / kSub; ++it) {
+            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+            float4 X[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) X[v] = ld_ro4(x + wb + v * 128 + lane * 4);
+            uint32_t B[4][4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                dd_acc(acc, fabsf(X[v].x)); dd_acc(acc, fabsf(X[v].y));
+                dd_acc(acc, fabsf(X[v].z)); dd_acc(acc, fabsf(X[v].w));
+                B[v][0] = __ballot_sync(kFull, X[v].x >= 0.0f);
+                B[v][1] = __ballot_sync(kFull, X[v].y >= 0.0f);
+                B[v][2] = __ballot_sync(kFull, X[v].z >= 0.0f);
+                B[v][3] = __ballot_sync(kFull, X[v].w >= 0.0f);
+            }
+            const uint32_t word = warp_words(B, lane);
+            if (lane < 16) bits[(wb >> 5) + lane] = word;
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[0] = acc;
+        return;
+    }
+
+    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
+    for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+        const bool valid = j < end;
+        const uint32_t word = __ballot_sync(kFull, valid && x[valid ? j : base] >= 0.0f);
+        if (lane == 0) bits[j >> 5] = word;
+    }
+    for (int r = first; r <= last; ++r) {
+        const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
+        dd acc = {0.0, 0.0};
+        for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock) dd_acc(acc, fabsf(x[j]));
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[r - first] = acc;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// launchers
+// ------------------------------------------------------------------------------------
+void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
+                        const float *scale_old, dd *wpart, const Tables &tb, int n,
+                        int64_t wp, bool vec_ok, cudaStream_t st)
+{
+    dim3 grid((unsigned)tb.ntiles, (unsigned)n);
+    k_worker_sign<<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+}
+
+void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
+                            cudaStream_t st)
+{
+    dim3 grid((unsigned)tb.q, (unsigned)rows);
+    k_finalize_scales<<<grid, kFinBlock, 0, st>>>(part, scales, tb);
+}
+
+void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
+                        const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
+                        int n, int64_t wp, bool vec_ok, cudaStream_t st)
+{
+    k_server_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+                                                          spart, tb, n, wp, vec_ok);
+}
+
+void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil, float *m,
+                        float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
+                        bool vec_ok, cudaStream_t st)
+{
+    k_update_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(sbits, sscale, gtil, m, v, vhat, x, tb,
+                                                          hp, vec_ok);
+}
+
+void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
+                       const Tables &tb, int n, int64_t wp, cudaStream_t st)
+{
+    dim3 grid((unsigned)tb.ntiles, (unsigned)n);
+    k_apply_sign<<<grid, kBlock, 0, st>>>(ghat_w, wbits, scales, tb, wp);
+}
+
+void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
+                      bool vec_ok, cudaStream_t st)
+{
+    k_pack_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(x, bits, part, tb, vec_ok);
+}
+
+}  // namespace cdadam

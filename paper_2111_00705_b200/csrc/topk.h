@@ -1,0 +1,37 @@
+// Top-k compressor (Appendix A) as an exact three-level radix select on the magnitude
+// bits, for `rows` independent vectors at once, plus the sparse server aggregation.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace cdadam {
+
+struct TopkWorkspace;
+
+// Scratch and payload buffers for selecting k of d coordinates in each of `rows` vectors.
+// If idx/val are NULL the workspace owns the payload arrays (rows x k each).
+int topk_workspace_create(TopkWorkspace **w, int64_t d, int64_t k, int rows,
+                          uint32_t *idx = nullptr, float *val = nullptr);
+void topk_workspace_destroy(TopkWorkspace *w);
+void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
+int topk_launches_per_step(int n);
+
+// For every row r: u = a_r - b_r (b may be NULL: u = a_r); keep the k coordinates of
+// largest |u| (ties: lower index); write their indices (increasing) and values u_j to the
+// payload; if update_b, b_r[j] += u_j at the kept coordinates.  a, b: rows x d.
+void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
+                 cudaStream_t st);
+
+// Worker stage, sparse server aggregation and server stage of Algorithm 1 with top-k:
+//   ghat_w[i] += C(g_i - ghat_w[i]);  ghat_s += (sum_i c_i) / n on the touched coordinates;
+//   gtil += C(ghat_s - gtil).
+// acc: d floats, all zero on entry and on exit.
+int topk_step(TopkWorkspace *ww, TopkWorkspace *ws, const float *grads, float *ghat_w,
+              float *ghat_s, float *gtil, float *acc, int64_t d, int n, bool vec_ok,
+              cudaStream_t st);
+
+// Stand-alone top-k of one vector into caller buffers (allocates and frees scratch).
+int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,
+                  cudaStream_t st);
+
+}  // namespace cdadam

@@ -1,0 +1,566 @@
+// Top-k compressor (Appendix A: keep the k coordinates of largest magnitude) for sm_100a.
+//
+// Exact selection without sorting: the magnitude bits key = bits(|u|) (31 bits; for finite
+// floats integer order = value order) are resolved by a three-level radix select,
+//   level 1: key bits 30..20, histogram over a dense pass;
+//   level 2: key bits 19..9 and level 3: key bits 8..0, histograms over the candidates only
+// which yields the exact k-th largest key T.  Coordinates with key > T are kept; among those
+// with key == T the ones of lowest index are kept until k is reached.  The selection lives in
+// bitmaps (1 bit per coordinate), so the ordered compaction (index-increasing payload) costs
+// d/8 bytes per pass instead of another pass over the data.  All counters are integer
+// atomics: the result does not depend on the order of execution.
+#include "topk.h"
+
+#include "../../include/cdadam.h"
+#include "common.cuh"
+
+namespace cdadam {
+
+constexpr uint32_t kFull = 0xffffffffu;
+constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
+constexpr int kHistStride = kBins1 + kBins2 + kBins3;
+constexpr int kTileWords = 1024;      // bitmap words per block in the sparse passes
+
+struct Sel {                          // outcome of the three levels for one row
+    uint32_t b1, k1, c1;              // bucket, entries still to take inside it, its size
+    uint32_t b2, k2, c2;
+    uint32_t b3, k3, c3;              // T = b1<<20 | b2<<9 | b3; take k3 of the c3 ties
+    uint32_t pad[3];
+};
+
+struct TopkWorkspace {
+    int64_t d, k, wp, nbt;
+    int rows;
+    uint32_t *hist;                   // rows x kHistStride
+    Sel *sel;                         // rows
+    uint32_t *bm_in, *bm_cand;        // rows x wp
+    uint32_t *cnt_tie, *cnt_fin;      // rows x nbt
+    uint32_t *idx;                    // rows x k
+    float *val;                       // rows x k
+    bool own_payload;
+};
+
+__device__ __forceinline__ uint32_t key_of(float u) { return __float_as_uint(u) & 0x7fffffffu; }
+
+template <bool HAS_B>
+__device__ __forceinline__ float diff1(const float *a, const float *b, int64_t j)
+{
+    return HAS_B ? __fsub_rn(a[j], b[j]) : a[j];
+}
+
+// exclusive prefix sum over the 256 threads of a block; all threads must call
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
+{
+    __shared__ uint32_t ws[kBlock / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    __syncthreads();
+    if (lane == 31) ws[warp] = inc;
+    __syncthreads();
+    uint32_t before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kBlock / 32; ++w) {
+        const uint32_t s = ws[w];
+        if (w < warp) before += s;
+        all += s;
+    }
+    total = all;
+    return before + inc - v;
+}
+
+// ------------------------------------------------------------------------------------
+// Level 1: histogram of key >> 20 over all coordinates.  grid = (ceil(d/4096), rows).
+// ------------------------------------------------------------------------------------
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
+             uint32_t *__restrict__ hist_all, int64_t d, int vec_ok)
+{
+    __shared__ uint32_t h[kBins1];
+    for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
+    __syncthreads();
+    const int row = blockIdx.y;
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const int64_t base = (int64_t)blockIdx.x * kSub;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (vec_ok && base + kSub <= d) {
+        const int64_t wb = base + warp * kWarpSpan;
+        float4 A[4], Bv[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int64_t j = wb + v * 128 + lane * 4;
+            A[v] = ld_ro4(a + j);
+            if (HAS_B) Bv[v] = ld_ro4(b + j);
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            if (HAS_B) {
+                A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
+                A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
+            }
+            atomicAdd(&h[key_of(A[v].x) >> 20], 1u);
+            atomicAdd(&h[key_of(A[v].y) >> 20], 1u);
+            atomicAdd(&h[key_of(A[v].z) >> 20], 1u);
+            atomicAdd(&h[key_of(A[v].w) >> 20], 1u);
+        }
+    } else {
+        const int64_t end = min(base + (int64_t)kSub, d);
+        for (int64_t j = base + threadIdx.x; j < end; j += kBlock)
+            atomicAdd(&h[key_of(diff1<HAS_B>(a, b, j)) >> 20], 1u);
+    }
+    __syncthreads();
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride;
+    for (int t = threadIdx.x; t < kBins1; t += kBlock)
+        if (h[t]) atomicAdd(&hist[t], h[t]);
+}
+
+// ------------------------------------------------------------------------------------
+// Pick the bucket that holds the `want`-th largest entry of a histogram: the bucket b with
+// count(bins > b) < want <= count(bins >= b).  grid = (rows), one block.
+// level 0/1/2 selects which histogram and which fields of Sel are read and written.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, int level,
+            uint32_t k)
+{
+    __shared__ uint32_t tot[kBlock];
+    const int row = blockIdx.x;
+    Sel *sel = sel_all + row;
+    const int nb = level == 2 ? kBins3 : kBins1;
+    const uint32_t *hist = hist_all + (int64_t)row * kHistStride +
+                           (level == 0 ? 0 : level == 1 ? kBins1 : kBins1 + kBins2);
+    const uint32_t want = level == 0 ? k : level == 1 ? sel->k1 : sel->k2;
+    const int per = nb / kBlock;                    // 8 or 2 contiguous bins per thread
+    const int lo = threadIdx.x * per;
+    uint32_t mine = 0;
+    for (int t = 0; t < per; ++t) mine += hist[lo + t];
+    tot[threadIdx.x] = mine;
+    __syncthreads();
+    uint32_t above = 0;                             // entries in bins owned by later threads
+    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+    for (int t = per - 1; t >= 0; --t) {
+        const uint32_t c = hist[lo + t];
+        if (above < want && above + c >= want) {
+            const uint32_t bucket = lo + t, rem = want - above;
+            if (level == 0) { sel->b1 = bucket; sel->k1 = rem; sel->c1 = c; }
+            else if (level == 1) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
+            else { sel->b3 = bucket; sel->k3 = rem; sel->c3 = c; }
+        }
+        above += c;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Second dense pass: bitmaps of "key >> 20 above the level-1 bucket" (certainly kept) and
+// "inside it" (candidates), and the level-2 histogram of the candidates.
+// grid = (ceil(d/4096), rows).
+// ------------------------------------------------------------------------------------
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
+            const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
+            uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
+            int64_t wp, int vec_ok)
+{
+    __shared__ uint32_t h[kBins2];
+    for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
+    __syncthreads();
+    const int row = blockIdx.y;
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
+    const uint32_t b1 = sel_all[row].b1;
+    const int64_t base = (int64_t)blockIdx.x * kSub;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (vec_ok && base + kSub <= d) {
+        const int64_t wb = base + warp * kWarpSpan;
+        float4 A[4], Bv[4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int64_t j = wb + v * 128 + lane * 4;
+            A[v] = ld_ro4(a + j);
+            if (HAS_B) Bv[v] = ld_ro4(b + j);
+        }
+        uint32_t BI[4][4], BC[4][4];
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            if (HAS_B) {
+                A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
+                A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
+            }
+            const uint32_t kx = key_of(A[v].x), ky = key_of(A[v].y);
+            const uint32_t kz = key_of(A[v].z), kw = key_of(A[v].w);
+            BI[v][0] = __ballot_sync(kFull, (kx >> 20) > b1);
+            BI[v][1] = __ballot_sync(kFull, (ky >> 20) > b1);
+            BI[v][2] = __ballot_sync(kFull, (kz >> 20) > b1);
+            BI[v][3] = __ballot_sync(kFull, (kw >> 20) > b1);
+            const bool cx = (kx >> 20) == b1, cy = (ky >> 20) == b1;
+            const bool cz = (kz >> 20) == b1, cw = (kw >> 20) == b1;
+            BC[v][0] = __ballot_sync(kFull, cx);
+            BC[v][1] = __ballot_sync(kFull, cy);
+            BC[v][2] = __ballot_sync(kFull, cz);
+            BC[v][3] = __ballot_sync(kFull, cw);
+            if (cx) atomicAdd(&h[(kx >> 9) & (kBins2 - 1)], 1u);
+            if (cy) atomicAdd(&h[(ky >> 9) & (kBins2 - 1)], 1u);
+            if (cz) atomicAdd(&h[(kz >> 9) & (kBins2 - 1)], 1u);
+            if (cw) atomicAdd(&h[(kw >> 9) & (kBins2 - 1)], 1u);
+        }
+        const uint32_t wi = warp_words(BI, lane), wc = warp_words(BC, lane);
+        if (lane < 16) { bm_in[(wb >> 5) + lane] = wi; bm_cand[(wb >> 5) + lane] = wc; }
+    } else {
+        const int64_t end = min(base + (int64_t)kSub, d);
+        for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+            const bool valid = j < end;
+            const uint32_t key = valid ? key_of(diff1<HAS_B>(a, b, j)) : 0u;
+            const bool in = valid && (key >> 20) > b1, cand = valid && (key >> 20) == b1;
+            const uint32_t wi = __ballot_sync(kFull, in), wc = __ballot_sync(kFull, cand);
+            if (lane == 0) { bm_in[j >> 5] = wi; bm_cand[j >> 5] = wc; }
+            if (cand) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
+    for (int t = threadIdx.x; t < kBins2; t += kBlock)
+        if (h[t]) atomicAdd(&hist[t], h[t]);
+}
+
+// ------------------------------------------------------------------------------------
+// Level 3: histogram of key & 511 over the candidates whose upper 22 key bits match.
+// grid = (nbt, rows); a thread walks the set bits of its bitmap words.
+// ------------------------------------------------------------------------------------
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
+             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ bm_cand_all,
+             uint32_t *__restrict__ hist_all, int64_t d, int64_t wp)
+{
+    __shared__ uint32_t h[kBins3];
+    for (int t = threadIdx.x; t < kBins3; t += kBlock) h[t] = 0;
+    __syncthreads();
+    const int row = blockIdx.y;
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const uint32_t *bm_cand = bm_cand_all + (int64_t)row * wp;
+    const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+        uint32_t word = bm_cand[w0 + t];
+        while (word) {
+            const int bit = __ffs(word) - 1;
+            word &= word - 1;
+            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+            if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+        }
+    }
+    __syncthreads();
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1 + kBins2;
+    for (int t = threadIdx.x; t < kBins3; t += kBlock)
+        if (h[t]) atomicAdd(&hist[t], h[t]);
+}
+
+// ------------------------------------------------------------------------------------
+// With the threshold key T known: bm_in |= candidates with key > T; bm_cand := candidates
+// with key == T (the ties).  If all ties are needed they are merged at once; otherwise the
+// per-tile tie counts feed the ordered pick below.  grid = (nbt, rows).
+// ------------------------------------------------------------------------------------
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
+               const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
+               uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ cnt_tie_all,
+               int64_t d, int64_t wp, int64_t nbt)
+{
+    const int row = blockIdx.y;
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
+    const Sel s = sel_all[row];
+    const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
+    const bool all_ties = s.k3 == s.c3;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+    uint32_t nt = 0;
+    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+        uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
+        while (word) {
+            const int bit = __ffs(word) - 1;
+            word &= word - 1;
+            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+            if (key > T) keep |= 1u << bit;
+            else if (key == T) tie |= 1u << bit;
+        }
+        if (all_ties) keep |= tie;
+        bm_in[w0 + t] = keep;
+        bm_cand[w0 + t] = tie;
+        nt += __popc(tie);
+    }
+    uint32_t total;
+    block_excl_scan(nt, total);
+    if (threadIdx.x == 0) cnt_tie_all[(int64_t)row * nbt + blockIdx.x] = total;
+}
+
+// exclusive scan of the per-tile counts of every row, in place.  grid = (rows).
+__global__ void __launch_bounds__(kBlock)
+k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt)
+{
+    uint32_t *cnt = cnt_all + (int64_t)blockIdx.x * nbt;
+    uint32_t carry = 0;
+    for (int64_t c = 0; c < nbt; c += kBlock) {
+        const int64_t t = c + threadIdx.x;
+        const uint32_t v = t < nbt ? cnt[t] : 0u;
+        uint32_t total;
+        const uint32_t ex = block_excl_scan(v, total);
+        if (t < nbt) cnt[t] = carry + ex;
+        carry += total;
+    }
+}
+
+__device__ __forceinline__ uint32_t lowest_set_bits(uint32_t word, uint32_t count)
+{
+    uint32_t m = 0;
+    for (uint32_t t = 0; t < count && word; ++t) {
+        const uint32_t lb = word & (0u - word);
+        m |= lb;
+        word ^= lb;
+    }
+    return m;
+}
+
+// ------------------------------------------------------------------------------------
+// Ties: keep those of global rank < k3 in index order (only if not all are kept), then
+// count the kept coordinates of every tile.  A thread owns 4 consecutive bitmap words.
+// grid = (nbt, rows).
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_topk_ties(const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
+            const uint32_t *__restrict__ bm_cand_all, const uint32_t *__restrict__ tie_off_all,
+            uint32_t *__restrict__ cnt_fin_all, int64_t wp, int64_t nbt)
+{
+    const int row = blockIdx.y;
+    uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
+    const uint32_t *bm_tie = bm_cand_all + (int64_t)row * wp;
+    const Sel s = sel_all[row];
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+    uint32_t keep[4], tie[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
+        tie[m] = w0 + m < wp ? bm_tie[w0 + m] : 0u;
+    }
+    if (s.k3 != s.c3) {                               // block-uniform
+        const uint32_t mine = __popc(tie[0]) + __popc(tie[1]) + __popc(tie[2]) + __popc(tie[3]);
+        uint32_t total;
+        uint32_t rank = block_excl_scan(mine, total) + tie_off_all[(int64_t)row * nbt + blockIdx.x];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            if (tie[m] && rank < s.k3) {
+                keep[m] |= lowest_set_bits(tie[m], s.k3 - rank);
+                bm_in[w0 + m] = keep[m];
+            }
+            rank += __popc(tie[m]);
+        }
+    }
+    uint32_t total;
+    block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total);
+    if (threadIdx.x == 0) cnt_fin_all[(int64_t)row * nbt + blockIdx.x] = total;
+}
+
+// ------------------------------------------------------------------------------------
+// Ordered compaction of the selection bitmap into the payload (index-increasing), and the
+// state update b_j += u_j at the kept coordinates (Algorithm 1 lines 6 / 10).
+// grid = (nbt, rows).
+// ------------------------------------------------------------------------------------
+template <bool HAS_B, bool UPDATE_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_emit(const float *__restrict__ a_all, float *__restrict__ b_all,
+            const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
+            uint32_t *__restrict__ idx_all, float *__restrict__ val_all, int64_t d, int64_t wp,
+            int64_t nbt, int64_t k)
+{
+    const int row = blockIdx.y;
+    const float *a = a_all + (int64_t)row * d;
+    float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
+    uint32_t *idx = idx_all + (int64_t)row * k;
+    float *val = val_all + (int64_t)row * k;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+    uint32_t keep[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
+    uint32_t total;
+    uint32_t rank = block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total) +
+                    fin_off_all[(int64_t)row * nbt + blockIdx.x];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        uint32_t word = keep[m];
+        while (word) {
+            const int bit = __ffs(word) - 1;
+            word &= word - 1;
+            const int64_t j = (w0 + m) * 32 + bit;
+            if (rank < k) {
+                float u;
+                if (HAS_B) {
+                    const float bj = b[j];
+                    u = __fsub_rn(a[j], bj);
+                    if (UPDATE_B) b[j] = __fadd_rn(bj, u);
+                } else {
+                    u = a[j];
+                }
+                idx[rank] = (uint32_t)j;
+                val[rank] = u;
+            }
+            ++rank;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// Sparse server aggregation (Algorithm 1 line 8).
+// ------------------------------------------------------------------------------------
+// acc[idx[t]] += val[t] for one worker's payload (its indices are distinct).
+__global__ void __launch_bounds__(kBlock)
+k_scatter_add(float *__restrict__ acc, const uint32_t *__restrict__ idx,
+              const float *__restrict__ val, int64_t k)
+{
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t < k) {
+        const uint32_t j = idx[t];
+        acc[j] = __fadd_rn(acc[j], val[t]);
+    }
+}
+
+// For every coordinate some worker sent: ghat_s += acc / n; acc = 0.  A thread owns one
+// bitmap word of the union of the n selection bitmaps.
+__global__ void __launch_bounds__(kBlock)
+k_server_apply(const uint32_t *__restrict__ bm_all, int n, int64_t wp, float *__restrict__ acc,
+               float *__restrict__ ghat_s, float fn)
+{
+    const int64_t w = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (w >= wp) return;
+    uint32_t word = 0;
+    for (int i = 0; i < n; ++i) word |= bm_all[(int64_t)i * wp + w];
+    while (word) {
+        const int bit = __ffs(word) - 1;
+        word &= word - 1;
+        const int64_t j = w * 32 + bit;
+        ghat_s[j] = __fadd_rn(ghat_s[j], __fdiv_rn(acc[j], fn));
+        acc[j] = 0.0f;
+    }
+}
+
+// ------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------
+static void free_ws(TopkWorkspace *w)
+{
+    cudaFree(w->hist); cudaFree(w->sel); cudaFree(w->bm_in); cudaFree(w->bm_cand);
+    cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
+    if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
+    delete w;
+}
+
+int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, uint32_t *idx,
+                          float *val)
+{
+    *out = nullptr;
+    TopkWorkspace *w = new TopkWorkspace();
+    w->d = d; w->k = k; w->rows = rows;
+    w->wp = (d + 31) / 32;
+    w->nbt = (w->wp + kTileWords - 1) / kTileWords;
+    w->own_payload = idx == nullptr;
+    w->idx = idx; w->val = val;
+    bool ok = true;
+    auto get = [&](void **p, size_t bytes) {
+        *p = nullptr;
+        if (ok && (cudaMalloc(p, bytes) != cudaSuccess || cudaMemset(*p, 0, bytes) != cudaSuccess)) ok = false;
+    };
+    get((void **)&w->hist, (size_t)rows * kHistStride * 4);
+    get((void **)&w->sel, (size_t)rows * sizeof(Sel));
+    get((void **)&w->bm_in, (size_t)rows * w->wp * 4);
+    get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
+    get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
+    get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
+    if (w->own_payload) {
+        get((void **)&w->idx, (size_t)rows * k * 4);
+        get((void **)&w->val, (size_t)rows * k * 4);
+    }
+    if (!ok) { cudaGetLastError(); free_ws(w); return CDADAM_ERR_ALLOC; }
+    *out = w;
+    return CDADAM_OK;
+}
+
+void topk_workspace_destroy(TopkWorkspace *w) { if (w) free_ws(w); }
+
+void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val)
+{
+    *idx = w->idx + (int64_t)row * w->k;
+    *val = w->val + (int64_t)row * w->k;
+}
+
+constexpr int kSelectLaunches = 11;
+int topk_launches_per_step(int n) { return 2 * kSelectLaunches + n + 1; }
+
+template <bool HAS_B>
+static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
+                        cudaStream_t st)
+{
+    const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
+    const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
+    cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
+    k_topk_hist1<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->hist, w->d, vec_ok);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k);
+    k_topk_mark<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->d, w->wp, vec_ok);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0);
+    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_cand, w->hist, w->d, w->wp);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0);
+    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt);
+    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt);
+    k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
+    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt);
+    if (HAS_B && update_b)
+        k_topk_emit<HAS_B, true><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->idx, w->val, w->d, w->wp, w->nbt, w->k);
+    else
+        k_topk_emit<HAS_B, false><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->idx, w->val, w->d, w->wp, w->nbt, w->k);
+}
+
+void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
+                 cudaStream_t st)
+{
+    if (b) select_impl<true>(w, a, b, update_b, vec_ok, st);
+    else select_impl<false>(w, a, nullptr, false, vec_ok, st);
+}
+
+int topk_step(TopkWorkspace *ww, TopkWorkspace *ws, const float *grads, float *ghat_w,
+              float *ghat_s, float *gtil, float *acc, int64_t d, int n, bool vec_ok,
+              cudaStream_t st)
+{
+    // workers: c_i = C(g_i - ghat_i), ghat_i += c_i
+    topk_select(ww, grads, ghat_w, true, vec_ok, st);
+    // server: workers added one after the other, i increasing, so that every coordinate
+    // sees the binary32 sum in the order 0, 1, ..., n-1
+    const unsigned gk = (unsigned)((ww->k + kBlock - 1) / kBlock);
+    for (int i = 0; i < n; ++i)
+        k_scatter_add<<<gk, kBlock, 0, st>>>(acc, ww->idx + (int64_t)i * ww->k, ww->val + (int64_t)i * ww->k, ww->k);
+    k_server_apply<<<(unsigned)((ww->wp + kBlock - 1) / kBlock), kBlock, 0, st>>>(ww->bm_in, n, ww->wp, acc, ghat_s, (float)n);
+    // server: c = C(ghat_s - gtil), gtil += c
+    topk_select(ws, ghat_s, gtil, true, d % 4 == 0, st);
+    return CDADAM_OK;
+}
+
+int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
+{
+    TopkWorkspace *w = nullptr;
+    int rc = topk_workspace_create(&w, d, k, 1, idx, val);
+    if (rc) return rc;
+    topk_select(w, x, nullptr, false, ((uintptr_t)x & 15u) == 0 && d % 4 == 0, st);
+    cudaError_t e = cudaStreamSynchronize(st);
+    topk_workspace_destroy(w);
+    return e == cudaSuccess ? CDADAM_OK : CDADAM_ERR_CUDA;
+}
+
+}  // namespace cdadam

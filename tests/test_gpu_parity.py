@@ -1,0 +1,276 @@
+"""GPU parity: the CUDA library (through its C interface) against the CPU oracle, element
+by element, on the same seeded inputs.
+
+Bar: sign words, scales, top-k index sets and values bit-exact after a single step from the
+same state; every float state vector within max relative error 1e-5 after every step of a
+free run and 1e-4 after the last one, relative error = max_j |a_j - b_j| / max(|b_j|, tau)
+with tau = 1e-6 * max_j |b_j| so that exact zeros do not dominate.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2111_00705_b200 import binding as cd
+from paper_2111_00705_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+STEP_TOL, FINAL_TOL = 1e-5, 1e-4
+
+
+def rel_err(a, b):
+    a = a.astype(np.float64).ravel(); b = b.astype(np.float64).ravel()
+    if a.size == 0:
+        return 0.0
+    tau = 1e-6 * max(np.abs(b).max(), 1e-300)
+    return float(np.max(np.abs(a - b) / np.maximum(np.abs(b), tau)))
+
+
+def u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def make_pair(w, x0=None, **kw):
+    dev = torch.device("cuda")
+    x0 = w.x0("cpu") if x0 is None else x0
+    args = dict(beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps)
+    args.update(kw)
+    g = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.to(dev), **args)
+    o = orc.Oracle(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.numpy(), **args)
+    return g, o
+
+
+def check_payloads(g, o, w):
+    if w.compressor == synth.IDENTITY:
+        return
+    for who in list(range(w.n)) + [cd.SERVER]:
+        a, b = g.last_payload(who)
+        oa, ob = o.payload(who)
+        assert np.array_equal(u32(a), oa), "payload words/indices of %s differ" % who
+        assert np.array_equal(b.cpu().numpy().view(np.uint32), ob.view(np.uint32)), \
+            "scales/values of %s differ" % who
+
+
+def check_state(g, o, tol, exact=False):
+    worst = 0.0
+    for name in orc.STATE_NAMES:
+        a = g.get_state(name).cpu().numpy()
+        b = o.state(name)
+        if exact:
+            assert np.array_equal(a.ravel(), b.ravel()), name
+        e = rel_err(a, b)
+        assert e <= tol, "%s: rel err %g" % (name, e)
+        worst = max(worst, e)
+    return worst
+
+
+def run_free(w, steps, exact=True, **kw):
+    """Free run: both sides step independently from the same inputs."""
+    g, o = make_pair(w, **kw)
+    for t in range(1, steps + 1):
+        grads = w.grads(t, "cpu")
+        g.step(grads.cuda())
+        o.step(grads.numpy())
+        torch.cuda.synchronize()
+        check_payloads(g, o, w)
+        # reading ghat_w applies the deferred payload: do it on alternate steps only so that
+        # both the deferred and the materialised path are exercised
+        if t % 2 == 0 or t == steps:
+            check_state(g, o, FINAL_TOL if t == steps else STEP_TOL, exact=exact)
+        else:
+            for name in ("x", "m", "v", "vhat", "gtil", "ghat_s"):
+                assert rel_err(g.get_state(name).cpu().numpy(), o.state(name)) <= STEP_TOL
+    g.close(); o.close()
+
+
+def run_teacher_forced(w, steps):
+    """Single-step parity: load the oracle's state into the GPU before every step."""
+    g, o = make_pair(w)
+    for t in range(1, steps + 1):
+        for name in orc.STATE_NAMES:
+            g.set_state(name, torch.from_numpy(o.state(name).copy()).cuda().reshape(-1))
+        grads = w.grads(t, "cpu")
+        g.step(grads.cuda())
+        o.step(grads.numpy())
+        check_payloads(g, o, w)
+        check_state(g, o, STEP_TOL, exact=True)
+    g.close(); o.close()
+
+
+# ---------------------------------------------------------------------------- configurations
+
+def test_c1_full_free_run():
+    run_free(synth.workload("C1"), 10)
+
+
+def test_c1_teacher_forced():
+    run_teacher_forced(synth.workload("C1"), 4)
+
+
+def test_c2_scaled_segments():
+    w = synth.workload("C2", scale=0.02)          # d = 224,000, 62 ragged segments, n = 8
+    assert w.q == 62
+    run_free(w, 6)
+
+
+def test_c3_scaled_topk():
+    w = synth.workload("C3", scale=0.01)          # d = 256,000, k = 2,560, n = 16
+    run_free(w, 5)
+
+
+def test_c3_teacher_forced():
+    run_teacher_forced(synth.workload("C3", scale=0.004), 3)
+
+
+def test_c4_scaled_heavy_tails():
+    w = synth.workload("C4", scale=0.004)         # d = 440,000, 15 segments, Student-t
+    assert w.q == 15
+    run_free(w, 5)
+
+
+def test_c5_scaled_flat():
+    w = synth.workload("C5", scale=0.0004)        # d = 600,000 flat, n = 4
+    run_free(w, 4)
+
+
+def test_identity_matches_oracle():
+    w = synth.Workload("ID", 5000, 3, synth.IDENTITY, 4)
+    run_free(w, 4)
+
+
+# ---------------------------------------------------------------------------- shapes and edges
+
+@pytest.mark.parametrize("d", list(range(1, 70)) + [127, 128, 129, 1023, 1024, 1025, 4095, 4096,
+                                                     4097, 8191, 8193, 12288, 12290])
+def test_sign_every_small_and_ragged_size(d):
+    w = synth.Workload("R", d, 2, synth.SIGN, 3, seed=d)
+    run_free(w, 3)
+
+
+@pytest.mark.parametrize("shift", range(0, 32, 3))
+def test_sign_segment_boundaries_at_every_residue(shift):
+    d = 3 * 4096 + 77
+    off = np.array([0, 5 + shift, 4096 + shift, 4096 + shift + 1, 2 * 4096 - shift, d])
+    w = synth.Workload("S", d, 3, synth.SIGN, 3, offsets=off, seed=shift)
+    run_free(w, 3)
+
+
+def test_many_tiny_segments_in_one_tile():
+    d = 9000
+    off = np.concatenate([np.arange(0, 640, 5), [700, 4096, 4100, 8192, d]])
+    w = synth.Workload("T", d, 2, synth.SIGN, 3, offsets=off)
+    run_free(w, 3)
+
+
+def test_unaligned_gradient_pointer_gives_same_bits():
+    w = synth.workload("C1", scale=0.25)
+    g, o = make_pair(w)
+    buf = torch.empty(w.n * w.d + 1, device="cuda")
+    for t in range(1, 4):
+        grads = w.grads(t, "cpu")
+        view = buf[1:]                              # 4-byte aligned only
+        view.copy_(grads.reshape(-1))
+        assert view.data_ptr() % 16 != 0
+        g.step(view)
+        o.step(grads.numpy())
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+
+
+@pytest.mark.parametrize("d,k", [(1, 1), (7, 7), (33, 1), (1000, 1000), (5000, 17), (40000, 400),
+                                 (32768 + 5, 300)])
+def test_topk_shapes(d, k):
+    w = synth.Workload("K", d, 3, synth.TOPK, 3, k=k, seed=d + k)
+    run_free(w, 3)
+
+
+def test_topk_ties_lower_index_wins():
+    """Few distinct magnitudes: most of the selection is decided by the tie rule."""
+    rng = np.random.default_rng(0)
+    d, n, k = 70000, 2, 900
+    g, o = None, None
+    w = synth.Workload("TIE", d, n, synth.TOPK, 3, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d))
+    for t in range(3):
+        grads = (rng.integers(-2, 3, (n, d)) * 0.5).astype(np.float32)
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    # all coordinates equal: the first k indices are kept
+    idx, val = cd.compress_topk(torch.full((5000,), -1.5, device="cuda"), 123)
+    assert idx.cpu().tolist() == list(range(123)) and torch.all(val == -1.5)
+    idx, val = cd.compress_topk(torch.zeros(4097, device="cuda"), 4097)
+    assert idx.cpu().tolist() == list(range(4097))
+
+
+def test_standalone_compressors_match_oracle():
+    rng = np.random.default_rng(1)
+    for d in (1, 31, 32, 33, 4096, 4097, 100003):
+        x = (rng.standard_normal(d) * np.exp2(rng.uniform(-20, 20, d))).astype(np.float32)
+        bits, scales = cd.compress_sign(torch.from_numpy(x).cuda())
+        ob, os_, _ = orc.compress_sign(x)
+        assert np.array_equal(u32(bits), ob) and np.array_equal(scales.cpu().numpy(), os_)
+        k = max(1, d // 50)
+        idx, val = cd.compress_topk(torch.from_numpy(x).cuda(), k)
+        oi, ov, _ = orc.compress_topk(x, k)
+        assert np.array_equal(u32(idx), oi) and np.array_equal(val.cpu().numpy(), ov)
+    off = np.array([0, 3, 4099, 50000, 100003])
+    bits, scales = cd.compress_sign(torch.from_numpy(x).cuda(), off)
+    ob, os_, _ = orc.compress_sign(x, off)
+    assert np.array_equal(u32(bits), ob) and np.array_equal(scales.cpu().numpy(), os_)
+
+
+def test_scale_is_correctly_rounded_on_hard_sums():
+    """Magnitudes spread over 80 binades defeat plain double accumulation; the scale must
+    still be the correctly rounded exact sum divided by d."""
+    rng = np.random.default_rng(2)
+    d = 1 << 20
+    x = (rng.standard_normal(d) * np.exp2(rng.uniform(-40, 40, d))).astype(np.float32)
+    _, scales = cd.compress_sign(torch.from_numpy(x).cuda())
+    want = np.float32(orc.l1_exact(x) / d)
+    assert scales.cpu().numpy()[0] == want
+
+
+def test_set_lr_and_step_host_and_params_view():
+    w = synth.workload("C1", scale=0.5)
+    g, o = make_pair(w)
+    grads = w.grads(1, "cpu")
+    xh = torch.empty(w.d).pin_memory()
+    g.step_host(grads.pin_memory(), xh)
+    o.step(grads.numpy())
+    assert np.array_equal(xh.numpy(), o.state("x"))
+    g.set_lr(5e-4); o.set_lr(5e-4)
+    grads = w.grads(2, "cpu")
+    g.step(grads.cuda()); o.step(grads.numpy())
+    torch.cuda.synchronize()
+    assert np.array_equal(g.params().cpu().numpy(), o.state("x"))
+    assert g.step_count() == 2 and g.launches_per_step() >= 3
+
+
+def test_argument_errors_are_reported_not_fatal():
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(0, 4)
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(100, 0)
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(100, 2, cd.TOPK, k=0)
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(100, 2, cd.TOPK, k=101)
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(100, 2, 7)
+    g = cd.CDAdam(100, 2)
+    with pytest.raises(cd.CdadamError):
+        g.set_segments([0, 50, 50, 100])
+    with pytest.raises(cd.CdadamError):
+        g.set_segments([0, 60, 40, 100])
+    with pytest.raises(cd.CdadamError):
+        g.set_segments([1, 100])
+    with pytest.raises(cd.CdadamError):
+        g.last_payload(0)                            # no step yet
+    g.step(torch.zeros(200, device="cuda"))
+    with pytest.raises(cd.CdadamError):
+        g.set_segments([0, 50, 100])                 # after the first step
+    with pytest.raises(cd.CdadamError):
+        g.last_payload(5)
+    torch.cuda.synchronize()
