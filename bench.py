@@ -1,0 +1,342 @@
+#!/usr/bin/env python
+"""Benchmark of the CD-Adam step (Algorithm 1, all stages) on synthetic gradients.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C4] [--impl cdadam|reference]
+
+A "step" is one call of cdadam_step: worker stage for all n workers, server stage and the
+worker-side AMSGrad update.  The default workload is C4 (d = 110,000,000, n = 8 workers,
+scaled sign per tensor, heavy-tailed gradients); C1..C5 can be chosen with --workload.
+The path is pinned to one GPU and does not shard: with --gpus N every rank runs an
+independent replica of the same problem ("replicas only"), value is the sum over ranks.
+
+Prints one JSON line (rank 0).  `value` is steps/s with the gradients already resident in
+device memory; `e2e` is the same through cdadam_step_host with pinned HOST gradients, the
+host->device copy of n*d floats and the device->host copy of x inside the timed region.
+`roofline` is for the dominant kernel (the worker pass), timed with CUDA events recorded by
+the library on the launching stream in a separate pass of the same K steps.
+`--impl reference` times the CPU oracle (tests/-only code, as it stands, one core) on a
+bounded sample of the same workload.
+"""
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "compressed-AMSGrad steps/s"
+UNIT = "steps/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# ncu capture of the dominant kernel: dram__bytes_read.sum + dram__bytes_write.sum per launch,
+# keyed by workload, with the hash of the kernel sources at capture time.  A changed source
+# makes the figure stale and bench reports null.
+NCU_TRAFFIC = {}
+
+
+def kernel_source_hash():
+    h = hashlib.sha256()
+    for f in ("common.cuh", "sign_kernels.cu", "topk_kernels.cu"):
+        with open(os.path.join(ROOT, "paper_2111_00705_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def algorithmic_bytes(w):
+    """Bytes Algorithm 1 must move per step with every vector touched once.
+    scaled sign: worker 4 (g) + 8 (ghat r/w) + 1/8 (bits) per worker element; server and
+    update n/8 + 48.25 per element.  top-k: 8 per worker element + 44 per element."""
+    from paper_2111_00705_b200 import synth
+    if w.compressor == synth.SIGN:
+        return w.d * (12.25 * w.n + 48.25), w.n * w.d * 12.125
+    if w.compressor == synth.TOPK:
+        return w.d * (8.0 * w.n + 44.0), w.n * w.d * 8.0
+    return w.d * (12.0 * w.n + 48.0), w.d * (12.0 * w.n + 48.0)
+
+
+class ClockSampler:
+    """nvidia-smi samples of SM clock and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush(); self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.f:
+            parts = [s.strip() for s in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+def oracle_sample(w, frac, steps):
+    """Time the CPU oracle on the first `frac` of the coordinates (same recipe) for `steps`
+    steps; returns seconds per step of the sample and the sample workload."""
+    import oracle as orc
+    from paper_2111_00705_b200 import synth
+    ws = synth.workload(w.name, scale=frac) if frac < 1.0 else w
+    o = orc.Oracle(ws.d, ws.n, ws.compressor, k=ws.k, offsets=ws.offsets, x0=ws.x0("cpu").numpy(),
+                   beta1=ws.beta1, beta2=ws.beta2, lr=ws.lr, eps=ws.eps)
+    grads = [ws.grads(t, "cpu").numpy() for t in (1, 2)]
+    t0 = time.perf_counter()
+    for t in range(steps):
+        o.step(grads[t % 2])
+    dt = (time.perf_counter() - t0) / steps
+    o.close()
+    return dt, ws
+
+
+SAMPLE = {"C1": (1.0, 20), "C2": (0.25, 4), "C3": (0.01, 4), "C4": (0.1, 5), "C5": (0.01, 5)}
+
+
+def run_reference(args, rank):
+    """The oracle, as it stands, on the host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    from paper_2111_00705_b200 import synth
+    w = synth.workload(args.workload)
+    frac, sample_steps = SAMPLE[w.name]
+    for _ in range(args.warmup and 1):
+        oracle_sample(w, frac, 1)
+    times = []
+    for _ in range(args.steps):
+        dt, ws = oracle_sample(w, frac, sample_steps)
+        times.append(dt)
+    sec_full = statistics.mean(times) / frac          # cost is linear in d
+    value = 1.0 / sec_full
+    sample = "first %g of the coordinates (d=%d, same recipe, n=%d), %d oracle steps per bench step; " \
+             "seconds per step scaled by 1/%g" % (frac, ws.d, ws.n, sample_steps, frac)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_full * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "params_per_s": value * w.d,
+            "config": {"workload": describe(w), "replicas": 1},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+def describe(w):
+    from paper_2111_00705_b200 import synth
+    comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity"}[w.compressor]
+    return "%s d=%d n=%d %s q=%d %s fp32" % (w.name, w.d, w.n, comp, w.q, w.dist)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="C4")
+    ap.add_argument("--impl", default="cdadam", choices=["cdadam", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--scale", type=float, default=1.0,
+                    help="shrink d (same recipe) for profiler captures; not a bench line")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2111_00705_b200 import binding as cd
+    from paper_2111_00705_b200 import synth
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = synth.workload(args.workload, scale=args.scale)
+    if args.warmup < 3:
+        args.warmup = 3
+    opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
+                    beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev)
+    # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
+    # flushed between steps instead
+    nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1
+    grads = [w.grads(t + 1, dev).reshape(-1) for t in range(nbuf)]
+    small = w.n * w.d * 4 < 512e6
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
+    stream = torch.cuda.current_stream()
+
+    def one_step(t):
+        if flush is not None:
+            flush.zero_()
+        opt.step(grads[t % nbuf], stream)
+
+    for t in range(args.warmup):
+        one_step(t)
+    barrier()
+
+    # ---- timed region: K steps, device time, max over ranks -----------------------------
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    if flush is None:
+        evs[0].record(stream)
+        for t in range(args.steps):
+            opt.step(grads[t % nbuf], stream)
+        evs[1].record(stream)
+        barrier()
+        total_ms = evs[0].elapsed_time(evs[1])
+    else:                       # time each step alone so that the L2 flush is not counted
+        pairs = []
+        for t in range(args.steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); opt.step(grads[t % nbuf], stream); b.record(stream)
+            pairs.append((a, b))
+        barrier()
+        total_ms = sum(a.elapsed_time(b) for a, b in pairs)
+    clocks = sampler.stop() if sampler else None
+    t_ms = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    total_ms = float(t_ms.item())
+    ms_per_step = total_ms / args.steps
+    value = world * args.steps / (total_ms * 1e-3)
+
+    # ---- per-kernel pass for the roofline ------------------------------------------------
+    opt.profile_enable(True)
+    for t in range(args.steps):
+        one_step(t)
+    stage_ms, psteps = opt.profile_read()
+    opt.profile_enable(False)
+    stage_ms = {k: v / max(psteps, 1) for k, v in stage_ms.items()}
+    step_bytes, dom_bytes = algorithmic_bytes(w)
+    dom_name = max(stage_ms, key=stage_ms.get)
+    peak, peak_kind = measured_peak()
+    achieved = dom_bytes / (stage_ms[dom_name] * 1e-3) / 1e9 if stage_ms[dom_name] > 0 else 0.0
+    traffic = None
+    cap = NCU_TRAFFIC.get(w.name)
+    if cap and cap.get("hash") == kernel_source_hash():
+        traffic = cap["bytes_per_launch"]
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
+                "traffic": traffic, "algorithmic_bytes_per_launch": dom_bytes,
+                "ms_per_launch": stage_ms[dom_name],
+                "timed": "separate pass of the same %d steps with events around every kernel" % args.steps}
+
+    # ---- end to end: host gradients in, x out, copies inside the timed region ------------
+    e2e = None
+    try:
+        if args.e2e_steps < 1:
+            raise RuntimeError("skipped (--e2e-steps 0)")
+        gh = [g.cpu().pin_memory() for g in grads[:1]]
+        xh = torch.empty(w.d, dtype=torch.float32).pin_memory()
+        opt.step_host(gh[0], xh, stream)                       # allocates the staging buffer
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for t in range(args.e2e_steps):
+            opt.step_host(gh[0], xh, stream)
+        b.record(stream)
+        barrier()
+        e_ms = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(e_ms, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * args.e2e_steps / (float(e_ms.item()) * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": w.n * w.d * 4, "d2h_bytes_per_step": w.d * 4,
+               "steps": args.e2e_steps}
+        del gh, xh
+    except Exception as exc:                                   # e.g. not enough pinned memory
+        e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+
+    launches = opt.launches_per_step() * args.steps
+    opt.close()
+    del grads
+    torch.cuda.empty_cache()
+
+    cpu = None
+    if rank == 0 and not args.no_cpu_baseline:
+        frac, sample_steps = SAMPLE[w.name]
+        dt, ws = oracle_sample(w, frac, sample_steps)
+        cpu = {"value": frac / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "host_cores": os.cpu_count(),
+               "sample": "first %g of the coordinates (d=%d, same recipe, n=%d), %d steps; "
+                         "seconds per step scaled by 1/%g" % (frac, ws.d, ws.n, sample_steps, frac)}
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale),
+                           "replicas": world,
+                           "l2": "flushed between steps" if flush is not None else
+                                 "inputs larger than L2 (%.2f GB of gradients per step)" % (w.n * w.d * 4 / 1e9)},
+                "params_per_s": value * w.d,
+                "step_hbm": {"algorithmic_bytes": step_bytes,
+                             "gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
+                             "frac_of_8tbs": step_bytes / (ms_per_step * 1e-3) / 8e12,
+                             "frac_of_measured": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
+                "stage_ms": stage_ms,
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
+                "clocks": clocks}
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

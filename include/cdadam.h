@@ -157,11 +157,24 @@ int64_t cdadam_step_count(cdadam_ctx *ctx);
 int cdadam_launches_per_step(cdadam_ctx *ctx);
 
 /*
+ * Optional per-stage timing for benchmarks.  While enabled, cdadam_step records CUDA events
+ * on its stream before the first and after every stage (a kernel or, for top-k, a group of
+ * kernels).  cdadam_profile_read waits for the recorded events, adds the elapsed
+ * milliseconds of every stage over all steps since the last read into ms[0..] (unused slots
+ * 0), stores the number of steps in *steps and forgets the events.  cdadam_profile_name
+ * gives a stage's name ("" if slot is out of range); the string is static.
+ */
+#define CDADAM_PROF_SLOTS 8
+int cdadam_profile_enable(cdadam_ctx *ctx, int on);
+int cdadam_profile_read(cdadam_ctx *ctx, double ms[CDADAM_PROF_SLOTS], int64_t *steps);
+const char *cdadam_profile_name(cdadam_ctx *ctx, int slot);
+
+/*
  * Stand-alone compressors of Appendix A on a device vector x of d floats.
  * Scaled sign: writes ceil(d/32) words to bits and q floats to scales (segments as in
  * cdadam_set_segments; offsets == NULL means one segment).  Top-k: writes k increasing
- * coordinates to idx and their values to val.  Scratch memory is taken from and returned
- * to the stream-ordered allocator of the current device inside the call.
+ * coordinates to idx and their values to val.  Both allocate their scratch memory on the
+ * current device inside the call and free it before returning, and may wait for `stream`.
  */
 int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offsets,
                          uint32_t *bits, float *scales, void *stream);

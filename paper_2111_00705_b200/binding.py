@@ -39,6 +39,9 @@ _SIGNATURES = {
                                         _c.c_void_p]),
     "cdadam_compress_topk": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int64, _c.c_void_p,
                                         _c.c_void_p, _c.c_void_p]),
+    "cdadam_profile_enable": (_c.c_int, [_c.c_void_p, _c.c_int]),
+    "cdadam_profile_read": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_double), _c.POINTER(_c.c_int64)]),
+    "cdadam_profile_name": (_c.c_char_p, [_c.c_void_p, _c.c_int]),
     "cdadam_last_error": (_c.c_char_p, []),
 }
 
@@ -193,6 +196,21 @@ class CDAdam:
                     _view(b.value, self.q, torch.float32, self.device))
         return (_view(a.value, self.k, torch.int32, self.device),
                 _view(b.value, self.k, torch.float32, self.device))
+
+    def profile_enable(self, on=True):
+        _check(lib().cdadam_profile_enable(self._h, 1 if on else 0))
+
+    def profile_read(self):
+        """({stage name: total ms}, steps) accumulated since the last read."""
+        ms = (ctypes.c_double * 8)()
+        steps = ctypes.c_int64()
+        _check(lib().cdadam_profile_read(self._h, ms, ctypes.byref(steps)))
+        out = {}
+        for s in range(8):
+            name = lib().cdadam_profile_name(self._h, s).decode()
+            if name:
+                out[name] = ms[s]
+        return out, steps.value
 
     def step_count(self):
         return lib().cdadam_step_count(self._h)

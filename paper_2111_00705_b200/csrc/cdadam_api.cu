@@ -127,6 +127,10 @@ struct cdadam_ctx {
     float *acc = nullptr;   // dense per-coordinate sum of the workers' sparse payloads
     // host-gradient staging
     float *stage = nullptr;
+    // optional per-kernel timing: events[step][0..nslots] recorded around every stage
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_ev;   // groups of (nslots + 1) events, one group per step
+    std::vector<cudaEvent_t> prof_pool;
 };
 
 namespace {
@@ -169,6 +173,22 @@ float *state_ptr(cdadam_ctx *c, int name)
     case CDADAM_STATE_X: return c->x;
     }
     return nullptr;
+}
+
+int prof_slots(const cdadam_ctx *c)
+{
+    return c->comp == CDADAM_SIGN ? 5 : c->comp == CDADAM_TOPK ? 4 : 1;
+}
+
+// Record the boundary event after a stage (or before the first one) when timing is on.
+void prof_mark(cdadam_ctx *c, cudaStream_t st)
+{
+    if (!c->prof_on) return;
+    cudaEvent_t e;
+    if (!c->prof_pool.empty()) { e = c->prof_pool.back(); c->prof_pool.pop_back(); }
+    else if (cudaEventCreate(&e) != cudaSuccess) return;
+    cudaEventRecord(e, st);
+    c->prof_ev.push_back(e);
 }
 
 int check_launch(const char *what)
@@ -234,6 +254,8 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->acc); cudaFree(c->stage);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
+    for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
+    for (cudaEvent_t e : c->prof_pool) cudaEventDestroy(e);
     c->ts.release(nullptr, false);
     delete c;
 }
@@ -244,23 +266,36 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     const bool vec = aligned16(grads) && c->d % 4 == 0;
+    prof_mark(c, st);
     if (c->comp == CDADAM_SIGN) {
         const Tables &tb = c->ts.tb;
+        const bool svec = c->d % 4 == 0;
         const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
         float *new_scale = c->wscale[c->cur ^ 1];
         launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, st);
+        prof_mark(c, st);
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
-        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, c->d % 4 == 0, st);
+        prof_mark(c, st);
+        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, svec, st);
+        prof_mark(c, st);
         launch_finalize_scales(c->spart, c->sscale, tb, 1, st);
-        launch_update_sign(c->sbits, c->sscale, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, c->d % 4 == 0, st);
+        prof_mark(c, st);
+        launch_update_sign(c->sbits, c->sscale, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, svec, st);
+        prof_mark(c, st);
         c->cur ^= 1;
         c->pending = true;
     } else if (c->comp == CDADAM_TOPK) {
-        int rc = topk_step(c->tk_w, c->tk_s, grads, c->ghat_w, c->ghat_s, c->gtil, c->acc, c->d, c->n, vec, st);
-        if (rc) return fail(rc, "top-k step failed");
+        topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
+        prof_mark(c, st);
+        topk_aggregate(c->tk_w, c->ghat_s, c->acc, c->n, st);              // line 8
+        prof_mark(c, st);
+        topk_select(c->tk_s, c->ghat_s, c->gtil, true, c->d % 4 == 0, st); // lines 9-10, 12
+        prof_mark(c, st);
         launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, c->d % 4 == 0, st);
+        prof_mark(c, st);
     } else {
         launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, st);
+        prof_mark(c, st);
     }
     int rc = check_launch("cdadam_step");
     if (rc) return rc;
@@ -375,6 +410,41 @@ int cdadam_launches_per_step(cdadam_ctx *c)
     if (c->comp == CDADAM_SIGN) return 5;
     if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1;
     return 1;
+}
+
+int cdadam_profile_enable(cdadam_ctx *c, int on)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_profile_enable: NULL context");
+    c->prof_on = on != 0;
+    return CDADAM_OK;
+}
+
+int cdadam_profile_read(cdadam_ctx *c, double *ms, int64_t *steps)
+{
+    if (!c || !ms || !steps) return fail(CDADAM_ERR_ARG, "cdadam_profile_read: NULL argument");
+    DeviceGuard guard(c->device);
+    const int ns = prof_slots(c), group = ns + 1;
+    for (int s = 0; s < CDADAM_PROF_SLOTS; ++s) ms[s] = 0.0;
+    *steps = (int64_t)(c->prof_ev.size() / group);
+    if (!c->prof_ev.empty()) CU_TRY(cudaEventSynchronize(c->prof_ev.back()));
+    for (int64_t t = 0; t < *steps; ++t)
+        for (int s = 0; s < ns; ++s) {
+            float f = 0.0f;
+            CU_TRY(cudaEventElapsedTime(&f, c->prof_ev[t * group + s], c->prof_ev[t * group + s + 1]));
+            ms[s] += f;
+        }
+    c->prof_pool.insert(c->prof_pool.end(), c->prof_ev.begin(), c->prof_ev.end());
+    c->prof_ev.clear();
+    return CDADAM_OK;
+}
+
+const char *cdadam_profile_name(cdadam_ctx *c, int slot)
+{
+    static const char *sign[] = {"k_worker_sign", "k_finalize_scales(workers)", "k_server_sign",
+                                 "k_finalize_scales(server)", "k_update_sign"};
+    static const char *topk[] = {"topk_select(workers)", "topk_aggregate", "topk_select(server)", "k_amsgrad"};
+    if (!c || slot < 0 || slot >= prof_slots(c)) return "";
+    return c->comp == CDADAM_SIGN ? sign[slot] : c->comp == CDADAM_TOPK ? topk[slot] : "k_step_identity";
 }
 
 int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offsets, uint32_t *bits,

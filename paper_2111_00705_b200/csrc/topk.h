@@ -22,13 +22,10 @@ int topk_launches_per_step(int n);
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                  cudaStream_t st);
 
-// Worker stage, sparse server aggregation and server stage of Algorithm 1 with top-k:
-//   ghat_w[i] += C(g_i - ghat_w[i]);  ghat_s += (sum_i c_i) / n on the touched coordinates;
-//   gtil += C(ghat_s - gtil).
-// acc: d floats, all zero on entry and on exit.
-int topk_step(TopkWorkspace *ww, TopkWorkspace *ws, const float *grads, float *ghat_w,
-              float *ghat_s, float *gtil, float *acc, int64_t d, int n, bool vec_ok,
-              cudaStream_t st);
+// Sparse server aggregation (Algorithm 1 line 8) from the n payloads held in `ww`:
+//   ghat_s += (sum_i c_i) / n on the coordinates some worker sent, workers added in the
+//   order 0, 1, ..., n-1.  acc: d floats, all zero on entry and on exit.
+void topk_aggregate(TopkWorkspace *ww, float *ghat_s, float *acc, int n, cudaStream_t st);
 
 // Stand-alone top-k of one vector into caller buffers (allocates and frees scratch).
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,

@@ -535,21 +535,14 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
     else select_impl<false>(w, a, nullptr, false, vec_ok, st);
 }
 
-int topk_step(TopkWorkspace *ww, TopkWorkspace *ws, const float *grads, float *ghat_w,
-              float *ghat_s, float *gtil, float *acc, int64_t d, int n, bool vec_ok,
-              cudaStream_t st)
+void topk_aggregate(TopkWorkspace *ww, float *ghat_s, float *acc, int n, cudaStream_t st)
 {
-    // workers: c_i = C(g_i - ghat_i), ghat_i += c_i
-    topk_select(ww, grads, ghat_w, true, vec_ok, st);
-    // server: workers added one after the other, i increasing, so that every coordinate
-    // sees the binary32 sum in the order 0, 1, ..., n-1
+    // one launch per worker, i increasing, so that every coordinate sees the binary32 sum
+    // in the order 0, 1, ..., n-1 (indices inside one payload are distinct: no atomics)
     const unsigned gk = (unsigned)((ww->k + kBlock - 1) / kBlock);
     for (int i = 0; i < n; ++i)
         k_scatter_add<<<gk, kBlock, 0, st>>>(acc, ww->idx + (int64_t)i * ww->k, ww->val + (int64_t)i * ww->k, ww->k);
     k_server_apply<<<(unsigned)((ww->wp + kBlock - 1) / kBlock), kBlock, 0, st>>>(ww->bm_in, n, ww->wp, acc, ghat_s, (float)n);
-    // server: c = C(ghat_s - gtil), gtil += c
-    topk_select(ws, ghat_s, gtil, true, d % 4 == 0, st);
-    return CDADAM_OK;
 }
 
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
