@@ -125,55 +125,105 @@ k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Table
 
 // ------------------------------------------------------------------------------------
 // Server pass A.  grid = (ntiles).
+//
+// Vector path: a warp owns 128*VPT consecutive coordinates per iteration.  The sign words
+// of up to kNC workers for that span are staged through shared memory, transposed so that a
+// thread fetches the words of all its VPT coordinate groups for one worker with a single
+// shared-memory load; the per-worker scales of the tile's segment sit in shared memory too.
 // ------------------------------------------------------------------------------------
+constexpr int kNC = 16;     // workers staged per chunk
+
+template <int VPT>
 __global__ void __launch_bounds__(kBlock)
 k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
               float *__restrict__ ghat_s, const float *__restrict__ gtil,
               uint32_t *__restrict__ sbits, dd *__restrict__ spart, Tables tb, int n,
-              int64_t wp, int vec_ok)
+              int64_t wp, int vec_ok, int n_pow2)
 {
+    __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
+    __shared__ float ssm[kNC];
     const int64_t T = blockIdx.x;
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
     dd *part = spart + tb.pbase[T];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float fn = (float)n;
+    const float rn = 1.0f / fn;               // exact when n is a power of two
 
     if (vec_ok && first == last && base + tb.tile <= tb.d) {
+        constexpr int kSpan = 128 * VPT;                  // coordinates per warp per iteration
+        constexpr int kIter = kSpan * (kBlock / 32);      // per block per iteration
+        const bool multi = n > kNC;
+        const int g = lane >> 3, sh = (lane & 7) * 4;
+        if (!multi) {
+            if (threadIdx.x < n) ssm[threadIdx.x] = wscale[(int64_t)threadIdx.x * tb.q + first];
+            __syncthreads();
+        }
         dd acc = {0.0, 0.0};
-        for (int it = 0; it < tb.tile / kSub; ++it) {
-            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
-            float4 H[4], Gt[4];
+        for (int it = 0; it < tb.tile / kIter; ++it) {
+            const int64_t wb = base + (int64_t)it * kIter + warp * kSpan;
+            float4 H[VPT], Gt[VPT];
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
+            for (int v = 0; v < VPT; ++v) {
                 const int64_t j = wb + v * 128 + lane * 4;
                 H[v] = ld_rw4(ghat_s + j);
                 Gt[v] = ld_ro4(gtil + j);
             }
-            float a[4][4];
+            float a[VPT][4];
 #pragma unroll
-            for (int v = 0; v < 4; ++v) a[v][0] = a[v][1] = a[v][2] = a[v][3] = 0.0f;
-            const uint32_t *wq = wbits + (wb >> 5) + (lane >> 3);
-            const int sh = (lane & 7) * 4;
+            for (int v = 0; v < VPT; ++v) a[v][0] = a[v][1] = a[v][2] = a[v][3] = 0.0f;
+            for (int i0 = 0; i0 < n; i0 += kNC) {        // workers in increasing order
+                const int nc = min(kNC, n - i0);
+                if (multi) {
+                    __syncthreads();
+                    if (threadIdx.x < nc) ssm[threadIdx.x] = wscale[(int64_t)(i0 + threadIdx.x) * tb.q + first];
+                } else {
+                    __syncwarp();
+                }
+                for (int idx = lane; idx < nc * 4 * VPT; idx += 32) {
+                    const int i = idx / (4 * VPT), wd = idx % (4 * VPT);
+                    wsm[warp][i][wd & 3][wd >> 2] = ld_ro_u32(wbits + (int64_t)(i0 + i) * wp + (wb >> 5) + wd);
+                }
+                if (multi) __syncthreads(); else __syncwarp();
 #pragma unroll 4
-            for (int i = 0; i < n; ++i) {            // workers in increasing order
-                const float s = __ldg(wscale + (int64_t)i * tb.q + first);
+                for (int i = 0; i < nc; ++i) {
+                    const float s = ssm[i];
+                    uint32_t W[VPT];
+                    if constexpr (VPT == 4) {
+                        const uint4 q4 = *reinterpret_cast<const uint4 *>(&wsm[warp][i][g][0]);
+                        W[0] = q4.x; W[1] = q4.y; W[2] = q4.z; W[3] = q4.w;
+                    } else {
+                        const uint2 q2 = *reinterpret_cast<const uint2 *>(&wsm[warp][i][g][0]);
+                        W[0] = q2.x; W[1] = q2.y;
+                    }
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const uint32_t nib = ld_ro_u32(wq + (int64_t)i * wp + v * 4) >> sh;
-                    a[v][0] = __fadd_rn(a[v][0], signed_scale(nib & 1u, s));
-                    a[v][1] = __fadd_rn(a[v][1], signed_scale(nib & 2u, s));
-                    a[v][2] = __fadd_rn(a[v][2], signed_scale(nib & 4u, s));
-                    a[v][3] = __fadd_rn(a[v][3], signed_scale(nib & 8u, s));
+                    for (int v = 0; v < VPT; ++v) {
+                        const uint32_t nib = W[v] >> sh;
+                        a[v][0] = __fadd_rn(a[v][0], signed_scale(nib & 1u, s));
+                        a[v][1] = __fadd_rn(a[v][1], signed_scale(nib & 2u, s));
+                        a[v][2] = __fadd_rn(a[v][2], signed_scale(nib & 4u, s));
+                        a[v][3] = __fadd_rn(a[v][3], signed_scale(nib & 8u, s));
+                    }
                 }
             }
             uint32_t B[4][4];
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                H[v].x = __fadd_rn(H[v].x, __fdiv_rn(a[v][0], fn));
-                H[v].y = __fadd_rn(H[v].y, __fdiv_rn(a[v][1], fn));
-                H[v].z = __fadd_rn(H[v].z, __fdiv_rn(a[v][2], fn));
-                H[v].w = __fadd_rn(H[v].w, __fdiv_rn(a[v][3], fn));
+            for (int v = 0; v < 4; ++v) B[v][0] = B[v][1] = B[v][2] = B[v][3] = 0u;
+#pragma unroll
+            for (int v = 0; v < VPT; ++v) {
+                // sum / n: multiplication by 1/n is the same correctly rounded value as the
+                // division when n is a power of two
+                if (n_pow2) {
+                    H[v].x = __fadd_rn(H[v].x, __fmul_rn(a[v][0], rn));
+                    H[v].y = __fadd_rn(H[v].y, __fmul_rn(a[v][1], rn));
+                    H[v].z = __fadd_rn(H[v].z, __fmul_rn(a[v][2], rn));
+                    H[v].w = __fadd_rn(H[v].w, __fmul_rn(a[v][3], rn));
+                } else {
+                    H[v].x = __fadd_rn(H[v].x, __fdiv_rn(a[v][0], fn));
+                    H[v].y = __fadd_rn(H[v].y, __fdiv_rn(a[v][1], fn));
+                    H[v].z = __fadd_rn(H[v].z, __fdiv_rn(a[v][2], fn));
+                    H[v].w = __fadd_rn(H[v].w, __fdiv_rn(a[v][3], fn));
+                }
                 st_rw4(ghat_s + wb + v * 128 + lane * 4, H[v]);
                 const float wx = __fsub_rn(H[v].x, Gt[v].x), wy = __fsub_rn(H[v].y, Gt[v].y);
                 const float wz = __fsub_rn(H[v].z, Gt[v].z), ww = __fsub_rn(H[v].w, Gt[v].w);
@@ -185,7 +235,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                 B[v][3] = __ballot_sync(kFull, ww >= 0.0f);
             }
             const uint32_t word = warp_words(B, lane);
-            if (lane < 16) sbits[(wb >> 5) + lane] = word;
+            if (lane < 4 * VPT) sbits[(wb >> 5) + lane] = word;
         }
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[0] = acc;
@@ -368,8 +418,9 @@ void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
                         int n, int64_t wp, bool vec_ok, cudaStream_t st)
 {
-    k_server_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                          spart, tb, n, wp, vec_ok);
+    const int pow2 = (n & (n - 1)) == 0;
+    k_server_sign<2><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+                                                             spart, tb, n, wp, vec_ok, pow2);
 }
 
 void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil, float *m,
