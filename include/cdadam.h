@@ -181,6 +181,28 @@ int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offset
 int cdadam_compress_topk(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,
                          void *stream);
 
+/*
+ * Scaled-sign compressor of one vector (one segment) that allocates nothing.  The paper has
+ * no counterpart: this entry point exists for callers that cannot allocate device memory
+ * when they call - code that must not risk the implicit device synchronisation of
+ * cudaMalloc / cudaFree, processes whose device memory is wholly reserved by a framework's
+ * pool, and latency-bound loops where an allocator call is an unbounded delay.
+ *   x      device, d floats;  bits  device, ceil(d/32) words;  scale  device, one float
+ *   d      1 <= d <= CDADAM_STATIC_MAX_D; larger sizes are rejected with CDADAM_ERR_ARG
+ * Same results as cdadam_compress_sign(x, d, 1, NULL, bits, scale, stream).  The partial
+ * sums of |x| go to a fixed 256 KiB array inside the library's device image (every GPU
+ * that loads the library holds it until the process exits) instead of allocated scratch;
+ * no cudaMalloc, cudaFree or other allocating call is made.  The first call on each device
+ * looks up the array's device address (cudaGetSymbolAddress); make that first call before
+ * any stream capture begins.  All calls on a device share the array and it keeps the last
+ * call's contents: every entry a call reads is first overwritten by that call, so nothing
+ * needs clearing, but two calls whose kernels overlap on the GPU (different streams, no
+ * ordering between them) race on it.  Calls on one stream are safe.
+ */
+#define CDADAM_STATIC_MAX_D ((int64_t)1 << 28)
+int cdadam_compress_sign_static(const float *x, int64_t d, uint32_t *bits, float *scale,
+                                void *stream);
+
 /* Message of the calling thread's most recent failure ("" if none).  Never NULL. */
 const char *cdadam_last_error(void);
 

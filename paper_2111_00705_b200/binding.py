@@ -39,6 +39,8 @@ _SIGNATURES = {
                                         _c.c_void_p]),
     "cdadam_compress_topk": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int64, _c.c_void_p,
                                         _c.c_void_p, _c.c_void_p]),
+    "cdadam_compress_sign_static": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_void_p, _c.c_void_p,
+                                               _c.c_void_p]),
     "cdadam_profile_enable": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_profile_read": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_double), _c.POINTER(_c.c_int64)]),
     "cdadam_profile_name": (_c.c_char_p, [_c.c_void_p, _c.c_int]),
@@ -241,3 +243,22 @@ def compress_topk(x, k, stream=None):
         _check(lib().cdadam_compress_topk(_dev_f32(x, d, "x"), d, k, ctypes.c_void_p(idx.data_ptr()),
                                           ctypes.c_void_p(val.data_ptr()), _stream(stream)))
     return idx, val
+
+
+STATIC_MAX_D = 1 << 28
+
+
+def compress_sign_static(x, bits=None, scale=None, stream=None):
+    """Flat scaled-sign compressor through the entry point that allocates nothing inside the
+    library (for callers that cannot allocate device memory at call time).  Pass preallocated
+    `bits` (int32[ceil(d/32)]) and `scale` (float32[1]) to keep the whole call free of
+    allocations; they are created here only when omitted.  Returns (bits, scale)."""
+    d = x.numel()
+    if bits is None:
+        bits = torch.empty((d + 31) // 32, dtype=torch.int32, device=x.device)
+    if scale is None:
+        scale = torch.empty(1, dtype=torch.float32, device=x.device)
+    with torch.cuda.device(x.device):
+        _check(lib().cdadam_compress_sign_static(_dev_f32(x, d, "x"), d, ctypes.c_void_p(bits.data_ptr()),
+                                                 ctypes.c_void_p(scale.data_ptr()), _stream(stream)))
+    return bits, scale

@@ -14,7 +14,8 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libcdadam.so")
-SOURCES = ["cdadam_api.cu", "sign_kernels.cu", "dense_kernels.cu", "topk_kernels.cu"]
+SOURCES = ["cdadam_api.cu", "sign_kernels.cu", "dense_kernels.cu", "topk_kernels.cu",
+           "static_scratch.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-fmad=false", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

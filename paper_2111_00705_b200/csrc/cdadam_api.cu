@@ -200,6 +200,10 @@ int check_launch(const char *what)
 
 }  // namespace
 
+namespace cdadam {
+void set_last_error(const char *message) { snprintf(g_err, sizeof g_err, "%s", message); }
+}  // namespace cdadam
+
 extern "C" {
 
 const char *cdadam_last_error(void) { return g_err; }

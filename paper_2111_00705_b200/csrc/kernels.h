@@ -41,4 +41,7 @@ void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, floa
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
                     Hyper hp, bool vec_ok, cudaStream_t st);
 
+// Store the message cdadam_last_error() returns for the calling thread.
+void set_last_error(const char *message);
+
 }  // namespace cdadam
