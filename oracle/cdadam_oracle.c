@@ -199,6 +199,9 @@ typedef struct oracle_ctx {
     float *s_scales;         /* q */
     uint32_t *s_idx;         /* k */
     float *s_val;            /* k */
+    /* sampled checks only: scales given from outside instead of computed (NULL = compute) */
+    float *force_w_scales;   /* n*q */
+    float *force_s_scales;   /* q */
 } oracle_ctx;
 
 static float *zeros(int64_t count) { return (float *)calloc((size_t)(count > 0 ? count : 1), sizeof(float)); }
@@ -211,6 +214,7 @@ void oracle_destroy(oracle_ctx *o)
     free(o->u); free(o->c); free(o->acc);
     free(o->w_bits); free(o->w_scales); free(o->w_idx); free(o->w_val);
     free(o->s_bits); free(o->s_scales); free(o->s_idx); free(o->s_val);
+    free(o->force_w_scales); free(o->force_s_scales);
     free(o);
 }
 
@@ -295,10 +299,50 @@ uint32_t *oracle_payload_idx(oracle_ctx *o, int who)
 float *oracle_payload_val(oracle_ctx *o, int who)
 { return who < 0 ? o->s_val : o->w_val + (int64_t)who * o->k; }
 
+/* For checks on a SAMPLE of the coordinates of a larger problem: the scaled-sign scales
+ * are global reductions that a sample cannot reproduce, so they are supplied (after having
+ * been verified on the full data with oracle_l1_exact) and only bits and the decoded vector
+ * are computed here.  Pass NULL to return to computed scales. */
+int oracle_force_scales(oracle_ctx *o, const float *worker_scales, const float *server_scales)
+{
+    if (!o || o->compressor != ORC_SIGN) return -1;
+    free(o->force_w_scales); free(o->force_s_scales);
+    o->force_w_scales = o->force_s_scales = NULL;
+    if (worker_scales) {
+        o->force_w_scales = (float *)malloc((size_t)o->n * o->q * sizeof(float));
+        memcpy(o->force_w_scales, worker_scales, (size_t)o->n * o->q * sizeof(float));
+    }
+    if (server_scales) {
+        o->force_s_scales = (float *)malloc((size_t)o->q * sizeof(float));
+        memcpy(o->force_s_scales, server_scales, (size_t)o->q * sizeof(float));
+    }
+    return 0;
+}
+
+static void sign_with_given_scales(oracle_ctx *o, const float *u, const float *given,
+                                   uint32_t *bits, float *scales, float *c)
+{
+    memset(bits, 0, (size_t)((o->d + 31) / 32) * sizeof(uint32_t));
+    for (int r = 0; r < o->q; ++r) {
+        const float s = given[r];
+        scales[r] = s;
+        for (int64_t j = o->off[r]; j < o->off[r + 1]; ++j) {
+            int nonneg = u[j] >= 0.0f;
+            if (nonneg) bits[j / 32] |= (uint32_t)1 << (j % 32);
+            c[j] = nonneg ? s : -s;
+        }
+    }
+}
+
 /* c = C(u) with the context's compressor; who selects where the payload is kept. */
 static void compress(oracle_ctx *o, const float *u, float *c, int who)
 {
-    if (o->compressor == ORC_SIGN)
+    const float *given = who < 0 ? o->force_s_scales
+                                 : (o->force_w_scales ? o->force_w_scales + (int64_t)who * o->q : NULL);
+    if (o->compressor == ORC_SIGN && given)
+        sign_with_given_scales(o, u, given, oracle_payload_bits(o, who),
+                               oracle_payload_scales(o, who), c);
+    else if (o->compressor == ORC_SIGN)
         oracle_compress_sign(u, o->d, o->q, o->off, oracle_payload_bits(o, who),
                              oracle_payload_scales(o, who), c);
     else if (o->compressor == ORC_TOPK)

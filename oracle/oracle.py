@@ -57,6 +57,8 @@ def _load():
     lib.oracle_set_mode.argtypes = [c.c_void_p, c.c_int]
     lib.oracle_set_lr.restype = c.c_int
     lib.oracle_set_lr.argtypes = [c.c_void_p, c.c_float]
+    lib.oracle_force_scales.restype = c.c_int
+    lib.oracle_force_scales.argtypes = [c.c_void_p, fp, fp]
     lib.oracle_state.restype = fp
     lib.oracle_state.argtypes = [c.c_void_p, c.c_int]
     lib.oracle_step.restype = c.c_int
@@ -147,6 +149,19 @@ class Oracle:
 
     def set_lr(self, lr):
         self._lib.oracle_set_lr(self._h, lr)
+
+    def force_scales(self, worker_scales=None, server_scales=None):
+        """Sampled checks only: use these scaled-sign scales (n x q, q) instead of computing
+        them from the (sampled, hence incomplete) data.  None returns to computed scales."""
+        ws = ss = None
+        if worker_scales is not None:
+            wa, ws = _f32(worker_scales)
+            assert wa.size == self.n * self.q
+        if server_scales is not None:
+            sa, ss = _f32(server_scales)
+            assert sa.size == self.q
+        if self._lib.oracle_force_scales(self._h, ws, ss) != 0:
+            raise ValueError("force_scales applies to the scaled-sign compressor")
 
     def state(self, name):
         """Writable numpy view of a state vector ('ghat_w' is n x d, the others d)."""

@@ -1,0 +1,188 @@
+"""Parity at the full sizes of the five configurations, in the launch configuration the
+benchmark times.
+
+Where the CPU oracle finishes in under a minute it runs on the whole problem and everything
+is compared element by element (C1 in test_gpu_parity, C2 and C4 here).  Where it cannot
+(C5: 1.5e9 coordinates; C3: seventeen 25.6 M-element sorts per step) the checks are
+ - scales: the oracle's exact l1 routine on the FULL data, bit for bit;
+ - sign words: against sign(u) on the full data;
+ - every state vector on a SAMPLE of coordinates (random, both ends, around the 2^29 / 2^30
+   / 2^31 element offsets and tile edges) with the oracle run on the gathered coordinates and
+   the (already verified) scales supplied;
+ - top-k: the selection is unique given the k-th largest magnitude, which an independent
+   library routine (torch.kthvalue) provides; index set, values and state updates follow.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+from paper_2111_00705_b200 import binding as cd
+from paper_2111_00705_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def u32(t):
+    return t.cpu().numpy().view(np.uint32)
+
+
+def full_oracle_run(w, steps):
+    x0 = w.x0(DEV)
+    g = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0)
+    o = orc.Oracle(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.cpu().numpy())
+    for t in range(1, steps + 1):
+        grads = w.grads(t, DEV)
+        g.step(grads.reshape(-1))
+        o.step(grads.cpu().numpy())
+        del grads
+        for who in list(range(w.n)) + [cd.SERVER]:
+            a, b = g.last_payload(who)
+            oa, ob = o.payload(who)
+            assert np.array_equal(u32(a), oa), (t, who)
+            assert np.array_equal(u32(b), ob.view(np.uint32)), (t, who)
+        names = orc.STATE_NAMES if t == steps else ("ghat_s", "gtil", "m", "v", "vhat", "x")
+        for name in names:                       # ghat_w only at the end: keeps the deferred path
+            a = g.get_state(name).cpu().numpy()
+            assert np.array_equal(a.ravel(), o.state(name).ravel()), (t, name)
+    g.close(); o.close()
+
+
+def test_c2_full_size_element_by_element():
+    full_oracle_run(synth.workload("C2"), 3)
+
+
+def test_c4_full_size_element_by_element():
+    full_oracle_run(synth.workload("C4"), 2)
+
+
+# ------------------------------------------------------------------------------ C5, sampled
+
+def sample_coordinates(d, count, seed):
+    rng = np.random.default_rng(seed)
+    parts = [rng.integers(0, d, count), np.arange(0, min(d, 2048)), np.arange(max(0, d - 2048), d)]
+    for center in (1 << 29, 1 << 30, 1 << 31, 3 << 29, 16384 * 1000, 16384 * 50001):
+        if center + 70 < d:
+            parts.append(np.arange(center - 70, center + 70))
+    return np.unique(np.concatenate(parts)).astype(np.int64)
+
+
+def unpack_bits(words, d):
+    """bool[d] from int32 sign words, in chunks to bound temporaries."""
+    out = torch.empty(d, dtype=torch.bool, device=words.device)
+    ar = torch.arange(32, device=words.device, dtype=torch.int32)
+    step = 1 << 22
+    for a in range(0, words.numel(), step):
+        wchunk = words[a:a + step]
+        b = ((wchunk.view(-1, 1) >> ar) & 1).bool().view(-1)
+        lo = a * 32
+        hi = min(d, lo + b.numel())
+        out[lo:hi] = b[:hi - lo]
+    return out
+
+
+def exact_scale(u):
+    """Correctly rounded scale of one flat segment with the oracle's exact l1 routine."""
+    return np.float32(orc.l1_exact(u.cpu().numpy()) / u.numel())
+
+
+def test_c5_full_size_scales_bits_and_sampled_state():
+    w = synth.workload("C5")
+    d, n = w.d, w.n
+    x0 = w.x0(DEV)
+    J = sample_coordinates(d, 300_000, 1)
+    Jt = torch.from_numpy(J).to(DEV)
+    g = cd.CDAdam(d, n, w.compressor, x0=x0)
+    o = orc.Oracle(J.size, n, orc.SIGN, x0=x0[Jt].cpu().numpy())
+    ghat_prev = None                 # worker states as they must be, rebuilt from the payloads
+    gtil_prev = torch.zeros(d, device=DEV)
+    grads = torch.empty((n, d), dtype=torch.float32, device=DEV)
+    for t in (1, 2):
+        w.grads(t, out=grads)
+        g.step(grads.reshape(-1))
+        wscales = np.zeros((n, 1), np.float32)
+        new_ghat = []
+        for i in range(n):
+            u = grads[i] if ghat_prev is None else grads[i] - ghat_prev[i]
+            bits, scale = g.last_payload(i)
+            assert scale.cpu().numpy()[0] == exact_scale(u), (t, i)
+            nonneg = unpack_bits(bits, d)
+            assert torch.equal(nonneg, u >= 0), (t, i)
+            wscales[i, 0] = scale.cpu().numpy()[0]
+            if t == 1:               # ghat_1 = 0 + c_1, needed to form u at step 2
+                s = scale[0]
+                new_ghat.append(torch.where(nonneg, s, -s))
+            del u, nonneg
+        if t == 1:
+            ghat_prev = new_ghat
+        ghat_s = g.get_state("ghat_s")
+        wv = ghat_s - gtil_prev
+        sbits, sscale = g.last_payload(cd.SERVER)
+        assert sscale.cpu().numpy()[0] == exact_scale(wv), t
+        assert torch.equal(unpack_bits(sbits, d), wv >= 0), t
+        del wv, ghat_s
+        o.force_scales(wscales, sscale.cpu().numpy())
+        o.step(grads[:, Jt].cpu().numpy())
+        gtil_prev = g.get_state("gtil")
+        for name in ("ghat_s", "gtil", "m", "v", "vhat", "x"):
+            a = g.get_state(name)[Jt].cpu().numpy()
+            assert np.array_equal(a, o.state(name)), (t, name)
+    del ghat_prev, new_ghat, gtil_prev
+    a = g.get_state("ghat_w")[:, Jt].cpu().numpy()       # applies the deferred payload
+    assert np.array_equal(a, o.state("ghat_w"))
+    g.close(); o.close()
+
+
+# ------------------------------------------------------------------------------ C3, properties
+
+def expected_topk(u, k):
+    """Index set the definition fixes: all |u| above the k-th largest magnitude and, among
+    those equal to it, the lowest indices."""
+    mag = u.abs()
+    thr = torch.kthvalue(mag, u.numel() - k + 1).values
+    above = torch.nonzero(mag > thr).view(-1)
+    ties = torch.nonzero(mag == thr).view(-1)[:k - above.numel()]
+    return torch.sort(torch.cat([above, ties])).values
+
+
+def test_c3_full_size_topk_selection_and_updates():
+    w = synth.workload("C3")
+    d, n, k = w.d, w.n, w.k
+    x0 = w.x0(DEV)
+    g = cd.CDAdam(d, n, w.compressor, k=k, x0=x0)
+    f = np.float32
+    b1, b2, lr, nu = f(w.beta1), f(w.beta2), f(w.lr), f(w.eps)
+    for t in (1, 2):
+        prev = {name: g.get_state(name) for name in orc.STATE_NAMES}
+        grads = w.grads(t, DEV)
+        g.step(grads.reshape(-1))
+        acc = torch.zeros(d, device=DEV)
+        ghat_w = g.get_state("ghat_w")
+        for i in range(n):
+            u = grads[i] - prev["ghat_w"][i]
+            idx, val = g.last_payload(i)
+            want = expected_topk(u, k)
+            assert torch.equal(idx.long(), want), (t, i)
+            assert torch.equal(val, u[want]), (t, i)
+            exp = prev["ghat_w"][i].clone()
+            exp[want] = exp[want] + u[want]
+            assert torch.equal(ghat_w[i], exp), (t, i)
+            acc[want] = acc[want] + u[want]               # workers in increasing order
+        ghat_s = prev["ghat_s"] + acc / float(n)
+        assert torch.equal(g.get_state("ghat_s"), ghat_s), t
+        wv = ghat_s - prev["gtil"]
+        idx, val = g.last_payload(cd.SERVER)
+        want = expected_topk(wv, k)
+        assert torch.equal(idx.long(), want) and torch.equal(val, wv[want]), t
+        gtil = prev["gtil"].clone()
+        gtil[want] = gtil[want] + wv[want]
+        assert torch.equal(g.get_state("gtil"), gtil), t
+        # AMSGrad of Section 3 on gtil, one rounding per operation (torch eager, no fusion)
+        m = float(b1) * prev["m"] + float(f(1) - b1) * gtil
+        v = float(b2) * prev["v"] + float(f(1) - b2) * (gtil * gtil)
+        vh = torch.maximum(prev["vhat"], v)
+        x = prev["x"] - (float(lr) * m) / torch.sqrt(vh + float(nu))
+        for name, exp in (("m", m), ("v", v), ("vhat", vh), ("x", x)):
+            assert torch.equal(g.get_state(name), exp), (t, name)
+    g.close()
