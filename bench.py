@@ -163,6 +163,22 @@ def run_reference(args, rank):
     print(json.dumps(line))
 
 
+def max_over_ranks_ms(ms, device):
+    """Device time of a region on this rank -> the maximum over all ranks (N = 1: itself)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_throughput(world, steps, total_ms):
+    """N independent replicas ("replicas only"): units all ranks processed over the slowest
+    rank's time."""
+    return world * steps / (total_ms * 1e-3)
+
+
 def describe(w):
     from paper_2111_00705_b200 import synth
     comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity"}[w.compressor]
@@ -250,12 +266,9 @@ def main():
         barrier()
         total_ms = sum(a.elapsed_time(b) for a, b in pairs)
     clocks = sampler.stop() if sampler else None
-    t_ms = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    total_ms = float(t_ms.item())
+    total_ms = max_over_ranks_ms(total_ms, dev)
     ms_per_step = total_ms / args.steps
-    value = world * args.steps / (total_ms * 1e-3)
+    value = replicas_throughput(world, args.steps, total_ms)
 
     # ---- per-kernel pass for the roofline ------------------------------------------------
     opt.profile_enable(True)
@@ -293,10 +306,8 @@ def main():
             opt.step_host(gh[0], xh, stream)
         b.record(stream)
         barrier()
-        e_ms = torch.tensor([a.elapsed_time(b)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(e_ms, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * args.e2e_steps / (float(e_ms.item()) * 1e-3), "unit": UNIT,
+        e_ms = max_over_ranks_ms(a.elapsed_time(b), dev)
+        e2e = {"value": replicas_throughput(world, args.e2e_steps, e_ms), "unit": UNIT,
                "h2d_bytes_per_step": w.n * w.d * 4, "d2h_bytes_per_step": w.d * 4,
                "steps": args.e2e_steps}
         del gh, xh
