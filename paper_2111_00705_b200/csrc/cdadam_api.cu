@@ -46,13 +46,14 @@ struct DeviceGuard {
     ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
 };
 
-// Tile size: a multiple of kSub; larger vectors use larger tiles so that the number of
-// partial sums per segment stays small.
-int choose_tile(int64_t d)
+// Tile size, a multiple of kSub.  Larger tiles amortise the per-block reduction and make the
+// streams longer, but every tile that contains a segment boundary takes the scalar path, so
+// the tile is kept small enough that such tiles hold at most about 2 % of the coordinates.
+int choose_tile(int64_t d, int q)
 {
-    if (d >= (int64_t)1 << 28) return 4 * kSub;
-    if (d >= (int64_t)1 << 24) return 2 * kSub;
-    return kSub;
+    int tile = kSub;
+    while (tile < 4 * kSub && (int64_t)(q - 1) * (2 * tile) * 50 <= d && d >= (int64_t)tile * 2 * 2048) tile *= 2;
+    return tile;
 }
 
 // Host tables + their device copies.
@@ -80,8 +81,15 @@ struct TableSet {
             pbase[T] = np;
             np += e - r + 1;
         }
+        std::vector<int32_t> order;
+        order.reserve(ntiles);
+        for (int pass = 0; pass < 2; ++pass)          // slow tiles first, then the rest in order
+            for (int64_t T = 0; T < ntiles; ++T) {
+                const bool slow = first[T] != last[T] || (T + 1) * (int64_t)tile > d;
+                if (slow == (pass == 0)) order.push_back((int32_t)T);
+            }
         const size_t b_off = (size_t)(q + 1) * 8, b_pb = (size_t)ntiles * 8, b_t = (size_t)ntiles * 4;
-        const size_t total = b_off + b_pb + 2 * b_t;
+        const size_t total = b_off + b_pb + 3 * b_t;
         cudaError_t e = async ? cudaMallocAsync(&dev, total, st) : cudaMalloc(&dev, total);
         if (e != cudaSuccess) { dev = nullptr; return fail(CDADAM_ERR_ALLOC, "table allocation: %s", cudaGetErrorString(e)); }
         char *p = (char *)dev;
@@ -90,12 +98,14 @@ struct TableSet {
         CU_TRY(cudaMemcpyAsync(p + b_off, pbase.data(), b_pb, cudaMemcpyHostToDevice, st));
         CU_TRY(cudaMemcpyAsync(p + b_off + b_pb, first.data(), b_t, cudaMemcpyHostToDevice, st));
         CU_TRY(cudaMemcpyAsync(p + b_off + b_pb + b_t, last.data(), b_t, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(p + b_off + b_pb + 2 * b_t, order.data(), b_t, cudaMemcpyHostToDevice, st));
         CU_TRY(cudaStreamSynchronize(st));
         tb.d = d; tb.q = q; tb.tile = tile; tb.ntiles = ntiles; tb.nparts = np;
         tb.off = (const int64_t *)p;
         tb.pbase = (const int64_t *)(p + b_off);
         tb.tile_first = (const int32_t *)(p + b_off + b_pb);
         tb.tile_last = (const int32_t *)(p + b_off + b_pb + b_t);
+        tb.order = (const int32_t *)(p + b_off + b_pb + 2 * b_t);
         return CDADAM_OK;
     }
     void release(cudaStream_t st, bool async)
@@ -235,7 +245,7 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
         if (compressor == CDADAM_SIGN) {
             if ((rc = dev_zalloc(&c->wbits, (size_t)n * c->wp))) break;
             if ((rc = dev_zalloc(&c->sbits, (size_t)c->wp))) break;
-            if ((rc = c->ts.build(d, 1, flat, choose_tile(d), nullptr, false))) break;
+            if ((rc = c->ts.build(d, 1, flat, choose_tile(d, 1), nullptr, false))) break;
             if ((rc = alloc_sign_buffers(c))) break;
         } else if (compressor == CDADAM_TOPK) {
             if ((rc = dev_zalloc(&c->acc, (size_t)d))) break;
@@ -344,7 +354,7 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
     DeviceGuard guard(c->device);
     CU_TRY(cudaDeviceSynchronize());
-    int rc = c->ts.build(c->d, q, offsets, choose_tile(c->d), nullptr, false);
+    int rc = c->ts.build(c->d, q, offsets, choose_tile(c->d, q), nullptr, false);
     if (rc) return rc;
     return alloc_sign_buffers(c);
 }
@@ -463,7 +473,7 @@ int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offset
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing");
     cudaStream_t st = (cudaStream_t)stream;
     TableSet ts;
-    int rc = ts.build(d, q, offsets, choose_tile(d), st, true);
+    int rc = ts.build(d, q, offsets, choose_tile(d, q), st, true);
     if (rc) return rc;
     dd *part = nullptr;
     cudaError_t e = cudaMallocAsync((void **)&part, (size_t)ts.tb.nparts * sizeof(dd), st);

@@ -15,7 +15,9 @@ constexpr int kWarpSpan = kSub / (kBlock / 32);   // 512 consecutive elements pe
 // Tile and segment tables (device pointers).  The index space [0, d) is cut into tiles of
 // `tile` elements (a multiple of kSub).  tile_first/tile_last give the first and last
 // segment that overlaps a tile; a tile writes one partial l1 sum per overlapped segment at
-// pbase[T] + (r - tile_first[T]).
+// pbase[T] + (r - tile_first[T]).  Block b of a streaming kernel works on tile order[b]:
+// the few tiles that need the slower scalar path (segment boundaries, the ragged tail) come
+// first so that they overlap with the bulk instead of forming the kernel's tail.
 // ------------------------------------------------------------------------------------
 struct Tables {
     int64_t d;
@@ -27,6 +29,7 @@ struct Tables {
     const int32_t *tile_first; // ntiles
     const int32_t *tile_last;  // ntiles
     const int64_t *pbase;      // ntiles
+    const int32_t *order;      // ntiles: permutation of the tiles, slow tiles first
 };
 
 // ------------------------------------------------------------------------------------

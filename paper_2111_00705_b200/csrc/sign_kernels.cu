@@ -17,13 +17,13 @@ __device__ __forceinline__ float signed_scale(uint32_t bit, float s) { return bi
 // ------------------------------------------------------------------------------------
 // Worker pass.  grid = (ntiles, n).
 // ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kBlock)
+__global__ void __launch_bounds__(kBlock, 4)
 k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
               uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
               dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
 {
     const int i = blockIdx.y;
-    const int64_t T = blockIdx.x;
+    const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
     const float *g = grads + (int64_t)i * tb.d;
@@ -74,20 +74,39 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
         return;
     }
 
-    // scalar path: lane L of a warp holds coordinate (word start + L), ballot = word
+    // scalar path: lane L of a warp holds coordinate (word start + L), ballot = word.
+    // Four rounds are loaded before any is processed to keep several loads in flight.
     const int64_t end = min(base + (int64_t)tb.tile, tb.d);
-    for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
-        const bool valid = j < end;
-        float u = -1.0f;
-        if (valid) {
-            const int r = find_segment(tb.off, first, last, j);
-            const uint32_t bit = (bw[j >> 5] >> (j & 31)) & 1u;
-            const float hn = __fadd_rn(gh[j], signed_scale(bit, so[r]));
-            gh[j] = hn;
-            u = __fsub_rn(g[j], hn);
+    for (int64_t j0 = base + threadIdx.x; j0 - lane < end; j0 += 4 * kBlock) {
+        float gv[4], hv[4], sv[4];
+        uint32_t wv[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int64_t j = j0 + t * kBlock;
+            gv[t] = hv[t] = sv[t] = 0.0f;
+            wv[t] = 0u;
+            if (j < end) {
+                gv[t] = g[j];
+                hv[t] = gh[j];
+                wv[t] = bw[j >> 5];
+                sv[t] = so[find_segment(tb.off, first, last, j)];
+            }
         }
-        const uint32_t word = __ballot_sync(kFull, valid && u >= 0.0f);
-        if (lane == 0) bw[j >> 5] = word;
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const int64_t j = j0 + t * kBlock;
+            if (j - lane < end) {                      // warp-uniform
+                const bool valid = j < end;
+                float u = -1.0f;
+                if (valid) {
+                    const float hn = __fadd_rn(hv[t], signed_scale((wv[t] >> (j & 31)) & 1u, sv[t]));
+                    gh[j] = hn;
+                    u = __fsub_rn(gv[t], hn);
+                }
+                const uint32_t word = __ballot_sync(kFull, valid && u >= 0.0f);
+                if (lane == 0) bw[j >> 5] = word;
+            }
+        }
     }
     __syncthreads();
     for (int r = first; r <= last; ++r) {
@@ -142,7 +161,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
 {
     __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
     __shared__ float ssm[kNC];
-    const int64_t T = blockIdx.x;
+    const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
     dd *part = spart + tb.pbase[T];
@@ -279,7 +298,7 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
               float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
               float *__restrict__ vhat, float *__restrict__ x, Tables tb, Hyper hp, int vec_ok)
 {
-    const int64_t T = blockIdx.x;
+    const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -331,7 +350,7 @@ k_apply_sign(float *__restrict__ ghat_w, const uint32_t *__restrict__ wbits,
              const float *__restrict__ scales, Tables tb, int64_t wp)
 {
     const int i = blockIdx.y;
-    const int64_t T = blockIdx.x;
+    const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile, end = min(base + (int64_t)tb.tile, tb.d);
     float *gh = ghat_w + (int64_t)i * tb.d;
@@ -350,7 +369,7 @@ __global__ void __launch_bounds__(kBlock)
 k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__restrict__ part_all,
             Tables tb, int vec_ok)
 {
-    const int64_t T = blockIdx.x;
+    const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
     dd *part = part_all + tb.pbase[T];
