@@ -315,6 +315,7 @@ def main():
         e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
 
     launches = opt.launches_per_step() * args.steps
+    opt.device_status()          # raises if a kernel reported a bounded wait that ran out
     opt.close()
     del grads
     torch.cuda.empty_cache()

@@ -52,7 +52,8 @@ enum {
     CDADAM_ERR_ARG = -1,     /* invalid argument; nothing was queued */
     CDADAM_ERR_ALLOC = -2,   /* device or host allocation failed */
     CDADAM_ERR_CUDA = -3,    /* a CUDA runtime call failed; see cdadam_last_error */
-    CDADAM_ERR_STATE = -4    /* call not allowed in the context's current state */
+    CDADAM_ERR_STATE = -4,   /* call not allowed in the context's current state */
+    CDADAM_ERR_TIMEOUT = -5  /* a kernel's bounded wait on an asynchronous copy ran out */
 };
 
 /* names of the state vectors for cdadam_get_state / cdadam_set_state */
@@ -152,6 +153,14 @@ int cdadam_last_payload(cdadam_ctx *ctx, int who, const void **a, const float **
 
 /* Number of completed calls of cdadam_step on this context. */
 int64_t cdadam_step_count(cdadam_ctx *ctx);
+
+/*
+ * Waits for `stream` and reports whether any kernel of this context has given up a bounded
+ * wait (the large-tile worker kernel waits, with an iteration limit, for its bulk
+ * asynchronous copies; it never spins without bound).  CDADAM_ERR_TIMEOUT means the state
+ * of the context is no longer valid; the device itself stays usable.
+ */
+int cdadam_device_status(cdadam_ctx *ctx, void *stream);
 
 /* Number of kernels one cdadam_step launches in the context's current configuration. */
 int cdadam_launches_per_step(cdadam_ctx *ctx);

@@ -12,7 +12,7 @@ import torch
 SIGN, TOPK, IDENTITY = 0, 1, 2
 SERVER = -1
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
-OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE = 0, -1, -2, -3, -4
+OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcdadam.so")
 _lib = None
@@ -33,6 +33,7 @@ _SIGNATURES = {
     "cdadam_last_payload": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_void_p),
                                        _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_int64)]),
     "cdadam_step_count": (_c.c_int64, [_c.c_void_p]),
+    "cdadam_device_status": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "cdadam_launches_per_step": (_c.c_int, [_c.c_void_p]),
     "cdadam_compress_sign": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int,
                                         _c.POINTER(_c.c_int64), _c.c_void_p, _c.c_void_p,
@@ -213,6 +214,10 @@ class CDAdam:
             if name:
                 out[name] = ms[s]
         return out, steps.value
+
+    def device_status(self, stream=None):
+        """Wait for the stream; raise if a kernel reported that a bounded wait ran out."""
+        _check(lib().cdadam_device_status(self._h, _stream(stream)))
 
     def step_count(self):
         return lib().cdadam_step_count(self._h)

@@ -130,6 +130,7 @@ struct cdadam_ctx {
     uint32_t *wbits = nullptr, *sbits = nullptr;
     float *wscale[2] = {nullptr, nullptr}, *sscale = nullptr, *zero_scale = nullptr;
     dd *wpart = nullptr, *spart = nullptr;
+    int *error_flag = nullptr;   // device word set by a kernel whose bounded wait ran out
     int cur = 0;            // wscale[cur] holds the scales of the last worker payloads
     bool pending = false;   // the last worker payloads are not yet added to ghat_w
     // top-k
@@ -242,6 +243,7 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
         if ((rc = dev_zalloc(&c->v, (size_t)d))) break;
         if ((rc = dev_zalloc(&c->vhat, (size_t)d))) break;
         if ((rc = dev_zalloc(&c->x, (size_t)d))) break;
+        if ((rc = dev_zalloc(&c->error_flag, 1))) break;
         if (compressor == CDADAM_SIGN) {
             if ((rc = dev_zalloc(&c->wbits, (size_t)n * c->wp))) break;
             if ((rc = dev_zalloc(&c->sbits, (size_t)c->wp))) break;
@@ -264,7 +266,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaDeviceSynchronize();
     cudaFree(c->ghat_w); cudaFree(c->ghat_s); cudaFree(c->gtil);
     cudaFree(c->m); cudaFree(c->v); cudaFree(c->vhat); cudaFree(c->x);
-    cudaFree(c->wbits); cudaFree(c->sbits);
+    cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->acc); cudaFree(c->stage);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
@@ -286,7 +288,7 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
         const bool svec = c->d % 4 == 0;
         const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
         float *new_scale = c->wscale[c->cur ^ 1];
-        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, st);
+        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, c->error_flag, st);
         prof_mark(c, st);
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
         prof_mark(c, st);
@@ -417,6 +419,17 @@ int cdadam_last_payload(cdadam_ctx *c, int who, const void **a, const float **b,
 }
 
 int64_t cdadam_step_count(cdadam_ctx *c) { return c ? c->steps : 0; }
+
+int cdadam_device_status(cdadam_ctx *c, void *stream)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_device_status: NULL context");
+    DeviceGuard guard(c->device);
+    int flag = 0;
+    CU_TRY(cudaMemcpyAsync(&flag, c->error_flag, sizeof flag, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    if (flag) return fail(CDADAM_ERR_TIMEOUT, "a kernel gave up waiting for an asynchronous copy; the state is not valid");
+    return CDADAM_OK;
+}
 
 int cdadam_launches_per_step(cdadam_ctx *c)
 {

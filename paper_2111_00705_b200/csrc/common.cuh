@@ -121,6 +121,51 @@ __device__ __forceinline__ void st_rw4(float *p, float4 v)
 __device__ __forceinline__ uint32_t ld_ro_u32(const uint32_t *p) { return __ldg(p); }
 
 // ------------------------------------------------------------------------------------
+// Bulk asynchronous copies (TMA, one-dimensional, no multicast) global -> shared, completed
+// on an mbarrier.  Addresses and sizes must be multiples of 16 bytes.  Every wait is
+// bounded: a barrier that does not complete makes the caller report an error and leave.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, int arrivals)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals));
+}
+__device__ __forceinline__ void mbar_fence_init()
+{
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile("{\n.reg .pred p;\n"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+                 "selp.u32 %0, 1, 0, p;\n}"
+                 : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+constexpr int kWaitLimit = 1 << 22;     // try_wait attempts before a wait gives up
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
+{
+    for (int spin = 0; spin < kWaitLimit; ++spin)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_copy_g2s(void *dst_smem, const void *src_gmem, uint32_t bytes,
+                                              uint64_t *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst_smem)), "l"(src_gmem), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+
+// ------------------------------------------------------------------------------------
 // Sign-bit packing.  In the vector kernels lane L of a warp holds the four consecutive
 // coordinates 4L..4L+3 of a 128-coordinate group, so the ballot over component c has bit L
 // = sign of coordinate 4L + c.  Word g (coordinates 32g..32g+31) of the group is the

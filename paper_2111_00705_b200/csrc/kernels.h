@@ -8,10 +8,12 @@ namespace cdadam {
 // ---- scaled sign -------------------------------------------------------------------
 // Worker pass (Algorithm 1 lines 5-6) for all n workers: applies the previous payload
 // (bits in wbits, scales in scale_old) to ghat_w, forms u = g - ghat_w, packs sign(u) into
-// wbits and writes per-tile double-double partial sums of |u| to wpart.
+// wbits and writes per-tile double-double partial sums of |u| to wpart.  For large tiles the
+// variant with a TMA prefetch ring runs; it sets *error_flag (device) if a bounded wait on
+// a copy ran out.
 void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, cudaStream_t st);
+                        int64_t wp, bool vec_ok, int *error_flag, cudaStream_t st);
 // Correctly rounded scale of every (row, segment) from the partial sums.
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
                             cudaStream_t st);

@@ -14,69 +14,17 @@ constexpr uint32_t kFull = 0xffffffffu;
 
 __device__ __forceinline__ float signed_scale(uint32_t bit, float s) { return bit ? s : -s; }
 
-// ------------------------------------------------------------------------------------
-// Worker pass.  grid = (ntiles, n).
-// ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kBlock, 4)
-k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
-              uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
-              dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
+// Scalar path of the worker pass for one tile (segment boundaries, the ragged last tile,
+// unaligned rows).  Kept out of line so that it does not shape the register allocation and
+// instruction schedule of the vector path.
+__device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, float *__restrict__ gh,
+                                                uint32_t *__restrict__ bw, const float *__restrict__ so,
+                                                dd *__restrict__ part, const int64_t *__restrict__ off,
+                                                int64_t base, int64_t end, int first, int last)
 {
-    const int i = blockIdx.y;
-    const int64_t T = tb.order[blockIdx.x];
-    const int first = tb.tile_first[T], last = tb.tile_last[T];
-    const int64_t base = T * tb.tile;
-    const float *g = grads + (int64_t)i * tb.d;
-    float *gh = ghat_w + (int64_t)i * tb.d;
-    uint32_t *bw = wbits + (int64_t)i * wp;
-    const float *so = scale_old + (int64_t)i * tb.q;
-    dd *part = wpart + (int64_t)i * tb.nparts + tb.pbase[T];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    if (vec_ok && first == last && base + tb.tile <= tb.d) {
-        const float s = so[first];
-        dd acc = {0.0, 0.0};
-        for (int it = 0; it < tb.tile / kSub; ++it) {
-            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
-            float4 G[4], H[4];
-            uint32_t ow[4];
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const int64_t j = wb + v * 128 + lane * 4;
-                G[v] = ld_ro4(g + j);
-                H[v] = ld_rw4(gh + j);
-                ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
-            }
-            uint32_t B[4][4];
-#pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const uint32_t nib = ow[v] >> ((lane & 7) * 4);
-                // ghat_{t-1} = ghat_{t-2} + c_{t-1}: the previous payload, applied now
-                H[v].x = __fadd_rn(H[v].x, signed_scale(nib & 1u, s));
-                H[v].y = __fadd_rn(H[v].y, signed_scale(nib & 2u, s));
-                H[v].z = __fadd_rn(H[v].z, signed_scale(nib & 4u, s));
-                H[v].w = __fadd_rn(H[v].w, signed_scale(nib & 8u, s));
-                st_rw4(gh + wb + v * 128 + lane * 4, H[v]);
-                const float ux = __fsub_rn(G[v].x, H[v].x), uy = __fsub_rn(G[v].y, H[v].y);
-                const float uz = __fsub_rn(G[v].z, H[v].z), uw = __fsub_rn(G[v].w, H[v].w);
-                dd_acc(acc, fabsf(ux)); dd_acc(acc, fabsf(uy));
-                dd_acc(acc, fabsf(uz)); dd_acc(acc, fabsf(uw));
-                B[v][0] = __ballot_sync(kFull, ux >= 0.0f);
-                B[v][1] = __ballot_sync(kFull, uy >= 0.0f);
-                B[v][2] = __ballot_sync(kFull, uz >= 0.0f);
-                B[v][3] = __ballot_sync(kFull, uw >= 0.0f);
-            }
-            const uint32_t word = warp_words(B, lane);
-            if (lane < 16) bw[(wb >> 5) + lane] = word;
-        }
-        acc = block_sum<kBlock>(acc);
-        if (threadIdx.x == 0) part[0] = acc;
-        return;
-    }
-
+    const int lane = threadIdx.x & 31;
     // scalar path: lane L of a warp holds coordinate (word start + L), ballot = word.
     // Four rounds are loaded before any is processed to keep several loads in flight.
-    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
     for (int64_t j0 = base + threadIdx.x; j0 - lane < end; j0 += 4 * kBlock) {
         float gv[4], hv[4], sv[4];
         uint32_t wv[4];
@@ -89,7 +37,7 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
                 gv[t] = g[j];
                 hv[t] = gh[j];
                 wv[t] = bw[j >> 5];
-                sv[t] = so[find_segment(tb.off, first, last, j)];
+                sv[t] = so[find_segment(off, first, last, j)];
             }
         }
 #pragma unroll
@@ -110,13 +58,181 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
     }
     __syncthreads();
     for (int r = first; r <= last; ++r) {
-        const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
+        const int64_t lo = max(off[r], base), hi = min(off[r + 1], end);
         dd acc = {0.0, 0.0};
         for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
             dd_acc(acc, fabsf(__fsub_rn(g[j], gh[j])));
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
+}
+
+// ------------------------------------------------------------------------------------
+// Worker pass.  grid = (ntiles, n).
+// ------------------------------------------------------------------------------------
+// The 16 coordinates a thread owns in one 4096-coordinate sub-tile: gradient, worker state
+// and the previous payload's sign words.
+struct WorkerRegs {
+    float4 G[4], H[4];
+    uint32_t ow[4];
+};
+
+__device__ __forceinline__ void worker_load(WorkerRegs &r, const float *__restrict__ g,
+                                            const float *__restrict__ gh,
+                                            const uint32_t *__restrict__ bw, int64_t wb, int lane)
+{
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        const int64_t j = wb + v * 128 + lane * 4;
+        r.G[v] = ld_ro4(g + j);
+        r.H[v] = ld_rw4(gh + j);
+        r.ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
+    }
+}
+
+__device__ __forceinline__ void worker_compute(WorkerRegs &r, float *__restrict__ gh,
+                                               uint32_t *__restrict__ bw, int64_t wb, int lane,
+                                               float s, dd &acc)
+{
+    uint32_t B[4][4];
+#pragma unroll
+    for (int v = 0; v < 4; ++v) {
+        const uint32_t nib = r.ow[v] >> ((lane & 7) * 4);
+        float4 H = r.H[v];
+        // ghat_{t-1} = ghat_{t-2} + c_{t-1}: the previous payload, applied now
+        H.x = __fadd_rn(H.x, signed_scale(nib & 1u, s));
+        H.y = __fadd_rn(H.y, signed_scale(nib & 2u, s));
+        H.z = __fadd_rn(H.z, signed_scale(nib & 4u, s));
+        H.w = __fadd_rn(H.w, signed_scale(nib & 8u, s));
+        st_rw4(gh + wb + v * 128 + lane * 4, H);
+        const float ux = __fsub_rn(r.G[v].x, H.x), uy = __fsub_rn(r.G[v].y, H.y);
+        const float uz = __fsub_rn(r.G[v].z, H.z), uw = __fsub_rn(r.G[v].w, H.w);
+        dd_acc(acc, fabsf(ux)); dd_acc(acc, fabsf(uy));
+        dd_acc(acc, fabsf(uz)); dd_acc(acc, fabsf(uw));
+        B[v][0] = __ballot_sync(kFull, ux >= 0.0f);
+        B[v][1] = __ballot_sync(kFull, uy >= 0.0f);
+        B[v][2] = __ballot_sync(kFull, uz >= 0.0f);
+        B[v][3] = __ballot_sync(kFull, uw >= 0.0f);
+    }
+    const uint32_t word = warp_words(B, lane);
+    if (lane < 16) bw[(wb >> 5) + lane] = word;
+}
+
+__global__ void __launch_bounds__(kBlock, 4)
+k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
+              uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
+              dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
+{
+    const int i = blockIdx.y;
+    const int64_t T = tb.order[blockIdx.x];
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    const float *g = grads + (int64_t)i * tb.d;
+    float *gh = ghat_w + (int64_t)i * tb.d;
+    uint32_t *bw = wbits + (int64_t)i * wp;
+    const float *so = scale_old + (int64_t)i * tb.q;
+
+    if (!(vec_ok && first == last && base + tb.tile <= tb.d)) {
+        worker_tile_scalar(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+                           min(base + (int64_t)tb.tile, tb.d), first, last);
+        return;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float s = so[first];
+    const int iters = tb.tile / kSub;
+    dd acc = {0.0, 0.0};
+    for (int it = 0; it < iters; ++it) {
+        WorkerRegs r;
+        const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+        worker_load(r, g, gh, bw, wb, lane);
+        worker_compute(r, gh, bw, wb, lane, s, acc);
+    }
+    acc = block_sum<kBlock>(acc);
+    if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
+}
+
+// ------------------------------------------------------------------------------------
+// Worker pass with a prefetch ring.  grid = (ntiles, n), tile >= 4 sub-tiles.
+//
+// Same arithmetic as k_worker_sign.  The gradient and worker-state sub-tiles are brought
+// into a two-stage shared-memory ring by bulk asynchronous copies (TMA), issued by one
+// thread, so the next sub-tile is in flight while the block works on the current one; each
+// thread moves its 16 coordinates from the ring to registers and the stage is refilled at
+// once.  Measured at the HBM ceiling for this 8-bytes-read / 4-bytes-written mix.
+// ------------------------------------------------------------------------------------
+constexpr int kRingStages = 2;
+constexpr int kRingStageBytes = 2 * kSub * (int)sizeof(float);    // g and ghat sub-tile: 32 KiB
+constexpr int kRingSmemBytes = kRingStages * kRingStageBytes;
+
+__global__ void __launch_bounds__(kBlock, 3)
+k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
+                   uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
+                   dd *__restrict__ wpart, Tables tb, int64_t wp, int *__restrict__ error_flag)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ __align__(8) uint64_t full[kRingStages];
+    const int i = blockIdx.y;
+    const int64_t T = tb.order[blockIdx.x];
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t base = T * tb.tile;
+    const float *g = grads + (int64_t)i * tb.d;
+    float *gh = ghat_w + (int64_t)i * tb.d;
+    uint32_t *bw = wbits + (int64_t)i * wp;
+    const float *so = scale_old + (int64_t)i * tb.q;
+
+    if (!(first == last && base + tb.tile <= tb.d)) {          // block-uniform
+        worker_tile_scalar(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+                           min(base + (int64_t)tb.tile, tb.d), first, last);
+        return;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int iters = tb.tile / kSub;
+    if (threadIdx.x == 0) {
+        for (int st = 0; st < kRingStages; ++st) mbar_init(&full[st], 1);
+        mbar_fence_init();
+    }
+    __syncthreads();
+    auto refill = [&](int it, int st) {                        // one thread
+        float *dst = reinterpret_cast<float *>(ring + st * kRingStageBytes);
+        mbar_arrive_expect_tx(&full[st], (uint32_t)kRingStageBytes);
+        bulk_copy_g2s(dst, g + base + (int64_t)it * kSub, kSub * sizeof(float), &full[st]);
+        bulk_copy_g2s(dst + kSub, gh + base + (int64_t)it * kSub, kSub * sizeof(float), &full[st]);
+    };
+    if (threadIdx.x == 0)
+        for (int st = 0; st < kRingStages && st < iters; ++st) refill(st, st);
+    const float s = so[first];
+    dd acc = {0.0, 0.0};
+    bool arrived = true;
+    for (int it = 0; it < iters; ++it) {
+        const int st = it % kRingStages;
+        arrived = mbar_wait_bounded(&full[st], (uint32_t)(it / kRingStages) & 1u);
+        if (!arrived) break;
+        const float *src = reinterpret_cast<const float *>(ring + st * kRingStageBytes);
+        const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+        WorkerRegs r;
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int e = warp * kWarpSpan + v * 128 + lane * 4;
+            r.G[v] = *reinterpret_cast<const float4 *>(src + e);
+            r.H[v] = *reinterpret_cast<const float4 *>(src + kSub + e);
+            r.ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
+        }
+        __syncthreads();                                       // the stage has been read by all
+        if (threadIdx.x == 0 && it + kRingStages < iters) refill(it + kRingStages, st);
+        worker_compute(r, gh, bw, wb, lane, s, acc);
+    }
+    if (!arrived) {
+        // A copy did not complete in time: report it, give the copies still in flight a
+        // bounded chance to land before this block's shared memory is released, and leave.
+        if (threadIdx.x == 0) atomicExch(error_flag, 1);
+        for (int st = 0; st < kRingStages; ++st) {
+            mbar_wait_bounded(&full[st], 0u);
+            mbar_wait_bounded(&full[st], 1u);
+        }
+        return;
+    }
+    acc = block_sum<kBlock>(acc);
+    if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
 }
 
 // ------------------------------------------------------------------------------------
@@ -291,45 +407,53 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
 }
 
 // ------------------------------------------------------------------------------------
-// Server pass B + worker update.  grid = (ntiles).
+// Server pass B + worker update.  grid = ceil(d / 1024): one float4 of each of the five
+// vectors per thread.  This kernel has no reduction, and short blocks at full occupancy
+// measured fastest for its ten streams (five read, five written).
 // ------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kBlock)
+constexpr int kUpdSpan = kBlock * 4;
+
+__global__ void __launch_bounds__(kBlock, 5)
 k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ sscale,
               float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
               float *__restrict__ vhat, float *__restrict__ x, Tables tb, Hyper hp, int vec_ok)
 {
-    const int64_t T = tb.order[blockIdx.x];
-    const int first = tb.tile_first[T], last = tb.tile_last[T];
-    const int64_t base = T * tb.tile;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t base = (int64_t)blockIdx.x * kUpdSpan;
+    const int64_t T = base / tb.tile;
 
-    if (vec_ok && first == last && base + tb.tile <= tb.d) {
-        const float s = __ldg(sscale + first);
-        for (int it = 0; it < tb.tile / kSub; ++it) {
-            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
-#pragma unroll 2
-            for (int v4 = 0; v4 < 4; ++v4) {
-                const int64_t j = wb + v4 * 128 + lane * 4;
-                float4 Gt = ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
-                float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
-                const uint32_t nib = ld_ro_u32(sbits + (wb >> 5) + v4 * 4 + (lane >> 3)) >>
-                                     ((lane & 7) * 4);
-                Gt.x = __fadd_rn(Gt.x, signed_scale(nib & 1u, s));
-                Gt.y = __fadd_rn(Gt.y, signed_scale(nib & 2u, s));
-                Gt.z = __fadd_rn(Gt.z, signed_scale(nib & 4u, s));
-                Gt.w = __fadd_rn(Gt.w, signed_scale(nib & 8u, s));
-                amsgrad1(Gt.x, M.x, V.x, Vh.x, X.x, hp);
-                amsgrad1(Gt.y, M.y, V.y, Vh.y, X.y, hp);
-                amsgrad1(Gt.z, M.z, V.z, Vh.z, X.z, hp);
-                amsgrad1(Gt.w, M.w, V.w, Vh.w, X.w, hp);
-                st_rw4(gtil + j, Gt); st_rw4(m + j, M); st_rw4(v + j, V);
-                st_rw4(vhat + j, Vh); st_rw4(x + j, X);
-            }
+    if (vec_ok && base + kUpdSpan <= tb.d) {
+        const int64_t j = base + threadIdx.x * 4;
+        float4 Gt = ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
+        float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
+        const uint32_t nib = ld_ro_u32(sbits + (j >> 5)) >> (j & 31);
+        const int first = tb.tile_first[T], last = tb.tile_last[T];
+        float s0, s1, s2, s3;
+        s0 = s1 = s2 = s3 = __ldg(sscale + first);
+        if (first != last) {                            // the tile spans several segments
+            int r = find_segment(tb.off, first, last, j);
+            s0 = __ldg(sscale + r);
+            while (r < last && j + 1 >= tb.off[r + 1]) ++r;
+            s1 = __ldg(sscale + r);
+            while (r < last && j + 2 >= tb.off[r + 1]) ++r;
+            s2 = __ldg(sscale + r);
+            while (r < last && j + 3 >= tb.off[r + 1]) ++r;
+            s3 = __ldg(sscale + r);
         }
+        Gt.x = __fadd_rn(Gt.x, signed_scale(nib & 1u, s0));
+        Gt.y = __fadd_rn(Gt.y, signed_scale(nib & 2u, s1));
+        Gt.z = __fadd_rn(Gt.z, signed_scale(nib & 4u, s2));
+        Gt.w = __fadd_rn(Gt.w, signed_scale(nib & 8u, s3));
+        amsgrad1(Gt.x, M.x, V.x, Vh.x, X.x, hp);
+        amsgrad1(Gt.y, M.y, V.y, Vh.y, X.y, hp);
+        amsgrad1(Gt.z, M.z, V.z, Vh.z, X.z, hp);
+        amsgrad1(Gt.w, M.w, V.w, Vh.w, X.w, hp);
+        st_rw4(gtil + j, Gt); st_rw4(m + j, M); st_rw4(v + j, V);
+        st_rw4(vhat + j, Vh); st_rw4(x + j, X);
         return;
     }
 
-    const int64_t end = min(base + (int64_t)tb.tile, tb.d);
+    const int first = tb.tile_first[T], last = tb.tile_last[T];
+    const int64_t end = min(base + (int64_t)kUpdSpan, tb.d);
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
         const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
@@ -420,10 +544,16 @@ k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__rest
 // ------------------------------------------------------------------------------------
 void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, cudaStream_t st)
+                        int64_t wp, bool vec_ok, int *error_flag, cudaStream_t st)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
-    k_worker_sign<<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+    if (vec_ok && tb.tile >= 4 * kSub) {
+        cudaFuncSetAttribute(k_worker_sign_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
+        k_worker_sign_ring<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb,
+                                                                 wp, error_flag);
+    } else {
+        k_worker_sign<<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+    }
 }
 
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
@@ -446,8 +576,8 @@ void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil,
                         float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
                         bool vec_ok, cudaStream_t st)
 {
-    k_update_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(sbits, sscale, gtil, m, v, vhat, x, tb,
-                                                          hp, vec_ok);
+    const unsigned blocks = (unsigned)((tb.d + kUpdSpan - 1) / kUpdSpan);
+    k_update_sign<<<blocks, kBlock, 0, st>>>(sbits, sscale, gtil, m, v, vhat, x, tb, hp, vec_ok);
 }
 
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,

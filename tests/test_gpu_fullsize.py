@@ -46,6 +46,7 @@ def full_oracle_run(w, steps):
         for name in names:                       # ghat_w only at the end: keeps the deferred path
             a = g.get_state(name).cpu().numpy()
             assert np.array_equal(a.ravel(), o.state(name).ravel()), (t, name)
+    g.device_status()
     g.close(); o.close()
 
 
@@ -131,6 +132,7 @@ def test_c5_full_size_scales_bits_and_sampled_state():
     del ghat_prev, new_ghat, gtil_prev
     a = g.get_state("ghat_w")[:, Jt].cpu().numpy()       # applies the deferred payload
     assert np.array_equal(a, o.state("ghat_w"))
+    g.device_status()
     g.close(); o.close()
 
 

@@ -81,6 +81,7 @@ def run_free(w, steps, exact=True, **kw):
         else:
             for name in ("x", "m", "v", "vhat", "gtil", "ghat_s"):
                 assert rel_err(g.get_state(name).cpu().numpy(), o.state(name)) <= STEP_TOL
+    g.device_status()                     # no kernel gave up a bounded wait
     g.close(); o.close()
 
 
