@@ -125,6 +125,14 @@ int cdadam_set_params(cdadam_ctx *ctx, const float *x0, void *stream);
  */
 int cdadam_set_segments(cdadam_ctx *ctx, int q, const int64_t *offsets);
 
+/*
+ * Tuning knob: the number of consecutive coordinates one thread block of the scaled-sign
+ * kernels owns (a multiple of 4096, at most 262144; 0 = chosen from d and q, the default).
+ * Results do not depend on it.  Tiles of 16384 coordinates or more select the worker kernel
+ * with the asynchronous-copy prefetch ring.  Only before the first step; synchronous.
+ */
+int cdadam_set_tile(cdadam_ctx *ctx, int tile);
+
 /* Step size alpha_t for the following steps (Algorithm 1 takes a non-increasing sequence;
  * monotonicity is not enforced). */
 int cdadam_set_lr(cdadam_ctx *ctx, float lr);

@@ -27,6 +27,7 @@ _SIGNATURES = {
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
+    "cdadam_set_tile": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
     "cdadam_get_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
@@ -172,6 +173,9 @@ class CDAdam:
         off = (ctypes.c_int64 * len(offsets))(*[int(v) for v in offsets])
         _check(lib().cdadam_set_segments(self._h, len(offsets) - 1, off))
         self.q = len(offsets) - 1
+
+    def set_tile(self, tile):
+        _check(lib().cdadam_set_tile(self._h, int(tile)))
 
     def set_lr(self, lr):
         _check(lib().cdadam_set_lr(self._h, lr))

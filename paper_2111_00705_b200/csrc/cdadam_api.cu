@@ -122,6 +122,7 @@ bool aligned16(const void *p) { return ((uintptr_t)p & 15u) == 0; }
 struct cdadam_ctx {
     int64_t d = 0, k = 0, wp = 0, steps = 0;
     int n = 0, comp = 0, device = 0;
+    int tile_override = 0;  // 0 = choose from d and q
     Hyper hp{};
     TableSet ts;
     float *ghat_w = nullptr, *ghat_s = nullptr, *gtil = nullptr;
@@ -356,9 +357,21 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
     DeviceGuard guard(c->device);
     CU_TRY(cudaDeviceSynchronize());
-    int rc = c->ts.build(c->d, q, offsets, choose_tile(c->d, q), nullptr, false);
+    int rc = c->ts.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q), nullptr, false);
     if (rc) return rc;
     return alloc_sign_buffers(c);
+}
+
+int cdadam_set_tile(cdadam_ctx *c, int tile)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_tile: NULL context");
+    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "tiles apply to the scaled-sign compressor only");
+    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the tile size must be set before the first step");
+    if (tile != 0 && (tile < kSub || tile % kSub != 0 || tile > 64 * kSub))
+        return fail(CDADAM_ERR_ARG, "tile must be 0 or a multiple of %d up to %d", kSub, 64 * kSub);
+    c->tile_override = tile;
+    std::vector<int64_t> off = c->ts.off;         // rebuild the tables for the current segments
+    return cdadam_set_segments(c, (int)off.size() - 1, off.data());
 }
 
 int cdadam_set_lr(cdadam_ctx *c, float lr)

@@ -65,9 +65,11 @@ def check_state(g, o, tol, exact=False):
     return worst
 
 
-def run_free(w, steps, exact=True, **kw):
+def run_free(w, steps, exact=True, tile=0, **kw):
     """Free run: both sides step independently from the same inputs."""
     g, o = make_pair(w, **kw)
+    if tile:
+        g.set_tile(tile)
     for t in range(1, steps + 1):
         grads = w.grads(t, "cpu")
         g.step(grads.cuda())
@@ -133,6 +135,16 @@ def test_c4_scaled_heavy_tails():
 def test_c5_scaled_flat():
     w = synth.workload("C5", scale=0.0004)        # d = 600,000 flat, n = 4
     run_free(w, 4)
+
+
+@pytest.mark.parametrize("tile", [8192, 16384, 32768])
+def test_large_tiles_and_prefetch_ring_give_the_same_bits(tile):
+    """Tiles of 16384+ coordinates run the worker kernel with the asynchronous-copy ring;
+    segments cut some tiles (scalar path) and d leaves a ragged last tile."""
+    d = 5 * 32768 + 4321 * 4
+    off = np.array([0, 1000, 40000, 40001, 3 * 32768, d])
+    run_free(synth.Workload("RING", d, 3, synth.SIGN, 4, offsets=off, seed=tile), 4, tile=tile)
+    run_free(synth.Workload("RINGF", 4 * 65536, 2, synth.SIGN, 3, seed=tile + 1), 3, tile=tile)
 
 
 def test_identity_matches_oracle():
