@@ -37,7 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 # ncu capture of the dominant kernel: dram__bytes_read.sum + dram__bytes_write.sum per launch,
 # keyed by workload, with the hash of the kernel sources at capture time.  A changed source
 # makes the figure stale and bench reports null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
+    "C4": {"hash": "95acb0a30d838775", "bytes_per_launch": 4 * (1.797066e9 + 0.856808e9)},
+}
 
 
 def kernel_source_hash():
@@ -194,6 +197,8 @@ def main():
     ap.add_argument("--impl", default="cdadam", choices=["cdadam", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tile", type=int, default=0,
+                    help="force the kernels' tile size (profiler captures of scaled-down cases)")
     ap.add_argument("--scale", type=float, default=1.0,
                     help="shrink d (same recipe) for profiler captures; not a bench line")
     args = ap.parse_args()
@@ -228,6 +233,8 @@ def main():
         args.warmup = 3
     opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
                     beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev)
+    if args.tile:
+        opt.set_tile(args.tile)
     # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
     # flushed between steps instead
     nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1
