@@ -147,6 +147,14 @@ def test_large_tiles_and_prefetch_ring_give_the_same_bits(tile):
     run_free(synth.Workload("RINGF", 4 * 65536, 2, synth.SIGN, 3, seed=tile + 1), 3, tile=tile)
 
 
+@pytest.mark.parametrize("n", [1, 5, 8, 9, 17, 32, 33, 40])
+def test_sign_worker_counts_cover_table_and_sequential_server_sums(n):
+    """n <= 8: the server sum comes from the pattern table alone; 9..32: table plus workers
+    added one by one; above 32: the staged kernel; odd n: true division by n."""
+    off = np.array([0, 5000, 3 * 4096 + 100, 5 * 4096])
+    run_free(synth.Workload("N", 5 * 4096, n, synth.SIGN, 3, offsets=off, seed=n), 3)
+
+
 def test_identity_matches_oracle():
     w = synth.Workload("ID", 5000, 3, synth.IDENTITY, 4)
     run_free(w, 4)
