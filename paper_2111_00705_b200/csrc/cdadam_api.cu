@@ -136,7 +136,6 @@ struct cdadam_ctx {
     bool pending = false;   // the last worker payloads are not yet added to ghat_w
     // top-k
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
-    float *acc = nullptr;   // dense per-coordinate sum of the workers' sparse payloads
     // host-gradient staging
     float *stage = nullptr;
     // optional per-kernel timing: events[step][0..nslots] recorded around every stage
@@ -251,7 +250,6 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
             if ((rc = c->ts.build(d, 1, flat, choose_tile(d, 1), nullptr, false))) break;
             if ((rc = alloc_sign_buffers(c))) break;
         } else if (compressor == CDADAM_TOPK) {
-            if ((rc = dev_zalloc(&c->acc, (size_t)d))) break;
             if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n))) { fail(rc, "top-k workspace allocation failed"); break; }
             if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1))) { fail(rc, "top-k workspace allocation failed"); break; }
         }
@@ -269,7 +267,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->m); cudaFree(c->v); cudaFree(c->vhat); cudaFree(c->x);
     cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
-    cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->acc); cudaFree(c->stage);
+    cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     for (cudaEvent_t e : c->prof_pool) cudaEventDestroy(e);
@@ -304,7 +302,7 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
     } else if (c->comp == CDADAM_TOPK) {
         topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
         prof_mark(c, st);
-        topk_aggregate(c->tk_w, c->ghat_s, c->acc, c->n, st);              // line 8
+        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);              // line 8
         prof_mark(c, st);
         topk_select(c->tk_s, c->ghat_s, c->gtil, true, c->d % 4 == 0, st); // lines 9-10, 12
         prof_mark(c, st);

@@ -24,8 +24,8 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
 
 // Sparse server aggregation (Algorithm 1 line 8) from the n payloads held in `ww`:
 //   ghat_s += (sum_i c_i) / n on the coordinates some worker sent, workers added in the
-//   order 0, 1, ..., n-1.  acc: d floats, all zero on entry and on exit.
-void topk_aggregate(TopkWorkspace *ww, float *ghat_s, float *acc, int n, cudaStream_t st);
+//   order 0, 1, ..., n-1.
+void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st);
 
 // Stand-alone top-k of one vector into caller buffers (allocates and frees scratch).
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,

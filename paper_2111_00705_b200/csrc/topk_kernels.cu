@@ -371,23 +371,17 @@ k_topk_ties(const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
 }
 
 // ------------------------------------------------------------------------------------
-// Ordered compaction of the selection bitmap into the payload (index-increasing), and the
-// state update b_j += u_j at the kept coordinates (Algorithm 1 lines 6 / 10).
+// Ordered compaction of the selection bitmap into the payload's index list (increasing).
+// A thread owns 4 consecutive bitmap words; ranks come from popcount scans.
 // grid = (nbt, rows).
 // ------------------------------------------------------------------------------------
-template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
-k_topk_emit(const float *__restrict__ a_all, float *__restrict__ b_all,
-            const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
-            uint32_t *__restrict__ idx_all, float *__restrict__ val_all, int64_t d, int64_t wp,
-            int64_t nbt, int64_t k)
+k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
+                uint32_t *__restrict__ idx_all, int64_t wp, int64_t nbt, int64_t k)
 {
     const int row = blockIdx.y;
-    const float *a = a_all + (int64_t)row * d;
-    float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     const uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
     uint32_t *idx = idx_all + (int64_t)row * k;
-    float *val = val_all + (int64_t)row * k;
     const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
     uint32_t keep[4];
 #pragma unroll
@@ -401,55 +395,104 @@ k_topk_emit(const float *__restrict__ a_all, float *__restrict__ b_all,
         while (word) {
             const int bit = __ffs(word) - 1;
             word &= word - 1;
-            const int64_t j = (w0 + m) * 32 + bit;
-            if (rank < k) {
-                float u;
-                if (HAS_B) {
-                    const float bj = b[j];
-                    u = __fsub_rn(a[j], bj);
-                    if (UPDATE_B) b[j] = __fadd_rn(bj, u);
-                } else {
-                    u = a[j];
-                }
-                idx[rank] = (uint32_t)j;
-                val[rank] = u;
-            }
+            if (rank < k) idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
             ++rank;
         }
     }
 }
 
 // ------------------------------------------------------------------------------------
-// Sparse server aggregation (Algorithm 1 line 8).
+// Payload values and the state update at the kept coordinates (Algorithm 1 lines 6 / 10):
+// val = u_j = a_j - b_j, b_j += u_j.  One thread per payload entry.  grid = (ceil(k/256), rows).
 // ------------------------------------------------------------------------------------
-// acc[idx[t]] += val[t] for one worker's payload (its indices are distinct).
+template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
-k_scatter_add(float *__restrict__ acc, const uint32_t *__restrict__ idx,
-              const float *__restrict__ val, int64_t k)
+k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
+              const uint32_t *__restrict__ idx_all, float *__restrict__ val_all, int64_t d, int64_t k)
 {
+    const int row = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
-    if (t < k) {
-        const uint32_t j = idx[t];
-        acc[j] = __fadd_rn(acc[j], val[t]);
+    if (t >= k) return;
+    const int64_t j = idx_all[(int64_t)row * k + t];
+    const float *a = a_all + (int64_t)row * d;
+    float u;
+    if (HAS_B) {
+        float *b = b_all + (int64_t)row * d;
+        const float bj = b[j];
+        u = __fsub_rn(a[j], bj);
+        if (UPDATE_B) b[j] = __fadd_rn(bj, u);
+    } else {
+        u = a[j];
     }
+    val_all[(int64_t)row * k + t] = u;
 }
 
-// For every coordinate some worker sent: ghat_s += acc / n; acc = 0.  A thread owns one
-// bitmap word of the union of the n selection bitmaps.
-__global__ void __launch_bounds__(kBlock)
-k_server_apply(const uint32_t *__restrict__ bm_all, int n, int64_t wp, float *__restrict__ acc,
-               float *__restrict__ ghat_s, float fn)
+// ------------------------------------------------------------------------------------
+// Sparse server aggregation (Algorithm 1 line 8): ghat_s += (sum_i c_i) / n.
+//
+// A block owns kAggSpan consecutive coordinates and keeps their sums in shared memory.
+// Every payload is sorted by index, so worker i's entries for the block are one contiguous
+// range found by binary search.  Workers are added one after the other (barrier between
+// them), so each coordinate sees the binary32 sum in the order 0, 1, ..., n-1; the indices
+// inside one payload are distinct, so no atomics are needed.  grid = ceil(d / kAggSpan).
+// ------------------------------------------------------------------------------------
+constexpr int kAggSpan = 8192;
+
+__device__ __forceinline__ int64_t lower_bound_u32(const uint32_t *p, int64_t count, uint32_t key)
 {
-    const int64_t w = (int64_t)blockIdx.x * kBlock + threadIdx.x;
-    if (w >= wp) return;
-    uint32_t word = 0;
-    for (int i = 0; i < n; ++i) word |= bm_all[(int64_t)i * wp + w];
-    while (word) {
-        const int bit = __ffs(word) - 1;
-        word &= word - 1;
-        const int64_t j = w * 32 + bit;
-        ghat_s[j] = __fadd_rn(ghat_s[j], __fdiv_rn(acc[j], fn));
-        acc[j] = 0.0f;
+    int64_t lo = 0, hi = count;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (p[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+constexpr int kAggChunk = 64;      // workers whose entry ranges are searched at once
+
+__global__ void __launch_bounds__(kBlock)
+k_topk_aggregate(const uint32_t *__restrict__ idx_all, const float *__restrict__ val_all,
+                 const uint32_t *__restrict__ fin_off_all, int64_t nbt, int n, int64_t k, int64_t d,
+                 float *__restrict__ ghat_s, int n_pow2)
+{
+    __shared__ float acc[kAggSpan];
+    __shared__ int64_t range[kAggChunk][2];
+    const int64_t base = (int64_t)blockIdx.x * kAggSpan;
+    const int64_t end = min(base + (int64_t)kAggSpan, d);
+    const int64_t tile = base / (kTileWords * 32);          // compaction tile of this span
+    for (int t = threadIdx.x; t < kAggSpan; t += kBlock) acc[t] = 0.0f;
+    for (int i0 = 0; i0 < n; i0 += kAggChunk) {
+        const int nc = min(kAggChunk, n - i0);
+        __syncthreads();
+        if (threadIdx.x < 2 * nc) {
+            // entries of worker i inside [base, end): searched only among its entries of the
+            // enclosing compaction tile, whose bounds are the scanned tile counts
+            const int i = i0 + (threadIdx.x >> 1), side = threadIdx.x & 1;
+            const uint32_t *idx = idx_all + (int64_t)i * k;
+            const int64_t t_lo = fin_off_all[(int64_t)i * nbt + tile];
+            const int64_t t_hi = tile + 1 < nbt ? (int64_t)fin_off_all[(int64_t)i * nbt + tile + 1] : k;
+            int64_t pos = t_hi;
+            if (side == 0 || end < (tile + 1) * (int64_t)(kTileWords * 32))
+                pos = t_lo + lower_bound_u32(idx + t_lo, min(t_hi, k) - t_lo, (uint32_t)(side == 0 ? base : end));
+            range[threadIdx.x >> 1][side] = min(pos, k);
+        }
+        __syncthreads();
+        for (int c = 0; c < nc; ++c) {                      // workers in increasing order
+            const uint32_t *idx = idx_all + (int64_t)(i0 + c) * k;
+            const float *val = val_all + (int64_t)(i0 + c) * k;
+            const int64_t lo = range[c][0], hi = range[c][1];
+            for (int64_t t = lo + threadIdx.x; t < hi; t += kBlock) {
+                const int e = (int)(idx[t] - base);
+                acc[e] = __fadd_rn(acc[e], val[t]);
+            }
+            __syncthreads();
+        }
+    }
+    const float fn = (float)n, rn = 1.0f / fn;
+    for (int t = threadIdx.x; t < (int)(end - base); t += kBlock) {
+        const float a = acc[t];
+        if (a != 0.0f)                         // adding an exact zero changes nothing
+            ghat_s[base + t] = __fadd_rn(ghat_s[base + t], n_pow2 ? __fmul_rn(a, rn) : __fdiv_rn(a, fn));
     }
 }
 
@@ -502,8 +545,8 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
     *val = w->val + (int64_t)row * w->k;
 }
 
-constexpr int kSelectLaunches = 11;
-int topk_launches_per_step(int n) { return 2 * kSelectLaunches + n + 1; }
+constexpr int kSelectLaunches = 12;
+int topk_launches_per_step(int) { return 2 * kSelectLaunches + 1; }
 
 template <bool HAS_B>
 static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
@@ -522,10 +565,12 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt);
     k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt);
+    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->idx, w->wp, w->nbt, w->k);
+    const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
-        k_topk_emit<HAS_B, true><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->idx, w->val, w->d, w->wp, w->nbt, w->k);
+        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
     else
-        k_topk_emit<HAS_B, false><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->idx, w->val, w->d, w->wp, w->nbt, w->k);
+        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
 }
 
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
@@ -535,14 +580,10 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
     else select_impl<false>(w, a, nullptr, false, vec_ok, st);
 }
 
-void topk_aggregate(TopkWorkspace *ww, float *ghat_s, float *acc, int n, cudaStream_t st)
+void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st)
 {
-    // one launch per worker, i increasing, so that every coordinate sees the binary32 sum
-    // in the order 0, 1, ..., n-1 (indices inside one payload are distinct: no atomics)
-    const unsigned gk = (unsigned)((ww->k + kBlock - 1) / kBlock);
-    for (int i = 0; i < n; ++i)
-        k_scatter_add<<<gk, kBlock, 0, st>>>(acc, ww->idx + (int64_t)i * ww->k, ww->val + (int64_t)i * ww->k, ww->k);
-    k_server_apply<<<(unsigned)((ww->wp + kBlock - 1) / kBlock), kBlock, 0, st>>>(ww->bm_in, n, ww->wp, acc, ghat_s, (float)n);
+    const unsigned blocks = (unsigned)((ww->d + kAggSpan - 1) / kAggSpan);
+    k_topk_aggregate<<<blocks, kBlock, 0, st>>>(ww->idx, ww->val, ww->cnt_fin, ww->nbt, n, ww->k, ww->d, ghat_s, (n & (n - 1)) == 0);
 }
 
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
