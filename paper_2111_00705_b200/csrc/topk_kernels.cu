@@ -11,6 +11,8 @@
 // atomics: the result does not depend on the order of execution.
 #include "topk.h"
 
+#include <algorithm>
+
 #include "../../include/cdadam.h"
 #include "common.cuh"
 
@@ -20,6 +22,7 @@ constexpr uint32_t kFull = 0xffffffffu;
 constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
 constexpr int kHistStride = kBins1 + kBins2 + kBins3;
 constexpr int kTileWords = 1024;      // bitmap words per block in the sparse passes
+constexpr uint32_t kGuessMargin = 2;  // level-1 buckets kept below the last threshold bucket
 
 struct Sel {                          // outcome of the three levels for one row
     uint32_t b1, k1, c1;              // bucket, entries still to take inside it, its size
@@ -34,6 +37,9 @@ struct TopkWorkspace {
     uint32_t *hist;                   // rows x kHistStride
     Sel *sel;                         // rows
     uint32_t *bm_in, *bm_cand;        // rows x wp
+    uint32_t *bm_ge;                  // rows x wp: coordinates at or above the guessed bucket
+    uint32_t *floor_bucket;           // rows: guessed level-1 bucket for the next selection
+    uint32_t *hit;                    // rows: 1 if the guess held in the current selection
     uint32_t *cnt_tie, *cnt_fin;      // rows x nbt
     uint32_t *idx;                    // rows x k
     float *val;                       // rows x k
@@ -79,40 +85,43 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
-             uint32_t *__restrict__ hist_all, int64_t d, int vec_ok)
+             uint32_t *__restrict__ hist_all, const uint32_t *__restrict__ hit, int64_t d, int vec_ok)
 {
     __shared__ uint32_t h[kBins1];
+    if (hit[blockIdx.y]) return;                      // the guessed bucket held: nothing to redo
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
     __syncthreads();
     const int row = blockIdx.y;
     const float *a = a_all + (int64_t)row * d;
     const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
-    const int64_t base = (int64_t)blockIdx.x * kSub;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (vec_ok && base + kSub <= d) {
-        const int64_t wb = base + warp * kWarpSpan;
-        float4 A[4], Bv[4];
+    // blocks loop over tiles: the grid is small, so rows whose guess held cost almost nothing
+    for (int64_t base = (int64_t)blockIdx.x * kSub; base < d; base += (int64_t)gridDim.x * kSub) {
+        if (vec_ok && base + kSub <= d) {
+            const int64_t wb = base + warp * kWarpSpan;
+            float4 A[4], Bv[4];
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const int64_t j = wb + v * 128 + lane * 4;
-            A[v] = ld_ro4(a + j);
-            if (HAS_B) Bv[v] = ld_ro4(b + j);
-        }
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            if (HAS_B) {
-                A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
-                A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
+            for (int v = 0; v < 4; ++v) {
+                const int64_t j = wb + v * 128 + lane * 4;
+                A[v] = ld_ro4(a + j);
+                if (HAS_B) Bv[v] = ld_ro4(b + j);
             }
-            atomicAdd(&h[key_of(A[v].x) >> 20], 1u);
-            atomicAdd(&h[key_of(A[v].y) >> 20], 1u);
-            atomicAdd(&h[key_of(A[v].z) >> 20], 1u);
-            atomicAdd(&h[key_of(A[v].w) >> 20], 1u);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                if (HAS_B) {
+                    A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
+                    A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
+                }
+                atomicAdd(&h[key_of(A[v].x) >> 20], 1u);
+                atomicAdd(&h[key_of(A[v].y) >> 20], 1u);
+                atomicAdd(&h[key_of(A[v].z) >> 20], 1u);
+                atomicAdd(&h[key_of(A[v].w) >> 20], 1u);
+            }
+        } else {
+            const int64_t end = min(base + (int64_t)kSub, d);
+            for (int64_t j = base + threadIdx.x; j < end; j += kBlock)
+                atomicAdd(&h[key_of(diff1<HAS_B>(a, b, j)) >> 20], 1u);
         }
-    } else {
-        const int64_t end = min(base + (int64_t)kSub, d);
-        for (int64_t j = base + threadIdx.x; j < end; j += kBlock)
-            atomicAdd(&h[key_of(diff1<HAS_B>(a, b, j)) >> 20], 1u);
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
@@ -127,10 +136,11 @@ k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
 k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, int level,
-            uint32_t k)
+            uint32_t k, const uint32_t *__restrict__ hit, uint32_t *__restrict__ floor_bucket)
 {
     __shared__ uint32_t tot[kBlock];
     const int row = blockIdx.x;
+    if (level == 0 && hit[row]) return;               // level 1 was settled by the guess
     Sel *sel = sel_all + row;
     const int nb = level == 2 ? kBins3 : kBins1;
     const uint32_t *hist = hist_all + (int64_t)row * kHistStride +
@@ -150,7 +160,11 @@ k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, in
             const uint32_t bucket = lo + t, rem = want - above;
             if (level == 0) { sel->b1 = bucket; sel->k1 = rem; sel->c1 = c; }
             else if (level == 1) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
-            else { sel->b3 = bucket; sel->k3 = rem; sel->c3 = c; }
+            else {
+                sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
+                // guess for the next selection of this row: a little below this threshold
+                floor_bucket[row] = sel->b1 > kGuessMargin ? sel->b1 - kGuessMargin : 1u;
+            }
         }
         above += c;
     }
@@ -165,10 +179,11 @@ template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
-            uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
-            int64_t wp, int vec_ok)
+            uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all,
+            const uint32_t *__restrict__ hit, int64_t d, int64_t wp, int vec_ok)
 {
     __shared__ uint32_t h[kBins2];
+    if (hit[blockIdx.y]) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
     const int row = blockIdx.y;
@@ -176,6 +191,85 @@ k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t b1 = sel_all[row].b1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    // blocks loop over tiles: the grid is small, so rows whose guess held cost almost nothing
+    for (int64_t base = (int64_t)blockIdx.x * kSub; base < d; base += (int64_t)gridDim.x * kSub) {
+        if (vec_ok && base + kSub <= d) {
+            const int64_t wb = base + warp * kWarpSpan;
+            float4 A[4], Bv[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int64_t j = wb + v * 128 + lane * 4;
+                A[v] = ld_ro4(a + j);
+                if (HAS_B) Bv[v] = ld_ro4(b + j);
+            }
+            uint32_t BI[4][4], BC[4][4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                if (HAS_B) {
+                    A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
+                    A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
+                }
+                const uint32_t kx = key_of(A[v].x), ky = key_of(A[v].y);
+                const uint32_t kz = key_of(A[v].z), kw = key_of(A[v].w);
+                BI[v][0] = __ballot_sync(kFull, (kx >> 20) > b1);
+                BI[v][1] = __ballot_sync(kFull, (ky >> 20) > b1);
+                BI[v][2] = __ballot_sync(kFull, (kz >> 20) > b1);
+                BI[v][3] = __ballot_sync(kFull, (kw >> 20) > b1);
+                const bool cx = (kx >> 20) == b1, cy = (ky >> 20) == b1;
+                const bool cz = (kz >> 20) == b1, cw = (kw >> 20) == b1;
+                BC[v][0] = __ballot_sync(kFull, cx);
+                BC[v][1] = __ballot_sync(kFull, cy);
+                BC[v][2] = __ballot_sync(kFull, cz);
+                BC[v][3] = __ballot_sync(kFull, cw);
+                if (cx) atomicAdd(&h[(kx >> 9) & (kBins2 - 1)], 1u);
+                if (cy) atomicAdd(&h[(ky >> 9) & (kBins2 - 1)], 1u);
+                if (cz) atomicAdd(&h[(kz >> 9) & (kBins2 - 1)], 1u);
+                if (cw) atomicAdd(&h[(kw >> 9) & (kBins2 - 1)], 1u);
+            }
+            const uint32_t wi = warp_words(BI, lane), wc = warp_words(BC, lane);
+            if (lane < 16) { bm_in[(wb >> 5) + lane] = wi; bm_cand[(wb >> 5) + lane] = wc; }
+        } else {
+            const int64_t end = min(base + (int64_t)kSub, d);
+            for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+                const bool valid = j < end;
+                const uint32_t key = valid ? key_of(diff1<HAS_B>(a, b, j)) : 0u;
+                const bool in = valid && (key >> 20) > b1, cand = valid && (key >> 20) == b1;
+                const uint32_t wi = __ballot_sync(kFull, in), wc = __ballot_sync(kFull, cand);
+                if (lane == 0) { bm_in[j >> 5] = wi; bm_cand[j >> 5] = wc; }
+                if (cand) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
+    for (int t = threadIdx.x; t < kBins2; t += kBlock)
+        if (h[t]) atomicAdd(&hist[t], h[t]);
+}
+
+// ------------------------------------------------------------------------------------
+// Speculative single dense pass.  The threshold moves little from one iteration to the
+// next, so the level-1 bucket of the previous selection, lowered by a margin, is taken as a
+// floor: this pass histograms only the coordinates at or above the floor (a few percent, so
+// few shared-memory atomics) and records them in a bitmap.  If at least k coordinates lie
+// at or above the floor, the threshold bucket is found from this histogram and the second
+// dense pass is not needed; otherwise the two classic passes run.  grid = (ceil(d/4096), rows).
+// ------------------------------------------------------------------------------------
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
+            const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ bm_ge_all,
+            uint32_t *__restrict__ hist_all, int64_t d, int64_t wp, int vec_ok)
+{
+    __shared__ uint32_t h[kBins1];
+    const int row = blockIdx.y;
+    const uint32_t fl = floor_bucket[row];
+    if (fl >= (uint32_t)kBins1) return;               // no guess for this row
+    for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
+    __syncthreads();
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    uint32_t *bm_ge = bm_ge_all + (int64_t)row * wp;
     const int64_t base = (int64_t)blockIdx.x * kSub;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (vec_ok && base + kSub <= d) {
@@ -187,42 +281,113 @@ k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
             A[v] = ld_ro4(a + j);
             if (HAS_B) Bv[v] = ld_ro4(b + j);
         }
-        uint32_t BI[4][4], BC[4][4];
+        uint32_t BG[4][4];
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             if (HAS_B) {
                 A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
                 A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
             }
-            const uint32_t kx = key_of(A[v].x), ky = key_of(A[v].y);
-            const uint32_t kz = key_of(A[v].z), kw = key_of(A[v].w);
-            BI[v][0] = __ballot_sync(kFull, (kx >> 20) > b1);
-            BI[v][1] = __ballot_sync(kFull, (ky >> 20) > b1);
-            BI[v][2] = __ballot_sync(kFull, (kz >> 20) > b1);
-            BI[v][3] = __ballot_sync(kFull, (kw >> 20) > b1);
-            const bool cx = (kx >> 20) == b1, cy = (ky >> 20) == b1;
-            const bool cz = (kz >> 20) == b1, cw = (kw >> 20) == b1;
-            BC[v][0] = __ballot_sync(kFull, cx);
-            BC[v][1] = __ballot_sync(kFull, cy);
-            BC[v][2] = __ballot_sync(kFull, cz);
-            BC[v][3] = __ballot_sync(kFull, cw);
-            if (cx) atomicAdd(&h[(kx >> 9) & (kBins2 - 1)], 1u);
-            if (cy) atomicAdd(&h[(ky >> 9) & (kBins2 - 1)], 1u);
-            if (cz) atomicAdd(&h[(kz >> 9) & (kBins2 - 1)], 1u);
-            if (cw) atomicAdd(&h[(kw >> 9) & (kBins2 - 1)], 1u);
+            const uint32_t hx = key_of(A[v].x) >> 20, hy = key_of(A[v].y) >> 20;
+            const uint32_t hz = key_of(A[v].z) >> 20, hw = key_of(A[v].w) >> 20;
+            BG[v][0] = __ballot_sync(kFull, hx >= fl);
+            BG[v][1] = __ballot_sync(kFull, hy >= fl);
+            BG[v][2] = __ballot_sync(kFull, hz >= fl);
+            BG[v][3] = __ballot_sync(kFull, hw >= fl);
+            if (hx >= fl) atomicAdd(&h[hx], 1u);
+            if (hy >= fl) atomicAdd(&h[hy], 1u);
+            if (hz >= fl) atomicAdd(&h[hz], 1u);
+            if (hw >= fl) atomicAdd(&h[hw], 1u);
         }
-        const uint32_t wi = warp_words(BI, lane), wc = warp_words(BC, lane);
-        if (lane < 16) { bm_in[(wb >> 5) + lane] = wi; bm_cand[(wb >> 5) + lane] = wc; }
+        const uint32_t wg = warp_words(BG, lane);
+        if (lane < 16) bm_ge[(wb >> 5) + lane] = wg;
     } else {
         const int64_t end = min(base + (int64_t)kSub, d);
         for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
             const bool valid = j < end;
-            const uint32_t key = valid ? key_of(diff1<HAS_B>(a, b, j)) : 0u;
-            const bool in = valid && (key >> 20) > b1, cand = valid && (key >> 20) == b1;
-            const uint32_t wi = __ballot_sync(kFull, in), wc = __ballot_sync(kFull, cand);
-            if (lane == 0) { bm_in[j >> 5] = wi; bm_cand[j >> 5] = wc; }
-            if (cand) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
+            const uint32_t hi = valid ? key_of(diff1<HAS_B>(a, b, j)) >> 20 : 0u;
+            const bool ge = valid && hi >= fl;
+            const uint32_t wg = __ballot_sync(kFull, ge);
+            if (lane == 0) bm_ge[j >> 5] = wg;
+            if (ge) atomicAdd(&h[hi], 1u);
         }
+    }
+    __syncthreads();
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride;
+    for (int t = threadIdx.x; t < kBins1; t += kBlock)
+        if (h[t]) atomicAdd(&hist[t], h[t]);
+}
+
+// Did the guess hold?  It did if at least k coordinates lie at or above the floor; then the
+// level-1 bucket follows from the histogram of those coordinates.  Otherwise the row's
+// level-1 histogram is cleared for the full pass.  grid = (rows), one block.
+__global__ void __launch_bounds__(kBlock)
+k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
+                 const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hit)
+{
+    __shared__ uint32_t tot[kBlock];
+    __shared__ uint32_t found;
+    const int row = blockIdx.x;
+    Sel *sel = sel_all + row;
+    uint32_t *hist = hist_all + (int64_t)row * kHistStride;
+    const uint32_t fl = floor_bucket[row];
+    if (threadIdx.x == 0) found = 0u;
+    const int per = kBins1 / kBlock, lo = threadIdx.x * per;
+    uint32_t mine = 0;
+    if (fl < (uint32_t)kBins1)
+        for (int t = 0; t < per; ++t) mine += hist[lo + t];
+    tot[threadIdx.x] = mine;
+    __syncthreads();
+    uint32_t above = 0;
+    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+    if (fl < (uint32_t)kBins1) {
+        for (int t = per - 1; t >= 0; --t) {
+            const uint32_t c = hist[lo + t];
+            if (above < k && above + c >= k) {
+                sel->b1 = lo + t; sel->k1 = k - above; sel->c1 = c;
+                found = 1u;
+            }
+            above += c;
+        }
+    }
+    __syncthreads();
+    const uint32_t ok = found;
+    if (threadIdx.x == 0) hit[row] = ok;
+    if (!ok)
+        for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
+}
+
+// After a successful guess: from the bitmap of coordinates at or above the floor, rebuild
+// what the second dense pass would have produced: bm_in (bucket above the threshold
+// bucket), bm_cand (inside it) and the level-2 histogram of the candidates.
+// grid = (nbt, rows); a thread walks the set bits of its bitmap words.
+template <bool HAS_B>
+__global__ void __launch_bounds__(kBlock)
+k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
+             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+             const uint32_t *__restrict__ bm_ge_all, uint32_t *__restrict__ bm_in_all,
+             uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d, int64_t wp)
+{
+    __shared__ uint32_t h[kBins2];
+    const int row = blockIdx.y;
+    if (!hit[row]) return;
+    for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
+    __syncthreads();
+    const float *a = a_all + (int64_t)row * d;
+    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const uint32_t b1 = sel_all[row].b1;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+        uint32_t word = bm_ge_all[(int64_t)row * wp + w0 + t], in = 0, cand = 0;
+        while (word) {
+            const int bit = __ffs(word) - 1;
+            word &= word - 1;
+            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+            if ((key >> 20) > b1) in |= 1u << bit;
+            else if ((key >> 20) == b1) { cand |= 1u << bit; atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u); }
+        }
+        bm_in_all[(int64_t)row * wp + w0 + t] = in;
+        bm_cand_all[(int64_t)row * wp + w0 + t] = cand;
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
@@ -503,6 +668,7 @@ static void free_ws(TopkWorkspace *w)
 {
     cudaFree(w->hist); cudaFree(w->sel); cudaFree(w->bm_in); cudaFree(w->bm_cand);
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
+    cudaFree(w->bm_ge); cudaFree(w->floor_bucket); cudaFree(w->hit);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
 }
@@ -526,6 +692,10 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
     get((void **)&w->sel, (size_t)rows * sizeof(Sel));
     get((void **)&w->bm_in, (size_t)rows * w->wp * 4);
     get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
+    get((void **)&w->bm_ge, (size_t)rows * w->wp * 4);
+    get((void **)&w->floor_bucket, (size_t)rows * 4);
+    get((void **)&w->hit, (size_t)rows * 4);
+    if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
     get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
     get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
     if (w->own_payload) {
@@ -545,7 +715,7 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
     *val = w->val + (int64_t)row * w->k;
 }
 
-constexpr int kSelectLaunches = 12;
+constexpr int kSelectLaunches = 15;
 int topk_launches_per_step(int) { return 2 * kSelectLaunches + 1; }
 
 template <bool HAS_B>
@@ -555,12 +725,18 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
     const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
     cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
-    k_topk_hist1<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->hist, w->d, vec_ok);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k);
-    k_topk_mark<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->d, w->wp, vec_ok);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0);
+    // one dense pass with the guessed floor; the two classic passes (small looping grids)
+    // do work only for rows whose guess failed
+    const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
+    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->bm_ge, w->hist, w->d, w->wp, vec_ok);
+    k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
+    k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
+    k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok);
+    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->bm_in, w->bm_cand, w->hist, w->d, w->wp);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
     k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_cand, w->hist, w->d, w->wp);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0);
+    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
     k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt);
     k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);

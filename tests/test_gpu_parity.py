@@ -206,6 +206,21 @@ def test_topk_shapes(d, k):
     run_free(w, 3)
 
 
+def test_topk_threshold_guess_hits_and_misses():
+    """The selection reuses the previous threshold bucket as a guess.  Gradients whose scale
+    stays, grows (guess holds) and collapses by 20x (guess fails, classic two passes) must
+    all give the oracle's payloads."""
+    rng = np.random.default_rng(3)
+    d, n, k = 150000, 3, 1500
+    w = synth.Workload("GUESS", d, n, synth.TOPK, 8, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d))
+    for scale in (1.0, 1.0, 0.9, 0.05, 0.05, 3.0, 3.0, 1e-30, 1e-30, 0.0, 1.0):
+        grads = (rng.standard_normal((n, d)) * scale).astype(np.float32)
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+
+
 def test_topk_ties_lower_index_wins():
     """Few distinct magnitudes: most of the selection is decided by the tie rule."""
     rng = np.random.default_rng(0)
