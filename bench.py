@@ -197,6 +197,8 @@ def main():
     ap.add_argument("--impl", default="cdadam", choices=["cdadam", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="markov", choices=["markov", "ef"],
+                    help="markov = Algorithm 1 (default); ef = classical error feedback (Section 4)")
     ap.add_argument("--tile", type=int, default=0,
                     help="force the kernels' tile size (profiler captures of scaled-down cases)")
     ap.add_argument("--scale", type=float, default=1.0,
@@ -232,7 +234,8 @@ def main():
     if args.warmup < 3:
         args.warmup = 3
     opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
-                    beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev)
+                    beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev,
+                    mode=cd.EF if args.mode == "ef" else cd.MARKOV)
     if args.tile:
         opt.set_tile(args.tile)
     # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
@@ -340,7 +343,8 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale),
+                "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale)
+                           + ("" if args.mode == "markov" else " [error-feedback mode]"),
                            "replicas": world,
                            "l2": "flushed between steps" if flush is not None else
                                  "inputs larger than L2 (%.2f GB of gradients per step)" % (w.n * w.d * 4 / 1e9)},

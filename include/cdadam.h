@@ -46,6 +46,12 @@ typedef struct cdadam_ctx cdadam_ctx;
 /* compressor C of Algorithm 1 (Appendix A) */
 enum { CDADAM_SIGN = 0, CDADAM_TOPK = 1, CDADAM_IDENTITY = 2 };
 
+/* recursion around the compressor */
+enum {
+    CDADAM_MARKOV = 0,   /* Algorithm 1: Markov compression sequences (Section 5), the default */
+    CDADAM_EF = 1        /* classical error feedback at workers and server (Section 4) */
+};
+
 /* status codes */
 enum {
     CDADAM_OK = 0,
@@ -124,6 +130,16 @@ int cdadam_set_params(cdadam_ctx *ctx, const float *x0, void *stream);
  * for CDADAM_SIGN.  Synchronous (re-allocates tables).
  */
 int cdadam_set_segments(cdadam_ctx *ctx, int q, const int64_t *offsets);
+
+/*
+ * Choose the recursion: CDADAM_MARKOV (Algorithm 1, default) or CDADAM_EF, the error-feedback
+ * scheme the paper compares against (Section 4), applied both ways:
+ *   worker: p = g + delta^(i), c^(i) = C(p), delta^(i) = p - c^(i);
+ *   server: p = (1/n) sum_i c^(i) + delta, c = C(p), delta = p - c; AMSGrad runs on c.
+ * In this mode the state named GHAT_W holds the worker errors delta^(i), GTIL the server
+ * error delta, and GHAT_S is scratch.  Only before the first step.
+ */
+int cdadam_set_mode(cdadam_ctx *ctx, int mode);
 
 /*
  * Tuning knob: the number of consecutive coordinates one thread block of the scaled-sign

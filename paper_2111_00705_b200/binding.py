@@ -10,6 +10,7 @@ import os
 import torch
 
 SIGN, TOPK, IDENTITY = 0, 1, 2
+MARKOV, EF = 0, 1
 SERVER = -1
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
 OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
@@ -27,6 +28,7 @@ _SIGNATURES = {
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
+    "cdadam_set_mode": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_tile": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
     "cdadam_get_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
@@ -116,17 +118,20 @@ class CDAdam:
     """One context of the library: n simulated workers and the server on one GPU."""
 
     def __init__(self, d, n, compressor=SIGN, k=0, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
-                 offsets=None, x0=None, device=None):
+                 offsets=None, x0=None, device=None, mode=MARKOV):
         self._h = None
         self.device = torch.device("cuda", torch.cuda.current_device()) if device is None \
             else torch.device(device)
         self.d, self.n, self.compressor, self.k = int(d), int(n), int(compressor), int(k)
         self.q = 1
+        self.mode = int(mode)
         with torch.cuda.device(self.device):
             self._h = lib().cdadam_create(self.d, self.n, self.compressor, self.k,
                                           beta1, beta2, lr, eps)
         if not self._h:
             raise CdadamError(ERR_ARG, last_error())
+        if mode != MARKOV:
+            _check(lib().cdadam_set_mode(self._h, int(mode)))
         if offsets is not None:
             self.set_segments(offsets)
         if x0 is not None:

@@ -123,6 +123,7 @@ struct cdadam_ctx {
     int64_t d = 0, k = 0, wp = 0, steps = 0;
     int n = 0, comp = 0, device = 0;
     int tile_override = 0;  // 0 = choose from d and q
+    int mode = CDADAM_MARKOV;
     Hyper hp{};
     TableSet ts;
     float *ghat_w = nullptr, *ghat_s = nullptr, *gtil = nullptr;
@@ -282,34 +283,57 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
     cudaStream_t st = (cudaStream_t)stream;
     const bool vec = aligned16(grads) && c->d % 4 == 0;
     prof_mark(c, st);
+    const bool ef = c->mode == CDADAM_EF;
+    const bool svec = c->d % 4 == 0;
     if (c->comp == CDADAM_SIGN) {
         const Tables &tb = c->ts.tb;
-        const bool svec = c->d % 4 == 0;
         const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
         float *new_scale = c->wscale[c->cur ^ 1];
-        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, c->error_flag, st);
+        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef, c->error_flag, st);
         prof_mark(c, st);
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
         prof_mark(c, st);
-        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, svec, st);
+        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, svec, ef, st);
         prof_mark(c, st);
         launch_finalize_scales(c->spart, c->sscale, tb, 1, st);
         prof_mark(c, st);
-        launch_update_sign(c->sbits, c->sscale, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, svec, st);
+        launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, svec, ef, st);
         prof_mark(c, st);
         c->cur ^= 1;
         c->pending = true;
-    } else if (c->comp == CDADAM_TOPK) {
+    } else if (c->comp == CDADAM_TOPK && !ef) {
         topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
         prof_mark(c, st);
-        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);              // line 8
+        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
         prof_mark(c, st);
-        topk_select(c->tk_s, c->ghat_s, c->gtil, true, c->d % 4 == 0, st); // lines 9-10, 12
+        topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // lines 9-10, 12
         prof_mark(c, st);
-        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, c->d % 4 == 0, st);
+        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+        prof_mark(c, st);
+    } else if (c->comp == CDADAM_TOPK) {
+        // classical error feedback: the delta buffers (ghat_w rows, gtil) first receive the
+        // compressor inputs p = g + delta and p = mean + delta, are compressed in place, and
+        // keep p - c, which is p outside the kept coordinates and 0 on them.  ghat_s is all
+        // zero between steps and carries the dense decoded server payload for AMSGrad.
+        const uint32_t *widx, *sidx;
+        const float *wval, *sval;
+        topk_payload(c->tk_w, 0, &widx, &wval);
+        topk_payload(c->tk_s, 0, &sidx, &sval);
+        launch_add_into(c->ghat_w, grads, (int64_t)c->n * c->d, vec, st);
+        topk_select(c->tk_w, c->ghat_w, nullptr, false, svec, st);
+        launch_scatter_set(c->ghat_w, widx, nullptr, c->k, c->d, c->n, st);
+        prof_mark(c, st);
+        topk_aggregate(c->tk_w, c->gtil, c->n, st);
+        prof_mark(c, st);
+        topk_select(c->tk_s, c->gtil, nullptr, false, svec, st);
+        launch_scatter_set(c->gtil, sidx, nullptr, c->k, c->d, 1, st);
+        launch_scatter_set(c->ghat_s, sidx, sval, c->k, c->d, 1, st);
+        prof_mark(c, st);
+        launch_amsgrad(c->ghat_s, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+        launch_scatter_set(c->ghat_s, sidx, nullptr, c->k, c->d, 1, st);
         prof_mark(c, st);
     } else {
-        launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, st);
+        launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, ef, st);
         prof_mark(c, st);
     }
     int rc = check_launch("cdadam_step");
@@ -372,6 +396,15 @@ int cdadam_set_tile(cdadam_ctx *c, int tile)
     return cdadam_set_segments(c, (int)off.size() - 1, off.data());
 }
 
+int cdadam_set_mode(cdadam_ctx *c, int mode)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_mode: NULL context");
+    if (mode != CDADAM_MARKOV && mode != CDADAM_EF) return fail(CDADAM_ERR_ARG, "unknown mode %d", mode);
+    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the mode must be set before the first step");
+    c->mode = mode;
+    return CDADAM_OK;
+}
+
 int cdadam_set_lr(cdadam_ctx *c, float lr)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_lr: NULL context");
@@ -387,7 +420,7 @@ int cdadam_get_state(cdadam_ctx *c, int name, float *dst, void *stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (name == CDADAM_STATE_GHAT_W && c->comp == CDADAM_SIGN && c->pending) {
-        launch_apply_sign(c->ghat_w, c->wbits, c->wscale[c->cur], c->ts.tb, c->n, c->wp, st);
+        launch_apply_sign(c->ghat_w, c->wbits, c->wscale[c->cur], c->ts.tb, c->n, c->wp, c->mode == CDADAM_EF, st);
         int rc = check_launch("apply deferred payload");
         if (rc) return rc;
         c->pending = false;
@@ -446,7 +479,7 @@ int cdadam_launches_per_step(cdadam_ctx *c)
 {
     if (!c) return 0;
     if (c->comp == CDADAM_SIGN) return 5;
-    if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1;
+    if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : 0);
     return 1;
 }
 

@@ -6,6 +6,8 @@
 namespace cdadam {
 
 // C(u) = u: every line of Algorithm 1 for one coordinate, workers in increasing order.
+// EF: the same with classical error feedback, whose error terms stay exactly zero.
+template <bool EF>
 __global__ void __launch_bounds__(kBlock)
 k_step_identity(const float *__restrict__ grads, float *__restrict__ ghat_w,
                 float *__restrict__ ghat_s, float *__restrict__ gtil, float *__restrict__ m,
@@ -19,15 +21,21 @@ k_step_identity(const float *__restrict__ grads, float *__restrict__ ghat_w,
         for (int i = 0; i < n; ++i) {
             const int64_t p = (int64_t)i * d + j;
             const float gh = ghat_w[p];
-            const float u = __fsub_rn(grads[p], gh);      // c^(i) = u
-            ghat_w[p] = __fadd_rn(gh, u);
+            const float u = EF ? __fadd_rn(grads[p], gh) : __fsub_rn(grads[p], gh);   // c^(i) = u
+            ghat_w[p] = EF ? __fsub_rn(u, u) : __fadd_rn(gh, u);
             a = __fadd_rn(a, u);
         }
-        const float hs = __fadd_rn(ghat_s[j], __fdiv_rn(a, fn));
-        ghat_s[j] = hs;
-        const float gt0 = gtil[j];
-        const float gt = __fadd_rn(gt0, __fsub_rn(hs, gt0));   // c = w
-        gtil[j] = gt;
+        float gt;
+        if (EF) {
+            gt = __fadd_rn(__fdiv_rn(a, fn), gtil[j]);         // c = p, the error p - c is zero
+            gtil[j] = __fsub_rn(gt, gt);
+        } else {
+            const float hs = __fadd_rn(ghat_s[j], __fdiv_rn(a, fn));
+            ghat_s[j] = hs;
+            const float gt0 = gtil[j];
+            gt = __fadd_rn(gt0, __fsub_rn(hs, gt0));           // c = w
+            gtil[j] = gt;
+        }
         float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
         amsgrad1(gt, mm, vv, vh, xx, hp);
         m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
@@ -67,10 +75,48 @@ static unsigned grid_for(int64_t items)
 
 void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
                           float *m, float *v, float *vhat, float *x, int64_t d, int n,
-                          Hyper hp, cudaStream_t st)
+                          Hyper hp, bool ef, cudaStream_t st)
 {
-    k_step_identity<<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x,
-                                                    d, n, hp);
+    if (ef) k_step_identity<true><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
+    else k_step_identity<false><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
+}
+
+// dst = src + dst
+__global__ void __launch_bounds__(kBlock)
+k_add_into(float *__restrict__ dst, const float *__restrict__ src, int64_t count, int vec_ok)
+{
+    const int64_t nvec = vec_ok ? count / 4 : 0;
+    const int64_t stride = (int64_t)gridDim.x * kBlock;
+    const int64_t t0 = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    for (int64_t q = t0; q < nvec; q += stride) {
+        const float4 a = ld_ro4(src + q * 4);
+        float4 b = ld_rw4(dst + q * 4);
+        b.x = __fadd_rn(a.x, b.x); b.y = __fadd_rn(a.y, b.y);
+        b.z = __fadd_rn(a.z, b.z); b.w = __fadd_rn(a.w, b.w);
+        st_rw4(dst + q * 4, b);
+    }
+    for (int64_t j = nvec * 4 + t0; j < count; j += stride) dst[j] = __fadd_rn(src[j], dst[j]);
+}
+
+void launch_add_into(float *dst, const float *src, int64_t count, bool vec_ok, cudaStream_t st)
+{
+    k_add_into<<<grid_for(vec_ok ? count / 4 : count), kBlock, 0, st>>>(dst, src, count, vec_ok);
+}
+
+__global__ void __launch_bounds__(kBlock)
+k_scatter_set(float *__restrict__ dst, const uint32_t *__restrict__ idx, const float *__restrict__ val,
+              int64_t k, int64_t d)
+{
+    const int row = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t < k) dst[(int64_t)row * d + idx[(int64_t)row * k + t]] = val ? val[(int64_t)row * k + t] : 0.0f;
+}
+
+void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d,
+                        int rows, cudaStream_t st)
+{
+    dim3 grid((unsigned)((k + kBlock - 1) / kBlock), (unsigned)rows);
+    k_scatter_set<<<grid, kBlock, 0, st>>>(dst, idx, val, k, d);
 }
 
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,

@@ -13,7 +13,7 @@ namespace cdadam {
 // a copy ran out.
 void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, int *error_flag, cudaStream_t st);
+                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st);
 // Correctly rounded scale of every (row, segment) from the partial sums.
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
                             cudaStream_t st);
@@ -21,14 +21,14 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 // sign(w) into sbits and writes partial sums of |w| to spart.
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, cudaStream_t st);
+                        int n, int64_t wp, bool vec_ok, bool ef, cudaStream_t st);
 // Server pass B and worker update (lines 10, 12-16): gtil += decode(c); AMSGrad.
-void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil, float *m,
-                        float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
-                        bool vec_ok, cudaStream_t st);
+void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
+                        float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
+                        bool vec_ok, bool ef, cudaStream_t st);
 // ghat_w += decode(bits, scales) for all workers (applies a deferred payload).
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
-                       const Tables &tb, int n, int64_t wp, cudaStream_t st);
+                       const Tables &tb, int n, int64_t wp, bool ef, cudaStream_t st);
 // Stand-alone scaled-sign compressor of one vector: bits and partial sums of |x|.
 void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
                       bool vec_ok, cudaStream_t st);
@@ -37,9 +37,16 @@ void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb
 // The whole iteration with C(u) = u, one fused pass.
 void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
                           float *m, float *v, float *vhat, float *x, int64_t d, int n,
-                          Hyper hp, cudaStream_t st);
+                          Hyper hp, bool ef, cudaStream_t st);
 
-// ---- AMSGrad alone (top-k path: gtil already updated) ---------------------------------
+// ---- pieces of the error-feedback iteration with the top-k compressor ---------------------
+// dst[j] = src[j] + dst[j] for count floats (p = g + delta, kept in the delta buffer).
+void launch_add_into(float *dst, const float *src, int64_t count, bool vec_ok, cudaStream_t st);
+// dst[idx[t]] = val ? val[t] : 0 for t < k, for `rows` rows (dst stride d, idx/val stride k).
+void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d,
+                        int rows, cudaStream_t st);
+
+// ---- AMSGrad alone on a dense gradient estimate (top-k path) ------------------------------
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
                     Hyper hp, bool vec_ok, cudaStream_t st);
 

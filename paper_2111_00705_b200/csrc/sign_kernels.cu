@@ -14,9 +14,64 @@ constexpr uint32_t kFull = 0xffffffffu;
 
 __device__ __forceinline__ float signed_scale(uint32_t bit, float s) { return bit ? s : -s; }
 
+// ------------------------------------------------------------------------------------
+// The two recursions a kernel can run (template parameter EF).
+//   EF = false, Algorithm 1 (Markov compression sequence): the worker buffer holds ghat^(i);
+//     ghat += c_prev, u = g - ghat; the server keeps ghat and gtil: ghat += mean,
+//     w = ghat - gtil, then gtil += c and AMSGrad runs on gtil.
+//   EF = true, classical error feedback (Section 4): the worker buffer holds the last
+//     compressor input p_prev = g_prev + delta_prev; delta = p_prev - c_prev, u = p = g + delta;
+//     the server keeps its error delta in the gtil buffer and its compressor input
+//     p = mean + delta in the ghat buffer; then delta = p - c and AMSGrad runs on c.
+// `stored` is what the buffer holds, `store` what is written back; the value returned is
+// the compressor input.
+// ------------------------------------------------------------------------------------
+template <bool EF>
+__device__ __forceinline__ float worker_step(float g, float stored, float c_prev, float &store)
+{
+    if (EF) {
+        store = __fadd_rn(g, __fsub_rn(stored, c_prev));
+        return store;
+    }
+    store = __fadd_rn(stored, c_prev);
+    return __fsub_rn(g, store);
+}
+template <bool EF>
+__device__ __forceinline__ float worker_input_from_memory(float g, float stored)
+{
+    return EF ? stored : __fsub_rn(g, stored);
+}
+template <bool EF>
+__device__ __forceinline__ float server_step(float mean, float ghat_stored, float gt, float &store)
+{
+    if (EF) {
+        store = __fadd_rn(mean, gt);
+        return store;
+    }
+    store = __fadd_rn(ghat_stored, mean);
+    return __fsub_rn(store, gt);
+}
+template <bool EF>
+__device__ __forceinline__ float server_input_from_memory(float ghat_stored, float gt)
+{
+    return EF ? ghat_stored : __fsub_rn(ghat_stored, gt);
+}
+// Returns the gradient estimate AMSGrad uses; gt_store is the new content of the gtil buffer.
+template <bool EF>
+__device__ __forceinline__ float update_step(float gt_stored, float p, float c, float &gt_store)
+{
+    if (EF) {
+        gt_store = __fsub_rn(p, c);
+        return c;
+    }
+    gt_store = __fadd_rn(gt_stored, c);
+    return gt_store;
+}
+
 // Scalar path of the worker pass for one tile (segment boundaries, the ragged last tile,
 // unaligned rows).  Kept out of line so that it does not shape the register allocation and
 // instruction schedule of the vector path.
+template <bool EF>
 __device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, float *__restrict__ gh,
                                                 uint32_t *__restrict__ bw, const float *__restrict__ so,
                                                 dd *__restrict__ part, const int64_t *__restrict__ off,
@@ -47,9 +102,9 @@ __device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, flo
                 const bool valid = j < end;
                 float u = -1.0f;
                 if (valid) {
-                    const float hn = __fadd_rn(hv[t], signed_scale((wv[t] >> (j & 31)) & 1u, sv[t]));
+                    float hn;
+                    u = worker_step<EF>(gv[t], hv[t], signed_scale((wv[t] >> (j & 31)) & 1u, sv[t]), hn);
                     gh[j] = hn;
-                    u = __fsub_rn(gv[t], hn);
                 }
                 const uint32_t word = __ballot_sync(kFull, valid && u >= 0.0f);
                 if (lane == 0) bw[j >> 5] = word;
@@ -61,7 +116,7 @@ __device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, flo
         const int64_t lo = max(off[r], base), hi = min(off[r + 1], end);
         dd acc = {0.0, 0.0};
         for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
-            dd_acc(acc, fabsf(__fsub_rn(g[j], gh[j])));
+            dd_acc(acc, fabsf(worker_input_from_memory<EF>(g[j], gh[j])));
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
@@ -90,6 +145,7 @@ __device__ __forceinline__ void worker_load(WorkerRegs &r, const float *__restri
     }
 }
 
+template <bool EF>
 __device__ __forceinline__ void worker_compute(WorkerRegs &r, float *__restrict__ gh,
                                                uint32_t *__restrict__ bw, int64_t wb, int lane,
                                                float s, dd &acc)
@@ -98,15 +154,13 @@ __device__ __forceinline__ void worker_compute(WorkerRegs &r, float *__restrict_
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
         const uint32_t nib = r.ow[v] >> ((lane & 7) * 4);
-        float4 H = r.H[v];
-        // ghat_{t-1} = ghat_{t-2} + c_{t-1}: the previous payload, applied now
-        H.x = __fadd_rn(H.x, signed_scale(nib & 1u, s));
-        H.y = __fadd_rn(H.y, signed_scale(nib & 2u, s));
-        H.z = __fadd_rn(H.z, signed_scale(nib & 4u, s));
-        H.w = __fadd_rn(H.w, signed_scale(nib & 8u, s));
+        // the previous payload (sign words + scale) is applied now, then the new input formed
+        float4 H;
+        const float ux = worker_step<EF>(r.G[v].x, r.H[v].x, signed_scale(nib & 1u, s), H.x);
+        const float uy = worker_step<EF>(r.G[v].y, r.H[v].y, signed_scale(nib & 2u, s), H.y);
+        const float uz = worker_step<EF>(r.G[v].z, r.H[v].z, signed_scale(nib & 4u, s), H.z);
+        const float uw = worker_step<EF>(r.G[v].w, r.H[v].w, signed_scale(nib & 8u, s), H.w);
         st_rw4(gh + wb + v * 128 + lane * 4, H);
-        const float ux = __fsub_rn(r.G[v].x, H.x), uy = __fsub_rn(r.G[v].y, H.y);
-        const float uz = __fsub_rn(r.G[v].z, H.z), uw = __fsub_rn(r.G[v].w, H.w);
         dd_acc(acc, fabsf(ux)); dd_acc(acc, fabsf(uy));
         dd_acc(acc, fabsf(uz)); dd_acc(acc, fabsf(uw));
         B[v][0] = __ballot_sync(kFull, ux >= 0.0f);
@@ -118,6 +172,7 @@ __device__ __forceinline__ void worker_compute(WorkerRegs &r, float *__restrict_
     if (lane < 16) bw[(wb >> 5) + lane] = word;
 }
 
+template <bool EF>
 __global__ void __launch_bounds__(kBlock, 4)
 k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
               uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
@@ -133,7 +188,7 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
     const float *so = scale_old + (int64_t)i * tb.q;
 
     if (!(vec_ok && first == last && base + tb.tile <= tb.d)) {
-        worker_tile_scalar(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+        worker_tile_scalar<EF>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
         return;
     }
@@ -145,7 +200,7 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
         WorkerRegs r;
         const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
         worker_load(r, g, gh, bw, wb, lane);
-        worker_compute(r, gh, bw, wb, lane, s, acc);
+        worker_compute<EF>(r, gh, bw, wb, lane, s, acc);
     }
     acc = block_sum<kBlock>(acc);
     if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
@@ -164,6 +219,7 @@ constexpr int kRingStages = 2;
 constexpr int kRingStageBytes = 2 * kSub * (int)sizeof(float);    // g and ghat sub-tile: 32 KiB
 constexpr int kRingSmemBytes = kRingStages * kRingStageBytes;
 
+template <bool EF>
 __global__ void __launch_bounds__(kBlock, 3)
 k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
                    uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
@@ -181,7 +237,7 @@ k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
     const float *so = scale_old + (int64_t)i * tb.q;
 
     if (!(first == last && base + tb.tile <= tb.d)) {          // block-uniform
-        worker_tile_scalar(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+        worker_tile_scalar<EF>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
         return;
     }
@@ -219,7 +275,7 @@ k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
         }
         __syncthreads();                                       // the stage has been read by all
         if (threadIdx.x == 0 && it + kRingStages < iters) refill(it + kRingStages, st);
-        worker_compute(r, gh, bw, wb, lane, s, acc);
+        worker_compute<EF>(r, gh, bw, wb, lane, s, acc);
     }
     if (!arrived) {
         // A copy did not complete in time: report it, give the copies still in flight a
@@ -268,7 +324,7 @@ k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Table
 // ------------------------------------------------------------------------------------
 constexpr int kNC = 16;     // workers staged per chunk
 
-template <int VPT>
+template <int VPT, bool EF>
 __global__ void __launch_bounds__(kBlock)
 k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
               float *__restrict__ ghat_s, const float *__restrict__ gtil,
@@ -301,7 +357,8 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
 #pragma unroll
             for (int v = 0; v < VPT; ++v) {
                 const int64_t j = wb + v * 128 + lane * 4;
-                H[v] = ld_rw4(ghat_s + j);
+                H[v] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                if (!EF) H[v] = ld_rw4(ghat_s + j);      // error feedback overwrites this buffer
                 Gt[v] = ld_ro4(gtil + j);
             }
             float a[VPT][4];
@@ -348,20 +405,20 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
             for (int v = 0; v < VPT; ++v) {
                 // sum / n: multiplication by 1/n is the same correctly rounded value as the
                 // division when n is a power of two
+                float m0, m1, m2, m3;
                 if (n_pow2) {
-                    H[v].x = __fadd_rn(H[v].x, __fmul_rn(a[v][0], rn));
-                    H[v].y = __fadd_rn(H[v].y, __fmul_rn(a[v][1], rn));
-                    H[v].z = __fadd_rn(H[v].z, __fmul_rn(a[v][2], rn));
-                    H[v].w = __fadd_rn(H[v].w, __fmul_rn(a[v][3], rn));
+                    m0 = __fmul_rn(a[v][0], rn); m1 = __fmul_rn(a[v][1], rn);
+                    m2 = __fmul_rn(a[v][2], rn); m3 = __fmul_rn(a[v][3], rn);
                 } else {
-                    H[v].x = __fadd_rn(H[v].x, __fdiv_rn(a[v][0], fn));
-                    H[v].y = __fadd_rn(H[v].y, __fdiv_rn(a[v][1], fn));
-                    H[v].z = __fadd_rn(H[v].z, __fdiv_rn(a[v][2], fn));
-                    H[v].w = __fadd_rn(H[v].w, __fdiv_rn(a[v][3], fn));
+                    m0 = __fdiv_rn(a[v][0], fn); m1 = __fdiv_rn(a[v][1], fn);
+                    m2 = __fdiv_rn(a[v][2], fn); m3 = __fdiv_rn(a[v][3], fn);
                 }
-                st_rw4(ghat_s + wb + v * 128 + lane * 4, H[v]);
-                const float wx = __fsub_rn(H[v].x, Gt[v].x), wy = __fsub_rn(H[v].y, Gt[v].y);
-                const float wz = __fsub_rn(H[v].z, Gt[v].z), ww = __fsub_rn(H[v].w, Gt[v].w);
+                float4 S;
+                const float wx = server_step<EF>(m0, H[v].x, Gt[v].x, S.x);
+                const float wy = server_step<EF>(m1, H[v].y, Gt[v].y, S.y);
+                const float wz = server_step<EF>(m2, H[v].z, Gt[v].z, S.z);
+                const float ww = server_step<EF>(m3, H[v].w, Gt[v].w, S.w);
+                st_rw4(ghat_s + wb + v * 128 + lane * 4, S);
                 dd_acc(acc, fabsf(wx)); dd_acc(acc, fabsf(wy));
                 dd_acc(acc, fabsf(wz)); dd_acc(acc, fabsf(ww));
                 B[v][0] = __ballot_sync(kFull, wx >= 0.0f);
@@ -388,9 +445,9 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                 const uint32_t bit = (wbits[(int64_t)i * wp + (j >> 5)] >> (j & 31)) & 1u;
                 a = __fadd_rn(a, signed_scale(bit, wscale[(int64_t)i * tb.q + r]));
             }
-            const float hn = __fadd_rn(ghat_s[j], __fdiv_rn(a, fn));
+            float hn;
+            w = server_step<EF>(__fdiv_rn(a, fn), EF ? 0.0f : ghat_s[j], gtil[j], hn);
             ghat_s[j] = hn;
-            w = __fsub_rn(hn, gtil[j]);
         }
         const uint32_t word = __ballot_sync(kFull, valid && w >= 0.0f);
         if (lane == 0) sbits[j >> 5] = word;
@@ -400,7 +457,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
         dd acc = {0.0, 0.0};
         for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
-            dd_acc(acc, fabsf(__fsub_rn(ghat_s[j], gtil[j])));
+            dd_acc(acc, fabsf(server_input_from_memory<EF>(ghat_s[j], gtil[j])));
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
@@ -413,9 +470,10 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
 // ------------------------------------------------------------------------------------
 constexpr int kUpdSpan = kBlock * 4;
 
+template <bool EF>
 __global__ void __launch_bounds__(kBlock, 5)
 k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ sscale,
-              float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
+              const float *__restrict__ ghat_s, float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
               float *__restrict__ vhat, float *__restrict__ x, Tables tb, Hyper hp, int vec_ok)
 {
     const int64_t base = (int64_t)blockIdx.x * kUpdSpan;
@@ -423,7 +481,8 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
 
     if (vec_ok && base + kUpdSpan <= tb.d) {
         const int64_t j = base + threadIdx.x * 4;
-        float4 Gt = ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
+        // error feedback reads the server's compressor input p (ghat buffer), not the old error
+        float4 Gt = EF ? ld_ro4(ghat_s + j) : ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
         float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
         const uint32_t nib = ld_ro_u32(sbits + (j >> 5)) >> (j & 31);
         const int first = tb.tile_first[T], last = tb.tile_last[T];
@@ -439,14 +498,14 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
             while (r < last && j + 3 >= tb.off[r + 1]) ++r;
             s3 = __ldg(sscale + r);
         }
-        Gt.x = __fadd_rn(Gt.x, signed_scale(nib & 1u, s0));
-        Gt.y = __fadd_rn(Gt.y, signed_scale(nib & 2u, s1));
-        Gt.z = __fadd_rn(Gt.z, signed_scale(nib & 4u, s2));
-        Gt.w = __fadd_rn(Gt.w, signed_scale(nib & 8u, s3));
-        amsgrad1(Gt.x, M.x, V.x, Vh.x, X.x, hp);
-        amsgrad1(Gt.y, M.y, V.y, Vh.y, X.y, hp);
-        amsgrad1(Gt.z, M.z, V.z, Vh.z, X.z, hp);
-        amsgrad1(Gt.w, M.w, V.w, Vh.w, X.w, hp);
+        const float ex = update_step<EF>(Gt.x, Gt.x, signed_scale(nib & 1u, s0), Gt.x);
+        const float ey = update_step<EF>(Gt.y, Gt.y, signed_scale(nib & 2u, s1), Gt.y);
+        const float ez = update_step<EF>(Gt.z, Gt.z, signed_scale(nib & 4u, s2), Gt.z);
+        const float ew = update_step<EF>(Gt.w, Gt.w, signed_scale(nib & 8u, s3), Gt.w);
+        amsgrad1(ex, M.x, V.x, Vh.x, X.x, hp);
+        amsgrad1(ey, M.y, V.y, Vh.y, X.y, hp);
+        amsgrad1(ez, M.z, V.z, Vh.z, X.z, hp);
+        amsgrad1(ew, M.w, V.w, Vh.w, X.w, hp);
         st_rw4(gtil + j, Gt); st_rw4(m + j, M); st_rw4(v + j, V);
         st_rw4(vhat + j, Vh); st_rw4(x + j, X);
         return;
@@ -457,10 +516,12 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
         const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
-        const float gt = __fadd_rn(gtil[j], signed_scale(bit, sscale[r]));
+        const float stored = EF ? ghat_s[j] : gtil[j];
+        float gt;
+        const float est = update_step<EF>(stored, stored, signed_scale(bit, sscale[r]), gt);
         gtil[j] = gt;
         float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
-        amsgrad1(gt, mm, vv, vh, xx, hp);
+        amsgrad1(est, mm, vv, vh, xx, hp);
         m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
     }
 }
@@ -469,6 +530,7 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
 // ghat_w += decode(bits, scales): applies a payload whose application was deferred.
 // grid = (ntiles, n).
 // ------------------------------------------------------------------------------------
+template <bool EF>
 __global__ void __launch_bounds__(kBlock)
 k_apply_sign(float *__restrict__ ghat_w, const uint32_t *__restrict__ wbits,
              const float *__restrict__ scales, Tables tb, int64_t wp)
@@ -482,7 +544,8 @@ k_apply_sign(float *__restrict__ ghat_w, const uint32_t *__restrict__ wbits,
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
         const uint32_t bit = (bw[j >> 5] >> (j & 31)) & 1u;
-        gh[j] = __fadd_rn(gh[j], signed_scale(bit, scales[(int64_t)i * tb.q + r]));
+        const float c = signed_scale(bit, scales[(int64_t)i * tb.q + r]);
+        gh[j] = EF ? __fsub_rn(gh[j], c) : __fadd_rn(gh[j], c);
     }
 }
 
@@ -544,15 +607,17 @@ k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__rest
 // ------------------------------------------------------------------------------------
 void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, int *error_flag, cudaStream_t st)
+                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
     if (vec_ok && tb.tile >= 4 * kSub) {
-        cudaFuncSetAttribute(k_worker_sign_ring, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
-        k_worker_sign_ring<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb,
-                                                                 wp, error_flag);
+        auto kern = ef ? k_worker_sign_ring<true> : k_worker_sign_ring<false>;
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
+        kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag);
+    } else if (ef) {
+        k_worker_sign<true><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
     } else {
-        k_worker_sign<<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+        k_worker_sign<false><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
     }
 }
 
@@ -565,26 +630,34 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, cudaStream_t st)
+                        int n, int64_t wp, bool vec_ok, bool ef, cudaStream_t st)
 {
     const int pow2 = (n & (n - 1)) == 0;
-    k_server_sign<2><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                             spart, tb, n, wp, vec_ok, pow2);
+    if (ef)
+        k_server_sign<2, true><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+                                                                       spart, tb, n, wp, vec_ok, pow2);
+    else
+        k_server_sign<2, false><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+                                                                        spart, tb, n, wp, vec_ok, pow2);
 }
 
-void launch_update_sign(const uint32_t *sbits, const float *sscale, float *gtil, float *m,
-                        float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
-                        bool vec_ok, cudaStream_t st)
+void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
+                        float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
+                        bool vec_ok, bool ef, cudaStream_t st)
 {
     const unsigned blocks = (unsigned)((tb.d + kUpdSpan - 1) / kUpdSpan);
-    k_update_sign<<<blocks, kBlock, 0, st>>>(sbits, sscale, gtil, m, v, vhat, x, tb, hp, vec_ok);
+    if (ef)
+        k_update_sign<true><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
+    else
+        k_update_sign<false><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
 }
 
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
-                       const Tables &tb, int n, int64_t wp, cudaStream_t st)
+                       const Tables &tb, int n, int64_t wp, bool ef, cudaStream_t st)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
-    k_apply_sign<<<grid, kBlock, 0, st>>>(ghat_w, wbits, scales, tb, wp);
+    if (ef) k_apply_sign<true><<<grid, kBlock, 0, st>>>(ghat_w, wbits, scales, tb, wp);
+    else k_apply_sign<false><<<grid, kBlock, 0, st>>>(ghat_w, wbits, scales, tb, wp);
 }
 
 void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
