@@ -5,8 +5,8 @@ paper's Algorithm 1 and Appendix A).  Nothing in the CUDA library or its Python 
 imports this package; it is used by the tests, the smoke check and the CPU-baseline leg of
 the benchmark only.
 """
-from .oracle import (Oracle, build, compress_sign, compress_topk, l1_exact,
-                     SIGN, TOPK, IDENTITY, MARKOV, EF, STATE_NAMES)
+from .oracle import (Oracle, build, compress_sign, compress_topk, compress_randk, l1_exact,
+                     SIGN, TOPK, IDENTITY, RANDK, MARKOV, EF, STATE_NAMES)
 
-__all__ = ["Oracle", "build", "compress_sign", "compress_topk", "l1_exact",
-           "SIGN", "TOPK", "IDENTITY", "MARKOV", "EF", "STATE_NAMES"]
+__all__ = ["Oracle", "build", "compress_sign", "compress_topk", "compress_randk", "l1_exact",
+           "SIGN", "TOPK", "IDENTITY", "RANDK", "MARKOV", "EF", "STATE_NAMES"]

@@ -28,7 +28,7 @@
 #include <string.h>
 #include <math.h>
 
-enum { ORC_SIGN = 0, ORC_TOPK = 1, ORC_IDENTITY = 2 };
+enum { ORC_SIGN = 0, ORC_TOPK = 1, ORC_IDENTITY = 2, ORC_RANDK = 3 };
 enum { ORC_MARKOV = 0, ORC_EF = 1 };
 
 /* ------------------------------------------------------------------------------------ */
@@ -173,6 +173,21 @@ void oracle_compress_topk(const float *x, int64_t d, int64_t k,
     free(key);
 }
 
+/* Rand-k: C(x) = sum_{j in S} x_j e_j for a set S of k distinct coordinates drawn uniformly at
+ * random.  The draw is an INPUT here (S, k increasing coordinates), so both sides of a
+ * comparison use the same set.  Payload: the k (index, value) pairs; c is x on S, 0 elsewhere. */
+void oracle_compress_randk(const float *x, int64_t d, int64_t k, const uint32_t *S,
+                           uint32_t *idx, float *val, float *c)
+{
+    memset(c, 0, (size_t)d * sizeof(float));
+    for (int64_t t = 0; t < k; ++t) {
+        uint32_t j = S[t];
+        idx[t] = j;
+        val[t] = x[j];
+        c[j] = x[j];
+    }
+}
+
 /* ------------------------------------------------------------------------------------ */
 /* Algorithm 1                                                                           */
 /* ------------------------------------------------------------------------------------ */
@@ -202,6 +217,9 @@ typedef struct oracle_ctx {
     /* sampled checks only: scales given from outside instead of computed (NULL = compute) */
     float *force_w_scales;   /* n*q */
     float *force_s_scales;   /* q */
+    /* rand-k: the coordinate sets of the coming iteration (inputs) */
+    uint32_t *rand_w;        /* n*k */
+    uint32_t *rand_s;        /* k */
 } oracle_ctx;
 
 static float *zeros(int64_t count) { return (float *)calloc((size_t)(count > 0 ? count : 1), sizeof(float)); }
@@ -215,6 +233,7 @@ void oracle_destroy(oracle_ctx *o)
     free(o->w_bits); free(o->w_scales); free(o->w_idx); free(o->w_val);
     free(o->s_bits); free(o->s_scales); free(o->s_idx); free(o->s_val);
     free(o->force_w_scales); free(o->force_s_scales);
+    free(o->rand_w); free(o->rand_s);
     free(o);
 }
 
@@ -240,11 +259,11 @@ static void alloc_payloads(oracle_ctx *o)
 oracle_ctx *oracle_create(int64_t d, int n, int compressor, int64_t k,
                           float beta1, float beta2, float lr, float nu)
 {
-    if (d < 1 || n < 1 || compressor < 0 || compressor > 2) return NULL;
-    if (compressor == ORC_TOPK && (k < 1 || k > d)) return NULL;
+    if (d < 1 || n < 1 || compressor < 0 || compressor > 3) return NULL;
+    if ((compressor == ORC_TOPK || compressor == ORC_RANDK) && (k < 1 || k > d)) return NULL;
     oracle_ctx *o = (oracle_ctx *)calloc(1, sizeof *o);
     o->d = d; o->n = n; o->compressor = compressor;
-    o->k = compressor == ORC_TOPK ? k : 0;
+    o->k = (compressor == ORC_TOPK || compressor == ORC_RANDK) ? k : 0;
     o->mode = ORC_MARKOV;
     o->beta1 = beta1; o->beta2 = beta2; o->lr = lr; o->nu = nu;
     o->q = 1;
@@ -334,6 +353,20 @@ static void sign_with_given_scales(oracle_ctx *o, const float *u, const float *g
     }
 }
 
+/* Rand-k: the coordinate sets (k increasing, distinct coordinates each) the n workers and the
+ * server use in the next call of oracle_step. */
+int oracle_set_random_sets(oracle_ctx *o, const uint32_t *workers, const uint32_t *server)
+{
+    if (!o || o->compressor != ORC_RANDK || !workers || !server) return -1;
+    if (!o->rand_w) {
+        o->rand_w = (uint32_t *)malloc((size_t)o->n * o->k * sizeof(uint32_t));
+        o->rand_s = (uint32_t *)malloc((size_t)o->k * sizeof(uint32_t));
+    }
+    memcpy(o->rand_w, workers, (size_t)o->n * o->k * sizeof(uint32_t));
+    memcpy(o->rand_s, server, (size_t)o->k * sizeof(uint32_t));
+    return 0;
+}
+
 /* c = C(u) with the context's compressor; who selects where the payload is kept. */
 static void compress(oracle_ctx *o, const float *u, float *c, int who)
 {
@@ -348,6 +381,9 @@ static void compress(oracle_ctx *o, const float *u, float *c, int who)
     else if (o->compressor == ORC_TOPK)
         oracle_compress_topk(u, o->d, o->k, oracle_payload_idx(o, who),
                              oracle_payload_val(o, who), c);
+    else if (o->compressor == ORC_RANDK)
+        oracle_compress_randk(u, o->d, o->k, who < 0 ? o->rand_s : o->rand_w + (int64_t)who * o->k,
+                              oracle_payload_idx(o, who), oracle_payload_val(o, who), c);
     else
         memcpy(c, u, (size_t)o->d * sizeof(float));
 }
@@ -422,6 +458,7 @@ static void step_ef(oracle_ctx *o, const float *g)
 int oracle_step(oracle_ctx *o, const float *g)
 {
     if (!o || !g) return -1;
+    if (o->compressor == ORC_RANDK && !o->rand_w) return -1;
     if (o->mode == ORC_MARKOV) step_markov(o, g); else step_ef(o, g);
     o->steps += 1;
     return 0;

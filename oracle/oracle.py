@@ -10,7 +10,7 @@ import subprocess
 
 import numpy as np
 
-SIGN, TOPK, IDENTITY = 0, 1, 2
+SIGN, TOPK, IDENTITY, RANDK = 0, 1, 2, 3
 MARKOV, EF = 0, 1
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
 
@@ -57,6 +57,10 @@ def _load():
     lib.oracle_set_mode.argtypes = [c.c_void_p, c.c_int]
     lib.oracle_set_lr.restype = c.c_int
     lib.oracle_set_lr.argtypes = [c.c_void_p, c.c_float]
+    lib.oracle_compress_randk.restype = None
+    lib.oracle_compress_randk.argtypes = [fp, c.c_int64, c.c_int64, up, up, fp, fp]
+    lib.oracle_set_random_sets.restype = c.c_int
+    lib.oracle_set_random_sets.argtypes = [c.c_void_p, up, up]
     lib.oracle_force_scales.restype = c.c_int
     lib.oracle_force_scales.argtypes = [c.c_void_p, fp, fp]
     lib.oracle_state.restype = fp
@@ -117,6 +121,22 @@ def compress_topk(x, k):
     return idx, val, c
 
 
+def compress_randk(x, S):
+    """Rand-k compressor of Appendix A on the given coordinate set S.  Returns (idx, val, c)."""
+    a, p = _f32(x)
+    d = a.size
+    S = np.ascontiguousarray(S, dtype=np.uint32)
+    k = S.size
+    idx = np.zeros(k, dtype=np.uint32)
+    val = np.zeros(k, dtype=np.float32)
+    c = np.zeros(d, dtype=np.float32)
+    up = ctypes.POINTER(ctypes.c_uint32)
+    _load().oracle_compress_randk(p, d, k, S.ctypes.data_as(up), idx.ctypes.data_as(up),
+                                  val.ctypes.data_as(ctypes.POINTER(ctypes.c_float)),
+                                  c.ctypes.data_as(ctypes.POINTER(ctypes.c_float)))
+    return idx, val, c
+
+
 class Oracle:
     """Algorithm 1 for n workers on the CPU.  State arrays are numpy views of the C memory."""
 
@@ -149,6 +169,15 @@ class Oracle:
 
     def set_lr(self, lr):
         self._lib.oracle_set_lr(self._h, lr)
+
+    def set_random_sets(self, workers, server):
+        """Rand-k: coordinate sets (n x k and k increasing distinct coordinates) of the next step."""
+        w = np.ascontiguousarray(workers, dtype=np.uint32)
+        s = np.ascontiguousarray(server, dtype=np.uint32)
+        assert w.size == self.n * self.k and s.size == self.k
+        up = ctypes.POINTER(ctypes.c_uint32)
+        if self._lib.oracle_set_random_sets(self._h, w.ctypes.data_as(up), s.ctypes.data_as(up)) != 0:
+            raise ValueError("set_random_sets applies to the rand-k compressor")
 
     def force_scales(self, worker_scales=None, server_scales=None):
         """Sampled checks only: use these scaled-sign scales (n x q, q) instead of computing
@@ -187,7 +216,7 @@ class Oracle:
             b = np.ctypeslib.as_array(self._lib.oracle_payload_bits(self._h, who), shape=(words,))
             s = np.ctypeslib.as_array(self._lib.oracle_payload_scales(self._h, who), shape=(self.q,))
             return b.copy(), s.copy()
-        if self.compressor == TOPK:
+        if self.compressor in (TOPK, RANDK):
             i = np.ctypeslib.as_array(self._lib.oracle_payload_idx(self._h, who), shape=(self.k,))
             v = np.ctypeslib.as_array(self._lib.oracle_payload_val(self._h, who), shape=(self.k,))
             return i.copy(), v.copy()

@@ -15,7 +15,7 @@ from typing import Optional
 import numpy as np
 import torch
 
-SIGN, TOPK, IDENTITY = 0, 1, 2
+SIGN, TOPK, IDENTITY, RANDK = 0, 1, 2, 3
 
 
 def _gen(device, *key):
@@ -113,6 +113,23 @@ class Workload:
                 if scale is not None:
                     row.mul_(scale)
         return out
+
+
+def random_sets(d, k, rows, seed, step):
+    """Rand-k draws: `rows` independent uniformly random k-subsets of range(d), each listed in
+    increasing order (uint32, rows x k).  Inputs of the method, not part of it."""
+    out = np.empty((rows, k), dtype=np.uint32)
+    for r in range(rows):
+        rng = np.random.default_rng([seed, step, r, 991])
+        if k * 4 > d:
+            pick = rng.permutation(d)[:k]
+        else:                                  # rejection-free for k << d: draw, dedupe, top up
+            pick = np.unique(rng.integers(0, d, size=int(k * 1.2) + 16))
+            while pick.size < k:
+                pick = np.unique(np.concatenate([pick, rng.integers(0, d, size=k)]))
+            pick = rng.permutation(pick)[:k]
+        out[r] = np.sort(pick).astype(np.uint32)
+    return out
 
 
 def workload(name, scale=1.0, steps=None, seed=0):

@@ -382,3 +382,55 @@ def test_planted_mistakes_are_caught():
     assert o.state("x").tolist() == gold["t1.x"]
     o.step(np.array([gold["t2.g0"], gold["t2.g1"]], dtype=np.float32))
     assert o.state("ghat_s").tolist() != gold["t2.s.ghat"]
+
+
+# ------------------------------------------------------------------ rand-k
+
+def test_randk_expected_error_appendix_a():
+    """E ||C(x) - x||^2 = (1 - k/d) ||x||^2 over the random set (Appendix A, rand-k)."""
+    from paper_2111_00705_b200 import synth
+    rng = np.random.default_rng(20)
+    d, k, draws = 400, 60, 4000
+    x = rng.standard_normal(d).astype(np.float32)
+    sets = synth.random_sets(d, k, draws, 5, 1)
+    err = 0.0
+    hits = np.zeros(d)
+    for S in sets:
+        idx, val, c = orc.compress_randk(x, S)
+        assert idx.tolist() == S.tolist() and np.array_equal(val, x[S])
+        dense = np.zeros(d, np.float32); dense[S] = x[S]
+        assert np.array_equal(c, dense)
+        err += np.sum((c.astype(np.float64) - x) ** 2)
+        hits[S] += 1
+    want = (1 - k / d) * np.sum(x.astype(np.float64) ** 2)
+    assert err / draws == pytest.approx(want, rel=0.02)
+    # every coordinate is drawn with probability k/d
+    assert np.all(np.abs(hits / draws - k / d) < 5 * math.sqrt(k / d * (1 - k / d) / draws))
+
+
+def test_randk_reduces_to_topk_and_identity_on_their_sets():
+    """With S = the top-k set the iteration equals the top-k one; with S = everything it
+    equals the identity compressor's (both already pinned), bit for bit."""
+    rng = np.random.default_rng(21)
+    d, n, k = 300, 3, 25
+    a = orc.Oracle(d, n, orc.TOPK, k=k)
+    b = orc.Oracle(d, n, orc.RANDK, k=k)
+    for t in range(4):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        # the sets top-k will choose, computed from the states before the step
+        W = np.stack([orc.compress_topk(g[i] - a.state("ghat_w")[i], k)[0] for i in range(n)])
+        a.step(g)
+        b.set_random_sets(W, a.payload(-1)[0])
+        b.step(g)
+        for name in orc.STATE_NAMES:
+            assert np.array_equal(a.state(name), b.state(name)), name
+        assert np.array_equal(a.payload(1)[1], b.payload(1)[1])
+    full = np.arange(d, dtype=np.uint32)
+    c = orc.Oracle(d, n, orc.IDENTITY)
+    e = orc.Oracle(d, n, orc.RANDK, k=d)
+    for t in range(3):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        e.set_random_sets(np.tile(full, (n, 1)), full)
+        c.step(g); e.step(g)
+        for name in orc.STATE_NAMES:
+            assert np.array_equal(c.state(name), e.state(name)), name
