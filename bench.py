@@ -68,6 +68,8 @@ def algorithmic_bytes(w):
         return w.d * (12.25 * w.n + 48.25), w.n * w.d * 12.125
     if w.compressor == synth.TOPK:
         return w.d * (8.0 * w.n + 44.0), w.n * w.d * 8.0
+    if w.compressor == synth.RANDK:      # sparse: 3 sectors-worth of floats per kept entry + dense AMSGrad
+        return w.d * 36.0 + (w.n + 1) * w.k * 20.0, w.d * 36.0
     return w.d * (12.0 * w.n + 48.0), w.d * (12.0 * w.n + 48.0)
 
 
@@ -184,7 +186,8 @@ def replicas_throughput(world, steps, total_ms):
 
 def describe(w):
     from paper_2111_00705_b200 import synth
-    comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity"}[w.compressor]
+    comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity",
+            synth.RANDK: "rand-k k=%d" % w.k}[w.compressor]
     return "%s d=%d n=%d %s q=%d %s fp32" % (w.name, w.d, w.n, comp, w.q, w.dist)
 
 
@@ -197,6 +200,8 @@ def main():
     ap.add_argument("--impl", default="cdadam", choices=["cdadam", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--compressor", default=None, choices=[None, "randk"],
+                    help="randk: run the workload's shapes with the rand-k compressor (k as in C3: d/100)")
     ap.add_argument("--mode", default="markov", choices=["markov", "ef"],
                     help="markov = Algorithm 1 (default); ef = classical error feedback (Section 4)")
     ap.add_argument("--tile", type=int, default=0,
@@ -231,6 +236,8 @@ def main():
         torch.cuda.synchronize()
 
     w = synth.workload(args.workload, scale=args.scale)
+    if args.compressor == "randk":
+        w.compressor, w.k, w.offsets = synth.RANDK, max(1, w.d // 100), None
     if args.warmup < 3:
         args.warmup = 3
     opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
@@ -238,6 +245,10 @@ def main():
                     mode=cd.EF if args.mode == "ef" else cd.MARKOV)
     if args.tile:
         opt.set_tile(args.tile)
+    if w.compressor == synth.RANDK:      # the draws are inputs; one set of draws serves all steps
+        import numpy as np
+        opt.set_random_sets(torch.from_numpy(synth.random_sets(w.d, w.k, w.n, w.seed, 1).view(np.int32)).to(dev),
+                            torch.from_numpy(synth.random_sets(w.d, w.k, 1, w.seed + 1, 1)[0].view(np.int32)).to(dev))
     # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
     # flushed between steps instead
     nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1

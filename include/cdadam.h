@@ -44,7 +44,7 @@ extern "C" {
 typedef struct cdadam_ctx cdadam_ctx;
 
 /* compressor C of Algorithm 1 (Appendix A) */
-enum { CDADAM_SIGN = 0, CDADAM_TOPK = 1, CDADAM_IDENTITY = 2 };
+enum { CDADAM_SIGN = 0, CDADAM_TOPK = 1, CDADAM_IDENTITY = 2, CDADAM_RANDK = 3 };
 
 /* recursion around the compressor */
 enum {
@@ -80,8 +80,8 @@ enum {
  *   d          model dimension, 1 <= d < 2^32
  *   n          number of simulated workers, 1 <= n <= 65535
  *   compressor CDADAM_SIGN, CDADAM_TOPK or CDADAM_IDENTITY
- *   k          entries kept by top-k at the workers and at the server, 1 <= k <= d;
- *              ignored for the other compressors
+ *   k          entries kept by top-k / rand-k at the workers and at the server,
+ *              1 <= k <= d; ignored for the other compressors
  * All state is allocated here, on the current device, and zero-initialised (Algorithm 1
  * line 1; x_1 = 0 until cdadam_set_params).  Scaled sign starts with one segment [0, d).
  * Synchronous.  Returns NULL on failure (see cdadam_last_error).  The caller destroys the
@@ -132,6 +132,17 @@ int cdadam_set_params(cdadam_ctx *ctx, const float *x0, void *stream);
 int cdadam_set_segments(cdadam_ctx *ctx, int q, const int64_t *offsets);
 
 /*
+ * Rand-k compressor (Appendix A: C(x) keeps x on k coordinates drawn uniformly at random).
+ * The draws are inputs: before each step give the coordinate sets the n workers (device,
+ * n x k uint32, row i = worker i) and the server (device, k uint32) use in that step.  Every
+ * set must be strictly increasing with all coordinates below d.  The sets are copied; they
+ * stay in force until replaced.  A malformed set is never dereferenced out of range; it is
+ * reported by cdadam_device_status (CDADAM_ERR_ARG) and invalidates the state.
+ */
+int cdadam_set_random_sets(cdadam_ctx *ctx, const uint32_t *workers, const uint32_t *server,
+                           void *stream);
+
+/*
  * Choose the recursion: CDADAM_MARKOV (Algorithm 1, default) or CDADAM_EF, the error-feedback
  * scheme the paper compares against (Section 4), applied both ways:
  *   worker: p = g + delta^(i), c^(i) = C(p), delta^(i) = p - c^(i);
@@ -168,7 +179,7 @@ int cdadam_set_state(cdadam_ctx *ctx, int name, const float *src, void *stream);
  *   scaled sign: *a = uint32 words, bit (j % 32) of word j / 32 is 1 iff u_j >= 0 (so a
  *                zero counts as positive), unused high bits of the last word are 0;
  *                *b = q float scales; *count = d.  The message is d + 32 q bits.
- *   top-k:       *a = k uint32 coordinates in increasing order, *b = their k float values
+ *   top-k, rand-k: *a = k uint32 coordinates in increasing order, *b = their k float values
  *                u_j; *count = k.  Among equal |u_j| the lower j is kept.
  * CDADAM_ERR_STATE before the first step or for the identity compressor.
  */

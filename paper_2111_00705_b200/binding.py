@@ -9,7 +9,7 @@ import os
 
 import torch
 
-SIGN, TOPK, IDENTITY = 0, 1, 2
+SIGN, TOPK, IDENTITY, RANDK = 0, 1, 2, 3
 MARKOV, EF = 0, 1
 SERVER = -1
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
@@ -28,6 +28,7 @@ _SIGNATURES = {
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
+    "cdadam_set_random_sets": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_mode": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_tile": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
@@ -178,6 +179,14 @@ class CDAdam:
         off = (ctypes.c_int64 * len(offsets))(*[int(v) for v in offsets])
         _check(lib().cdadam_set_segments(self._h, len(offsets) - 1, off))
         self.q = len(offsets) - 1
+
+    def set_random_sets(self, workers, server, stream=None):
+        """Rand-k: CUDA int32/uint32 tensors with n*k and k increasing coordinates."""
+        for t, cnt in ((workers, self.n * self.k), (server, self.k)):
+            if not (t.is_cuda and t.is_contiguous() and t.element_size() == 4 and t.numel() == cnt):
+                raise ValueError("sets must be contiguous CUDA 32-bit integer tensors of n*k and k elements")
+        _check(lib().cdadam_set_random_sets(self._h, ctypes.c_void_p(workers.data_ptr()),
+                                            ctypes.c_void_p(server.data_ptr()), _stream(stream)))
 
     def set_tile(self, tile):
         _check(lib().cdadam_set_tile(self._h, int(tile)))

@@ -135,6 +135,7 @@ struct cdadam_ctx {
     int *error_flag = nullptr;   // device word set by a kernel whose bounded wait ran out
     int cur = 0;            // wscale[cur] holds the scales of the last worker payloads
     bool pending = false;   // the last worker payloads are not yet added to ghat_w
+    bool sets_given = false;   // rand-k: coordinate sets have been supplied
     // top-k
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
     // host-gradient staging
@@ -189,7 +190,7 @@ float *state_ptr(cdadam_ctx *c, int name)
 
 int prof_slots(const cdadam_ctx *c)
 {
-    return c->comp == CDADAM_SIGN ? 5 : c->comp == CDADAM_TOPK ? 4 : 1;
+    return c->comp == CDADAM_SIGN ? 5 : (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK) ? 4 : 1;
 }
 
 // Record the boundary event after a stage (or before the first one) when timing is on.
@@ -225,11 +226,11 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
 {
     if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
     if (n < 1 || n > 65535) { fail(CDADAM_ERR_ARG, "n must be in [1, 65535]"); return nullptr; }
-    if (compressor < CDADAM_SIGN || compressor > CDADAM_IDENTITY) { fail(CDADAM_ERR_ARG, "unknown compressor %d", compressor); return nullptr; }
-    if (compressor == CDADAM_TOPK && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k needs 1 <= k <= d"); return nullptr; }
+    if (compressor < CDADAM_SIGN || compressor > CDADAM_RANDK) { fail(CDADAM_ERR_ARG, "unknown compressor %d", compressor); return nullptr; }
+    if ((compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k and rand-k need 1 <= k <= d"); return nullptr; }
     cdadam_ctx *c = new (std::nothrow) cdadam_ctx;
     if (!c) { fail(CDADAM_ERR_ALLOC, "out of host memory"); return nullptr; }
-    c->d = d; c->n = n; c->comp = compressor; c->k = compressor == CDADAM_TOPK ? k : 0;
+    c->d = d; c->n = n; c->comp = compressor; c->k = (compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) ? k : 0;
     c->wp = (d + 31) / 32;
     c->hp.beta1 = beta1; c->hp.beta2 = beta2; c->hp.lr = lr; c->hp.nu = eps;
     c->hp.omb1 = 1.0f - beta1; c->hp.omb2 = 1.0f - beta2;
@@ -250,6 +251,9 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
             if ((rc = dev_zalloc(&c->sbits, (size_t)c->wp))) break;
             if ((rc = c->ts.build(d, 1, flat, choose_tile(d, 1), nullptr, false))) break;
             if ((rc = alloc_sign_buffers(c))) break;
+        } else if (compressor == CDADAM_RANDK) {
+            if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n, nullptr, nullptr, false))) { fail(rc, "rand-k payload allocation failed"); break; }
+            if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1, nullptr, nullptr, false))) { fail(rc, "rand-k payload allocation failed"); break; }
         } else if (compressor == CDADAM_TOPK) {
             if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n))) { fail(rc, "top-k workspace allocation failed"); break; }
             if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1))) { fail(rc, "top-k workspace allocation failed"); break; }
@@ -332,6 +336,36 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
         launch_amsgrad(c->ghat_s, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
         launch_scatter_set(c->ghat_s, sidx, nullptr, c->k, c->d, 1, st);
         prof_mark(c, st);
+    } else if (c->comp == CDADAM_RANDK) {
+        if (!c->sets_given) return fail(CDADAM_ERR_STATE, "rand-k needs cdadam_set_random_sets before the first step");
+        const uint32_t *widx, *sidx;
+        const float *wval, *sval;
+        topk_payload(c->tk_w, 0, &widx, &wval);
+        topk_payload(c->tk_s, 0, &sidx, &sval);
+        if (!ef) {
+            randk_gather(c->tk_w, grads, c->ghat_w, true, st);                 // lines 5-6
+            prof_mark(c, st);
+            topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
+            prof_mark(c, st);
+            randk_gather(c->tk_s, c->ghat_s, c->gtil, true, st);               // lines 9-10, 12
+            prof_mark(c, st);
+            launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+            prof_mark(c, st);
+        } else {                                                               // as top-k above
+            launch_add_into(c->ghat_w, grads, (int64_t)c->n * c->d, vec, st);
+            randk_gather(c->tk_w, c->ghat_w, nullptr, false, st);
+            launch_scatter_set(c->ghat_w, widx, nullptr, c->k, c->d, c->n, st);
+            prof_mark(c, st);
+            topk_aggregate(c->tk_w, c->gtil, c->n, st);
+            prof_mark(c, st);
+            randk_gather(c->tk_s, c->gtil, nullptr, false, st);
+            launch_scatter_set(c->gtil, sidx, nullptr, c->k, c->d, 1, st);
+            launch_scatter_set(c->ghat_s, sidx, sval, c->k, c->d, 1, st);
+            prof_mark(c, st);
+            launch_amsgrad(c->ghat_s, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+            launch_scatter_set(c->ghat_s, sidx, nullptr, c->k, c->d, 1, st);
+            prof_mark(c, st);
+        }
     } else {
         launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, ef, st);
         prof_mark(c, st);
@@ -396,6 +430,17 @@ int cdadam_set_tile(cdadam_ctx *c, int tile)
     return cdadam_set_segments(c, (int)off.size() - 1, off.data());
 }
 
+int cdadam_set_random_sets(cdadam_ctx *c, const uint32_t *workers, const uint32_t *server, void *stream)
+{
+    if (!c || !workers || !server) return fail(CDADAM_ERR_ARG, "cdadam_set_random_sets: NULL argument");
+    if (c->comp != CDADAM_RANDK) return fail(CDADAM_ERR_STATE, "random sets apply to the rand-k compressor only");
+    DeviceGuard guard(c->device);
+    randk_set(c->tk_w, workers, c->error_flag, (cudaStream_t)stream);
+    randk_set(c->tk_s, server, c->error_flag, (cudaStream_t)stream);
+    c->sets_given = true;
+    return check_launch("cdadam_set_random_sets");
+}
+
 int cdadam_set_mode(cdadam_ctx *c, int mode)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_mode: NULL context");
@@ -453,7 +498,7 @@ int cdadam_last_payload(cdadam_ctx *c, int who, const void **a, const float **b,
         *count = c->d;
         return CDADAM_OK;
     }
-    if (c->comp == CDADAM_TOPK) {
+    if (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK) {
         TopkWorkspace *w = who == CDADAM_SERVER ? c->tk_s : c->tk_w;
         topk_payload(w, who == CDADAM_SERVER ? 0 : who, (const uint32_t **)a, b);
         *count = c->k;
@@ -471,6 +516,7 @@ int cdadam_device_status(cdadam_ctx *c, void *stream)
     int flag = 0;
     CU_TRY(cudaMemcpyAsync(&flag, c->error_flag, sizeof flag, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    if (flag == 2) return fail(CDADAM_ERR_ARG, "a rand-k coordinate set was not strictly increasing or had a coordinate >= d; the state is not valid");
     if (flag) return fail(CDADAM_ERR_TIMEOUT, "a kernel gave up waiting for an asynchronous copy; the state is not valid");
     return CDADAM_OK;
 }
@@ -480,6 +526,7 @@ int cdadam_launches_per_step(cdadam_ctx *c)
     if (!c) return 0;
     if (c->comp == CDADAM_SIGN) return 5;
     if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : 0);
+    if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : 4;
     return 1;
 }
 
@@ -515,6 +562,8 @@ const char *cdadam_profile_name(cdadam_ctx *c, int slot)
                                  "k_finalize_scales(server)", "k_update_sign"};
     static const char *topk[] = {"topk_select(workers)", "topk_aggregate", "topk_select(server)", "k_amsgrad"};
     if (!c || slot < 0 || slot >= prof_slots(c)) return "";
+    static const char *randk[] = {"randk_gather(workers)", "topk_aggregate", "randk_gather(server)", "k_amsgrad"};
+    if (c->comp == CDADAM_RANDK) return randk[slot];
     return c->comp == CDADAM_SIGN ? sign[slot] : c->comp == CDADAM_TOPK ? topk[slot] : "k_step_identity";
 }
 

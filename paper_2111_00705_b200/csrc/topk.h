@@ -10,8 +10,9 @@ struct TopkWorkspace;
 
 // Scratch and payload buffers for selecting k of d coordinates in each of `rows` vectors.
 // If idx/val are NULL the workspace owns the payload arrays (rows x k each).
+// with_select = false allocates the payload arrays only (rand-k needs no selection scratch).
 int topk_workspace_create(TopkWorkspace **w, int64_t d, int64_t k, int rows,
-                          uint32_t *idx = nullptr, float *val = nullptr);
+                          uint32_t *idx = nullptr, float *val = nullptr, bool with_select = true);
 void topk_workspace_destroy(TopkWorkspace *w);
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
 int topk_launches_per_step(int n);
@@ -26,6 +27,13 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
 //   ghat_s += (sum_i c_i) / n on the coordinates some worker sent, workers added in the
 //   order 0, 1, ..., n-1.
 void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st);
+
+// Rand-k (Appendix A): the k coordinates of every row are given by the caller.
+// randk_set copies rows x k device indices into the payload and checks them (strictly
+// increasing, below d; *error_flag = 2 otherwise).  randk_gather fills the payload values
+// u_j = a_j - b_j (b may be NULL) and, if update_b, adds them to b at those coordinates.
+void randk_set(TopkWorkspace *w, const uint32_t *sets, int *error_flag, cudaStream_t st);
+void randk_gather(TopkWorkspace *w, const float *a, float *b, bool update_b, cudaStream_t st);
 
 // Stand-alone top-k of one vector into caller buffers (allocates and frees scratch).
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val,

@@ -12,6 +12,7 @@
 #include "topk.h"
 
 #include <algorithm>
+#include <cstring>
 
 #include "../../include/cdadam.h"
 #include "common.cuh"
@@ -579,6 +580,7 @@ k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
     if (t >= k) return;
     const int64_t j = idx_all[(int64_t)row * k + t];
+    if (j >= d) return;                       // caller-supplied sets are checked separately
     const float *a = a_all + (int64_t)row * d;
     float u;
     if (HAS_B) {
@@ -634,11 +636,16 @@ k_topk_aggregate(const uint32_t *__restrict__ idx_all, const float *__restrict__
             // enclosing compaction tile, whose bounds are the scanned tile counts
             const int i = i0 + (threadIdx.x >> 1), side = threadIdx.x & 1;
             const uint32_t *idx = idx_all + (int64_t)i * k;
-            const int64_t t_lo = fin_off_all[(int64_t)i * nbt + tile];
-            const int64_t t_hi = tile + 1 < nbt ? (int64_t)fin_off_all[(int64_t)i * nbt + tile + 1] : k;
+            int64_t t_lo = 0, t_hi = k;       // without tile counts (rand-k): the whole payload
+            if (fin_off_all) {
+                t_lo = fin_off_all[(int64_t)i * nbt + tile];
+                t_hi = tile + 1 < nbt ? (int64_t)fin_off_all[(int64_t)i * nbt + tile + 1] : k;
+            }
             int64_t pos = t_hi;
-            if (side == 0 || end < (tile + 1) * (int64_t)(kTileWords * 32))
-                pos = t_lo + lower_bound_u32(idx + t_lo, min(t_hi, k) - t_lo, (uint32_t)(side == 0 ? base : end));
+            if (!fin_off_all || side == 0 || end < (tile + 1) * (int64_t)(kTileWords * 32))
+                pos = (side == 1 && end >= ((int64_t)1 << 32))
+                          ? min(t_hi, k)
+                          : t_lo + lower_bound_u32(idx + t_lo, min(t_hi, k) - t_lo, (uint32_t)(side == 0 ? base : end));
             range[threadIdx.x >> 1][side] = min(pos, k);
         }
         __syncthreads();
@@ -647,8 +654,8 @@ k_topk_aggregate(const uint32_t *__restrict__ idx_all, const float *__restrict__
             const float *val = val_all + (int64_t)(i0 + c) * k;
             const int64_t lo = range[c][0], hi = range[c][1];
             for (int64_t t = lo + threadIdx.x; t < hi; t += kBlock) {
-                const int e = (int)(idx[t] - base);
-                acc[e] = __fadd_rn(acc[e], val[t]);
+                const uint32_t e = idx[t] - (uint32_t)base;
+                if (e < (uint32_t)kAggSpan) acc[e] = __fadd_rn(acc[e], val[t]);
             }
             __syncthreads();
         }
@@ -674,10 +681,11 @@ static void free_ws(TopkWorkspace *w)
 }
 
 int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, uint32_t *idx,
-                          float *val)
+                          float *val, bool with_select)
 {
     *out = nullptr;
     TopkWorkspace *w = new TopkWorkspace();
+    memset(w, 0, sizeof *w);
     w->d = d; w->k = k; w->rows = rows;
     w->wp = (d + 31) / 32;
     w->nbt = (w->wp + kTileWords - 1) / kTileWords;
@@ -688,16 +696,18 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         *p = nullptr;
         if (ok && (cudaMalloc(p, bytes) != cudaSuccess || cudaMemset(*p, 0, bytes) != cudaSuccess)) ok = false;
     };
-    get((void **)&w->hist, (size_t)rows * kHistStride * 4);
-    get((void **)&w->sel, (size_t)rows * sizeof(Sel));
-    get((void **)&w->bm_in, (size_t)rows * w->wp * 4);
-    get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
-    get((void **)&w->bm_ge, (size_t)rows * w->wp * 4);
-    get((void **)&w->floor_bucket, (size_t)rows * 4);
-    get((void **)&w->hit, (size_t)rows * 4);
-    if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
-    get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
-    get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
+    if (with_select) {
+        get((void **)&w->hist, (size_t)rows * kHistStride * 4);
+        get((void **)&w->sel, (size_t)rows * sizeof(Sel));
+        get((void **)&w->bm_in, (size_t)rows * w->wp * 4);
+        get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
+        get((void **)&w->bm_ge, (size_t)rows * w->wp * 4);
+        get((void **)&w->floor_bucket, (size_t)rows * 4);
+        get((void **)&w->hit, (size_t)rows * 4);
+        if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
+        get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
+        get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
+    }
     if (w->own_payload) {
         get((void **)&w->idx, (size_t)rows * k * 4);
         get((void **)&w->val, (size_t)rows * k * 4);
@@ -762,10 +772,37 @@ void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st)
     k_topk_aggregate<<<blocks, kBlock, 0, st>>>(ww->idx, ww->val, ww->cnt_fin, ww->nbt, n, ww->k, ww->d, ghat_s, (n & (n - 1)) == 0);
 }
 
+// ---- rand-k: the coordinate sets come from the caller -------------------------------------
+// Every row's set must be strictly increasing and below d; a violation sets *error_flag.
+__global__ void __launch_bounds__(kBlock)
+k_check_sets(const uint32_t *__restrict__ idx_all, int64_t k, int64_t d, int *__restrict__ error_flag)
+{
+    const int row = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t >= k) return;
+    const uint32_t *idx = idx_all + (int64_t)row * k;
+    if ((int64_t)idx[t] >= d || (t > 0 && idx[t - 1] >= idx[t])) atomicExch(error_flag, 2);
+}
+
+void randk_set(TopkWorkspace *w, const uint32_t *sets, int *error_flag, cudaStream_t st)
+{
+    cudaMemcpyAsync(w->idx, sets, (size_t)w->rows * w->k * 4, cudaMemcpyDeviceToDevice, st);
+    const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+    k_check_sets<<<entries, kBlock, 0, st>>>(w->idx, w->k, w->d, error_flag);
+}
+
+void randk_gather(TopkWorkspace *w, const float *a, float *b, bool update_b, cudaStream_t st)
+{
+    const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
+    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
+    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, w->d, w->k);
+}
+
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
 {
     TopkWorkspace *w = nullptr;
-    int rc = topk_workspace_create(&w, d, k, 1, idx, val);
+    int rc = topk_workspace_create(&w, d, k, 1, idx, val, true);
     if (rc) return rc;
     topk_select(w, x, nullptr, false, ((uintptr_t)x & 15u) == 0 && d % 4 == 0, st);
     cudaError_t e = cudaStreamSynchronize(st);

@@ -176,6 +176,40 @@ def test_error_feedback_mode_matches_oracle(case):
         run_free(synth.Workload("EF5", 5000, 3, synth.IDENTITY, 4), 4, mode=cd.EF)
 
 
+@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
+@pytest.mark.parametrize("d,n,k", [(50000, 4, 500), (4097, 3, 4097), (70001, 2, 1)])
+def test_randk_matches_oracle(mode, d, n, k):
+    """Rand-k (Appendix A) with the random coordinate sets supplied to both sides."""
+    w = synth.Workload("RK", d, n, synth.RANDK, 4, k=k, seed=d)
+    g, o = make_pair(w, mode=mode)
+    for t in range(1, 5):
+        W = synth.random_sets(d, k, n, w.seed, t)
+        S = synth.random_sets(d, k, 1, w.seed + 1, t)[0]
+        g.set_random_sets(torch.from_numpy(W.view(np.int32)).cuda(),
+                          torch.from_numpy(S.view(np.int32)).cuda())
+        o.set_random_sets(W, S)
+        grads = w.grads(t, "cpu")
+        g.step(grads.cuda()); o.step(grads.numpy())
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.device_status()
+
+
+def test_randk_malformed_sets_are_reported_not_dereferenced():
+    d, n, k = 1000, 2, 5
+    g = cd.CDAdam(d, n, cd.RANDK, k=k)
+    with pytest.raises(cd.CdadamError):
+        g.step(torch.zeros(n * d, device="cuda"))            # no sets yet
+    bad = torch.tensor([[1, 2, 3, 4, 5], [9, 8, 7, 6, 2_000_000_000]], dtype=torch.int32, device="cuda")
+    g.set_random_sets(bad, torch.arange(k, dtype=torch.int32, device="cuda"))
+    g.step(torch.ones(n * d, device="cuda"))
+    with pytest.raises(cd.CdadamError) as e:
+        g.device_status()
+    assert e.value.code == cd.ERR_ARG
+    torch.cuda.synchronize()                                 # the device is still usable
+    assert torch.ones(4, device="cuda").sum().item() == 4
+
+
 def test_identity_matches_oracle():
     w = synth.Workload("ID", 5000, 3, synth.IDENTITY, 4)
     run_free(w, 4)
