@@ -560,6 +560,8 @@ const char *cdadam_profile_name(cdadam_ctx *c, int slot)
 {
     static const char *sign[] = {"k_worker_sign", "k_finalize_scales(workers)", "k_server_sign",
                                  "k_finalize_scales(server)", "k_update_sign"};
+    if (c && c->comp == CDADAM_SIGN && slot == 0 && c->ts.tb.tile >= 4 * kSub && c->d % 4 == 0)
+        return "k_worker_sign_ring";
     static const char *topk[] = {"topk_select(workers)", "topk_aggregate", "topk_select(server)", "k_amsgrad"};
     if (!c || slot < 0 || slot >= prof_slots(c)) return "";
     static const char *randk[] = {"randk_gather(workers)", "topk_aggregate", "randk_gather(server)", "k_amsgrad"};
