@@ -39,13 +39,13 @@ FALLBACK_HBM_GBS = 6650.0
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
     # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "95acb0a30d838775", "bytes_per_launch": 4 * (1.797066e9 + 0.856808e9)},
+    "C4": {"hash": "4838b8045026de76", "bytes_per_launch": 4 * (1.797152e9 + 0.857482e9)},
 }
 
 
 def kernel_source_hash():
     h = hashlib.sha256()
-    for f in ("common.cuh", "sign_kernels.cu", "topk_kernels.cu"):
+    for f in ("common.cuh", "sign_kernels.cu"):
         with open(os.path.join(ROOT, "paper_2111_00705_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
