@@ -23,6 +23,7 @@ constexpr uint32_t kFull = 0xffffffffu;
 constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
 constexpr int kHistStride = kBins1 + kBins2 + kBins3;
 constexpr int kTileWords = 1024;      // bitmap words per block in the sparse passes
+constexpr int kStashCap = 512;        // values kept per 4096-coordinate tile by the dense pass
 constexpr uint32_t kGuessMargin = 2;  // level-1 buckets kept below the last threshold bucket
 
 struct Sel {                          // outcome of the three levels for one row
@@ -41,6 +42,9 @@ struct TopkWorkspace {
     uint32_t *bm_ge;                  // rows x wp: coordinates at or above the guessed bucket
     uint32_t *floor_bucket;           // rows: guessed level-1 bucket for the next selection
     uint32_t *hit;                    // rows: 1 if the guess held in the current selection
+    uint32_t *ovf;                    // rows: 1 if some tile had more than kStashCap values to keep
+    float *stash;                     // rows x ceil(d/4096) x kStashCap: u of the coordinates in bm_ge
+    int64_t nt4k;                     // ceil(d / 4096)
     uint32_t *cnt_tie, *cnt_fin;      // rows x nbt
     uint32_t *idx;                    // rows x k
     float *val;                       // rows x k
@@ -260,9 +264,11 @@ template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ bm_ge_all,
-            uint32_t *__restrict__ hist_all, int64_t d, int64_t wp, int vec_ok)
+            uint32_t *__restrict__ hist_all, float *__restrict__ stash_all, uint32_t *__restrict__ ovf,
+            int64_t d, int64_t wp, int vec_ok)
 {
     __shared__ uint32_t h[kBins1];
+    __shared__ uint32_t wcnt[kBlock / 32];
     const int row = blockIdx.y;
     const uint32_t fl = floor_bucket[row];
     if (fl >= (uint32_t)kBins1) return;               // no guess for this row
@@ -271,8 +277,12 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const float *a = a_all + (int64_t)row * d;
     const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     uint32_t *bm_ge = bm_ge_all + (int64_t)row * wp;
+    // the values u of the coordinates at or above the floor, in index order, so that the
+    // sparse passes that follow read them back sequentially instead of gathering a and b
+    float *stash = stash_all + ((int64_t)row * gridDim.x + blockIdx.x) * kStashCap;
     const int64_t base = (int64_t)blockIdx.x * kSub;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t lt = (1u << lane) - 1u;
     if (vec_ok && base + kSub <= d) {
         const int64_t wb = base + warp * kWarpSpan;
         float4 A[4], Bv[4];
@@ -283,6 +293,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if (HAS_B) Bv[v] = ld_ro4(b + j);
         }
         uint32_t BG[4][4];
+        uint32_t mine = 0;
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             if (HAS_B) {
@@ -299,19 +310,54 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if (hy >= fl) atomicAdd(&h[hy], 1u);
             if (hz >= fl) atomicAdd(&h[hz], 1u);
             if (hw >= fl) atomicAdd(&h[hw], 1u);
+            mine += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
         }
         const uint32_t wg = warp_words(BG, lane);
         if (lane < 16) bm_ge[(wb >> 5) + lane] = wg;
+        if (lane == 0) wcnt[warp] = mine;             // the same in every lane
+        __syncthreads();
+        uint32_t rank = 0, total = 0;
+#pragma unroll
+        for (int w8 = 0; w8 < kBlock / 32; ++w8) {
+            if (w8 < warp) rank += wcnt[w8];
+            total += wcnt[w8];
+        }
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            uint32_t r = rank + __popc(BG[v][0] & lt) + __popc(BG[v][1] & lt) + __popc(BG[v][2] & lt) +
+                         __popc(BG[v][3] & lt);
+            if ((BG[v][0] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].x; ++r; }
+            if ((BG[v][1] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].y; ++r; }
+            if ((BG[v][2] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].z; ++r; }
+            if ((BG[v][3] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].w; }
+            rank += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
+        }
+        if (threadIdx.x == 0 && total > (uint32_t)kStashCap) ovf[row] = 1u;
     } else {
         const int64_t end = min(base + (int64_t)kSub, d);
-        for (int64_t j = base + threadIdx.x; j - lane < end; j += kBlock) {
+        uint32_t run = 0;                             // coordinates kept so far, block-uniform
+        for (int64_t j0 = base; j0 < end; j0 += kBlock) {
+            const int64_t j = j0 + threadIdx.x;
             const bool valid = j < end;
-            const uint32_t hi = valid ? key_of(diff1<HAS_B>(a, b, j)) >> 20 : 0u;
+            const float u = valid ? diff1<HAS_B>(a, b, j) : 0.0f;
+            const uint32_t hi = key_of(u) >> 20;
             const bool ge = valid && hi >= fl;
             const uint32_t wg = __ballot_sync(kFull, ge);
-            if (lane == 0) bm_ge[j >> 5] = wg;
+            if (lane == 0 && j < end) bm_ge[j >> 5] = wg;
             if (ge) atomicAdd(&h[hi], 1u);
+            if (lane == 0) wcnt[warp] = __popc(wg);
+            __syncthreads();
+            uint32_t r = run + __popc(wg & lt), total = 0;
+#pragma unroll
+            for (int w8 = 0; w8 < kBlock / 32; ++w8) {
+                if (w8 < warp) r += wcnt[w8];
+                total += wcnt[w8];
+            }
+            if (ge && r < (uint32_t)kStashCap) stash[r] = u;
+            run += total;
+            __syncthreads();
         }
+        if (threadIdx.x == 0 && run > (uint32_t)kStashCap) ovf[row] = 1u;
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
@@ -319,12 +365,14 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
         if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
-// Did the guess hold?  It did if at least k coordinates lie at or above the floor; then the
+// Did the guess hold?  It did if at least k coordinates lie at or above the floor (and every
+// tile could keep the values of its coordinates at or above the floor); then the
 // level-1 bucket follows from the histogram of those coordinates.  Otherwise the row's
 // level-1 histogram is cleared for the full pass.  grid = (rows), one block.
 __global__ void __launch_bounds__(kBlock)
 k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
-                 const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hit)
+                 const uint32_t *__restrict__ floor_bucket, const uint32_t *__restrict__ ovf,
+                 uint32_t *__restrict__ hit)
 {
     __shared__ uint32_t tot[kBlock];
     __shared__ uint32_t found;
@@ -352,43 +400,64 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
         }
     }
     __syncthreads();
-    const uint32_t ok = found;
+    const uint32_t ok = found && !ovf[row];             // a tile that could not keep its values: redo
     if (threadIdx.x == 0) hit[row] = ok;
     if (!ok)
         for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
+}
+
+// In the passes below a thread owns 4 consecutive bitmap words and a warp therefore one
+// 4096-coordinate tile of the dense pass.  The k-th set bit of the tile's bm_ge words has its
+// value at stash[k]; a thread's first rank is the warp-exclusive sum of the popcounts.
+__device__ __forceinline__ uint32_t warp_excl_sum(uint32_t v)
+{
+    const int lane = threadIdx.x & 31;
+    uint32_t inc = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(kFull, inc, o);
+        if (lane >= o) inc += t;
+    }
+    return inc - v;
 }
 
 // After a successful guess: from the bitmap of coordinates at or above the floor, rebuild
 // what the second dense pass would have produced: bm_in (bucket above the threshold
 // bucket), bm_cand (inside it) and the level-2 histogram of the candidates.
 // grid = (nbt, rows); a thread walks the set bits of its bitmap words.
-template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
-k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
-             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-             const uint32_t *__restrict__ bm_ge_all, uint32_t *__restrict__ bm_in_all,
-             uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d, int64_t wp)
+k_topk_split(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+             const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
+             uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
+             uint32_t *__restrict__ hist_all, int64_t wp, int64_t nt4k)
 {
     __shared__ uint32_t h[kBins2];
     const int row = blockIdx.y;
     if (!hit[row]) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     const uint32_t b1 = sel_all[row].b1;
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
-    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
-        uint32_t word = bm_ge_all[(int64_t)row * wp + w0 + t], in = 0, cand = 0;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+    const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
+    const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
+    uint32_t ge[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
+    uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
+#pragma unroll
+    for (int m = 0; m < 4; ++m) {
+        uint32_t word = ge[m], in = 0, cand = 0;
         while (word) {
             const int bit = __ffs(word) - 1;
             word &= word - 1;
-            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+            const uint32_t key = key_of(stash[rank++]);
             if ((key >> 20) > b1) in |= 1u << bit;
             else if ((key >> 20) == b1) { cand |= 1u << bit; atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u); }
         }
-        bm_in_all[(int64_t)row * wp + w0 + t] = in;
-        bm_cand_all[(int64_t)row * wp + w0 + t] = cand;
+        if (w0 + m < wp) {
+            bm_in_all[(int64_t)row * wp + w0 + m] = in;
+            bm_cand_all[(int64_t)row * wp + w0 + m] = cand;
+        }
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
@@ -403,25 +472,51 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
-             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ bm_cand_all,
-             uint32_t *__restrict__ hist_all, int64_t d, int64_t wp)
+             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+             const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
+             const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
+             int64_t wp, int64_t nt4k)
 {
     __shared__ uint32_t h[kBins3];
     for (int t = threadIdx.x; t < kBins3; t += kBlock) h[t] = 0;
     __syncthreads();
     const int row = blockIdx.y;
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     const uint32_t *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
-    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
-        uint32_t word = bm_cand[w0 + t];
-        while (word) {
-            const int bit = __ffs(word) - 1;
-            word &= word - 1;
-            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
-            if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+    if (hit[row]) {                                   // values come from the dense pass's stash
+        const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+        const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
+        const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
+        uint32_t ge[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
+        uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            const uint32_t cand = ge[m] ? bm_cand[w0 + m] : 0u;
+            uint32_t word = ge[m];
+            while (word) {
+                const int bit = __ffs(word) - 1;
+                word &= word - 1;
+                if ((cand >> bit) & 1u) {
+                    const uint32_t key = key_of(stash[rank]);
+                    if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+                }
+                ++rank;
+            }
+        }
+    } else {                                          // classic path: gather a and b
+        const float *a = a_all + (int64_t)row * d;
+        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+        for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+            uint32_t word = bm_cand[w0 + t];
+            while (word) {
+                const int bit = __ffs(word) - 1;
+                word &= word - 1;
+                const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+                if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+            }
         }
     }
     __syncthreads();
@@ -438,32 +533,63 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
-               const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
-               uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ cnt_tie_all,
-               int64_t d, int64_t wp, int64_t nbt)
+               const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+               const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
+               uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
+               uint32_t *__restrict__ cnt_tie_all, int64_t d, int64_t wp, int64_t nbt, int64_t nt4k)
 {
     const int row = blockIdx.y;
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
     const Sel s = sel_all[row];
     const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
     const bool all_ties = s.k3 == s.c3;
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
     uint32_t nt = 0;
-    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
-        uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
-        while (word) {
-            const int bit = __ffs(word) - 1;
-            word &= word - 1;
-            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
-            if (key > T) keep |= 1u << bit;
-            else if (key == T) tie |= 1u << bit;
+    if (hit[row]) {                                   // values come from the dense pass's stash
+        const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+        const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
+        const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
+        uint32_t ge[4];
+#pragma unroll
+        for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
+        uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            if (w0 + m >= wp) continue;
+            const uint32_t cand = bm_cand[w0 + m];
+            uint32_t word = ge[m], keep = bm_in[w0 + m], tie = 0;
+            while (word) {
+                const int bit = __ffs(word) - 1;
+                word &= word - 1;
+                if ((cand >> bit) & 1u) {
+                    const uint32_t key = key_of(stash[rank]);
+                    if (key > T) keep |= 1u << bit;
+                    else if (key == T) tie |= 1u << bit;
+                }
+                ++rank;
+            }
+            if (all_ties) keep |= tie;
+            bm_in[w0 + m] = keep;
+            bm_cand[w0 + m] = tie;
+            nt += __popc(tie);
         }
-        if (all_ties) keep |= tie;
-        bm_in[w0 + t] = keep;
-        bm_cand[w0 + t] = tie;
-        nt += __popc(tie);
+    } else {
+        const float *a = a_all + (int64_t)row * d;
+        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+        for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+            uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
+            while (word) {
+                const int bit = __ffs(word) - 1;
+                word &= word - 1;
+                const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+                if (key > T) keep |= 1u << bit;
+                else if (key == T) tie |= 1u << bit;
+            }
+            if (all_ties) keep |= tie;
+            bm_in[w0 + t] = keep;
+            bm_cand[w0 + t] = tie;
+            nt += __popc(tie);
+        }
     }
     uint32_t total;
     block_excl_scan(nt, total);
@@ -543,26 +669,42 @@ k_topk_ties(const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
 k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
-                uint32_t *__restrict__ idx_all, int64_t wp, int64_t nbt, int64_t k)
+                const uint32_t *__restrict__ hit, const uint32_t *__restrict__ bm_ge_all,
+                const float *__restrict__ stash_all, uint32_t *__restrict__ idx_all,
+                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k)
 {
     const int row = blockIdx.y;
     const uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
     uint32_t *idx = idx_all + (int64_t)row * k;
+    float *val = val_all + (int64_t)row * k;
     const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
-    uint32_t keep[4];
+    const bool stashed = hit[row] != 0;               // then the values are at hand as well
+    const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
+    const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
+    uint32_t keep[4], ge[4];
 #pragma unroll
-    for (int m = 0; m < 4; ++m) keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
+    for (int m = 0; m < 4; ++m) {
+        keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
+        ge[m] = stashed && w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
+    }
     uint32_t total;
     uint32_t rank = block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total) +
                     fin_off_all[(int64_t)row * nbt + blockIdx.x];
+    uint32_t srank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
 #pragma unroll
     for (int m = 0; m < 4; ++m) {
-        uint32_t word = keep[m];
+        uint32_t word = stashed ? ge[m] : keep[m];
         while (word) {
             const int bit = __ffs(word) - 1;
             word &= word - 1;
-            if (rank < k) idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
-            ++rank;
+            if ((keep[m] >> bit) & 1u) {
+                if (rank < k) {
+                    idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
+                    if (stashed) val[rank] = stash[srank];
+                }
+                ++rank;
+            }
+            ++srank;
         }
     }
 }
@@ -570,11 +712,13 @@ k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restri
 // ------------------------------------------------------------------------------------
 // Payload values and the state update at the kept coordinates (Algorithm 1 lines 6 / 10):
 // val = u_j = a_j - b_j, b_j += u_j.  One thread per payload entry.  grid = (ceil(k/256), rows).
+// Rows whose values were already written from the stash only update b.
 // ------------------------------------------------------------------------------------
 template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
-              const uint32_t *__restrict__ idx_all, float *__restrict__ val_all, int64_t d, int64_t k)
+              const uint32_t *__restrict__ idx_all, float *__restrict__ val_all,
+              const uint32_t *__restrict__ have_val, int64_t d, int64_t k)
 {
     const int row = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
@@ -582,6 +726,13 @@ k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
     const int64_t j = idx_all[(int64_t)row * k + t];
     if (j >= d) return;                       // caller-supplied sets are checked separately
     const float *a = a_all + (int64_t)row * d;
+    if (have_val && have_val[row]) {          // the payload values were written with the indices
+        if (HAS_B && UPDATE_B) {
+            float *b = b_all + (int64_t)row * d;
+            b[j] = __fadd_rn(b[j], val_all[(int64_t)row * k + t]);
+        }
+        return;
+    }
     float u;
     if (HAS_B) {
         float *b = b_all + (int64_t)row * d;
@@ -675,7 +826,7 @@ static void free_ws(TopkWorkspace *w)
 {
     cudaFree(w->hist); cudaFree(w->sel); cudaFree(w->bm_in); cudaFree(w->bm_cand);
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
-    cudaFree(w->bm_ge); cudaFree(w->floor_bucket); cudaFree(w->hit);
+    cudaFree(w->bm_ge); cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->ovf); cudaFree(w->stash);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
 }
@@ -704,6 +855,9 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         get((void **)&w->bm_ge, (size_t)rows * w->wp * 4);
         get((void **)&w->floor_bucket, (size_t)rows * 4);
         get((void **)&w->hit, (size_t)rows * 4);
+        get((void **)&w->ovf, (size_t)rows * 4);
+        w->nt4k = (d + kSub - 1) / kSub;
+        get((void **)&w->stash, (size_t)rows * w->nt4k * kStashCap * 4);
         if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
         get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
         get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
@@ -735,28 +889,29 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
     const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
     cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
+    cudaMemsetAsync(w->ovf, 0, (size_t)w->rows * 4, st);
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
-    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->bm_ge, w->hist, w->d, w->wp, vec_ok);
-    k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
+    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->bm_ge, w->hist, w->stash, w->ovf, w->d, w->wp, vec_ok);
+    k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->ovf, w->hit);
     k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
     k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok);
-    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->bm_in, w->bm_cand, w->hist, w->d, w->wp);
+    k_topk_split<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_ge, w->stash, w->bm_in, w->bm_cand, w->hist, w->wp, w->nt4k);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
-    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_cand, w->hist, w->d, w->wp);
+    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->stash, w->bm_cand, w->hist, w->d, w->wp, w->nt4k);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
-    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt);
+    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->stash, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt);
     k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt);
-    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->idx, w->wp, w->nbt, w->k);
+    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->hit, w->bm_ge, w->stash, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
-        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
+        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);
     else
-        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
+        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);
 }
 
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
@@ -794,9 +949,9 @@ void randk_set(TopkWorkspace *w, const uint32_t *sets, int *error_flag, cudaStre
 void randk_gather(TopkWorkspace *w, const float *a, float *b, bool update_b, cudaStream_t st)
 {
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
-    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
-    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->d, w->k);
-    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, w->d, w->k);
+    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k);
+    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k);
+    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, nullptr, w->d, w->k);
 }
 
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
