@@ -136,6 +136,39 @@ def test_c5_full_size_scales_bits_and_sampled_state():
     g.close(); o.close()
 
 
+def test_largest_dimension_one_step():
+    """d = 2^32 - 33 (the interface allows d < 2^32; uint32 coordinates, 64-bit offsets,
+    ragged last tile), n = 1, scaled sign, one step from zero state: the scale against the
+    oracle's exact l1 on the full vector, every sign word against sign(g), and the state at
+    both ends and around 2^31 against the oracle on the gathered coordinates."""
+    d = (1 << 32) - 33
+    gen = torch.Generator(device=DEV).manual_seed(77)
+    grads = torch.empty(d, dtype=torch.float32, device=DEV)
+    grads.normal_(0.0, 1e-2, generator=gen)
+    x0 = torch.zeros(d, device=DEV)
+    g = cd.CDAdam(d, 1, cd.SIGN, x0=x0)
+    del x0
+    g.step(grads)
+    bits, scale = g.last_payload(0)
+    assert scale.cpu().numpy()[0] == exact_scale(grads)
+    assert torch.equal(unpack_bits(bits, d), grads >= 0)
+    J = np.unique(np.concatenate([np.arange(0, 5000), np.arange(d - 5000, d),
+                                  np.arange((1 << 31) - 300, (1 << 31) + 300),
+                                  np.random.default_rng(5).integers(0, d, 100000)])).astype(np.int64)
+    Jt = torch.from_numpy(J).to(DEV)
+    sscale = g.last_payload(cd.SERVER)[1].cpu().numpy()
+    o = orc.Oracle(J.size, 1, orc.SIGN)
+    o.force_scales(scale.cpu().numpy().reshape(1, 1), sscale)
+    o.step(grads[Jt].cpu().numpy()[None, :])
+    del grads
+    for name in ("ghat_s", "gtil", "m", "v", "vhat", "x"):
+        assert np.array_equal(g.get_state(name)[Jt].cpu().numpy(), o.state(name)), name
+    # with n = 1 the server aggregate is the worker's payload: its scale is the worker's
+    assert sscale[0] == scale.cpu().numpy()[0]
+    g.device_status()
+    g.close(); o.close()
+
+
 # ------------------------------------------------------------------------------ C3, properties
 
 def expected_topk(u, k):
