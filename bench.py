@@ -59,13 +59,14 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def algorithmic_bytes(w):
+def algorithmic_bytes(w, bf16=False):
     """Bytes Algorithm 1 must move per step with every vector touched once.
     scaled sign: worker 4 (g) + 8 (ghat r/w) + 1/8 (bits) per worker element; server and
     update n/8 + 48.25 per element.  top-k: 8 per worker element + 44 per element."""
     from paper_2111_00705_b200 import synth
     if w.compressor == synth.SIGN:
-        return w.d * (12.25 * w.n + 48.25), w.n * w.d * 12.125
+        gb = 2.0 if bf16 else 4.0
+        return w.d * ((8.25 + gb) * w.n + 48.25), w.n * w.d * (8.125 + gb)
     if w.compressor == synth.TOPK:
         return w.d * (8.0 * w.n + 44.0), w.n * w.d * 8.0
     if w.compressor == synth.RANDK:      # sparse: 3 sectors-worth of floats per kept entry + dense AMSGrad
@@ -202,6 +203,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--compressor", default=None, choices=[None, "randk"],
                     help="randk: run the workload's shapes with the rand-k compressor (k as in C3: d/100)")
+    ap.add_argument("--grads", default="f32", choices=["f32", "bf16"],
+                    help="bf16: gradients given in bfloat16 through cdadam_step_bf16 (not the headline config)")
     ap.add_argument("--mode", default="markov", choices=["markov", "ef"],
                     help="markov = Algorithm 1 (default); ef = classical error feedback (Section 4)")
     ap.add_argument("--tile", type=int, default=0,
@@ -253,6 +256,9 @@ def main():
     # flushed between steps instead
     nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1
     grads = [w.grads(t + 1, dev).reshape(-1) for t in range(nbuf)]
+    if args.grads == "bf16":
+        grads = [g.to(torch.bfloat16) for g in grads]
+        opt.step = opt.step_bf16
     small = w.n * w.d * 4 < 512e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
     stream = torch.cuda.current_stream()
@@ -298,7 +304,7 @@ def main():
     stage_ms, psteps = opt.profile_read()
     opt.profile_enable(False)
     stage_ms = {k: v / max(psteps, 1) for k, v in stage_ms.items()}
-    step_bytes, dom_bytes = algorithmic_bytes(w)
+    step_bytes, dom_bytes = algorithmic_bytes(w, args.grads == "bf16")
     dom_name = max(stage_ms, key=stage_ms.get)
     peak, peak_kind = measured_peak()
     achieved = dom_bytes / (stage_ms[dom_name] * 1e-3) / 1e9 if stage_ms[dom_name] > 0 else 0.0
@@ -317,6 +323,8 @@ def main():
     try:
         if args.e2e_steps < 1:
             raise RuntimeError("skipped (--e2e-steps 0)")
+        if args.grads != "f32":
+            raise RuntimeError("skipped (host path takes binary32 gradients)")
         gh = [g.cpu().pin_memory() for g in grads[:1]]
         xh = torch.empty(w.d, dtype=torch.float32).pin_memory()
         opt.step_host(gh[0], xh, stream)                       # allocates the staging buffer
@@ -355,7 +363,8 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale)
-                           + ("" if args.mode == "markov" else " [error-feedback mode]"),
+                           + ("" if args.mode == "markov" else " [error-feedback mode]")
+                           + ("" if args.grads == "f32" else " [bf16 gradients]"),
                            "replicas": world,
                            "l2": "flushed between steps" if flush is not None else
                                  "inputs larger than L2 (%.2f GB of gradients per step)" % (w.n * w.d * 4 / 1e9)},

@@ -105,6 +105,16 @@ void cdadam_destroy(cdadam_ctx *ctx);
 int cdadam_step(cdadam_ctx *ctx, const float *grads, void *stream);
 
 /*
+ * The same iteration with the gradients given in bfloat16 (device, n x d 16-bit values, the
+ * upper halves of binary32 numbers).  Widening is exact, so the result is that of
+ * cdadam_step on the widened values.  The scaled-sign worker kernels read the 16-bit values
+ * directly (2 instead of 4 bytes per gradient; vectorised when the base address is a multiple
+ * of 16 bytes and d % 8 == 0); the other compressors first widen into a staging buffer owned
+ * by the context (allocated at the first such call).
+ */
+int cdadam_step_bf16(cdadam_ctx *ctx, const void *grads_bf16, void *stream);
+
+/*
  * The same iteration with the gradients in HOST memory: copies n x d floats host->device
  * into a staging buffer owned by the context (allocated at the first call), runs the step,
  * copies x_{t+1} (d floats) into x_out (host; may be NULL to skip) and waits for `stream`.

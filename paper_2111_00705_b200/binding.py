@@ -24,6 +24,7 @@ _SIGNATURES = {
                                     _c.c_float, _c.c_float, _c.c_float, _c.c_float]),
     "cdadam_destroy": (None, [_c.c_void_p]),
     "cdadam_step": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_step_bf16": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_host": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
@@ -153,6 +154,13 @@ class CDAdam:
     def step(self, grads, stream=None):
         """One iteration of Algorithm 1 on the n x d device gradients."""
         _check(lib().cdadam_step(self._h, _dev_f32(grads, self.n * self.d, "grads"), _stream(stream)))
+
+    def step_bf16(self, grads, stream=None):
+        """One iteration on n x d device gradients in bfloat16."""
+        if not (grads.is_cuda and grads.dtype == torch.bfloat16 and grads.is_contiguous()
+                and grads.numel() == self.n * self.d):
+            raise ValueError("grads must be a contiguous CUDA bfloat16 tensor of n*d elements")
+        _check(lib().cdadam_step_bf16(self._h, ctypes.c_void_p(grads.data_ptr()), _stream(stream)))
 
     def step_host(self, grads_host, x_out_host=None, stream=None):
         """The same with host gradients (pinned or pageable) and x copied back to the host."""

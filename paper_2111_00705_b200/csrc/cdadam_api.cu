@@ -280,12 +280,31 @@ void cdadam_destroy(cdadam_ctx *c)
     delete c;
 }
 
-int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
+static int ensure_stage(cdadam_ctx *c)
 {
-    if (!c || !grads) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
+    if (c->stage) return CDADAM_OK;
+    const size_t bytes = (size_t)c->n * c->d * sizeof(float);
+    cudaError_t e = cudaMalloc((void **)&c->stage, bytes);
+    if (e != cudaSuccess) { c->stage = nullptr; return fail(CDADAM_ERR_ALLOC, "staging buffer: %s", cudaGetErrorString(e)); }
+    return CDADAM_OK;
+}
+
+static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *stream)
+{
+    if (!c || !grads_in) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
-    const bool vec = aligned16(grads) && c->d % 4 == 0;
+    const float *grads = static_cast<const float *>(grads_in);
+    if (bf16 && c->comp != CDADAM_SIGN) {
+        // only the scaled-sign worker pass reads bfloat16 directly; the other compressors
+        // get an exact binary32 copy in the context's staging buffer
+        int rc = ensure_stage(c);
+        if (rc) return rc;
+        launch_widen_bf16(c->stage, grads_in, (int64_t)c->n * c->d, st);
+        grads = c->stage;
+        bf16 = false;
+    }
+    const bool vec = aligned16(grads_in) && c->d % (bf16 ? 8 : 4) == 0;
     prof_mark(c, st);
     const bool ef = c->mode == CDADAM_EF;
     const bool svec = c->d % 4 == 0;
@@ -293,7 +312,7 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
         const Tables &tb = c->ts.tb;
         const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
         float *new_scale = c->wscale[c->cur ^ 1];
-        launch_worker_sign(grads, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef, c->error_flag, st);
+        launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef, c->error_flag, st);
         prof_mark(c, st);
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
         prof_mark(c, st);
@@ -376,16 +395,18 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream)
     return CDADAM_OK;
 }
 
+int cdadam_step(cdadam_ctx *c, const float *grads, void *stream) { return step_impl(c, grads, false, stream); }
+
+int cdadam_step_bf16(cdadam_ctx *c, const void *grads, void *stream) { return step_impl(c, grads, true, stream); }
+
 int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, void *stream)
 {
     if (!c || !grads_host) return fail(CDADAM_ERR_ARG, "cdadam_step_host: NULL argument");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     const size_t bytes = (size_t)c->n * c->d * sizeof(float);
-    if (!c->stage) {
-        cudaError_t e = cudaMalloc((void **)&c->stage, bytes);
-        if (e != cudaSuccess) { c->stage = nullptr; return fail(CDADAM_ERR_ALLOC, "staging buffer: %s", cudaGetErrorString(e)); }
-    }
+    int rc0 = ensure_stage(c);
+    if (rc0) return rc0;
     CU_TRY(cudaMemcpyAsync(c->stage, grads_host, bytes, cudaMemcpyHostToDevice, st));
     int rc = cdadam_step(c, c->stage, stream);
     if (rc) return rc;

@@ -81,6 +81,19 @@ void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, floa
     else k_step_identity<false><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
 }
 
+// exact widening bfloat16 -> binary32
+__global__ void __launch_bounds__(kBlock)
+k_widen_bf16(float *__restrict__ dst, const uint16_t *__restrict__ src, int64_t count)
+{
+    for (int64_t j = (int64_t)blockIdx.x * kBlock + threadIdx.x; j < count; j += (int64_t)gridDim.x * kBlock)
+        dst[j] = __uint_as_float((uint32_t)src[j] << 16);
+}
+
+void launch_widen_bf16(float *dst, const void *src, int64_t count, cudaStream_t st)
+{
+    k_widen_bf16<<<grid_for(count), kBlock, 0, st>>>(dst, static_cast<const uint16_t *>(src), count);
+}
+
 // dst = src + dst
 __global__ void __launch_bounds__(kBlock)
 k_add_into(float *__restrict__ dst, const float *__restrict__ src, int64_t count, int vec_ok)

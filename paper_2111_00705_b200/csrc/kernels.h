@@ -7,11 +7,11 @@ namespace cdadam {
 
 // ---- scaled sign -------------------------------------------------------------------
 // Worker pass (Algorithm 1 lines 5-6) for all n workers: applies the previous payload
-// (bits in wbits, scales in scale_old) to ghat_w, forms u = g - ghat_w, packs sign(u) into
+// (bits in wbits, scales in scale_old) to ghat_w (grads: n x d binary32 or bfloat16), forms u = g - ghat_w, packs sign(u) into
 // wbits and writes per-tile double-double partial sums of |u| to wpart.  For large tiles the
 // variant with a TMA prefetch ring runs; it sets *error_flag (device) if a bounded wait on
 // a copy ran out.
-void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
+void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
                         int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st);
 // Correctly rounded scale of every (row, segment) from the partial sums.
@@ -40,6 +40,8 @@ void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, floa
                           Hyper hp, bool ef, cudaStream_t st);
 
 // ---- pieces of the error-feedback iteration with the top-k compressor ---------------------
+// dst[j] = (float)src[j] for count bfloat16 values (exact widening).
+void launch_widen_bf16(float *dst, const void *src, int64_t count, cudaStream_t st);
 // dst[j] = src[j] + dst[j] for count floats (p = g + delta, kept in the delta buffer).
 void launch_add_into(float *dst, const float *src, int64_t count, bool vec_ok, cudaStream_t st);
 // dst[idx[t]] = val ? val[t] : 0 for t < k, for `rows` rows (dst stride d, idx/val stride k).

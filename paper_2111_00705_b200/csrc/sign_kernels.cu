@@ -68,11 +68,36 @@ __device__ __forceinline__ float update_step(float gt_stored, float p, float c, 
     return gt_store;
 }
 
+// Gradient element types: binary32, or bfloat16 (the upper 16 bits of a binary32, so the
+// conversion is exact and the arithmetic that follows is unchanged).
+typedef uint16_t bf16_t;
+__device__ __forceinline__ float grad_at(const float *g, int64_t j) { return g[j]; }
+__device__ __forceinline__ float grad_at(const bf16_t *g, int64_t j)
+{
+    return __uint_as_float((uint32_t)g[j] << 16);
+}
+__device__ __forceinline__ float4 grad_ld4(const float *g) { return ld_ro4(g); }
+__device__ __forceinline__ float4 grad_ld4(const bf16_t *g)
+{
+    uint2 raw;
+    asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(raw.x), "=r"(raw.y) : "l"(g));
+    return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                       __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+}
+// four consecutive gradients from a shared-memory copy of a sub-tile
+__device__ __forceinline__ float4 grad_lds4(const float *g) { return *reinterpret_cast<const float4 *>(g); }
+__device__ __forceinline__ float4 grad_lds4(const bf16_t *g)
+{
+    const uint2 raw = *reinterpret_cast<const uint2 *>(g);
+    return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
+                       __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
+}
+
 // Scalar path of the worker pass for one tile (segment boundaries, the ragged last tile,
 // unaligned rows).  Kept out of line so that it does not shape the register allocation and
 // instruction schedule of the vector path.
-template <bool EF>
-__device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, float *__restrict__ gh,
+template <bool EF, typename G>
+__device__ __noinline__ void worker_tile_scalar(const G *__restrict__ g, float *__restrict__ gh,
                                                 uint32_t *__restrict__ bw, const float *__restrict__ so,
                                                 dd *__restrict__ part, const int64_t *__restrict__ off,
                                                 int64_t base, int64_t end, int first, int last)
@@ -89,7 +114,7 @@ __device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, flo
             gv[t] = hv[t] = sv[t] = 0.0f;
             wv[t] = 0u;
             if (j < end) {
-                gv[t] = g[j];
+                gv[t] = grad_at(g, j);
                 hv[t] = gh[j];
                 wv[t] = bw[j >> 5];
                 sv[t] = so[find_segment(off, first, last, j)];
@@ -116,7 +141,7 @@ __device__ __noinline__ void worker_tile_scalar(const float *__restrict__ g, flo
         const int64_t lo = max(off[r], base), hi = min(off[r + 1], end);
         dd acc = {0.0, 0.0};
         for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
-            dd_acc(acc, fabsf(worker_input_from_memory<EF>(g[j], gh[j])));
+            dd_acc(acc, fabsf(worker_input_from_memory<EF>(grad_at(g, j), gh[j])));
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
@@ -132,14 +157,15 @@ struct WorkerRegs {
     uint32_t ow[4];
 };
 
-__device__ __forceinline__ void worker_load(WorkerRegs &r, const float *__restrict__ g,
+template <typename G>
+__device__ __forceinline__ void worker_load(WorkerRegs &r, const G *__restrict__ g,
                                             const float *__restrict__ gh,
                                             const uint32_t *__restrict__ bw, int64_t wb, int lane)
 {
 #pragma unroll
     for (int v = 0; v < 4; ++v) {
         const int64_t j = wb + v * 128 + lane * 4;
-        r.G[v] = ld_ro4(g + j);
+        r.G[v] = grad_ld4(g + j);
         r.H[v] = ld_rw4(gh + j);
         r.ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
     }
@@ -172,9 +198,9 @@ __device__ __forceinline__ void worker_compute(WorkerRegs &r, float *__restrict_
     if (lane < 16) bw[(wb >> 5) + lane] = word;
 }
 
-template <bool EF>
+template <bool EF, typename G>
 __global__ void __launch_bounds__(kBlock, 4)
-k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
+k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
               uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
               dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
 {
@@ -182,13 +208,13 @@ k_worker_sign(const float *__restrict__ grads, float *__restrict__ ghat_w,
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
-    const float *g = grads + (int64_t)i * tb.d;
+    const G *g = grads + (int64_t)i * tb.d;
     float *gh = ghat_w + (int64_t)i * tb.d;
     uint32_t *bw = wbits + (int64_t)i * wp;
     const float *so = scale_old + (int64_t)i * tb.q;
 
     if (!(vec_ok && first == last && base + tb.tile <= tb.d)) {
-        worker_tile_scalar<EF>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+        worker_tile_scalar<EF, G>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
         return;
     }
@@ -219,9 +245,9 @@ constexpr int kRingStages = 2;
 constexpr int kRingStageBytes = 2 * kSub * (int)sizeof(float);    // g and ghat sub-tile: 32 KiB
 constexpr int kRingSmemBytes = kRingStages * kRingStageBytes;
 
-template <bool EF>
+template <bool EF, typename G>
 __global__ void __launch_bounds__(kBlock, 3)
-k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
+k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
                    uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
                    dd *__restrict__ wpart, Tables tb, int64_t wp, int *__restrict__ error_flag)
 {
@@ -231,13 +257,13 @@ k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
-    const float *g = grads + (int64_t)i * tb.d;
+    const G *g = grads + (int64_t)i * tb.d;
     float *gh = ghat_w + (int64_t)i * tb.d;
     uint32_t *bw = wbits + (int64_t)i * wp;
     const float *so = scale_old + (int64_t)i * tb.q;
 
     if (!(first == last && base + tb.tile <= tb.d)) {          // block-uniform
-        worker_tile_scalar<EF>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
+        worker_tile_scalar<EF, G>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
         return;
     }
@@ -249,10 +275,11 @@ k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
     }
     __syncthreads();
     auto refill = [&](int it, int st) {                        // one thread
+        // stage layout: the worker-state sub-tile (16 KiB), then the gradient sub-tile
         float *dst = reinterpret_cast<float *>(ring + st * kRingStageBytes);
-        mbar_arrive_expect_tx(&full[st], (uint32_t)kRingStageBytes);
-        bulk_copy_g2s(dst, g + base + (int64_t)it * kSub, kSub * sizeof(float), &full[st]);
-        bulk_copy_g2s(dst + kSub, gh + base + (int64_t)it * kSub, kSub * sizeof(float), &full[st]);
+        mbar_arrive_expect_tx(&full[st], (uint32_t)(kSub * (sizeof(float) + sizeof(G))));
+        bulk_copy_g2s(dst, gh + base + (int64_t)it * kSub, kSub * sizeof(float), &full[st]);
+        bulk_copy_g2s(dst + kSub, g + base + (int64_t)it * kSub, kSub * sizeof(G), &full[st]);
     };
     if (threadIdx.x == 0)
         for (int st = 0; st < kRingStages && st < iters; ++st) refill(st, st);
@@ -269,8 +296,8 @@ k_worker_sign_ring(const float *__restrict__ grads, float *__restrict__ ghat_w,
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             const int e = warp * kWarpSpan + v * 128 + lane * 4;
-            r.G[v] = *reinterpret_cast<const float4 *>(src + e);
-            r.H[v] = *reinterpret_cast<const float4 *>(src + kSub + e);
+            r.H[v] = *reinterpret_cast<const float4 *>(src + e);
+            r.G[v] = grad_lds4(reinterpret_cast<const G *>(src + kSub) + e);
             r.ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
         }
         __syncthreads();                                       // the stage has been read by all
@@ -605,20 +632,33 @@ k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__rest
 // ------------------------------------------------------------------------------------
 // launchers
 // ------------------------------------------------------------------------------------
-void launch_worker_sign(const float *grads, float *ghat_w, uint32_t *wbits,
-                        const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
+template <typename G>
+static void launch_worker_sign_t(const G *grads, float *ghat_w, uint32_t *wbits,
+                                 const float *scale_old, dd *wpart, const Tables &tb, int n,
+                                 int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
     if (vec_ok && tb.tile >= 4 * kSub) {
-        auto kern = ef ? k_worker_sign_ring<true> : k_worker_sign_ring<false>;
+        auto kern = ef ? k_worker_sign_ring<true, G> : k_worker_sign_ring<false, G>;
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
         kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag);
     } else if (ef) {
-        k_worker_sign<true><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+        k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
     } else {
-        k_worker_sign<false><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+        k_worker_sign<false, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
     }
+}
+
+void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
+                        const float *scale_old, dd *wpart, const Tables &tb, int n,
+                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
+{
+    if (grads_bf16)
+        launch_worker_sign_t(static_cast<const bf16_t *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
+                             vec_ok, ef, error_flag, st);
+    else
+        launch_worker_sign_t(static_cast<const float *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
+                             vec_ok, ef, error_flag, st);
 }
 
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,

@@ -210,6 +210,38 @@ def test_randk_malformed_sets_are_reported_not_dereferenced():
     assert torch.ones(4, device="cuda").sum().item() == 4
 
 
+@pytest.mark.parametrize("case", ["sign_ragged", "sign_segments", "sign_ring", "sign_ef", "topk", "identity"])
+def test_bf16_gradients_equal_the_widened_fp32_run(case):
+    """Gradients given in bfloat16: widening is exact, so payloads and state must equal the
+    oracle's on the widened values, whichever kernel reads the 16-bit data."""
+    tile, mode = 0, cd.MARKOV
+    if case == "sign_ragged":
+        w = synth.Workload("B1", 3 * 4096 + 77, 3, synth.SIGN, 4, seed=1)        # d % 8 != 0: scalar reads
+    elif case == "sign_segments":
+        w = synth.workload("C2", scale=0.01)
+    elif case == "sign_ring":
+        off = np.array([0, 1000, 40000, 3 * 32768, 5 * 32768 + 448])
+        w = synth.Workload("B3", 5 * 32768 + 448, 3, synth.SIGN, 4, offsets=off, seed=3)
+        tile = 16384
+    elif case == "sign_ef":
+        w = synth.Workload("B4", 8 * 4096, 4, synth.SIGN, 4, seed=4)
+        mode = cd.EF
+    elif case == "topk":
+        w = synth.workload("C3", scale=0.004)
+    else:
+        w = synth.Workload("B6", 5000, 3, synth.IDENTITY, 4)
+    g, o = make_pair(w, mode=mode)
+    if tile:
+        g.set_tile(tile)
+    for t in range(1, 5):
+        gb = w.grads(t, "cpu").to(torch.bfloat16)
+        g.step_bf16(gb.cuda().reshape(-1))
+        o.step(gb.to(torch.float32).numpy())
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.device_status()
+
+
 def test_identity_matches_oracle():
     w = synth.Workload("ID", 5000, 3, synth.IDENTITY, 4)
     run_free(w, 4)
