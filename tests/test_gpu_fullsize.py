@@ -24,6 +24,18 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
+@pytest.fixture(autouse=True)
+def release_cached_device_memory():
+    """These tests hold tens of GB each; the library allocates with cudaMalloc, outside torch's
+    caching allocator, so torch's cache must be returned to the driver between tests."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    yield
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
 def u32(t):
     return t.cpu().numpy().view(np.uint32)
 
