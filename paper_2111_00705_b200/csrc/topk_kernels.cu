@@ -9,6 +9,13 @@
 // bitmaps (1 bit per coordinate), so the ordered compaction (index-increasing payload) costs
 // d/8 bytes per pass instead of another pass over the data.  All counters are integer
 // atomics: the result does not depend on the order of execution.
+//
+// Normally ONE dense pass suffices: the level-1 bucket of the previous selection, lowered by
+// a margin, serves as a floor; the pass histograms and bitmaps only the coordinates at or
+// above it and keeps their values per tile, so every later pass is sparse and reads those
+// values back in order.  If fewer than k coordinates lie above the floor (or a tile cannot
+// keep its values) the classic two dense passes run instead.  The same file holds the sparse
+// server aggregation and the rand-k path, which shares the payload kernels.
 #include "topk.h"
 
 #include <algorithm>
