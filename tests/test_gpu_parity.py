@@ -371,6 +371,24 @@ def test_set_lr_and_step_host_and_params_view():
     assert g.step_count() == 2 and g.launches_per_step() >= 3
 
 
+@pytest.mark.parametrize("comp", [cd.SIGN, cd.TOPK, cd.IDENTITY])
+def test_non_finite_gradients_neither_hang_nor_fault(comp):
+    """The contract asks for finite gradients; NaN and infinities give an unspecified result
+    but must leave the device usable (no out-of-range access, no endless wait)."""
+    d, n = 3 * 4096 + 5, 3
+    g = cd.CDAdam(d, n, comp, k=100 if comp == cd.TOPK else 0)
+    grads = torch.randn(n, d, device="cuda")
+    grads[0, 5] = float("nan"); grads[1, 4097] = float("inf"); grads[2, d - 1] = -float("inf")
+    for _ in range(3):
+        g.step(grads.reshape(-1))
+    g.device_status()
+    torch.cuda.synchronize()
+    g.close()
+    ok = cd.CDAdam(64, 1, cd.SIGN)
+    ok.step(torch.ones(64, device="cuda"))
+    assert torch.isfinite(ok.params()).all()
+
+
 def test_argument_errors_are_reported_not_fatal():
     with pytest.raises(cd.CdadamError):
         cd.CDAdam(0, 4)
