@@ -164,7 +164,8 @@ int cdadam_set_mode(cdadam_ctx *ctx, int mode);
 
 /*
  * Tuning knob: the number of consecutive coordinates one thread block of the scaled-sign
- * kernels owns (a multiple of 4096, at most 262144; 0 = chosen from d and q, the default).
+ * kernels owns (a multiple of 4096, at most 262144; 0 = chosen from d and q, separately for
+ * the worker pass and for the server side, the default).
  * Results do not depend on it.  Tiles of 16384 coordinates or more select the worker kernel
  * with the asynchronous-copy prefetch ring.  Only before the first step; synchronous.
  */

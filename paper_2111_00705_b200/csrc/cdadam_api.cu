@@ -46,13 +46,19 @@ struct DeviceGuard {
     ~DeviceGuard() { if (switched) cudaSetDevice(prev); }
 };
 
-// Tile size, a multiple of kSub.  Larger tiles amortise the per-block reduction and make the
-// streams longer, but every tile that contains a segment boundary takes the scalar path, so
-// the tile is kept small enough that such tiles hold at most about 2 % of the coordinates.
-int choose_tile(int64_t d, int q)
+// Tile sizes, multiples of kSub.  Larger tiles amortise the per-block reduction, make the
+// streams longer and (from 4 sub-tiles on) enable the worker pass's prefetch ring; but every
+// tile that contains a segment boundary takes the scalar path, and a row needs enough tiles
+// to fill the machine.  The scalar path of the server pass loops over the n workers per
+// coordinate and is the costlier one, so the server side (server pass, update pass) gets its
+// own, more cautious, tile size: `slack` bounds 1 / (share of coordinates in cut tiles).
+int choose_tile(int64_t d, int q, bool server_side)
 {
+    const int64_t slack = server_side ? 50 : 16;
     int tile = kSub;
-    while (tile < 4 * kSub && (int64_t)(q - 1) * (2 * tile) * 50 <= d && d >= (int64_t)tile * 2 * 2048) tile *= 2;
+    if (d >= ((int64_t)1 << 23) && (int64_t)(q - 1) * (2 * kSub) * slack <= d && !server_side) tile = 2 * kSub;
+    if (d >= ((int64_t)1 << 24) && (int64_t)(q - 1) * (2 * kSub) * slack <= d) tile = 2 * kSub;
+    if (d >= ((int64_t)1 << 25) && (int64_t)(q - 1) * (4 * kSub) * slack <= d) tile = 4 * kSub;
     return tile;
 }
 
@@ -125,7 +131,8 @@ struct cdadam_ctx {
     int tile_override = 0;  // 0 = choose from d and q
     int mode = CDADAM_MARKOV;
     Hyper hp{};
-    TableSet ts;
+    TableSet ts;            // worker pass
+    TableSet ts_s;          // server pass and update pass
     float *ghat_w = nullptr, *ghat_s = nullptr, *gtil = nullptr;
     float *m = nullptr, *v = nullptr, *vhat = nullptr, *x = nullptr;
     // scaled sign
@@ -170,7 +177,7 @@ int alloc_sign_buffers(cdadam_ctx *c)
     if ((rc = dev_zalloc(&c->zero_scale, (size_t)c->n * q))) return rc;
     if ((rc = dev_zalloc(&c->sscale, (size_t)q))) return rc;
     if ((rc = dev_zalloc(&c->wpart, (size_t)c->n * c->ts.tb.nparts))) return rc;
-    if ((rc = dev_zalloc(&c->spart, (size_t)c->ts.tb.nparts))) return rc;
+    if ((rc = dev_zalloc(&c->spart, (size_t)c->ts_s.tb.nparts))) return rc;
     return CDADAM_OK;
 }
 
@@ -249,7 +256,8 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
         if (compressor == CDADAM_SIGN) {
             if ((rc = dev_zalloc(&c->wbits, (size_t)n * c->wp))) break;
             if ((rc = dev_zalloc(&c->sbits, (size_t)c->wp))) break;
-            if ((rc = c->ts.build(d, 1, flat, choose_tile(d, 1), nullptr, false))) break;
+            if ((rc = c->ts.build(d, 1, flat, choose_tile(d, 1, false), nullptr, false))) break;
+            if ((rc = c->ts_s.build(d, 1, flat, choose_tile(d, 1, true), nullptr, false))) break;
             if ((rc = alloc_sign_buffers(c))) break;
         } else if (compressor == CDADAM_RANDK) {
             if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n, nullptr, nullptr, false))) { fail(rc, "rand-k payload allocation failed"); break; }
@@ -277,6 +285,7 @@ void cdadam_destroy(cdadam_ctx *c)
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     for (cudaEvent_t e : c->prof_pool) cudaEventDestroy(e);
     c->ts.release(nullptr, false);
+    c->ts_s.release(nullptr, false);
     delete c;
 }
 
@@ -309,18 +318,18 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
     const bool ef = c->mode == CDADAM_EF;
     const bool svec = c->d % 4 == 0;
     if (c->comp == CDADAM_SIGN) {
-        const Tables &tb = c->ts.tb;
+        const Tables &tb = c->ts.tb, &tbs = c->ts_s.tb;
         const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
         float *new_scale = c->wscale[c->cur ^ 1];
         launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef, c->error_flag, st);
         prof_mark(c, st);
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
         prof_mark(c, st);
-        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tb, c->n, c->wp, svec, ef, st);
+        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, ef, st);
         prof_mark(c, st);
-        launch_finalize_scales(c->spart, c->sscale, tb, 1, st);
+        launch_finalize_scales(c->spart, c->sscale, tbs, 1, st);
         prof_mark(c, st);
-        launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tb, c->hp, svec, ef, st);
+        launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, ef, st);
         prof_mark(c, st);
         c->cur ^= 1;
         c->pending = true;
@@ -434,7 +443,9 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
     DeviceGuard guard(c->device);
     CU_TRY(cudaDeviceSynchronize());
-    int rc = c->ts.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q), nullptr, false);
+    int rc = c->ts.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q, false), nullptr, false);
+    if (rc) return rc;
+    rc = c->ts_s.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q, true), nullptr, false);
     if (rc) return rc;
     return alloc_sign_buffers(c);
 }
@@ -602,7 +613,7 @@ int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offset
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing");
     cudaStream_t st = (cudaStream_t)stream;
     TableSet ts;
-    int rc = ts.build(d, q, offsets, choose_tile(d, q), st, true);
+    int rc = ts.build(d, q, offsets, choose_tile(d, q, false), st, true);
     if (rc) return rc;
     dd *part = nullptr;
     cudaError_t e = cudaMallocAsync((void **)&part, (size_t)ts.tb.nparts * sizeof(dd), st);
