@@ -389,6 +389,33 @@ def test_non_finite_gradients_neither_hang_nor_fault(comp):
     assert torch.isfinite(ok.params()).all()
 
 
+def test_stage_timing_and_late_configuration_calls():
+    g = cd.CDAdam(3 * 4096, 2, cd.SIGN)
+    grads = torch.randn(2 * 3 * 4096, device="cuda")
+    g.profile_enable(True)
+    for _ in range(4):
+        g.step(grads)
+    ms, steps = g.profile_read()
+    assert steps == 4 and set(ms) == {"k_worker_sign", "k_finalize_scales(workers)", "k_server_sign",
+                                      "k_finalize_scales(server)", "k_update_sign"}
+    assert all(v > 0 for v in ms.values())
+    assert g.profile_read()[1] == 0                       # reading forgets the events
+    g.profile_enable(False)
+    assert g.launches_per_step() == 5
+    with pytest.raises(cd.CdadamError):
+        g.set_tile(8192)                                  # after the first step
+    assert cd.lib().cdadam_set_mode(g._h, cd.EF) == cd.ERR_STATE
+    h = cd.CDAdam(100, 2, cd.TOPK, k=3)
+    with pytest.raises(cd.CdadamError):
+        h.set_tile(4096)                                  # tiles belong to scaled sign
+    f = cd.CDAdam(100, 2, cd.SIGN)
+    with pytest.raises(cd.CdadamError):
+        f.set_tile(1000)                                  # not a multiple of 4096
+    assert cd.lib().cdadam_set_mode(f._h, 7) == cd.ERR_ARG
+    with pytest.raises(ValueError):
+        f.step_bf16(torch.zeros(200, device="cuda"))      # wrong dtype is caught by the binding
+
+
 def test_argument_errors_are_reported_not_fatal():
     with pytest.raises(cd.CdadamError):
         cd.CDAdam(0, 4)
