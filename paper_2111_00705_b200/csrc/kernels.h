@@ -10,18 +10,23 @@ namespace cdadam {
 // (bits in wbits, scales in scale_old) to ghat_w (grads: n x d binary32 or bfloat16), forms u = g - ghat_w, packs sign(u) into
 // wbits and writes per-tile double-double partial sums of |u| to wpart.  For large tiles the
 // variant with a TMA prefetch ring runs; it sets *error_flag (device) if a bounded wait on
-// a copy ran out.
+// a copy ran out.  With scale_new != NULL the block that completes a (worker, segment) also
+// turns its partial sums into the scale (done: n x q zeroed counters, left zeroed), and no
+// launch_finalize_scales is needed.
 void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st);
+                        int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
+                        unsigned int *done, cudaStream_t st);
 // Correctly rounded scale of every (row, segment) from the partial sums.
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
                             cudaStream_t st);
 // Server pass A (lines 8-9): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
-// sign(w) into sbits and writes partial sums of |w| to spart.
+// sign(w) into sbits and writes partial sums of |w| to spart.  sscale != NULL: the scales are
+// finished in the same launch (done: q zeroed counters), as in the worker pass.
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, bool ef, cudaStream_t st);
+                        int n, int64_t wp, bool vec_ok, bool ef, float *sscale, unsigned int *done,
+                        cudaStream_t st);
 // Server pass B and worker update (lines 10, 12-16): gtil += decode(c); AMSGrad.
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
                         float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,

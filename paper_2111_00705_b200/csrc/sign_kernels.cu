@@ -97,6 +97,48 @@ __device__ __forceinline__ float4 grad_lds4(const bf16_t *g)
                        __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
 }
 
+// ------------------------------------------------------------------------------------
+// Scale of one (row, segment) without a launch of its own: every block that has written a
+// partial l1 sum of the segment takes a ticket, and the block that takes the last one adds
+// the partial sums (fixed thread mapping and tree, hence the same result whichever block
+// it is), rounds and divides as k_finalize_scales does, and puts the counter back to zero.
+// No block waits for another.  `part`, `scales` and `done` are the row's.  All threads of the
+// block call it, after thread 0 has written the block's partial sum.
+// ------------------------------------------------------------------------------------
+__device__ __noinline__ void finish_segment(const dd *part, float *scales, unsigned int *done, int r,
+                                            const int64_t *__restrict__ off,
+                                            const int32_t *__restrict__ tile_first,
+                                            const int64_t *__restrict__ pbase, int tile)
+{
+    __shared__ int is_last;
+    const int64_t lo = off[r], hi = off[r + 1];
+    const int64_t T0 = lo / tile, T1 = (hi - 1) / tile;
+    __syncthreads();                 // the previous call's readers of is_last are done
+    if (threadIdx.x == 0) {
+        __threadfence();             // this block's partial sum is visible before its ticket
+        is_last = atomicAdd(done + r, 1u) == (unsigned int)(T1 - T0);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    dd a0 = {0.0, 0.0}, a1 = {0.0, 0.0};
+    for (int64_t T = T0 + threadIdx.x; T <= T1; T += 2 * kBlock) {
+        const double2 p0 = __ldcg(reinterpret_cast<const double2 *>(part + pbase[T] + (r - tile_first[T])));
+        a0 = dd_add(a0, dd{p0.x, p0.y});
+        const int64_t U = T + kBlock;
+        if (U <= T1) {
+            const double2 p1 = __ldcg(reinterpret_cast<const double2 *>(part + pbase[U] + (r - tile_first[U])));
+            a1 = dd_add(a1, dd{p1.x, p1.y});
+        }
+    }
+    a0 = block_sum<kBlock>(dd_add(a0, a1));
+    if (threadIdx.x == 0) {
+        const double l1 = __dadd_rn(a0.hi, a0.lo);
+        scales[r] = __double2float_rn(__ddiv_rn(l1, (double)(hi - lo)));
+        done[r] = 0u;
+    }
+}
+
 // Scalar path of the worker pass for one tile (segment boundaries, the ragged last tile,
 // unaligned rows).  Kept out of line so that it does not shape the register allocation and
 // instruction schedule of the vector path.
@@ -206,7 +248,8 @@ template <bool EF, typename G>
 __global__ void __launch_bounds__(kBlock, 4)
 k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
               uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
-              dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok)
+              dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok,
+              float *__restrict__ scale_new, unsigned int *__restrict__ done)
 {
     const int i = blockIdx.y;
     const int64_t T = tb.order[blockIdx.x];
@@ -220,20 +263,24 @@ k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
     if (!(vec_ok && first == last && base + tb.tile <= tb.d)) {
         worker_tile_scalar<EF, G>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
-        return;
+    } else {
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const float s = so[first];
+        const int iters = tb.tile / kSub;
+        dd acc = {0.0, 0.0};
+        for (int it = 0; it < iters; ++it) {
+            WorkerRegs r;
+            const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
+            worker_load(r, g, gh, bw, wb, lane);
+            worker_compute<EF>(r, gh, bw, wb, lane, s, acc);
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
     }
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const float s = so[first];
-    const int iters = tb.tile / kSub;
-    dd acc = {0.0, 0.0};
-    for (int it = 0; it < iters; ++it) {
-        WorkerRegs r;
-        const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
-        worker_load(r, g, gh, bw, wb, lane);
-        worker_compute<EF>(r, gh, bw, wb, lane, s, acc);
-    }
-    acc = block_sum<kBlock>(acc);
-    if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
+    if (scale_new)                                             // launch-uniform
+        for (int r = first; r <= last; ++r)
+            finish_segment(wpart + (int64_t)i * tb.nparts, scale_new + (int64_t)i * tb.q,
+                           done + (int64_t)i * tb.q, r, tb.off, tb.tile_first, tb.pbase, tb.tile);
 }
 
 // ------------------------------------------------------------------------------------
@@ -253,7 +300,8 @@ template <bool EF, typename G>
 __global__ void __launch_bounds__(kBlock, 3)
 k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
                    uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
-                   dd *__restrict__ wpart, Tables tb, int64_t wp, int *__restrict__ error_flag)
+                   dd *__restrict__ wpart, Tables tb, int64_t wp, int *__restrict__ error_flag,
+                   float *__restrict__ scale_new, unsigned int *__restrict__ done)
 {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) uint64_t full[kRingStages];
@@ -269,6 +317,10 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
     if (!(first == last && base + tb.tile <= tb.d)) {          // block-uniform
         worker_tile_scalar<EF, G>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
+        if (scale_new)
+            for (int r = first; r <= last; ++r)
+                finish_segment(wpart + (int64_t)i * tb.nparts, scale_new + (int64_t)i * tb.q,
+                               done + (int64_t)i * tb.q, r, tb.off, tb.tile_first, tb.pbase, tb.tile);
         return;
     }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -310,7 +362,8 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
     }
     if (!arrived) {
         // A copy did not complete in time: report it, give the copies still in flight a
-        // bounded chance to land before this block's shared memory is released, and leave.
+        // bounded chance to land before this block's shared memory is released, and leave
+        // (the step's results are void; the scale of this segment is not finished).
         if (threadIdx.x == 0) atomicExch(error_flag, 1);
         for (int st = 0; st < kRingStages; ++st) {
             mbar_wait_bounded(&full[st], 0u);
@@ -320,6 +373,9 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
     }
     acc = block_sum<kBlock>(acc);
     if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
+    if (scale_new)
+        finish_segment(wpart + (int64_t)i * tb.nparts, scale_new + (int64_t)i * tb.q,
+                       done + (int64_t)i * tb.q, first, tb.off, tb.tile_first, tb.pbase, tb.tile);
 }
 
 // ------------------------------------------------------------------------------------
@@ -360,7 +416,8 @@ __global__ void __launch_bounds__(kBlock)
 k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
               float *__restrict__ ghat_s, const float *__restrict__ gtil,
               uint32_t *__restrict__ sbits, dd *__restrict__ spart, Tables tb, int n,
-              int64_t wp, int vec_ok, int n_pow2)
+              int64_t wp, int vec_ok, int n_pow2, float *__restrict__ sscale,
+              unsigned int *__restrict__ done)
 {
     __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
     __shared__ float ssm[kNC];
@@ -462,6 +519,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         }
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[0] = acc;
+        if (sscale) finish_segment(spart, sscale, done, first, tb.off, tb.tile_first, tb.pbase, tb.tile);
         return;
     }
 
@@ -492,6 +550,9 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
+    if (sscale)
+        for (int r = first; r <= last; ++r)
+            finish_segment(spart, sscale, done, r, tb.off, tb.tile_first, tb.pbase, tb.tile);
 }
 
 // ------------------------------------------------------------------------------------
@@ -639,30 +700,35 @@ k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__rest
 template <typename G>
 static void launch_worker_sign_t(const G *grads, float *ghat_w, uint32_t *wbits,
                                  const float *scale_old, dd *wpart, const Tables &tb, int n,
-                                 int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
+                                 int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
+                                 unsigned int *done, cudaStream_t st)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
     if (vec_ok && tb.tile >= 4 * kSub) {
         auto kern = ef ? k_worker_sign_ring<true, G> : k_worker_sign_ring<false, G>;
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
-        kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag);
+        kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag,
+                                                   scale_new, done);
     } else if (ef) {
-        k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+        k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
+                                                        scale_new, done);
     } else {
-        k_worker_sign<false, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok);
+        k_worker_sign<false, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
+                                                         scale_new, done);
     }
 }
 
 void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
-                        int64_t wp, bool vec_ok, bool ef, int *error_flag, cudaStream_t st)
+                        int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
+                        unsigned int *done, cudaStream_t st)
 {
     if (grads_bf16)
         launch_worker_sign_t(static_cast<const bf16_t *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
-                             vec_ok, ef, error_flag, st);
+                             vec_ok, ef, error_flag, scale_new, done, st);
     else
         launch_worker_sign_t(static_cast<const float *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
-                             vec_ok, ef, error_flag, st);
+                             vec_ok, ef, error_flag, scale_new, done, st);
 }
 
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
@@ -674,15 +740,16 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, bool ef, cudaStream_t st)
+                        int n, int64_t wp, bool vec_ok, bool ef, float *sscale, unsigned int *done,
+                        cudaStream_t st)
 {
     const int pow2 = (n & (n - 1)) == 0;
     if (ef)
         k_server_sign<2, true><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                                       spart, tb, n, wp, vec_ok, pow2);
+                                                                       spart, tb, n, wp, vec_ok, pow2, sscale, done);
     else
         k_server_sign<2, false><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                                        spart, tb, n, wp, vec_ok, pow2);
+                                                                        spart, tb, n, wp, vec_ok, pow2, sscale, done);
 }
 
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,

@@ -67,11 +67,13 @@ def check_state(g, o, tol, exact=False):
     return worst
 
 
-def run_free(w, steps, exact=True, tile=0, **kw):
+def run_free(w, steps, exact=True, tile=0, launches=None, **kw):
     """Free run: both sides step independently from the same inputs."""
     g, o = make_pair(w, **kw)
     if tile:
         g.set_tile(tile)
+    if launches is not None:
+        assert g.launches_per_step() == launches
     for t in range(1, steps + 1):
         grads = w.grads(t, "cpu")
         g.step(grads.cuda())
@@ -155,6 +157,18 @@ def test_sign_worker_counts_cover_table_and_sequential_server_sums(n):
     added one by one; above 32: the staged kernel; odd n: true division by n."""
     off = np.array([0, 5000, 3 * 4096 + 100, 5 * 4096])
     run_free(synth.Workload("N", 5 * 4096, n, synth.SIGN, 3, offsets=off, seed=n), 3)
+
+
+@pytest.mark.parametrize("n,launches", [(4, 3), (5, 5)])
+@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
+def test_scales_finished_in_the_passes_or_by_their_own_kernel(n, launches, mode):
+    """148 tiles per worker: with 4 workers the worker pass is one wave of blocks and finishes
+    its scales itself (tickets, last block adds); with 5 the separate kernel does.  Segments
+    that cut tiles put several tickets on one block."""
+    d = 148 * 4096
+    off = np.array([0, 5, 4096, 9000, 300001, 300002, d - 4097, d])
+    run_free(synth.Workload("F1", d, n, synth.SIGN, 4, offsets=off, seed=11), 4, mode=mode, launches=launches)
+    run_free(synth.Workload("F2", d - 3, n, synth.SIGN, 3, seed=12), 3, mode=mode, launches=launches)
 
 
 @pytest.mark.parametrize("case", ["sign_flat", "sign_segments", "sign_ring", "topk", "identity"])
@@ -390,18 +404,22 @@ def test_non_finite_gradients_neither_hang_nor_fault(comp):
 
 
 def test_stage_timing_and_late_configuration_calls():
-    g = cd.CDAdam(3 * 4096, 2, cd.SIGN)
-    grads = torch.randn(2 * 3 * 4096, device="cuda")
-    g.profile_enable(True)
-    for _ in range(4):
-        g.step(grads)
-    ms, steps = g.profile_read()
-    assert steps == 4 and set(ms) == {"k_worker_sign", "k_finalize_scales(workers)", "k_server_sign",
-                                      "k_finalize_scales(server)", "k_update_sign"}
-    assert all(v > 0 for v in ms.values())
-    assert g.profile_read()[1] == 0                       # reading forgets the events
-    g.profile_enable(False)
-    assert g.launches_per_step() == 5
+    # a grid of one wave finishes its scales inside the passes (3 launches); larger ones
+    # use the separate scale kernel (5 launches)
+    for d, names in ((3 * 4096, {"k_worker_sign", "k_server_sign", "k_update_sign"}),
+                     (400 * 4096, {"k_worker_sign", "k_finalize_scales(workers)", "k_server_sign",
+                                   "k_finalize_scales(server)", "k_update_sign"})):
+        g = cd.CDAdam(d, 2, cd.SIGN)
+        grads = torch.randn(2 * d, device="cuda")
+        g.profile_enable(True)
+        for _ in range(4):
+            g.step(grads)
+        ms, steps = g.profile_read()
+        assert steps == 4 and set(ms) == names
+        assert all(v > 0 for v in ms.values())
+        assert g.profile_read()[1] == 0                   # reading forgets the events
+        g.profile_enable(False)
+        assert g.launches_per_step() == len(names)
     with pytest.raises(cd.CdadamError):
         g.set_tile(8192)                                  # after the first step
     assert cd.lib().cdadam_set_mode(g._h, cd.EF) == cd.ERR_STATE
