@@ -99,8 +99,14 @@ void cdadam_destroy(cdadam_ctx *ctx);
  *           the work queued on `stream` has completed; never written.  A base address
  *           that is a multiple of 16 bytes together with d % 4 == 0 selects the
  *           vectorised kernels; any other alignment is accepted and gives the same result.
- *   stream  cudaStream_t
- * Allocates nothing.  After the stream has completed, cdadam_params() holds x_{t+1}.
+ *   stream  cudaStream_t; must not be under stream capture (CDADAM_ERR_STATE, nothing
+ *           queued): launch arguments alternate between steps, so a step replayed from a
+ *           caller's graph would be wrong
+ * Allocates no device memory.  Where the step is launch-bound (scaled sign, every pass a
+ * single wave of blocks, about n*d <= 2.4e6) the scales are finished inside the passes
+ * (3 launches instead of 5) and, from the second step on the same gradient buffer, the
+ * launches are replayed from a CUDA graph owned by the context.  After the stream has
+ * completed, cdadam_params() holds x_{t+1}.
  */
 int cdadam_step(cdadam_ctx *ctx, const float *grads, void *stream);
 

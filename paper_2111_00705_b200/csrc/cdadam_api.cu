@@ -151,6 +151,20 @@ struct cdadam_ctx {
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
     // host-gradient staging
     float *stage = nullptr;
+    // Replay of the scaled-sign step as a CUDA graph where the step is launch-bound (grids of
+    // one wave).  A graph is recorded for a gradient buffer seen twice; the key holds every
+    // launch argument that changes between steps.
+    struct StepGraph {
+        const void *grads = nullptr;
+        bool bf16 = false, pending = false;
+        int cur = 0, hits = 0;
+        uint64_t stamp = 0;
+        cudaGraphExec_t exec = nullptr;
+    };
+    StepGraph graphs[4];
+    uint64_t graph_clock = 0;
+    cudaStream_t cap_stream = nullptr;
+    bool graphs_ok = true;       // cleared for good when recording fails once
     // optional per-kernel timing: events[step][0..nslots] recorded around every stage
     bool prof_on = false;
     std::vector<cudaEvent_t> prof_ev;   // groups of (nslots + 1) events, one group per step
@@ -219,6 +233,86 @@ void prof_mark(cdadam_ctx *c, cudaStream_t st)
     else if (cudaEventCreate(&e) != cudaSuccess) return;
     cudaEventRecord(e, st);
     c->prof_ev.push_back(e);
+}
+
+void drop_graphs(cdadam_ctx *c)
+{
+    for (auto &g : c->graphs) {
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+        g = cdadam_ctx::StepGraph{};
+    }
+}
+
+// The three to five launches of one scaled-sign step, queued on st.  Changes no host state.
+void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
+{
+    const Tables &tb = c->ts.tb, &tbs = c->ts_s.tb;
+    const bool ef = c->mode == CDADAM_EF;
+    const bool svec = c->d % 4 == 0;
+    const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
+    float *new_scale = c->wscale[c->cur ^ 1];
+    const bool fuse = c->fuse_finish;
+    launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef,
+                       c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
+    prof_mark(c, st);
+    if (!fuse) {
+        launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
+        prof_mark(c, st);
+    }
+    launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, ef,
+                       fuse ? c->sscale : nullptr, c->sdone, st);
+    prof_mark(c, st);
+    if (!fuse) {
+        launch_finalize_scales(c->spart, c->sscale, tbs, 1, st);
+        prof_mark(c, st);
+    }
+    launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, ef, st);
+    prof_mark(c, st);
+}
+
+// Launch-bound steps: replays the recorded graph of this step on st and returns true, or
+// returns false when the step has to be queued launch by launch (first sighting of the
+// gradient buffer, timing on, recording unavailable).
+bool replay_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
+{
+    if (!c->fuse_finish || !c->graphs_ok || c->prof_on) return false;
+    cdadam_ctx::StepGraph *slot = nullptr, *oldest = &c->graphs[0];
+    for (auto &g : c->graphs) {
+        if (g.hits && g.grads == grads_in && g.bf16 == bf16 && g.pending == c->pending && g.cur == c->cur) slot = &g;
+        if (g.stamp < oldest->stamp) oldest = &g;
+    }
+    if (!slot) {                                               // remember the sighting only
+        if (oldest->exec) cudaGraphExecDestroy(oldest->exec);
+        *oldest = cdadam_ctx::StepGraph{};
+        oldest->grads = grads_in; oldest->bf16 = bf16; oldest->pending = c->pending; oldest->cur = c->cur;
+        oldest->hits = 1; oldest->stamp = ++c->graph_clock;
+        return false;
+    }
+    slot->hits += 1;
+    slot->stamp = ++c->graph_clock;
+    if (!slot->exec) {
+        cudaGraph_t graph = nullptr;
+        bool ok = c->cap_stream || cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) == cudaSuccess;
+        ok = ok && cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+        if (ok) {
+            enqueue_sign_step(c, grads_in, bf16, vec, c->cap_stream);
+            ok = cudaStreamEndCapture(c->cap_stream, &graph) == cudaSuccess && graph;
+        }
+        ok = ok && cudaGraphInstantiate(&slot->exec, graph, 0) == cudaSuccess;
+        if (graph) cudaGraphDestroy(graph);
+        if (!ok) {
+            cudaGetLastError();
+            slot->exec = nullptr;
+            c->graphs_ok = false;
+            return false;
+        }
+    }
+    if (cudaGraphLaunch(slot->exec, st) != cudaSuccess) {
+        cudaGetLastError();
+        c->graphs_ok = false;
+        return false;
+    }
+    return true;
 }
 
 int check_launch(const char *what)
@@ -293,6 +387,8 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     cudaFree(c->wdone); cudaFree(c->sdone);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
+    drop_graphs(c);
+    if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     for (cudaEvent_t e : c->prof_pool) cudaEventDestroy(e);
     c->ts.release(nullptr, false);
@@ -314,6 +410,14 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
     if (!c || !grads_in) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
+    {
+        // Launch arguments alternate from step to step (double-buffered scales, the deferred
+        // payload), so a step recorded into a caller's graph would replay wrongly.
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) cudaGetLastError();
+        else if (cs != cudaStreamCaptureStatusNone)
+            return fail(CDADAM_ERR_STATE, "cdadam_step: the stream is being captured; a step cannot be part of a caller's graph");
+    }
     const float *grads = static_cast<const float *>(grads_in);
     if (bf16 && c->comp != CDADAM_SIGN) {
         // only the scaled-sign worker pass reads bfloat16 directly; the other compressors
@@ -329,26 +433,7 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
     const bool ef = c->mode == CDADAM_EF;
     const bool svec = c->d % 4 == 0;
     if (c->comp == CDADAM_SIGN) {
-        const Tables &tb = c->ts.tb, &tbs = c->ts_s.tb;
-        const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
-        float *new_scale = c->wscale[c->cur ^ 1];
-        const bool fuse = c->fuse_finish;
-        launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef,
-                           c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
-        prof_mark(c, st);
-        if (!fuse) {
-            launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
-            prof_mark(c, st);
-        }
-        launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, ef,
-                           fuse ? c->sscale : nullptr, c->sdone, st);
-        prof_mark(c, st);
-        if (!fuse) {
-            launch_finalize_scales(c->spart, c->sscale, tbs, 1, st);
-            prof_mark(c, st);
-        }
-        launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, ef, st);
-        prof_mark(c, st);
+        if (!replay_sign_step(c, grads_in, bf16, vec, st)) enqueue_sign_step(c, grads_in, bf16, vec, st);
         c->cur ^= 1;
         c->pending = true;
     } else if (c->comp == CDADAM_TOPK && !ef) {
@@ -503,6 +588,7 @@ int cdadam_set_mode(cdadam_ctx *c, int mode)
 int cdadam_set_lr(cdadam_ctx *c, float lr)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_lr: NULL context");
+    if (lr != c->hp.lr) drop_graphs(c);       // the step size is a launch argument
     c->hp.lr = lr;
     return CDADAM_OK;
 }

@@ -6,6 +6,8 @@ same state; every float state vector within max relative error 1e-5 after every 
 free run and 1e-4 after the last one, relative error = max_j |a_j - b_j| / max(|b_j|, tau)
 with tau = 1e-6 * max_j |b_j| so that exact zeros do not dominate.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -401,6 +403,58 @@ def test_non_finite_gradients_neither_hang_nor_fault(comp):
     ok = cd.CDAdam(64, 1, cd.SIGN)
     ok.step(torch.ones(64, device="cuda"))
     assert torch.isfinite(ok.params()).all()
+
+
+@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
+def test_replayed_launch_bound_steps_match_oracle(mode):
+    """Small problems replay their launches from a recorded graph once a gradient buffer has
+    been seen twice.  Two buffers in turn, a side stream, a read of the worker states (which
+    applies the deferred payload and changes the next step's arguments) and a change of step
+    size (a launch argument) in between: every payload and state vector against the oracle."""
+    w = synth.Workload("G1", 5 * 4096 + 13, 4, synth.SIGN, 14, offsets=np.array([0, 4000, 9000, 5 * 4096 + 13]), seed=21)
+    g, o = make_pair(w, mode=mode)
+    bufs = [torch.empty(w.n * w.d, device="cuda") for _ in range(2)]
+    side = torch.cuda.Stream()
+    for t in range(1, 15):
+        grads = w.grads(t, "cpu")
+        buf = bufs[0] if t < 6 else bufs[t % 2]
+        buf.copy_(grads.reshape(-1))
+        if t == 9:
+            g.set_lr(5e-4); o.set_lr(5e-4)
+        if t in (7, 8, 12):
+            torch.cuda.synchronize()
+            with torch.cuda.stream(side):
+                g.step(buf, stream=side)
+            side.synchronize()
+        else:
+            g.step(buf)
+        o.step(grads.numpy())
+        torch.cuda.synchronize()
+        check_payloads(g, o, w)
+        if t in (4, 10, 14):
+            check_state(g, o, STEP_TOL, exact=True)
+        else:
+            for name in ("x", "m", "v", "vhat", "gtil"):
+                assert np.array_equal(g.get_state(name).cpu().numpy().ravel(), o.state(name).ravel()), (t, name)
+    g.device_status()
+    g.close(); o.close()
+
+
+def test_step_on_a_capturing_stream_is_refused():
+    g = cd.CDAdam(4096, 2, cd.SIGN)
+    grads = torch.randn(2 * 4096, device="cuda")
+    g.step(grads)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        graph.capture_begin()
+        rc = cd.lib().cdadam_step(g._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(side.cuda_stream))
+        graph.capture_end()
+    assert rc == cd.ERR_STATE and "captur" in cd.last_error()
+    g.step(grads)                                         # the context is unharmed
+    assert g.step_count() == 2
+    g.close()
 
 
 def test_stage_timing_and_late_configuration_calls():
