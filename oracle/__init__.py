@@ -6,7 +6,7 @@ imports this package; it is used by the tests, the smoke check and the CPU-basel
 the benchmark only.
 """
 from .oracle import (Oracle, build, compress_sign, compress_topk, compress_randk, l1_exact,
-                     SIGN, TOPK, IDENTITY, RANDK, MARKOV, EF, STATE_NAMES)
+                     SIGN, TOPK, IDENTITY, RANDK, MARKOV, EF, NAIVE, STATE_NAMES)
 
 __all__ = ["Oracle", "build", "compress_sign", "compress_topk", "compress_randk", "l1_exact",
-           "SIGN", "TOPK", "IDENTITY", "RANDK", "MARKOV", "EF", "STATE_NAMES"]
+           "SIGN", "TOPK", "IDENTITY", "RANDK", "MARKOV", "EF", "NAIVE", "STATE_NAMES"]

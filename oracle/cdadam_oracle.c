@@ -21,7 +21,10 @@
  * Parity pins (tests/, CPU only): exact rational worked examples, math.fsum for the exact
  * l1 sum, brute-force sort for top-k, the closed form of Appendix A for the scaled-sign
  * error, the Markov identity ghat_t - ghat_{t-1} = c_t, and an independently written
- * vanilla AMSGrad for the identity compressor.  No function here is "parity unpinned".
+ * vanilla AMSGrad for the identity compressor; for the naive-compression mode a second
+ * hand-worked step and its statelessness; for the decoupled weight decay and the step-size
+ * milestones the closed form x_t = x_1 prod (1 - alpha_t lambda) at zero gradients and an
+ * independently written recursion.  No function here is "parity unpinned".
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -29,7 +32,7 @@
 #include <math.h>
 
 enum { ORC_SIGN = 0, ORC_TOPK = 1, ORC_IDENTITY = 2, ORC_RANDK = 3 };
-enum { ORC_MARKOV = 0, ORC_EF = 1 };
+enum { ORC_MARKOV = 0, ORC_EF = 1, ORC_NAIVE = 2 };
 
 /* ------------------------------------------------------------------------------------ */
 /* Exact l1 norm of binary32 data.                                                        */
@@ -195,6 +198,10 @@ void oracle_compress_randk(const float *x, int64_t d, int64_t k, const uint32_t 
 typedef struct oracle_ctx {
     int64_t d, k;
     int n, compressor, mode, q;
+    float wd;                /* decoupled weight decay lambda (0 = none) */
+    float base_lr, gamma;    /* step-size milestones */
+    int n_milestones;
+    int64_t milestones[64];
     float beta1, beta2, lr, nu;
     int64_t *off;            /* q+1 segment offsets */
     int64_t steps;
@@ -291,12 +298,37 @@ int oracle_set_segments(oracle_ctx *o, int q, const int64_t *off)
 
 int oracle_set_mode(oracle_ctx *o, int mode)
 {
-    if (!o || (mode != ORC_MARKOV && mode != ORC_EF) || o->steps != 0) return -1;
+    if (!o || (mode != ORC_MARKOV && mode != ORC_EF && mode != ORC_NAIVE) || o->steps != 0) return -1;
     o->mode = mode;
     return 0;
 }
 
-int oracle_set_lr(oracle_ctx *o, float lr) { if (!o) return -1; o->lr = lr; return 0; }
+int oracle_set_lr(oracle_ctx *o, float lr) { if (!o) return -1; o->lr = lr; o->n_milestones = 0; return 0; }
+
+/* Decoupled weight decay lambda (the image-classification experiments of Section 6 use a
+ * weight decay; the paper does not print the formula, the decoupled form is the reading):
+ *   x_{t+1} = x_t - alpha_t m_t / sqrt(vhat_t + nu) - (alpha_t lambda) x_t. */
+int oracle_set_weight_decay(oracle_ctx *o, float lambda)
+{
+    if (!o || !(lambda >= 0.0f)) return -1;
+    o->wd = lambda;
+    return 0;
+}
+
+/* Step-size milestones (Section 6: the step size is multiplied by 0.1 at two points of the
+ * run): the step with 1-based number t uses alpha_t = base * gamma^(number of milestones
+ * < t), the product taken by repeated binary32 multiplication.  Milestones count completed
+ * steps and must be increasing; gamma in (0, 1] keeps alpha_t non-increasing (Algorithm 1). */
+int oracle_set_lr_milestones(oracle_ctx *o, float base, int count, const int64_t *after_steps, float gamma)
+{
+    if (!o || count < 0 || count > 64 || !(gamma > 0.0f && gamma <= 1.0f)) return -1;
+    for (int i = 0; i < count; ++i)
+        if (after_steps[i] < 0 || (i > 0 && after_steps[i] <= after_steps[i - 1])) return -1;
+    o->base_lr = base; o->gamma = gamma; o->n_milestones = count;
+    for (int i = 0; i < count; ++i) o->milestones[i] = after_steps[i];
+    if (count == 0) o->lr = base;
+    return 0;
+}
 
 /* name: 0 ghat_w (n*d), 1 ghat_s, 2 gtil, 3 m, 4 v, 5 vhat, 6 x */
 float *oracle_state(oracle_ctx *o, int name)
@@ -395,6 +427,7 @@ static void amsgrad(oracle_ctx *o, const float *ge)
 {
     const float b1 = o->beta1, b2 = o->beta2;
     const float omb1 = 1.0f - b1, omb2 = 1.0f - b2;
+    const float lrwd = o->lr * o->wd;
     for (int64_t j = 0; j < o->d; ++j) {
         float g = ge[j];
         float m1 = b1 * o->m[j];
@@ -407,7 +440,13 @@ static void amsgrad(oracle_ctx *o, const float *ge)
         o->vhat[j] = o->vhat[j] >= o->v[j] ? o->vhat[j] : o->v[j];
         float den = sqrtf(o->vhat[j] + o->nu);
         float num = o->lr * o->m[j];
-        o->x[j] = o->x[j] - num / den;
+        float xold = o->x[j];
+        float xnew = xold - num / den;
+        if (o->wd != 0.0f) {                         /* decoupled weight decay */
+            float decay = lrwd * xold;
+            xnew = xnew - decay;
+        }
+        o->x[j] = xnew;
     }
 }
 
@@ -455,11 +494,39 @@ static void step_ef(oracle_ctx *o, const float *g)
     amsgrad(o, o->c);
 }
 
+/* Naive compression (Section 4, first paragraph) carried over to AMSGrad, the third
+ * comparison scheme of the experiments of Section 6: no state on either side,
+ *   worker: c^(i) = C(g^(i));   server: c = C(mean_i c^(i));   AMSGrad on c.
+ * (The section prints the SGD form with the uplink compressed; compressing the downlink with
+ * the same C is the reading that puts it under the same communication budget as the other
+ * schemes.)  ghat_w, ghat_s and gtil stay zero. */
+static void step_naive(oracle_ctx *o, const float *g)
+{
+    const int64_t d = o->d;
+    memset(o->acc, 0, (size_t)d * sizeof(float));
+    for (int i = 0; i < o->n; ++i) {
+        compress(o, g + (int64_t)i * d, o->c, i);
+        for (int64_t j = 0; j < d; ++j) o->acc[j] = o->acc[j] + o->c[j];
+    }
+    const float fn = (float)o->n;
+    for (int64_t j = 0; j < d; ++j) o->u[j] = o->acc[j] / fn;
+    compress(o, o->u, o->c, -1);
+    amsgrad(o, o->c);
+}
+
 int oracle_step(oracle_ctx *o, const float *g)
 {
     if (!o || !g) return -1;
     if (o->compressor == ORC_RANDK && !o->rand_w) return -1;
-    if (o->mode == ORC_MARKOV) step_markov(o, g); else step_ef(o, g);
+    if (o->n_milestones > 0) {
+        float lr = o->base_lr;
+        for (int i = 0; i < o->n_milestones; ++i)
+            if (o->milestones[i] <= o->steps) lr = lr * o->gamma;
+        o->lr = lr;
+    }
+    if (o->mode == ORC_MARKOV) step_markov(o, g);
+    else if (o->mode == ORC_EF) step_ef(o, g);
+    else step_naive(o, g);
     o->steps += 1;
     return 0;
 }

@@ -11,7 +11,7 @@ import subprocess
 import numpy as np
 
 SIGN, TOPK, IDENTITY, RANDK = 0, 1, 2, 3
-MARKOV, EF = 0, 1
+MARKOV, EF, NAIVE = 0, 1, 2
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -57,6 +57,10 @@ def _load():
     lib.oracle_set_mode.argtypes = [c.c_void_p, c.c_int]
     lib.oracle_set_lr.restype = c.c_int
     lib.oracle_set_lr.argtypes = [c.c_void_p, c.c_float]
+    lib.oracle_set_weight_decay.restype = c.c_int
+    lib.oracle_set_weight_decay.argtypes = [c.c_void_p, c.c_float]
+    lib.oracle_set_lr_milestones.restype = c.c_int
+    lib.oracle_set_lr_milestones.argtypes = [c.c_void_p, c.c_float, c.c_int, ip, c.c_float]
     lib.oracle_compress_randk.restype = None
     lib.oracle_compress_randk.argtypes = [fp, c.c_int64, c.c_int64, up, up, fp, fp]
     lib.oracle_set_random_sets.restype = c.c_int
@@ -169,6 +173,17 @@ class Oracle:
 
     def set_lr(self, lr):
         self._lib.oracle_set_lr(self._h, lr)
+
+    def set_weight_decay(self, weight_decay):
+        if self._lib.oracle_set_weight_decay(self._h, weight_decay) != 0:
+            raise ValueError("bad weight decay")
+
+    def set_lr_milestones(self, base_lr, after_steps, gamma):
+        """alpha_t = base_lr * gamma^(number of entries of after_steps that are <= t - 1)."""
+        ms = np.ascontiguousarray(after_steps, dtype=np.int64)
+        ip = ctypes.POINTER(ctypes.c_int64)
+        if self._lib.oracle_set_lr_milestones(self._h, base_lr, ms.size, ms.ctypes.data_as(ip), gamma) != 0:
+            raise ValueError("bad milestones")
 
     def set_random_sets(self, workers, server):
         """Rand-k: coordinate sets (n x k and k increasing distinct coordinates) of the next step."""

@@ -434,3 +434,141 @@ def test_randk_reduces_to_topk_and_identity_on_their_sets():
         c.step(g); e.step(g)
         for name in orc.STATE_NAMES:
             assert np.array_equal(c.state(name), e.state(name)), name
+
+
+# ------------------------------------------------------------------ naive compression mode
+
+def test_naive_mode_worked_example():
+    """AMSGrad with naive compression, both directions, hand-worked (golden file)."""
+    gold = read_golden("worked_example_naive.txt")
+    n, d = int(gold["n"][0]), int(gold["d"][0])
+    o = orc.Oracle(d, n, orc.SIGN, beta1=gold["beta1"][0], beta2=gold["beta2"][0],
+                   lr=gold["alpha"][0], eps=gold["nu"][0], x0=gold["x1"], mode=orc.NAIVE)
+    for t in (1, 2):
+        p = "t%d." % t
+        o.step(np.array([gold[p + "g0"], gold[p + "g1"]], dtype=np.float32))
+        for i in range(n):
+            bits, scales = o.payload(i)
+            assert scales[0] == gold[p + "w%d.scale" % i][0] and bits[0] == gold[p + "w%d.word" % i][0]
+        bits, scales = o.payload(-1)
+        assert scales[0] == gold[p + "s.scale"][0] and bits[0] == gold[p + "s.word"][0]
+        for name in ("m", "v", "vhat"):
+            assert o.state(name).tolist() == gold[p + name]
+        if t == 1:
+            assert o.state("x").tolist() == gold[p + "x"]
+        else:
+            np.testing.assert_allclose(o.state("x"), gold[p + "x"], rtol=0, atol=1.5e-7)
+            r = 0.5 * 0.8125 / math.sqrt(77 / 64)
+            np.testing.assert_allclose(o.state("x"), [0.75 - r, 1.25 + r, 0.75 - r, 1.25 + r], rtol=2e-7)
+        for name in ("ghat_w", "ghat_s", "gtil"):
+            assert not o.state(name).any()             # the scheme keeps no compression state
+
+
+@pytest.mark.parametrize("comp", [orc.SIGN, orc.TOPK, orc.IDENTITY])
+def test_naive_mode_is_stateless_and_first_step_equals_algorithm_1(comp):
+    rng = np.random.default_rng(31)
+    d, n, k = 300, 3, 17
+    G = rng.standard_normal((4, n, d)).astype(np.float32)
+    x0 = rng.standard_normal(d).astype(np.float32)
+    a = orc.Oracle(d, n, comp, k=k, x0=x0, mode=orc.NAIVE)
+    b = orc.Oracle(d, n, comp, k=k, x0=x0, mode=orc.MARKOV)
+    a.step(G[0]); b.step(G[0])
+    for name in ("m", "v", "vhat", "x"):               # from zero state Algorithm 1 sends C(g) too
+        assert np.array_equal(a.state(name), b.state(name)), name
+    # payloads of a later step depend on that step's gradients only: a fresh context that is
+    # given the moments and x reproduces step 3 without having seen steps 1 and 2
+    a.step(G[1])
+    snap = {name: a.state(name).copy() for name in ("m", "v", "vhat", "x")}
+    a.step(G[2])
+    c = orc.Oracle(d, n, comp, k=k, mode=orc.NAIVE)
+    for name, val in snap.items():
+        c.state(name)[:] = val
+    c.step(G[2])
+    for name in ("m", "v", "vhat", "x"):
+        assert np.array_equal(a.state(name), c.state(name)), name
+    if comp != orc.IDENTITY:
+        for who in list(range(n)) + [-1]:
+            pa, pc = a.payload(who), c.payload(who)
+            assert np.array_equal(pa[0], pc[0]) and np.array_equal(pa[1], pc[1])
+        # worker payload = the compressor applied to the gradient itself
+        if comp == orc.SIGN:
+            bits, scales, _ = orc.compress_sign(G[2, 1])
+            assert np.array_equal(a.payload(1)[0], bits) and np.array_equal(a.payload(1)[1], scales)
+        else:
+            order = sorted(range(d), key=lambda j: (-abs(float(G[2, 1, j])), j))[:k]
+            assert sorted(order) == a.payload(1)[0].tolist()
+    else:                                              # identity: vanilla AMSGrad, bit for bit
+        means = []
+        for t in range(3):
+            acc = np.zeros(d, np.float32)
+            for i in range(n):
+                acc = acc + G[t, i]
+            means.append(acc / np.float32(n))
+        x, m, v, vh = vanilla_amsgrad(x0, means, 0.9, 0.999, 1e-3, 1e-8)
+        assert np.array_equal(a.state("x"), x) and np.array_equal(a.state("vhat"), vh)
+
+
+# ------------------------------------------------------------------ weight decay, milestones
+
+def test_weight_decay_closed_form_at_zero_gradient():
+    """With g = 0 the moments stay 0 and x_{t+1} = x_t - (alpha lambda) x_t: for
+    alpha = lambda = 1/2 every x_t = (3/4)^(t-1) x_1 is exact in binary32 for small t."""
+    d, n = 5, 2
+    x1 = np.array([1.0, -2.0, 0.5, 3.0, 0.0], np.float32)
+    o = orc.Oracle(d, n, orc.IDENTITY, lr=0.5, eps=1.0, x0=x1)
+    o.set_weight_decay(0.5)
+    for t in range(1, 11):
+        o.step(np.zeros((n, d), np.float32))
+        want = [float(Fraction(3, 4) ** t * Fraction(float(x))) for x in x1]
+        assert o.state("x").tolist() == want
+        assert not o.state("m").any() and not o.state("vhat").any()
+
+
+def decayed_amsgrad(x0, grads, lrs, b1, b2, nu, wd):
+    """AMSGrad with decoupled weight decay and a per-step step size, written independently."""
+    f = np.float32
+    x = x0.astype(f).copy()
+    m = np.zeros_like(x); v = np.zeros_like(x); vh = np.zeros_like(x)
+    b1, b2, nu, wd = f(b1), f(b2), f(nu), f(wd)
+    for g, lr in zip(grads, lrs):
+        lr = f(lr)
+        m = b1 * m + (f(1) - b1) * g
+        v = b2 * v + (f(1) - b2) * (g * g)
+        vh = np.maximum(vh, v)
+        step = (lr * m) / np.sqrt(vh + nu)
+        x = (x - step) - (lr * wd) * x if wd != 0 else x - step
+    return x, m, v, vh
+
+
+@pytest.mark.parametrize("wd", [0.0, 5e-4, 0.1])
+def test_weight_decay_and_lr_milestones_against_independent_recursion(wd):
+    rng = np.random.default_rng(44)
+    d, T = 257, 7
+    x0 = rng.standard_normal(d).astype(np.float32)
+    G = rng.standard_normal((T, 1, d)).astype(np.float32)
+    f = np.float32
+    base, gamma = f(1e-2), f(0.1)
+    # milestones after 2 and after 5 completed steps: steps 1-2 base, 3-5 base*gamma, 6-7 base*gamma^2
+    lrs = [base] * 2 + [base * gamma] * 3 + [(base * gamma) * gamma] * 2
+    o = orc.Oracle(d, 1, orc.IDENTITY, beta2=0.99, lr=123.0, x0=x0, mode=orc.EF)   # EF + identity: exact
+    o.set_weight_decay(wd)
+    o.set_lr_milestones(base, [2, 5], gamma)
+    p = orc.Oracle(d, 1, orc.IDENTITY, beta2=0.99, lr=float(base), x0=x0, mode=orc.EF)
+    p.set_weight_decay(wd)
+    for t in range(T):
+        o.step(G[t])
+        p.set_lr(float(lrs[t]))                        # the same schedule by explicit calls
+        p.step(G[t])
+    x, m, v, vh = decayed_amsgrad(x0, G[:, 0], lrs, 0.9, 0.99, 1e-8, wd)
+    for side in (o, p):
+        assert np.array_equal(side.state("x"), x) and np.array_equal(side.state("m"), m)
+        assert np.array_equal(side.state("vhat"), vh)
+    if wd:                                             # the decay really acts
+        q = decayed_amsgrad(x0, G[:, 0], lrs, 0.9, 0.99, 1e-8, 0.0)[0]
+        assert not np.array_equal(q, x)
+    with pytest.raises(ValueError):
+        o.set_lr_milestones(base, [5, 2], gamma)       # not increasing
+    with pytest.raises(ValueError):
+        o.set_lr_milestones(base, [2], 1.5)            # alpha_t must not increase
+    with pytest.raises(ValueError):
+        o.set_weight_decay(-1.0)
