@@ -205,8 +205,10 @@ def main():
                     help="randk: run the workload's shapes with the rand-k compressor (k as in C3: d/100)")
     ap.add_argument("--grads", default="f32", choices=["f32", "bf16"],
                     help="bf16: gradients given in bfloat16 through cdadam_step_bf16 (not the headline config)")
-    ap.add_argument("--mode", default="markov", choices=["markov", "ef"],
-                    help="markov = Algorithm 1 (default); ef = classical error feedback (Section 4)")
+    ap.add_argument("--mode", default="markov", choices=["markov", "ef", "naive"],
+                    help="markov = Algorithm 1 (default); ef = classical error feedback, naive = naive "
+                         "compression (the comparison schemes of Section 4; their bytes differ, so the "
+                         "roofline figures of such a run are not the headline's)")
     ap.add_argument("--tile", type=int, default=0,
                     help="force the kernels' tile size (profiler captures of scaled-down cases)")
     ap.add_argument("--scale", type=float, default=1.0,
@@ -245,7 +247,7 @@ def main():
         args.warmup = 3
     opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
                     beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev,
-                    mode=cd.EF if args.mode == "ef" else cd.MARKOV)
+                    mode={"markov": cd.MARKOV, "ef": cd.EF, "naive": cd.NAIVE}[args.mode])
     if args.tile:
         opt.set_tile(args.tile)
     if w.compressor == synth.RANDK:      # the draws are inputs; one set of draws serves all steps
@@ -363,7 +365,7 @@ def main():
                 "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
                 "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale)
-                           + ("" if args.mode == "markov" else " [error-feedback mode]")
+                           + {"markov": "", "ef": " [error-feedback mode]", "naive": " [naive-compression mode]"}[args.mode]
                            + ("" if args.grads == "f32" else " [bf16 gradients]"),
                            "replicas": world,
                            "l2": "flushed between steps" if flush is not None else

@@ -49,7 +49,8 @@ enum { CDADAM_SIGN = 0, CDADAM_TOPK = 1, CDADAM_IDENTITY = 2, CDADAM_RANDK = 3 }
 /* recursion around the compressor */
 enum {
     CDADAM_MARKOV = 0,   /* Algorithm 1: Markov compression sequences (Section 5), the default */
-    CDADAM_EF = 1        /* classical error feedback at workers and server (Section 4) */
+    CDADAM_EF = 1,       /* classical error feedback at workers and server (Section 4) */
+    CDADAM_NAIVE = 2     /* naive compression (Section 4): no state, C applied both ways */
 };
 
 /* status codes */
@@ -164,7 +165,12 @@ int cdadam_set_random_sets(cdadam_ctx *ctx, const uint32_t *workers, const uint3
  *   worker: p = g + delta^(i), c^(i) = C(p), delta^(i) = p - c^(i);
  *   server: p = (1/n) sum_i c^(i) + delta, c = C(p), delta = p - c; AMSGrad runs on c.
  * In this mode the state named GHAT_W holds the worker errors delta^(i), GTIL the server
- * error delta, and GHAT_S is scratch.  Only before the first step.
+ * error delta, and GHAT_S is scratch.
+ * CDADAM_NAIVE is AMSGrad with naive compression (first paragraph of Section 4; the third
+ * scheme compared in Section 6), compressed both ways like the other two:
+ *   worker: c^(i) = C(g^(i));   server: c = C((1/n) sum_i c^(i));   AMSGrad runs on c.
+ * GHAT_W and GTIL stay zero; GHAT_S is scratch.
+ * Only before the first step.
  */
 int cdadam_set_mode(cdadam_ctx *ctx, int mode);
 
@@ -178,8 +184,27 @@ int cdadam_set_mode(cdadam_ctx *ctx, int mode);
 int cdadam_set_tile(cdadam_ctx *ctx, int tile);
 
 /* Step size alpha_t for the following steps (Algorithm 1 takes a non-increasing sequence;
- * monotonicity is not enforced). */
+ * monotonicity is not enforced).  Ends a schedule set by cdadam_set_lr_milestones. */
 int cdadam_set_lr(cdadam_ctx *ctx, float lr);
+
+/*
+ * Step-size milestones (Section 6 multiplies the step size by 0.1 at two points of the run):
+ * the step with 1-based number t uses alpha_t = base_lr * gamma^(number of after_steps[i]
+ * <= t - 1), the product formed by repeated binary32 multiplication.  after_steps: host,
+ * `count` (0..64) increasing non-negative numbers of completed steps; gamma in (0, 1].
+ * count = 0 sets the constant step size base_lr.  Invalid arguments: CDADAM_ERR_ARG, nothing
+ * changed.
+ */
+int cdadam_set_lr_milestones(cdadam_ctx *ctx, float base_lr, int count, const int64_t *after_steps,
+                             float gamma);
+
+/*
+ * Decoupled weight decay lambda >= 0 for the following steps (Section 6 trains with a weight
+ * decay; the paper does not print the formula, and the decoupled form is used):
+ *   x_{t+1} = x_t - alpha_t m_t / sqrt(vhat_t + nu) - (alpha_t lambda) x_t,
+ * with alpha_t lambda rounded once to binary32.  0 (the default) is Algorithm 1 as printed.
+ */
+int cdadam_set_weight_decay(cdadam_ctx *ctx, float lambda);
 
 /*
  * Copy a state vector to / from device memory (dst / src: n*d floats for GHAT_W, else d).

@@ -10,7 +10,7 @@ import os
 import torch
 
 SIGN, TOPK, IDENTITY, RANDK = 0, 1, 2, 3
-MARKOV, EF = 0, 1
+MARKOV, EF, NAIVE = 0, 1, 2
 SERVER = -1
 STATE_NAMES = ("ghat_w", "ghat_s", "gtil", "m", "v", "vhat", "x")
 OK, ERR_ARG, ERR_ALLOC, ERR_CUDA, ERR_STATE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
@@ -33,6 +33,8 @@ _SIGNATURES = {
     "cdadam_set_mode": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_tile": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
+    "cdadam_set_lr_milestones": (_c.c_int, [_c.c_void_p, _c.c_float, _c.c_int, _c.POINTER(_c.c_int64), _c.c_float]),
+    "cdadam_set_weight_decay": (_c.c_int, [_c.c_void_p, _c.c_float]),
     "cdadam_get_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_state": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
     "cdadam_last_payload": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_void_p),
@@ -201,6 +203,14 @@ class CDAdam:
 
     def set_lr(self, lr):
         _check(lib().cdadam_set_lr(self._h, lr))
+
+    def set_lr_milestones(self, base_lr, after_steps, gamma):
+        """alpha_t = base_lr * gamma^(number of entries of after_steps that are <= t - 1)."""
+        ms = (ctypes.c_int64 * len(after_steps))(*[int(a) for a in after_steps])
+        _check(lib().cdadam_set_lr_milestones(self._h, base_lr, len(after_steps), ms, gamma))
+
+    def set_weight_decay(self, weight_decay):
+        _check(lib().cdadam_set_weight_decay(self._h, weight_decay))
 
     def get_state(self, name, stream=None):
         count = self.n * self.d if name == "ghat_w" else self.d

@@ -133,6 +133,9 @@ struct cdadam_ctx {
     int tile_override = 0;  // 0 = choose from d and q
     int mode = CDADAM_MARKOV;
     Hyper hp{};
+    float wd = 0.0f;             // decoupled weight decay lambda
+    float base_lr = 0.0f, gamma = 1.0f;          // step-size milestones
+    std::vector<int64_t> milestones;
     TableSet ts;            // worker pass
     TableSet ts_s;          // server pass and update pass
     float *ghat_w = nullptr, *ghat_s = nullptr, *gtil = nullptr;
@@ -221,7 +224,7 @@ float *state_ptr(cdadam_ctx *c, int name)
 
 int prof_slots(const cdadam_ctx *c)
 {
-    return c->comp == CDADAM_SIGN ? (c->fuse_finish ? 3 : 5) : (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK) ? 4 : 1;
+    return c->comp == CDADAM_SIGN ? (c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5) : (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK) ? 4 : 1;
 }
 
 // Record the boundary event after a stage (or before the first one) when timing is on.
@@ -233,6 +236,19 @@ void prof_mark(cdadam_ctx *c, cudaStream_t st)
     else if (cudaEventCreate(&e) != cudaSuccess) return;
     cudaEventRecord(e, st);
     c->prof_ev.push_back(e);
+}
+
+void drop_graphs(cdadam_ctx *c);
+
+// The step size and everything derived from it (launch arguments, hence recorded graphs).
+void apply_lr(cdadam_ctx *c, float lr)
+{
+    const float lrwd = lr * c->wd;
+    if (lr == c->hp.lr && lrwd == c->hp.lrwd && (c->wd != 0.0f) == (c->hp.decay != 0)) return;
+    drop_graphs(c);
+    c->hp.lr = lr;
+    c->hp.lrwd = lrwd;
+    c->hp.decay = c->wd != 0.0f;
 }
 
 void drop_graphs(cdadam_ctx *c)
@@ -251,22 +267,26 @@ void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec,
     const bool svec = c->d % 4 == 0;
     const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
     float *new_scale = c->wscale[c->cur ^ 1];
-    const bool fuse = c->fuse_finish;
-    launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef,
-                       c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
+    const bool naive = c->mode == CDADAM_NAIVE;
+    const bool fuse = c->fuse_finish && !naive;
+    if (naive)      // the payload is C(g) itself: no worker state is read or written
+        launch_pack_sign(static_cast<const float *>(grads_in), c->wbits, c->wpart, tb, c->n, c->wp, vec, st);
+    else
+        launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef,
+                           c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
     prof_mark(c, st);
     if (!fuse) {
         launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
         prof_mark(c, st);
     }
-    launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, ef,
+    launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, c->mode,
                        fuse ? c->sscale : nullptr, c->sdone, st);
     prof_mark(c, st);
     if (!fuse) {
         launch_finalize_scales(c->spart, c->sscale, tbs, 1, st);
         prof_mark(c, st);
     }
-    launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, ef, st);
+    launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, c->mode, st);
     prof_mark(c, st);
 }
 
@@ -275,7 +295,7 @@ void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec,
 // gradient buffer, timing on, recording unavailable).
 bool replay_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
 {
-    if (!c->fuse_finish || !c->graphs_ok || c->prof_on) return false;
+    if (!c->fuse_finish || !c->graphs_ok || c->prof_on || c->mode == CDADAM_NAIVE) return false;
     cdadam_ctx::StepGraph *slot = nullptr, *oldest = &c->graphs[0];
     for (auto &g : c->graphs) {
         if (g.hits && g.grads == grads_in && g.bf16 == bf16 && g.pending == c->pending && g.cur == c->cur) slot = &g;
@@ -419,23 +439,55 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
             return fail(CDADAM_ERR_STATE, "cdadam_step: the stream is being captured; a step cannot be part of a caller's graph");
     }
     const float *grads = static_cast<const float *>(grads_in);
-    if (bf16 && c->comp != CDADAM_SIGN) {
+    if (bf16 && (c->comp != CDADAM_SIGN || c->mode == CDADAM_NAIVE)) {
         // only the scaled-sign worker pass reads bfloat16 directly; the other compressors
-        // get an exact binary32 copy in the context's staging buffer
+        // (and naive compression) get an exact binary32 copy in the context's staging buffer
         int rc = ensure_stage(c);
         if (rc) return rc;
         launch_widen_bf16(c->stage, grads_in, (int64_t)c->n * c->d, st);
         grads = c->stage;
         bf16 = false;
     }
-    const bool vec = aligned16(grads_in) && c->d % (bf16 ? 8 : 4) == 0;
+    const bool vec = aligned16(grads) && c->d % (bf16 ? 8 : 4) == 0;
+    if (!c->milestones.empty()) {
+        // alpha_t = base * gamma^(milestones already passed), by repeated binary32 products
+        float lr = c->base_lr;
+        for (int64_t after : c->milestones)
+            if (after <= c->steps) lr = lr * c->gamma;
+        apply_lr(c, lr);
+    }
     prof_mark(c, st);
     const bool ef = c->mode == CDADAM_EF;
+    const bool naive = c->mode == CDADAM_NAIVE;
     const bool svec = c->d % 4 == 0;
     if (c->comp == CDADAM_SIGN) {
-        if (!replay_sign_step(c, grads_in, bf16, vec, st)) enqueue_sign_step(c, grads_in, bf16, vec, st);
+        const void *gin = bf16 ? grads_in : grads;
+        if (!replay_sign_step(c, gin, bf16, vec, st)) enqueue_sign_step(c, gin, bf16, vec, st);
         c->cur ^= 1;
-        c->pending = true;
+        c->pending = !naive;             // naive compression has no worker state to bring up to date
+    } else if (naive && (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK)) {
+        // Naive compression (Section 4): c^(i) = C(g^(i)), c = C(mean_i c^(i)), AMSGrad on c.
+        // ghat_s is all zero between steps: it receives the sparse mean, is compressed, then
+        // carries the dense decoded server payload for AMSGrad and is cleared again.
+        if (c->comp == CDADAM_RANDK && !c->sets_given)
+            return fail(CDADAM_ERR_STATE, "rand-k needs cdadam_set_random_sets before the first step");
+        const uint32_t *widx, *sidx;
+        const float *wval, *sval;
+        topk_payload(c->tk_w, 0, &widx, &wval);
+        topk_payload(c->tk_s, 0, &sidx, &sval);
+        if (c->comp == CDADAM_TOPK) topk_select(c->tk_w, grads, nullptr, false, vec, st);
+        else randk_gather(c->tk_w, grads, nullptr, false, st);
+        prof_mark(c, st);
+        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);
+        prof_mark(c, st);
+        if (c->comp == CDADAM_TOPK) topk_select(c->tk_s, c->ghat_s, nullptr, false, svec, st);
+        else randk_gather(c->tk_s, c->ghat_s, nullptr, false, st);
+        launch_scatter_zero_shared(c->ghat_s, widx, c->k, c->n, st);
+        launch_scatter_set(c->ghat_s, sidx, sval, c->k, c->d, 1, st);
+        prof_mark(c, st);
+        launch_amsgrad(c->ghat_s, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+        launch_scatter_set(c->ghat_s, sidx, nullptr, c->k, c->d, 1, st);
+        prof_mark(c, st);
     } else if (c->comp == CDADAM_TOPK && !ef) {
         topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
         prof_mark(c, st);
@@ -498,7 +550,7 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
             prof_mark(c, st);
         }
     } else {
-        launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, ef, st);
+        launch_step_identity(grads, c->ghat_w, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->n, c->hp, c->mode, st);
         prof_mark(c, st);
     }
     int rc = check_launch("cdadam_step");
@@ -579,7 +631,7 @@ int cdadam_set_random_sets(cdadam_ctx *c, const uint32_t *workers, const uint32_
 int cdadam_set_mode(cdadam_ctx *c, int mode)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_mode: NULL context");
-    if (mode != CDADAM_MARKOV && mode != CDADAM_EF) return fail(CDADAM_ERR_ARG, "unknown mode %d", mode);
+    if (mode != CDADAM_MARKOV && mode != CDADAM_EF && mode != CDADAM_NAIVE) return fail(CDADAM_ERR_ARG, "unknown mode %d", mode);
     if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the mode must be set before the first step");
     c->mode = mode;
     return CDADAM_OK;
@@ -588,8 +640,32 @@ int cdadam_set_mode(cdadam_ctx *c, int mode)
 int cdadam_set_lr(cdadam_ctx *c, float lr)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_lr: NULL context");
-    if (lr != c->hp.lr) drop_graphs(c);       // the step size is a launch argument
-    c->hp.lr = lr;
+    c->milestones.clear();                    // an explicit step size ends a schedule
+    apply_lr(c, lr);
+    return CDADAM_OK;
+}
+
+int cdadam_set_weight_decay(cdadam_ctx *c, float lambda)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_weight_decay: NULL context");
+    if (!(lambda >= 0.0f)) return fail(CDADAM_ERR_ARG, "the weight decay must be >= 0");
+    c->wd = lambda;
+    apply_lr(c, c->hp.lr);
+    return CDADAM_OK;
+}
+
+int cdadam_set_lr_milestones(cdadam_ctx *c, float base_lr, int count, const int64_t *after_steps, float gamma)
+{
+    if (!c || (count > 0 && !after_steps)) return fail(CDADAM_ERR_ARG, "cdadam_set_lr_milestones: NULL argument");
+    if (count < 0 || count > 64) return fail(CDADAM_ERR_ARG, "between 0 and 64 milestones");
+    if (!(gamma > 0.0f && gamma <= 1.0f)) return fail(CDADAM_ERR_ARG, "gamma must be in (0, 1]: the step sizes of Algorithm 1 do not increase");
+    for (int i = 0; i < count; ++i)
+        if (after_steps[i] < 0 || (i > 0 && after_steps[i] <= after_steps[i - 1]))
+            return fail(CDADAM_ERR_ARG, "milestones must be non-negative and increasing");
+    c->base_lr = base_lr;
+    c->gamma = gamma;
+    c->milestones.assign(after_steps, after_steps + count);
+    if (count == 0) apply_lr(c, base_lr);
     return CDADAM_OK;
 }
 
@@ -660,9 +736,10 @@ int cdadam_device_status(cdadam_ctx *c, void *stream)
 int cdadam_launches_per_step(cdadam_ctx *c)
 {
     if (!c) return 0;
-    if (c->comp == CDADAM_SIGN) return c->fuse_finish ? 3 : 5;
-    if (c->comp == CDADAM_TOPK) return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : 0);
-    if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : 4;
+    if (c->comp == CDADAM_SIGN) return c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5;
+    if (c->comp == CDADAM_TOPK)
+        return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : c->mode == CDADAM_NAIVE ? 3 : 0);
+    if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : c->mode == CDADAM_NAIVE ? 7 : 4;
     return 1;
 }
 
@@ -703,6 +780,9 @@ const char *cdadam_profile_name(cdadam_ctx *c, int slot)
     if (!c || slot < 0 || slot >= prof_slots(c)) return "";
     static const char *randk[] = {"randk_gather(workers)", "topk_aggregate", "randk_gather(server)", "k_amsgrad"};
     if (c->comp == CDADAM_RANDK) return randk[slot];
+    static const char *nsign[] = {"k_pack_sign", "k_finalize_scales(workers)", "k_server_sign",
+                                  "k_finalize_scales(server)", "k_update_sign"};
+    if (c->comp == CDADAM_SIGN && c->mode == CDADAM_NAIVE) return nsign[slot];
     return c->comp == CDADAM_SIGN ? (c->fuse_finish ? fused[slot] : sign[slot]) : c->comp == CDADAM_TOPK ? topk[slot] : "k_step_identity";
 }
 
@@ -723,7 +803,7 @@ int cdadam_compress_sign(const float *x, int64_t d, int q, const int64_t *offset
     dd *part = nullptr;
     cudaError_t e = cudaMallocAsync((void **)&part, (size_t)ts.tb.nparts * sizeof(dd), st);
     if (e != cudaSuccess) { ts.release(st, true); return fail(CDADAM_ERR_ALLOC, "scratch allocation: %s", cudaGetErrorString(e)); }
-    launch_pack_sign(x, bits, part, ts.tb, aligned16(x) && d % 4 == 0, st);
+    launch_pack_sign(x, bits, part, ts.tb, 1, (d + 31) / 32, aligned16(x) && d % 4 == 0, st);
     launch_finalize_scales(part, scales, ts.tb, 1, st);
     rc = check_launch("cdadam_compress_sign");
     cudaFreeAsync(part, st);

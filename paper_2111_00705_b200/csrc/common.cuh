@@ -210,10 +210,13 @@ __device__ __forceinline__ int find_segment(const int64_t *off, int lo, int hi, 
 
 // ------------------------------------------------------------------------------------
 // AMSGrad update of one coordinate (Algorithm 1 lines 13-16): nu inside the root, no bias
-// correction, one rounding per operation, no fused multiply-add.
+// correction, one rounding per operation, no fused multiply-add.  With a weight decay
+// lambda (Section 6; decoupled form) x also loses (alpha lambda) x_t.
 // ------------------------------------------------------------------------------------
 struct Hyper {
     float beta1, beta2, omb1, omb2, lr, nu;   // omb = 1 - beta, rounded once in binary32
+    float lrwd;                               // alpha * lambda, rounded once in binary32
+    int decay;                                // lambda != 0
 };
 
 __device__ __forceinline__ void amsgrad1(float gt, float &m, float &v, float &vh, float &x,
@@ -222,7 +225,9 @@ __device__ __forceinline__ void amsgrad1(float gt, float &m, float &v, float &vh
     m = __fadd_rn(__fmul_rn(hp.beta1, m), __fmul_rn(hp.omb1, gt));
     v = __fadd_rn(__fmul_rn(hp.beta2, v), __fmul_rn(hp.omb2, __fmul_rn(gt, gt)));
     vh = vh >= v ? vh : v;
-    x = __fsub_rn(x, __fdiv_rn(__fmul_rn(hp.lr, m), __fsqrt_rn(__fadd_rn(vh, hp.nu))));
+    const float xo = x;
+    x = __fsub_rn(xo, __fdiv_rn(__fmul_rn(hp.lr, m), __fsqrt_rn(__fadd_rn(vh, hp.nu))));
+    if (hp.decay) x = __fsub_rn(x, __fmul_rn(hp.lrwd, xo));
 }
 
 }  // namespace cdadam

@@ -7,26 +7,30 @@ namespace cdadam {
 
 // C(u) = u: every line of Algorithm 1 for one coordinate, workers in increasing order.
 // EF: the same with classical error feedback, whose error terms stay exactly zero.
-template <bool EF>
+template <int MODE>      // 0 = Algorithm 1, 1 = error feedback, 2 = naive (no state)
 __global__ void __launch_bounds__(kBlock)
 k_step_identity(const float *__restrict__ grads, float *__restrict__ ghat_w,
                 float *__restrict__ ghat_s, float *__restrict__ gtil, float *__restrict__ m,
                 float *__restrict__ v, float *__restrict__ vhat, float *__restrict__ x,
                 int64_t d, int n, Hyper hp)
 {
+    constexpr bool EF = MODE == 1;
     const float fn = (float)n;
     for (int64_t j = (int64_t)blockIdx.x * kBlock + threadIdx.x; j < d;
          j += (int64_t)gridDim.x * kBlock) {
         float a = 0.0f;
         for (int i = 0; i < n; ++i) {
             const int64_t p = (int64_t)i * d + j;
+            if (MODE == 2) { a = __fadd_rn(a, grads[p]); continue; }
             const float gh = ghat_w[p];
             const float u = EF ? __fadd_rn(grads[p], gh) : __fsub_rn(grads[p], gh);   // c^(i) = u
             ghat_w[p] = EF ? __fsub_rn(u, u) : __fadd_rn(gh, u);
             a = __fadd_rn(a, u);
         }
         float gt;
-        if (EF) {
+        if (MODE == 2) {
+            gt = __fdiv_rn(a, fn);
+        } else if (EF) {
             gt = __fadd_rn(__fdiv_rn(a, fn), gtil[j]);         // c = p, the error p - c is zero
             gtil[j] = __fsub_rn(gt, gt);
         } else {
@@ -75,10 +79,11 @@ static unsigned grid_for(int64_t items)
 
 void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
                           float *m, float *v, float *vhat, float *x, int64_t d, int n,
-                          Hyper hp, bool ef, cudaStream_t st)
+                          Hyper hp, int mode, cudaStream_t st)
 {
-    if (ef) k_step_identity<true><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
-    else k_step_identity<false><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
+    if (mode == 2) k_step_identity<2><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
+    else if (mode == 1) k_step_identity<1><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
+    else k_step_identity<0><<<grid_for(d), kBlock, 0, st>>>(grads, ghat_w, ghat_s, gtil, m, v, vhat, x, d, n, hp);
 }
 
 // exact widening bfloat16 -> binary32
@@ -123,6 +128,20 @@ k_scatter_set(float *__restrict__ dst, const uint32_t *__restrict__ idx, const f
     const int row = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
     if (t < k) dst[(int64_t)row * d + idx[(int64_t)row * k + t]] = val ? val[(int64_t)row * k + t] : 0.0f;
+}
+
+// dst[idx[row][t]] = 0 for every row: one vector, the coordinate sets of all rows
+__global__ void __launch_bounds__(kBlock)
+k_scatter_zero_shared(float *__restrict__ dst, const uint32_t *__restrict__ idx, int64_t k)
+{
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t < k) dst[idx[(int64_t)blockIdx.y * k + t]] = 0.0f;
+}
+
+void launch_scatter_zero_shared(float *dst, const uint32_t *idx, int64_t k, int rows, cudaStream_t st)
+{
+    dim3 grid((unsigned)((k + kBlock - 1) / kBlock), (unsigned)rows);
+    k_scatter_zero_shared<<<grid, kBlock, 0, st>>>(dst, idx, k);
 }
 
 void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d,

@@ -23,26 +23,28 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 // Server pass A (lines 8-9): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
 // sign(w) into sbits and writes partial sums of |w| to spart.  sscale != NULL: the scales are
 // finished in the same launch (done: q zeroed counters), as in the worker pass.
+// mode: 0 Algorithm 1, 1 error feedback, 2 naive compression (w = mean; gtil is not read).
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, bool ef, float *sscale, unsigned int *done,
+                        int n, int64_t wp, bool vec_ok, int mode, float *sscale, unsigned int *done,
                         cudaStream_t st);
 // Server pass B and worker update (lines 10, 12-16): gtil += decode(c); AMSGrad.
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
                         float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
-                        bool vec_ok, bool ef, cudaStream_t st);
+                        bool vec_ok, int mode, cudaStream_t st);
 // ghat_w += decode(bits, scales) for all workers (applies a deferred payload).
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
                        const Tables &tb, int n, int64_t wp, bool ef, cudaStream_t st);
-// Stand-alone scaled-sign compressor of one vector: bits and partial sums of |x|.
-void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
-                      bool vec_ok, cudaStream_t st);
+// Scaled-sign compressor without state for `rows` vectors (x rows x d, bits rows x wp, part
+// rows x nparts): bits and partial sums of |x|.
+void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb, int rows,
+                      int64_t wp, bool vec_ok, cudaStream_t st);
 
 // ---- identity ----------------------------------------------------------------------
 // The whole iteration with C(u) = u, one fused pass.
 void launch_step_identity(const float *grads, float *ghat_w, float *ghat_s, float *gtil,
                           float *m, float *v, float *vhat, float *x, int64_t d, int n,
-                          Hyper hp, bool ef, cudaStream_t st);
+                          Hyper hp, int mode, cudaStream_t st);
 
 // ---- pieces of the error-feedback iteration with the top-k compressor ---------------------
 // dst[j] = (float)src[j] for count bfloat16 values (exact widening).
@@ -52,6 +54,8 @@ void launch_add_into(float *dst, const float *src, int64_t count, bool vec_ok, c
 // dst[idx[t]] = val ? val[t] : 0 for t < k, for `rows` rows (dst stride d, idx/val stride k).
 void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d,
                         int rows, cudaStream_t st);
+// dst[idx[t]] = 0 for t < rows * k: one vector, the coordinate sets of all rows.
+void launch_scatter_zero_shared(float *dst, const uint32_t *idx, int64_t k, int rows, cudaStream_t st);
 
 // ---- AMSGrad alone on a dense gradient estimate (top-k path) ------------------------------
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,

@@ -29,6 +29,9 @@ __device__ __forceinline__ float signed_scale(uint32_t bit, float s) { return bi
 //     p = mean + delta in the ghat buffer; then delta = p - c and AMSGrad runs on c.
 // `stored` is what the buffer holds, `store` what is written back; the value returned is
 // the compressor input.
+// The server-side kernels take MODE: 0 = Algorithm 1, 1 = error feedback, 2 = naive
+// compression (Section 4: no state; as error feedback with the error held at zero and
+// never written; the workers' payloads come from k_pack_sign on the gradients).
 // ------------------------------------------------------------------------------------
 template <bool EF>
 __device__ __forceinline__ float worker_step(float g, float stored, float c_prev, float &store)
@@ -411,7 +414,7 @@ k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Table
 // ------------------------------------------------------------------------------------
 constexpr int kNC = 16;     // workers staged per chunk
 
-template <int VPT, bool EF>
+template <int VPT, int MODE>
 __global__ void __launch_bounds__(kBlock)
 k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
               float *__restrict__ ghat_s, const float *__restrict__ gtil,
@@ -419,6 +422,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
               int64_t wp, int vec_ok, int n_pow2, float *__restrict__ sscale,
               unsigned int *__restrict__ done)
 {
+    constexpr bool EF = MODE != 0;
     __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
     __shared__ float ssm[kNC];
     const int64_t T = tb.order[blockIdx.x];
@@ -447,7 +451,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                 const int64_t j = wb + v * 128 + lane * 4;
                 H[v] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
                 if (!EF) H[v] = ld_rw4(ghat_s + j);      // error feedback overwrites this buffer
-                Gt[v] = ld_ro4(gtil + j);
+                Gt[v] = MODE == 2 ? make_float4(0.0f, 0.0f, 0.0f, 0.0f) : ld_ro4(gtil + j);
             }
             float a[VPT][4];
 #pragma unroll
@@ -535,7 +539,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                 a = __fadd_rn(a, signed_scale(bit, wscale[(int64_t)i * tb.q + r]));
             }
             float hn;
-            w = server_step<EF>(__fdiv_rn(a, fn), EF ? 0.0f : ghat_s[j], gtil[j], hn);
+            w = server_step<EF>(__fdiv_rn(a, fn), EF ? 0.0f : ghat_s[j], MODE == 2 ? 0.0f : gtil[j], hn);
             ghat_s[j] = hn;
         }
         const uint32_t word = __ballot_sync(kFull, valid && w >= 0.0f);
@@ -546,7 +550,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         const int64_t lo = max(tb.off[r], base), hi = min(tb.off[r + 1], end);
         dd acc = {0.0, 0.0};
         for (int64_t j = lo + threadIdx.x; j < hi; j += kBlock)
-            dd_acc(acc, fabsf(server_input_from_memory<EF>(ghat_s[j], gtil[j])));
+            dd_acc(acc, fabsf(server_input_from_memory<EF>(ghat_s[j], EF ? 0.0f : gtil[j])));
         acc = block_sum<kBlock>(acc);
         if (threadIdx.x == 0) part[r - first] = acc;
     }
@@ -562,19 +566,22 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
 // ------------------------------------------------------------------------------------
 constexpr int kUpdSpan = kBlock * 4;
 
-template <bool EF>
+template <int MODE>
 __global__ void __launch_bounds__(kBlock, 5)
 k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ sscale,
               const float *__restrict__ ghat_s, float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
               float *__restrict__ vhat, float *__restrict__ x, Tables tb, Hyper hp, int vec_ok)
 {
+    constexpr bool EF = MODE == 1;
     const int64_t base = (int64_t)blockIdx.x * kUpdSpan;
     const int64_t T = base / tb.tile;
 
     if (vec_ok && base + kUpdSpan <= tb.d) {
         const int64_t j = base + threadIdx.x * 4;
-        // error feedback reads the server's compressor input p (ghat buffer), not the old error
-        float4 Gt = EF ? ld_ro4(ghat_s + j) : ld_rw4(gtil + j), M = ld_rw4(m + j), V = ld_rw4(v + j);
+        // error feedback reads the server's compressor input p (ghat buffer), not the old error;
+        // naive compression reads and writes no compression state
+        float4 Gt = MODE == 2 ? make_float4(0.0f, 0.0f, 0.0f, 0.0f) : EF ? ld_ro4(ghat_s + j) : ld_rw4(gtil + j);
+        float4 M = ld_rw4(m + j), V = ld_rw4(v + j);
         float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
         const uint32_t nib = ld_ro_u32(sbits + (j >> 5)) >> (j & 31);
         const int first = tb.tile_first[T], last = tb.tile_last[T];
@@ -590,15 +597,16 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
             while (r < last && j + 3 >= tb.off[r + 1]) ++r;
             s3 = __ldg(sscale + r);
         }
-        const float ex = update_step<EF>(Gt.x, Gt.x, signed_scale(nib & 1u, s0), Gt.x);
-        const float ey = update_step<EF>(Gt.y, Gt.y, signed_scale(nib & 2u, s1), Gt.y);
-        const float ez = update_step<EF>(Gt.z, Gt.z, signed_scale(nib & 4u, s2), Gt.z);
-        const float ew = update_step<EF>(Gt.w, Gt.w, signed_scale(nib & 8u, s3), Gt.w);
+        const float ex = update_step<MODE != 0>(Gt.x, Gt.x, signed_scale(nib & 1u, s0), Gt.x);
+        const float ey = update_step<MODE != 0>(Gt.y, Gt.y, signed_scale(nib & 2u, s1), Gt.y);
+        const float ez = update_step<MODE != 0>(Gt.z, Gt.z, signed_scale(nib & 4u, s2), Gt.z);
+        const float ew = update_step<MODE != 0>(Gt.w, Gt.w, signed_scale(nib & 8u, s3), Gt.w);
         amsgrad1(ex, M.x, V.x, Vh.x, X.x, hp);
         amsgrad1(ey, M.y, V.y, Vh.y, X.y, hp);
         amsgrad1(ez, M.z, V.z, Vh.z, X.z, hp);
         amsgrad1(ew, M.w, V.w, Vh.w, X.w, hp);
-        st_rw4(gtil + j, Gt); st_rw4(m + j, M); st_rw4(v + j, V);
+        if (MODE != 2) st_rw4(gtil + j, Gt);
+        st_rw4(m + j, M); st_rw4(v + j, V);
         st_rw4(vhat + j, Vh); st_rw4(x + j, X);
         return;
     }
@@ -608,10 +616,10 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
         const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
-        const float stored = EF ? ghat_s[j] : gtil[j];
+        const float stored = MODE == 2 ? 0.0f : EF ? ghat_s[j] : gtil[j];
         float gt;
-        const float est = update_step<EF>(stored, stored, signed_scale(bit, sscale[r]), gt);
-        gtil[j] = gt;
+        const float est = update_step<MODE != 0>(stored, stored, signed_scale(bit, sscale[r]), gt);
+        if (MODE != 2) gtil[j] = gt;
         float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
         amsgrad1(est, mm, vv, vh, xx, hp);
         m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
@@ -642,16 +650,19 @@ k_apply_sign(float *__restrict__ ghat_w, const uint32_t *__restrict__ wbits,
 }
 
 // ------------------------------------------------------------------------------------
-// Stand-alone compressor: sign bits of x and partial sums of |x|.  grid = (ntiles).
+// Compressor without state: sign bits of x and partial sums of |x|, for each of the rows of
+// x (rows x d; bits rows x wp; partial sums rows x nparts).  grid = (ntiles, rows).
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
-k_pack_sign(const float *__restrict__ x, uint32_t *__restrict__ bits, dd *__restrict__ part_all,
-            Tables tb, int vec_ok)
+k_pack_sign(const float *__restrict__ x_all, uint32_t *__restrict__ bits_all, dd *__restrict__ part_all,
+            Tables tb, int64_t wp, int vec_ok)
 {
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
-    dd *part = part_all + tb.pbase[T];
+    const float *x = x_all + (int64_t)blockIdx.y * tb.d;
+    uint32_t *bits = bits_all + (int64_t)blockIdx.y * wp;
+    dd *part = part_all + (int64_t)blockIdx.y * tb.nparts + tb.pbase[T];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     if (vec_ok && first == last && base + tb.tile <= tb.d) {
@@ -740,27 +751,32 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
-                        int n, int64_t wp, bool vec_ok, bool ef, float *sscale, unsigned int *done,
+                        int n, int64_t wp, bool vec_ok, int mode, float *sscale, unsigned int *done,
                         cudaStream_t st)
 {
     const int pow2 = (n & (n - 1)) == 0;
-    if (ef)
-        k_server_sign<2, true><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+    if (mode == 2)
+        k_server_sign<2, 2><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+                                                                    spart, tb, n, wp, vec_ok, pow2, sscale, done);
+    else if (mode == 1)
+        k_server_sign<2, 1><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
                                                                        spart, tb, n, wp, vec_ok, pow2, sscale, done);
     else
-        k_server_sign<2, false><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
+        k_server_sign<2, 0><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
                                                                         spart, tb, n, wp, vec_ok, pow2, sscale, done);
 }
 
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
                         float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
-                        bool vec_ok, bool ef, cudaStream_t st)
+                        bool vec_ok, int mode, cudaStream_t st)
 {
     const unsigned blocks = (unsigned)((tb.d + kUpdSpan - 1) / kUpdSpan);
-    if (ef)
-        k_update_sign<true><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
+    if (mode == 2)
+        k_update_sign<2><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
+    else if (mode == 1)
+        k_update_sign<1><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
     else
-        k_update_sign<false><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
+        k_update_sign<0><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
 }
 
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
@@ -771,10 +787,11 @@ void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales
     else k_apply_sign<false><<<grid, kBlock, 0, st>>>(ghat_w, wbits, scales, tb, wp);
 }
 
-void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb,
-                      bool vec_ok, cudaStream_t st)
+void launch_pack_sign(const float *x, uint32_t *bits, dd *part, const Tables &tb, int rows,
+                      int64_t wp, bool vec_ok, cudaStream_t st)
 {
-    k_pack_sign<<<(unsigned)tb.ntiles, kBlock, 0, st>>>(x, bits, part, tb, vec_ok);
+    dim3 grid((unsigned)tb.ntiles, (unsigned)rows);
+    k_pack_sign<<<grid, kBlock, 0, st>>>(x, bits, part, tb, wp, vec_ok);
 }
 
 }  // namespace cdadam
