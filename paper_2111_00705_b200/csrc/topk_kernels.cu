@@ -11,10 +11,12 @@
 // atomics: the result does not depend on the order of execution.
 //
 // Normally ONE dense pass suffices: the level-1 bucket of the previous selection, lowered by
-// a margin, serves as a floor; the pass histograms and bitmaps only the coordinates at or
-// above it and keeps their values per tile, so every later pass is sparse and reads those
-// values back in order.  If fewer than k coordinates lie above the floor (or a tile cannot
-// keep its values) the classic two dense passes run instead.  The same file holds the sparse
+// a margin, serves as a floor; the pass histograms only the coordinates at or above it and
+// keeps them per 4096-coordinate tile as a short list (position in the tile, value) in index
+// order.  Every later pass of such a row walks these lists, one warp per tile, with coalesced
+// reads; selection, ties and the ordered compaction follow from per-tile counts and two
+// scans, without bitmaps.  If fewer than k coordinates lie above the floor (or a tile cannot
+// keep its list) the classic two dense passes and the bitmap passes run instead.  The same file holds the sparse
 // server aggregation and the rand-k path, which shares the payload kernels.
 #include "topk.h"
 
@@ -45,12 +47,16 @@ struct TopkWorkspace {
     int rows;
     uint32_t *hist;                   // rows x kHistStride
     Sel *sel;                         // rows
-    uint32_t *bm_in, *bm_cand;        // rows x wp
-    uint32_t *bm_ge;                  // rows x wp: coordinates at or above the guessed bucket
+    uint32_t *bm_in, *bm_cand;        // rows x wp (rows whose guess failed)
     uint32_t *floor_bucket;           // rows: guessed level-1 bucket for the next selection
     uint32_t *hit;                    // rows: 1 if the guess held in the current selection
     uint32_t *ovf;                    // rows: 1 if some tile had more than kStashCap values to keep
-    float *stash;                     // rows x ceil(d/4096) x kStashCap: u of the coordinates in bm_ge
+    // lists of the coordinates at or above the guessed bucket, per 4096-coordinate tile:
+    float *stash;                     // rows x nt4k x kStashCap: values u, in index order
+    uint16_t *stash_pos;              // rows x nt4k x kStashCap: positions inside the tile
+    uint32_t *stash_cnt;              // rows x nt4k: list lengths (may exceed kStashCap: ovf)
+    uint32_t *cnt_gt, *cnt_eq;        // rows x nt4k: per tile, keys above / equal to the threshold;
+                                      // after the scans: payload offset / tie rank of the tile
     int64_t nt4k;                     // ceil(d / 4096)
     uint32_t *cnt_tie, *cnt_fin;      // rows x nbt
     uint32_t *idx;                    // rows x k
@@ -263,16 +269,17 @@ k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
 // Speculative single dense pass.  The threshold moves little from one iteration to the
 // next, so the level-1 bucket of the previous selection, lowered by a margin, is taken as a
 // floor: this pass histograms only the coordinates at or above the floor (a few percent, so
-// few shared-memory atomics) and records them in a bitmap.  If at least k coordinates lie
-// at or above the floor, the threshold bucket is found from this histogram and the second
-// dense pass is not needed; otherwise the two classic passes run.  grid = (ceil(d/4096), rows).
+// few shared-memory atomics) and keeps them as the tile's list (position, value) in index
+// order.  If at least k coordinates lie at or above the floor, the threshold bucket is found
+// from this histogram and the second dense pass is not needed; otherwise the two classic
+// passes run.  grid = (ceil(d/4096), rows).
 // ------------------------------------------------------------------------------------
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
-            const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ bm_ge_all,
-            uint32_t *__restrict__ hist_all, float *__restrict__ stash_all, uint32_t *__restrict__ ovf,
-            int64_t d, int64_t wp, int vec_ok)
+            const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
+            float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
+            uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ ovf, int64_t d, int vec_ok)
 {
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
@@ -283,10 +290,9 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
     __syncthreads();
     const float *a = a_all + (int64_t)row * d;
     const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
-    uint32_t *bm_ge = bm_ge_all + (int64_t)row * wp;
-    // the values u of the coordinates at or above the floor, in index order, so that the
-    // sparse passes that follow read them back sequentially instead of gathering a and b
-    float *stash = stash_all + ((int64_t)row * gridDim.x + blockIdx.x) * kStashCap;
+    const int64_t tile = (int64_t)row * gridDim.x + blockIdx.x;
+    float *stash = stash_all + tile * kStashCap;
+    uint16_t *spos = stash_pos_all + tile * kStashCap;
     const int64_t base = (int64_t)blockIdx.x * kSub;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
@@ -319,8 +325,6 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if (hw >= fl) atomicAdd(&h[hw], 1u);
             mine += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
         }
-        const uint32_t wg = warp_words(BG, lane);
-        if (lane < 16) bm_ge[(wb >> 5) + lane] = wg;
         if (lane == 0) wcnt[warp] = mine;             // the same in every lane
         __syncthreads();
         uint32_t rank = 0, total = 0;
@@ -329,17 +333,22 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if (w8 < warp) rank += wcnt[w8];
             total += wcnt[w8];
         }
+        // index order: coordinate = warp * 512 + v * 128 + lane * 4 + component
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             uint32_t r = rank + __popc(BG[v][0] & lt) + __popc(BG[v][1] & lt) + __popc(BG[v][2] & lt) +
                          __popc(BG[v][3] & lt);
-            if ((BG[v][0] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].x; ++r; }
-            if ((BG[v][1] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].y; ++r; }
-            if ((BG[v][2] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].z; ++r; }
-            if ((BG[v][3] >> lane) & 1u) { if (r < kStashCap) stash[r] = A[v].w; }
+            const uint32_t p0 = (uint32_t)(warp * kWarpSpan + v * 128 + lane * 4);
+            if ((BG[v][0] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].x; spos[r] = (uint16_t)p0; } ++r; }
+            if ((BG[v][1] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].y; spos[r] = (uint16_t)(p0 + 1); } ++r; }
+            if ((BG[v][2] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].z; spos[r] = (uint16_t)(p0 + 2); } ++r; }
+            if ((BG[v][3] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].w; spos[r] = (uint16_t)(p0 + 3); } }
             rank += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
         }
-        if (threadIdx.x == 0 && total > (uint32_t)kStashCap) ovf[row] = 1u;
+        if (threadIdx.x == 0) {
+            stash_cnt_all[tile] = total;
+            if (total > (uint32_t)kStashCap) ovf[row] = 1u;
+        }
     } else {
         const int64_t end = min(base + (int64_t)kSub, d);
         uint32_t run = 0;                             // coordinates kept so far, block-uniform
@@ -350,7 +359,6 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const uint32_t hi = key_of(u) >> 20;
             const bool ge = valid && hi >= fl;
             const uint32_t wg = __ballot_sync(kFull, ge);
-            if (lane == 0 && j < end) bm_ge[j >> 5] = wg;
             if (ge) atomicAdd(&h[hi], 1u);
             if (lane == 0) wcnt[warp] = __popc(wg);
             __syncthreads();
@@ -360,11 +368,14 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
                 if (w8 < warp) r += wcnt[w8];
                 total += wcnt[w8];
             }
-            if (ge && r < (uint32_t)kStashCap) stash[r] = u;
+            if (ge && r < (uint32_t)kStashCap) { stash[r] = u; spos[r] = (uint16_t)(j - base); }
             run += total;
             __syncthreads();
         }
-        if (threadIdx.x == 0 && run > (uint32_t)kStashCap) ovf[row] = 1u;
+        if (threadIdx.x == 0) {
+            stash_cnt_all[tile] = run;
+            if (run > (uint32_t)kStashCap) ovf[row] = 1u;
+        }
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
@@ -413,30 +424,37 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
         for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
 }
 
-// In the passes below a thread owns 4 consecutive bitmap words and a warp therefore one
-// 4096-coordinate tile of the dense pass.  The k-th set bit of the tile's bm_ge words has its
-// value at stash[k]; a thread's first rank is the warp-exclusive sum of the popcounts.
-__device__ __forceinline__ uint32_t warp_excl_sum(uint32_t v)
+// In the list passes below a block owns the 8 tiles of one 32768-coordinate span and a warp
+// one tile: lane L reads entries L, L + 32, ... of the tile's list (coalesced).
+constexpr int kTilesPerBlock = kTileWords * 32 / kSub;
+
+struct TileList {
+    const float *val;
+    const uint16_t *pos;
+    uint32_t cnt;
+    int64_t tile;        // index of the tile inside its row
+    bool any;
+};
+
+__device__ __forceinline__ TileList tile_list(const float *stash_all, const uint16_t *stash_pos_all,
+                                              const uint32_t *stash_cnt_all, int row, int64_t nt4k)
 {
-    const int lane = threadIdx.x & 31;
-    uint32_t inc = v;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const uint32_t t = __shfl_up_sync(kFull, inc, o);
-        if (lane >= o) inc += t;
-    }
-    return inc - v;
+    TileList t;
+    t.tile = (int64_t)blockIdx.x * kTilesPerBlock + (threadIdx.x >> 5);
+    t.any = t.tile < nt4k;
+    const int64_t g = (int64_t)row * nt4k + (t.any ? t.tile : 0);
+    t.val = stash_all + g * kStashCap;
+    t.pos = stash_pos_all + g * kStashCap;
+    t.cnt = t.any ? min(stash_cnt_all[g], (uint32_t)kStashCap) : 0u;
+    return t;
 }
 
-// After a successful guess: from the bitmap of coordinates at or above the floor, rebuild
-// what the second dense pass would have produced: bm_in (bucket above the threshold
-// bucket), bm_cand (inside it) and the level-2 histogram of the candidates.
-// grid = (nbt, rows); a thread walks the set bits of its bitmap words.
+// After a successful guess: the level-2 histogram of the listed values that fall into the
+// threshold bucket (what the second dense pass would have produced).  grid = (nbt, rows).
 __global__ void __launch_bounds__(kBlock)
 k_topk_split(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-             const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
-             uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
-             uint32_t *__restrict__ hist_all, int64_t wp, int64_t nt4k)
+             const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
+             const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all, int64_t nt4k)
 {
     __shared__ uint32_t h[kBins2];
     const int row = blockIdx.y;
@@ -444,27 +462,10 @@ k_topk_split(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
     const uint32_t b1 = sel_all[row].b1;
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
-    const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
-    const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
-    uint32_t ge[4];
-#pragma unroll
-    for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
-    uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        uint32_t word = ge[m], in = 0, cand = 0;
-        while (word) {
-            const int bit = __ffs(word) - 1;
-            word &= word - 1;
-            const uint32_t key = key_of(stash[rank++]);
-            if ((key >> 20) > b1) in |= 1u << bit;
-            else if ((key >> 20) == b1) { cand |= 1u << bit; atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u); }
-        }
-        if (w0 + m < wp) {
-            bm_in_all[(int64_t)row * wp + w0 + m] = in;
-            bm_cand_all[(int64_t)row * wp + w0 + m] = cand;
-        }
+    const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+    for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
+        const uint32_t key = key_of(tl.val[e]);
+        if ((key >> 20) == b1) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
@@ -480,7 +481,8 @@ template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-             const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
+             const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
+             const uint32_t *__restrict__ stash_cnt_all,
              const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
              int64_t wp, int64_t nt4k)
 {
@@ -490,27 +492,11 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const int row = blockIdx.y;
     const uint32_t *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
-    if (hit[row]) {                                   // values come from the dense pass's stash
-        const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
-        const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
-        const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
-        uint32_t ge[4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
-        uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
-#pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            const uint32_t cand = ge[m] ? bm_cand[w0 + m] : 0u;
-            uint32_t word = ge[m];
-            while (word) {
-                const int bit = __ffs(word) - 1;
-                word &= word - 1;
-                if ((cand >> bit) & 1u) {
-                    const uint32_t key = key_of(stash[rank]);
-                    if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
-                }
-                ++rank;
-            }
+    if (hit[row]) {                                   // the tiles' lists hold the values
+        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
+            const uint32_t key = key_of(tl.val[e]);
+            if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
         }
     } else {                                          // classic path: gather a and b
         const float *a = a_all + (int64_t)row * d;
@@ -533,15 +519,19 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
 }
 
 // ------------------------------------------------------------------------------------
-// With the threshold key T known: bm_in |= candidates with key > T; bm_cand := candidates
-// with key == T (the ties).  If all ties are needed they are merged at once; otherwise the
-// per-tile tie counts feed the ordered pick below.  grid = (nbt, rows).
+// With the threshold key T known.  Rows with lists: per tile, the number of keys above T and
+// the number equal to T (the ties); the scans below turn them into payload offsets.  Other
+// rows: bm_in |= candidates with key > T; bm_cand := candidates with key == T; if all ties
+// are needed they are merged at once, otherwise the per-tile tie counts feed the ordered
+// pick below.  grid = (nbt, rows).
 // ------------------------------------------------------------------------------------
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
                const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-               const uint32_t *__restrict__ bm_ge_all, const float *__restrict__ stash_all,
+               const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
+               const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ cnt_gt_all,
+               uint32_t *__restrict__ cnt_eq_all,
                uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
                uint32_t *__restrict__ cnt_tie_all, int64_t d, int64_t wp, int64_t nbt, int64_t nt4k)
 {
@@ -551,34 +541,24 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
     const bool all_ties = s.k3 == s.c3;
     uint32_t nt = 0;
-    if (hit[row]) {                                   // values come from the dense pass's stash
-        const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
-        const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
-        const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
-        uint32_t ge[4];
-#pragma unroll
-        for (int m = 0; m < 4; ++m) ge[m] = w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
-        uint32_t rank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
-#pragma unroll
-        for (int m = 0; m < 4; ++m) {
-            if (w0 + m >= wp) continue;
-            const uint32_t cand = bm_cand[w0 + m];
-            uint32_t word = ge[m], keep = bm_in[w0 + m], tie = 0;
-            while (word) {
-                const int bit = __ffs(word) - 1;
-                word &= word - 1;
-                if ((cand >> bit) & 1u) {
-                    const uint32_t key = key_of(stash[rank]);
-                    if (key > T) keep |= 1u << bit;
-                    else if (key == T) tie |= 1u << bit;
-                }
-                ++rank;
-            }
-            if (all_ties) keep |= tie;
-            bm_in[w0 + m] = keep;
-            bm_cand[w0 + m] = tie;
-            nt += __popc(tie);
+    if (hit[row]) {                                   // the tiles' lists hold the values
+        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        uint32_t gt = 0, eq = 0;
+        for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
+            const uint32_t key = key_of(tl.val[e]);
+            gt += key > T;
+            eq += key == T;
         }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            gt += __shfl_xor_sync(kFull, gt, o);
+            eq += __shfl_xor_sync(kFull, eq, o);
+        }
+        if (tl.any && (threadIdx.x & 31) == 0) {
+            cnt_gt_all[(int64_t)row * nt4k + tl.tile] = gt;
+            cnt_eq_all[(int64_t)row * nt4k + tl.tile] = eq;
+        }
+        return;
     } else {
         const float *a = a_all + (int64_t)row * d;
         const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
@@ -603,10 +583,12 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
     if (threadIdx.x == 0) cnt_tie_all[(int64_t)row * nbt + blockIdx.x] = total;
 }
 
-// exclusive scan of the per-tile counts of every row, in place.  grid = (rows).
+// Exclusive scan of the per-tile counts of the rows whose guess failed, in place
+// (skip_hit: rows with lists are left alone).  grid = (rows).
 __global__ void __launch_bounds__(kBlock)
-k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt)
+k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__restrict__ hit)
 {
+    if (hit[blockIdx.x]) return;
     uint32_t *cnt = cnt_all + (int64_t)blockIdx.x * nbt;
     uint32_t carry = 0;
     for (int64_t c = 0; c < nbt; c += kBlock) {
@@ -616,6 +598,48 @@ k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt)
         const uint32_t ex = block_excl_scan(v, total);
         if (t < nbt) cnt[t] = carry + ex;
         carry += total;
+    }
+}
+
+// Rows with lists: from the per-tile counts of keys above / equal to the threshold to, per
+// tile, the rank of its first tie among the row's ties (cnt_eq) and the payload offset of its
+// first kept coordinate (cnt_gt); a tile keeps its keys above T and those of its ties whose
+// rank is below k3.  Every eighth tile's offset is also the offset of its 32768-coordinate
+// span (cnt_fin), which the server aggregation uses.  A thread owns a contiguous run of
+// tiles.  grid = (rows).
+__global__ void __launch_bounds__(kBlock)
+k_scan_lists(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+             uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all,
+             uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt)
+{
+    const int row = blockIdx.x;
+    if (!hit[row]) return;
+    const Sel s = sel_all[row];
+    const bool all_ties = s.k3 == s.c3;
+    uint32_t *gt = cnt_gt_all + (int64_t)row * nt4k, *eq = cnt_eq_all + (int64_t)row * nt4k;
+    uint32_t *fin = cnt_fin_all + (int64_t)row * nbt;
+    const int64_t per = (nt4k + kBlock - 1) / kBlock;
+    const int64_t t0 = min((int64_t)threadIdx.x * per, nt4k), t1 = min(t0 + per, nt4k);
+    uint32_t sum_eq = 0;
+    for (int64_t t = t0; t < t1; ++t) sum_eq += eq[t];
+    uint32_t total;
+    uint32_t tie_rank = block_excl_scan(sum_eq, total);
+    uint32_t sum_keep = 0;
+    for (int64_t t = t0; t < t1; ++t) {
+        const uint32_t e = eq[t];
+        const uint32_t take = all_ties ? e : (tie_rank >= s.k3 ? 0u : min(e, s.k3 - tie_rank));
+        eq[t] = tie_rank;
+        tie_rank += e;
+        const uint32_t keep = gt[t] + take;
+        gt[t] = keep;
+        sum_keep += keep;
+    }
+    uint32_t off = block_excl_scan(sum_keep, total);
+    for (int64_t t = t0; t < t1; ++t) {
+        const uint32_t keep = gt[t];
+        gt[t] = off;
+        if (t % kTilesPerBlock == 0) fin[t / kTilesPerBlock] = off;
+        off += keep;
     }
 }
 
@@ -631,16 +655,18 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t word, uint32_t coun
 }
 
 // ------------------------------------------------------------------------------------
-// Ties: keep those of global rank < k3 in index order (only if not all are kept), then
-// count the kept coordinates of every tile.  A thread owns 4 consecutive bitmap words.
-// grid = (nbt, rows).
+// Ties (rows whose guess failed): keep those of global rank < k3 in index order (only if
+// not all are kept), then count the kept coordinates of every tile.  A thread owns 4
+// consecutive bitmap words.  grid = (nbt, rows).
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
-k_topk_ties(const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
+k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+            uint32_t *__restrict__ bm_in_all,
             const uint32_t *__restrict__ bm_cand_all, const uint32_t *__restrict__ tie_off_all,
             uint32_t *__restrict__ cnt_fin_all, int64_t wp, int64_t nbt)
 {
     const int row = blockIdx.y;
+    if (hit[row]) return;                             // rows with lists have no bitmaps
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
     const uint32_t *bm_tie = bm_cand_all + (int64_t)row * wp;
     const Sel s = sel_all[row];
@@ -670,48 +696,69 @@ k_topk_ties(const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
 }
 
 // ------------------------------------------------------------------------------------
-// Ordered compaction of the selection bitmap into the payload's index list (increasing).
-// A thread owns 4 consecutive bitmap words; ranks come from popcount scans.
-// grid = (nbt, rows).
+// Ordered compaction into the payload (indices increasing).  grid = (nbt, rows).
+// Rows with lists: a warp walks its tile's list in order; an entry is kept if its key is
+// above T, or equal to T with tie rank below k3; positions come from ballots, and the value
+// is written with the index.  Other rows: from the selection bitmap; a thread owns 4
+// consecutive bitmap words, ranks come from popcount scans, values follow in k_topk_gather.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
 k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
-                const uint32_t *__restrict__ hit, const uint32_t *__restrict__ bm_ge_all,
-                const float *__restrict__ stash_all, uint32_t *__restrict__ idx_all,
+                const uint32_t *__restrict__ hit, const Sel *__restrict__ sel_all,
+                const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
+                const uint32_t *__restrict__ stash_cnt_all, const uint32_t *__restrict__ cnt_gt_all,
+                const uint32_t *__restrict__ cnt_eq_all, uint32_t *__restrict__ idx_all,
                 float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k)
 {
     const int row = blockIdx.y;
-    const uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
-    const bool stashed = hit[row] != 0;               // then the values are at hand as well
-    const int64_t tile = (int64_t)blockIdx.x * (kTileWords / 128) + (threadIdx.x >> 5);
-    const float *stash = stash_all + ((int64_t)row * nt4k + tile) * kStashCap;
-    uint32_t keep[4], ge[4];
-#pragma unroll
-    for (int m = 0; m < 4; ++m) {
-        keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
-        ge[m] = stashed && w0 + m < wp ? bm_ge_all[(int64_t)row * wp + w0 + m] : 0u;
+    if (hit[row]) {
+        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        if (!tl.any) return;
+        const Sel s = sel_all[row];
+        const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
+        const bool all_ties = s.k3 == s.c3;
+        const int lane = threadIdx.x & 31;
+        const uint32_t lt = (1u << lane) - 1u;
+        uint32_t out = cnt_gt_all[(int64_t)row * nt4k + tl.tile];
+        uint32_t tie_rank = cnt_eq_all[(int64_t)row * nt4k + tl.tile];
+        const uint32_t base = (uint32_t)(tl.tile * kSub);
+        for (uint32_t e0 = 0; e0 < tl.cnt; e0 += 32) {          // warp-uniform bounds
+            const uint32_t e = e0 + lane;
+            const bool valid = e < tl.cnt;
+            const float v = valid ? tl.val[e] : 0.0f;
+            const uint32_t key = key_of(v);
+            const bool eq = valid && key == T;
+            const uint32_t eqm = __ballot_sync(kFull, eq);
+            const bool keep = valid && (key > T || (eq && (all_ties || tie_rank + __popc(eqm & lt) < s.k3)));
+            const uint32_t km = __ballot_sync(kFull, keep);
+            const uint32_t at = out + __popc(km & lt);
+            if (keep && at < k) {
+                idx[at] = base + tl.pos[e];
+                val[at] = v;
+            }
+            out += __popc(km);
+            tie_rank += __popc(eqm);
+        }
+        return;
     }
+    const uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+    uint32_t keep[4];
+#pragma unroll
+    for (int m = 0; m < 4; ++m) keep[m] = w0 + m < wp ? bm_in[w0 + m] : 0u;
     uint32_t total;
     uint32_t rank = block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total) +
                     fin_off_all[(int64_t)row * nbt + blockIdx.x];
-    uint32_t srank = warp_excl_sum(__popc(ge[0]) + __popc(ge[1]) + __popc(ge[2]) + __popc(ge[3]));
 #pragma unroll
     for (int m = 0; m < 4; ++m) {
-        uint32_t word = stashed ? ge[m] : keep[m];
+        uint32_t word = keep[m];
         while (word) {
             const int bit = __ffs(word) - 1;
             word &= word - 1;
-            if ((keep[m] >> bit) & 1u) {
-                if (rank < k) {
-                    idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
-                    if (stashed) val[rank] = stash[srank];
-                }
-                ++rank;
-            }
-            ++srank;
+            if (rank < k) idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
+            ++rank;
         }
     }
 }
@@ -833,7 +880,8 @@ static void free_ws(TopkWorkspace *w)
 {
     cudaFree(w->hist); cudaFree(w->sel); cudaFree(w->bm_in); cudaFree(w->bm_cand);
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
-    cudaFree(w->bm_ge); cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->ovf); cudaFree(w->stash);
+    cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->ovf); cudaFree(w->stash);
+    cudaFree(w->stash_pos); cudaFree(w->stash_cnt); cudaFree(w->cnt_gt); cudaFree(w->cnt_eq);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
 }
@@ -859,12 +907,15 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         get((void **)&w->sel, (size_t)rows * sizeof(Sel));
         get((void **)&w->bm_in, (size_t)rows * w->wp * 4);
         get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
-        get((void **)&w->bm_ge, (size_t)rows * w->wp * 4);
         get((void **)&w->floor_bucket, (size_t)rows * 4);
         get((void **)&w->hit, (size_t)rows * 4);
         get((void **)&w->ovf, (size_t)rows * 4);
         w->nt4k = (d + kSub - 1) / kSub;
         get((void **)&w->stash, (size_t)rows * w->nt4k * kStashCap * 4);
+        get((void **)&w->stash_pos, (size_t)rows * w->nt4k * kStashCap * 2);
+        get((void **)&w->stash_cnt, (size_t)rows * w->nt4k * 4);
+        get((void **)&w->cnt_gt, (size_t)rows * w->nt4k * 4);
+        get((void **)&w->cnt_eq, (size_t)rows * w->nt4k * 4);
         if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
         get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
         get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
@@ -886,7 +937,7 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
     *val = w->val + (int64_t)row * w->k;
 }
 
-constexpr int kSelectLaunches = 15;
+constexpr int kSelectLaunches = 16;
 int topk_launches_per_step(int) { return 2 * kSelectLaunches + 1; }
 
 template <bool HAS_B>
@@ -900,20 +951,21 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
-    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->bm_ge, w->hist, w->stash, w->ovf, w->d, w->wp, vec_ok);
+    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->ovf, w->d, vec_ok);
     k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->ovf, w->hit);
     k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
     k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok);
-    k_topk_split<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_ge, w->stash, w->bm_in, w->bm_cand, w->hist, w->wp, w->nt4k);
+    k_topk_split<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
-    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->stash, w->bm_cand, w->hist, w->d, w->wp, w->nt4k);
+    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->bm_cand, w->hist, w->d, w->wp, w->nt4k);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
-    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_ge, w->stash, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k);
-    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt);
-    k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
-    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt);
-    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->hit, w->bm_ge, w->stash, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k);
+    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k);
+    k_scan_lists<<<w->rows, kBlock, 0, st>>>(w->sel, w->hit, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt);
+    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
+    k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
+    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit);
+    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
         k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);
