@@ -424,30 +424,75 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
         for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
 }
 
-// In the list passes below a block owns the 8 tiles of one 32768-coordinate span and a warp
-// one tile: lane L reads entries L, L + 32, ... of the tile's list (coalesced).
-constexpr int kTilesPerBlock = kTileWords * 32 / kSub;
+// In the list passes below a warp owns kWarpTiles consecutive tiles and a block
+// kListTiles; lane L reads entries L, L + 32, ... of a tile's list (coalesced).  The passes
+// are bound by memory latency, so the first kPre chunks of every tile of the warp are loaded
+// before any is used.  Blocks beyond the last tile return (the grid is sized for the
+// bitmap passes of the rows whose guess failed).
+constexpr int kTilesPerBlock = kTileWords * 32 / kSub;      // tiles per 32768-coordinate span
+constexpr int kWarpTiles = 2;
+constexpr int kListTiles = kWarpTiles * (kBlock / 32);
+constexpr int kPre = 4;
 
-struct TileList {
-    const float *val;
-    const uint16_t *pos;
-    uint32_t cnt;
-    int64_t tile;        // index of the tile inside its row
-    bool any;
+struct WarpLists {
+    const float *val[kWarpTiles];
+    const uint16_t *pos[kWarpTiles];
+    uint32_t cnt[kWarpTiles];
+    int64_t tile[kWarpTiles];      // index of the tile inside its row (>= nt4k: none, cnt = 0)
 };
 
-__device__ __forceinline__ TileList tile_list(const float *stash_all, const uint16_t *stash_pos_all,
-                                              const uint32_t *stash_cnt_all, int row, int64_t nt4k)
+__device__ __forceinline__ WarpLists warp_lists(const float *stash_all, const uint16_t *stash_pos_all,
+                                                const uint32_t *stash_cnt_all, int row, int64_t nt4k)
 {
-    TileList t;
-    t.tile = (int64_t)blockIdx.x * kTilesPerBlock + (threadIdx.x >> 5);
-    t.any = t.tile < nt4k;
-    const int64_t g = (int64_t)row * nt4k + (t.any ? t.tile : 0);
-    t.val = stash_all + g * kStashCap;
-    t.pos = stash_pos_all + g * kStashCap;
-    t.cnt = t.any ? min(stash_cnt_all[g], (uint32_t)kStashCap) : 0u;
-    return t;
+    WarpLists w;
+    const int64_t t0 = ((int64_t)blockIdx.x * (kBlock / 32) + (threadIdx.x >> 5)) * kWarpTiles;
+#pragma unroll
+    for (int m = 0; m < kWarpTiles; ++m) {
+        w.tile[m] = t0 + m;
+        const bool any = w.tile[m] < nt4k;
+        const int64_t g = (int64_t)row * nt4k + (any ? w.tile[m] : 0);
+        w.val[m] = stash_all + g * kStashCap;
+        w.pos[m] = stash_pos_all + g * kStashCap;
+        w.cnt[m] = any ? min(stash_cnt_all[g], (uint32_t)kStashCap) : 0u;
+    }
+    return w;
 }
+
+// f(value) for every entry of the warp's lists.
+template <typename F>
+__device__ __forceinline__ void for_each_listed(const WarpLists &w, F f)
+{
+    const uint32_t lane = threadIdx.x & 31;
+    float v[kWarpTiles][kPre];
+#pragma unroll
+    for (int m = 0; m < kWarpTiles; ++m)
+#pragma unroll
+        for (int i = 0; i < kPre; ++i) v[m][i] = lane + 32 * i < w.cnt[m] ? w.val[m][lane + 32 * i] : 0.0f;
+#pragma unroll
+    for (int m = 0; m < kWarpTiles; ++m) {
+#pragma unroll
+        for (int i = 0; i < kPre; ++i)
+            if (lane + 32 * i < w.cnt[m]) f(v[m][i]);
+        for (uint32_t e = lane + 32 * kPre; e < w.cnt[m]; e += 32) f(w.val[m][e]);
+    }
+}
+
+struct HistLevel2 {
+    uint32_t *h, b1;
+    __device__ __forceinline__ void operator()(float v) const
+    {
+        const uint32_t key = key_of(v);
+        if ((key >> 20) == b1) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
+    }
+};
+struct HistLevel3 {
+    uint32_t *h, pre;
+    __device__ __forceinline__ void operator()(float v) const
+    {
+        const uint32_t key = key_of(v);
+        if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+    }
+};
 
 // After a successful guess: the level-2 histogram of the listed values that fall into the
 // threshold bucket (what the second dense pass would have produced).  grid = (nbt, rows).
@@ -458,15 +503,11 @@ k_topk_split(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
 {
     __shared__ uint32_t h[kBins2];
     const int row = blockIdx.y;
-    if (!hit[row]) return;
+    if (!hit[row] || (int64_t)blockIdx.x * kListTiles >= nt4k) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
-    const uint32_t b1 = sel_all[row].b1;
-    const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
-    for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
-        const uint32_t key = key_of(tl.val[e]);
-        if ((key >> 20) == b1) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
-    }
+    for_each_listed(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k),
+                    HistLevel2{h, sel_all[row].b1});
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
     for (int t = threadIdx.x; t < kBins2; t += kBlock)
@@ -493,11 +534,8 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const uint32_t *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
     if (hit[row]) {                                   // the tiles' lists hold the values
-        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
-        for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
-            const uint32_t key = key_of(tl.val[e]);
-            if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
-        }
+        if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
+        for_each_listed(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k), HistLevel3{h, pre});
     } else {                                          // classic path: gather a and b
         const float *a = a_all + (int64_t)row * d;
         const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
@@ -542,21 +580,34 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const bool all_ties = s.k3 == s.c3;
     uint32_t nt = 0;
     if (hit[row]) {                                   // the tiles' lists hold the values
-        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
-        uint32_t gt = 0, eq = 0;
-        for (uint32_t e = threadIdx.x & 31; e < tl.cnt; e += 32) {
-            const uint32_t key = key_of(tl.val[e]);
-            gt += key > T;
-            eq += key == T;
-        }
+        if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
+        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        const uint32_t lane = threadIdx.x & 31;
+        float v[kWarpTiles][kPre];
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) {
-            gt += __shfl_xor_sync(kFull, gt, o);
-            eq += __shfl_xor_sync(kFull, eq, o);
-        }
-        if (tl.any && (threadIdx.x & 31) == 0) {
-            cnt_gt_all[(int64_t)row * nt4k + tl.tile] = gt;
-            cnt_eq_all[(int64_t)row * nt4k + tl.tile] = eq;
+        for (int m = 0; m < kWarpTiles; ++m)
+#pragma unroll
+            for (int i = 0; i < kPre; ++i) v[m][i] = lane + 32 * i < w.cnt[m] ? w.val[m][lane + 32 * i] : 0.0f;
+#pragma unroll
+        for (int m = 0; m < kWarpTiles; ++m) {
+            uint32_t gt = 0, eq = 0;
+#pragma unroll
+            for (int i = 0; i < kPre; ++i)
+                if (lane + 32 * i < w.cnt[m]) { gt += key_of(v[m][i]) > T; eq += key_of(v[m][i]) == T; }
+            for (uint32_t e = lane + 32 * kPre; e < w.cnt[m]; e += 32) {
+                const uint32_t key = key_of(w.val[m][e]);
+                gt += key > T;
+                eq += key == T;
+            }
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) {
+                gt += __shfl_xor_sync(kFull, gt, o);
+                eq += __shfl_xor_sync(kFull, eq, o);
+            }
+            if (w.tile[m] < nt4k && lane == 0) {
+                cnt_gt_all[(int64_t)row * nt4k + w.tile[m]] = gt;
+                cnt_eq_all[(int64_t)row * nt4k + w.tile[m]] = eq;
+            }
         }
         return;
     } else {
@@ -714,32 +765,55 @@ k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restri
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
     if (hit[row]) {
-        const TileList tl = tile_list(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
-        if (!tl.any) return;
+        if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
+        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
         const Sel s = sel_all[row];
         const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
         const bool all_ties = s.k3 == s.c3;
-        const int lane = threadIdx.x & 31;
+        const uint32_t lane = threadIdx.x & 31;
         const uint32_t lt = (1u << lane) - 1u;
-        uint32_t out = cnt_gt_all[(int64_t)row * nt4k + tl.tile];
-        uint32_t tie_rank = cnt_eq_all[(int64_t)row * nt4k + tl.tile];
-        const uint32_t base = (uint32_t)(tl.tile * kSub);
-        for (uint32_t e0 = 0; e0 < tl.cnt; e0 += 32) {          // warp-uniform bounds
-            const uint32_t e = e0 + lane;
-            const bool valid = e < tl.cnt;
-            const float v = valid ? tl.val[e] : 0.0f;
-            const uint32_t key = key_of(v);
-            const bool eq = valid && key == T;
-            const uint32_t eqm = __ballot_sync(kFull, eq);
-            const bool keep = valid && (key > T || (eq && (all_ties || tie_rank + __popc(eqm & lt) < s.k3)));
-            const uint32_t km = __ballot_sync(kFull, keep);
-            const uint32_t at = out + __popc(km & lt);
-            if (keep && at < k) {
-                idx[at] = base + tl.pos[e];
-                val[at] = v;
+        float v[kWarpTiles][kPre];
+        uint32_t ps[kWarpTiles][kPre], out[kWarpTiles], tie_rank[kWarpTiles];
+#pragma unroll
+        for (int m = 0; m < kWarpTiles; ++m) {
+            const int64_t g = (int64_t)row * nt4k + (w.tile[m] < nt4k ? w.tile[m] : 0);
+            out[m] = cnt_gt_all[g];
+            tie_rank[m] = cnt_eq_all[g];
+#pragma unroll
+            for (int i = 0; i < kPre; ++i) {
+                const bool valid = lane + 32 * i < w.cnt[m];
+                v[m][i] = valid ? w.val[m][lane + 32 * i] : 0.0f;
+                ps[m][i] = valid ? w.pos[m][lane + 32 * i] : 0u;
             }
-            out += __popc(km);
-            tie_rank += __popc(eqm);
+        }
+#pragma unroll
+        for (int m = 0; m < kWarpTiles; ++m) {
+            const uint32_t base = (uint32_t)(w.tile[m] * kSub);
+            // one chunk of 32 entries in index order: ballots give the tie ranks and the
+            // payload positions
+            auto chunk = [&](uint32_t e, float val_e, uint32_t pos_e) {
+                const bool valid = e < w.cnt[m];
+                const uint32_t key = key_of(val_e);
+                const bool eq = valid && key == T;
+                const uint32_t eqm = __ballot_sync(kFull, eq);
+                const bool keep = valid && (key > T || (eq && (all_ties || tie_rank[m] + __popc(eqm & lt) < s.k3)));
+                const uint32_t km = __ballot_sync(kFull, keep);
+                const uint32_t at = out[m] + __popc(km & lt);
+                if (keep && at < k) {
+                    idx[at] = base + pos_e;
+                    val[at] = val_e;
+                }
+                out[m] += __popc(km);
+                tie_rank[m] += __popc(eqm);
+            };
+#pragma unroll
+            for (int i = 0; i < kPre; ++i)
+                if (32u * i < w.cnt[m]) chunk(lane + 32 * i, v[m][i], ps[m][i]);       // warp-uniform
+            for (uint32_t e0 = 32 * kPre; e0 < w.cnt[m]; e0 += 32) {
+                const uint32_t e = e0 + lane;
+                const bool valid = e < w.cnt[m];
+                chunk(e, valid ? w.val[m][e] : 0.0f, valid ? (uint32_t)w.pos[m][e] : 0u);
+            }
         }
         return;
     }
@@ -766,7 +840,7 @@ k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restri
 // ------------------------------------------------------------------------------------
 // Payload values and the state update at the kept coordinates (Algorithm 1 lines 6 / 10):
 // val = u_j = a_j - b_j, b_j += u_j.  One thread per payload entry.  grid = (ceil(k/256), rows).
-// Rows whose values were already written from the stash only update b.
+// Rows whose values were already written from the lists only update b.
 // ------------------------------------------------------------------------------------
 template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
