@@ -106,8 +106,9 @@ void cdadam_destroy(cdadam_ctx *ctx);
  * Allocates no device memory.  Where the step is launch-bound (scaled sign, every pass a
  * single wave of blocks, about n*d <= 2.4e6) the scales are finished inside the passes
  * (3 launches instead of 5) and, from the second step on the same gradient buffer, the
- * launches are replayed from a CUDA graph owned by the context.  After the stream has
- * completed, cdadam_params() holds x_{t+1}.
+ * launches are replayed from a CUDA graph owned by the context; so are the some thirty
+ * launches of every top-k step of Algorithm 1.  After the stream has completed,
+ * cdadam_params() holds x_{t+1}.
  */
 int cdadam_step(cdadam_ctx *ctx, const float *grads, void *stream);
 

@@ -154,9 +154,10 @@ struct cdadam_ctx {
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
     // host-gradient staging
     float *stage = nullptr;
-    // Replay of the scaled-sign step as a CUDA graph where the step is launch-bound (grids of
-    // one wave).  A graph is recorded for a gradient buffer seen twice; the key holds every
-    // launch argument that changes between steps.
+    // Replay of a step as a CUDA graph where launches matter: scaled sign with grids of one
+    // wave, and top-k (some thirty launches, most of them short).  A graph is recorded for a
+    // gradient buffer seen twice; the key holds every launch argument that changes between
+    // steps.
     struct StepGraph {
         const void *grads = nullptr;
         bool bf16 = false, pending = false;
@@ -290,12 +291,29 @@ void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec,
     prof_mark(c, st);
 }
 
+// One iteration of Algorithm 1 with the top-k compressor, queued on st.  No host state changes.
+void enqueue_topk_step(cdadam_ctx *c, const void *grads_in, bool, bool vec, cudaStream_t st)
+{
+    const float *grads = static_cast<const float *>(grads_in);
+    const bool svec = c->d % 4 == 0;
+    topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
+    prof_mark(c, st);
+    topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
+    prof_mark(c, st);
+    topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // lines 9-10, 12
+    prof_mark(c, st);
+    launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+    prof_mark(c, st);
+}
+
 // Launch-bound steps: replays the recorded graph of this step on st and returns true, or
 // returns false when the step has to be queued launch by launch (first sighting of the
 // gradient buffer, timing on, recording unavailable).
-bool replay_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
+typedef void (*enqueue_fn)(cdadam_ctx *, const void *, bool, bool, cudaStream_t);
+
+bool replay_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st, enqueue_fn enqueue)
 {
-    if (!c->fuse_finish || !c->graphs_ok || c->prof_on || c->mode == CDADAM_NAIVE) return false;
+    if (!c->graphs_ok || c->prof_on) return false;
     cdadam_ctx::StepGraph *slot = nullptr, *oldest = &c->graphs[0];
     for (auto &g : c->graphs) {
         if (g.hits && g.grads == grads_in && g.bf16 == bf16 && g.pending == c->pending && g.cur == c->cur) slot = &g;
@@ -315,7 +333,7 @@ bool replay_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, 
         bool ok = c->cap_stream || cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) == cudaSuccess;
         ok = ok && cudaStreamBeginCapture(c->cap_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
         if (ok) {
-            enqueue_sign_step(c, grads_in, bf16, vec, c->cap_stream);
+            enqueue(c, grads_in, bf16, vec, c->cap_stream);
             ok = cudaStreamEndCapture(c->cap_stream, &graph) == cudaSuccess && graph;
         }
         ok = ok && cudaGraphInstantiate(&slot->exec, graph, 0) == cudaSuccess;
@@ -462,7 +480,8 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
     const bool svec = c->d % 4 == 0;
     if (c->comp == CDADAM_SIGN) {
         const void *gin = bf16 ? grads_in : grads;
-        if (!replay_sign_step(c, gin, bf16, vec, st)) enqueue_sign_step(c, gin, bf16, vec, st);
+        const bool launch_bound = c->fuse_finish && !naive;
+        if (!(launch_bound && replay_step(c, gin, bf16, vec, st, enqueue_sign_step))) enqueue_sign_step(c, gin, bf16, vec, st);
         c->cur ^= 1;
         c->pending = !naive;             // naive compression has no worker state to bring up to date
     } else if (naive && (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK)) {
@@ -489,14 +508,8 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
         launch_scatter_set(c->ghat_s, sidx, nullptr, c->k, c->d, 1, st);
         prof_mark(c, st);
     } else if (c->comp == CDADAM_TOPK && !ef) {
-        topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
-        prof_mark(c, st);
-        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
-        prof_mark(c, st);
-        topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // lines 9-10, 12
-        prof_mark(c, st);
-        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
-        prof_mark(c, st);
+        // some thirty launches, most of them short: replayed from a graph where possible
+        if (!replay_step(c, grads, false, vec, st, enqueue_topk_step)) enqueue_topk_step(c, grads, false, vec, st);
     } else if (c->comp == CDADAM_TOPK) {
         // classical error feedback: the delta buffers (ghat_w rows, gtil) first receive the
         // compressor inputs p = g + delta and p = mean + delta, are compressed in place, and

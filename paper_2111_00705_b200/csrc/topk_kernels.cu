@@ -33,7 +33,7 @@ constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
 constexpr int kHistStride = kBins1 + kBins2 + kBins3;
 constexpr int kTileWords = 1024;      // bitmap words per block in the sparse passes
 constexpr int kStashCap = 512;        // values kept per 4096-coordinate tile by the dense pass
-constexpr uint32_t kGuessMargin = 2;  // level-1 buckets kept below the last threshold bucket
+constexpr uint32_t kGuessMargin = 1;  // level-1 buckets kept below the last threshold bucket
 
 struct Sel {                          // outcome of the three levels for one row
     uint32_t b1, k1, c1;              // bucket, entries still to take inside it, its size

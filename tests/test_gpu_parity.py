@@ -462,13 +462,18 @@ def test_non_finite_gradients_neither_hang_nor_fault(comp):
     assert torch.isfinite(ok.params()).all()
 
 
-@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
-def test_replayed_launch_bound_steps_match_oracle(mode):
-    """Small problems replay their launches from a recorded graph once a gradient buffer has
-    been seen twice.  Two buffers in turn, a side stream, a read of the worker states (which
-    applies the deferred payload and changes the next step's arguments) and a change of step
-    size (a launch argument) in between: every payload and state vector against the oracle."""
-    w = synth.Workload("G1", 5 * 4096 + 13, 4, synth.SIGN, 14, offsets=np.array([0, 4000, 9000, 5 * 4096 + 13]), seed=21)
+@pytest.mark.parametrize("comp,mode", [(cd.SIGN, cd.MARKOV), (cd.SIGN, cd.EF), (cd.TOPK, cd.MARKOV)])
+def test_replayed_steps_match_oracle(comp, mode):
+    """Launch-bound scaled-sign problems and every top-k step of Algorithm 1 replay their
+    launches from a recorded graph once a gradient buffer has been seen twice.  Two buffers
+    in turn, a side stream, a read of the worker states (which applies the deferred payload
+    and changes the next step's arguments) and a change of step size (a launch argument) in
+    between: every payload and state vector against the oracle."""
+    d = 5 * 4096 + 13
+    if comp == cd.SIGN:
+        w = synth.Workload("G1", d, 4, synth.SIGN, 14, offsets=np.array([0, 4000, 9000, d]), seed=21)
+    else:
+        w = synth.Workload("G2", d, 4, synth.TOPK, 14, k=300, seed=22)
     g, o = make_pair(w, mode=mode)
     bufs = [torch.empty(w.n * w.d, device="cuda") for _ in range(2)]
     side = torch.cuda.Stream()
