@@ -168,7 +168,10 @@ struct cdadam_ctx {
     StepGraph graphs[4];
     uint64_t graph_clock = 0;
     cudaStream_t cap_stream = nullptr;
-    bool graphs_ok = true;       // cleared for good when recording fails once
+    bool graphs_ok = true;       // cleared for good when recording fails once, or when graphs go
+                                 // stale too often (a step size that changes every step)
+    int graph_drops = 0;
+    std::vector<cudaGraphExec_t> retired;   // stale graphs, possibly still running: freed with the context
     // optional per-kernel timing: events[step][0..nslots] recorded around every stage
     bool prof_on = false;
     std::vector<cudaEvent_t> prof_ev;   // groups of (nslots + 1) events, one group per step
@@ -252,12 +255,22 @@ void apply_lr(cdadam_ctx *c, float lr)
     c->hp.decay = c->wd != 0.0f;
 }
 
+constexpr int kMaxGraphDrops = 4;
+
+// A recorded graph whose launch arguments are stale.  It may still be running, so it is only
+// set aside; a context that keeps invalidating its graphs stops recording them.
+void retire_graph(cdadam_ctx *c, cdadam_ctx::StepGraph &g)
+{
+    if (g.exec) {
+        c->retired.push_back(g.exec);
+        if (++c->graph_drops > kMaxGraphDrops * 4) c->graphs_ok = false;
+    }
+    g = cdadam_ctx::StepGraph{};
+}
+
 void drop_graphs(cdadam_ctx *c)
 {
-    for (auto &g : c->graphs) {
-        if (g.exec) cudaGraphExecDestroy(g.exec);
-        g = cdadam_ctx::StepGraph{};
-    }
+    for (auto &g : c->graphs) retire_graph(c, g);
 }
 
 // The three to five launches of one scaled-sign step, queued on st.  Changes no host state.
@@ -320,8 +333,7 @@ bool replay_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaS
         if (g.stamp < oldest->stamp) oldest = &g;
     }
     if (!slot) {                                               // remember the sighting only
-        if (oldest->exec) cudaGraphExecDestroy(oldest->exec);
-        *oldest = cdadam_ctx::StepGraph{};
+        retire_graph(c, *oldest);
         oldest->grads = grads_in; oldest->bf16 = bf16; oldest->pending = c->pending; oldest->cur = c->cur;
         oldest->hits = 1; oldest->stamp = ++c->graph_clock;
         return false;
@@ -426,6 +438,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wdone); cudaFree(c->sdone);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
     drop_graphs(c);
+    for (cudaGraphExec_t e : c->retired) cudaGraphExecDestroy(e);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
     for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
     for (cudaEvent_t e : c->prof_pool) cudaEventDestroy(e);

@@ -33,7 +33,7 @@ constexpr int kBins1 = 2048, kBins2 = 2048, kBins3 = 512;
 constexpr int kHistStride = kBins1 + kBins2 + kBins3;
 constexpr int kTileWords = 1024;      // bitmap words per block in the sparse passes
 constexpr int kStashCap = 512;        // values kept per 4096-coordinate tile by the dense pass
-constexpr uint32_t kGuessMargin = 1;  // level-1 buckets kept below the last threshold bucket
+constexpr uint32_t kGuessMargin = 1;  // level-1 buckets (1/8 octave each) kept below the last threshold bucket
 
 struct Sel {                          // outcome of the three levels for one row
     uint32_t b1, k1, c1;              // bucket, entries still to take inside it, its size
@@ -180,8 +180,10 @@ k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, in
             else if (level == 1) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
             else {
                 sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
-                // guess for the next selection of this row: a little below this threshold
-                floor_bucket[row] = sel->b1 > kGuessMargin ? sel->b1 - kGuessMargin : 1u;
+                // guess for the next selection of this row: a little below this threshold,
+                // one bucket more after a guess that failed
+                const uint32_t margin = hit[row] ? kGuessMargin : kGuessMargin + 1u;
+                floor_bucket[row] = sel->b1 > margin ? sel->b1 - margin : 1u;
             }
         }
         above += c;

@@ -502,6 +502,32 @@ def test_replayed_steps_match_oracle(comp, mode):
     g.close(); o.close()
 
 
+@pytest.mark.parametrize("comp", [cd.SIGN, cd.TOPK])
+def test_replay_with_a_step_size_per_step_and_many_buffers(comp):
+    """A step size that changes every step makes recorded graphs stale every step (they are set
+    aside, and recording stops after a few rounds); six gradient buffers in rotation exceed
+    the four graphs a context keeps.  Results stay those of the oracle."""
+    d = 2 * 4096 + 5
+    w = synth.Workload("G3", d, 3, comp, 40, k=64 if comp == cd.TOPK else 0, seed=23)
+    g, o = make_pair(w)
+    bufs = [torch.empty(w.n * d, device="cuda") for _ in range(6)]
+    for t in range(1, 41):
+        grads = w.grads(t, "cpu")
+        buf = bufs[t % 6] if t > 12 else bufs[t % 2]
+        buf.copy_(grads.reshape(-1))
+        if t <= 24:
+            lr = 1e-3 / t
+            g.set_lr(lr); o.set_lr(lr)
+        g.step(buf)
+        o.step(grads.numpy())
+        if t % 8 == 0:
+            check_payloads(g, o, w)
+            for name in ("x", "m", "vhat", "gtil"):
+                assert np.array_equal(g.get_state(name).cpu().numpy().ravel(), o.state(name).ravel()), (t, name)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.close(); o.close()
+
+
 def test_step_on_a_capturing_stream_is_refused():
     g = cd.CDAdam(4096, 2, cd.SIGN)
     grads = torch.randn(2 * 4096, device="cuda")
