@@ -535,8 +535,11 @@ def test_step_on_a_capturing_stream_is_refused():
     torch.cuda.synchronize()
     side = torch.cuda.Stream()
     graph = torch.cuda.CUDAGraph()
+    other = torch.zeros(8, device="cuda")
+    torch.cuda.synchronize()
     with torch.cuda.stream(side):
         graph.capture_begin()
+        other.add_(1.0)                                   # the caller's own work is recorded
         rc = cd.lib().cdadam_step(g._h, ctypes.c_void_p(grads.data_ptr()), ctypes.c_void_p(side.cuda_stream))
         graph.capture_end()
     assert rc == cd.ERR_STATE and "captur" in cd.last_error()
