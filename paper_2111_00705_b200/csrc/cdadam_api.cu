@@ -1,5 +1,6 @@
 // C interface of the CD-Adam library (see include/cdadam.h): context, state buffers and the
 // per-step launch sequence.  No arithmetic of the method lives here.
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
@@ -145,6 +146,8 @@ struct cdadam_ctx {
     float *wscale[2] = {nullptr, nullptr}, *sscale = nullptr, *zero_scale = nullptr;
     dd *wpart = nullptr, *spart = nullptr;
     unsigned int *wdone = nullptr, *sdone = nullptr;   // tickets of the in-kernel scale finish
+    int wsplit = 1, ssplit = 1;  // blocks that share a segment in the separate scale kernel
+    dd *wsums = nullptr, *ssums = nullptr;
     bool fuse_finish = false;    // scales finished inside the worker / server pass
     int *error_flag = nullptr;   // device word set by a kernel whose bounded wait ran out
     int cur = 0;            // wscale[cur] holds the scales of the last worker payloads
@@ -191,11 +194,22 @@ int dev_zalloc(T **p, size_t count)
     return CDADAM_OK;
 }
 
+// Blocks of the separate scale kernel that share one segment: one per 4096 tiles, up to 32.
+int finalize_split(const TableSet &ts)
+{
+    int64_t most = 1;
+    for (size_t r = 0; r + 1 < ts.off.size(); ++r)
+        most = std::max(most, (ts.off[r + 1] - 1) / ts.tb.tile - ts.off[r] / ts.tb.tile + 1);
+    return (int)std::min<int64_t>(32, (most + 4095) / 4096);
+}
+
 int alloc_sign_buffers(cdadam_ctx *c)
 {
     const int q = c->ts.tb.q;
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->wdone); cudaFree(c->sdone);
+    cudaFree(c->wsums); cudaFree(c->ssums);
+    c->wsums = c->ssums = nullptr;
     int rc;
     if ((rc = dev_zalloc(&c->wscale[0], (size_t)c->n * q))) return rc;
     if ((rc = dev_zalloc(&c->wscale[1], (size_t)c->n * q))) return rc;
@@ -209,6 +223,11 @@ int alloc_sign_buffers(cdadam_ctx *c)
     // a fence and an atomic round trip: measured 12 % faster when all blocks of a pass are
     // resident at once (d = 65,536, n = 4) and 4 to 13 % slower on grids of many waves.
     c->fuse_finish = (int64_t)c->n * c->ts.tb.ntiles <= kFuseMaxBlocks && c->ts_s.tb.ntiles <= kFuseMaxBlocks;
+    // a segment of more than 4096 tiles is shared by several blocks of the scale kernel
+    c->wsplit = finalize_split(c->ts);
+    c->ssplit = finalize_split(c->ts_s);
+    if (c->wsplit > 1 && (rc = dev_zalloc(&c->wsums, (size_t)c->n * q * c->wsplit))) return rc;
+    if (c->ssplit > 1 && (rc = dev_zalloc(&c->ssums, (size_t)q * c->ssplit))) return rc;
     return CDADAM_OK;
 }
 
@@ -290,14 +309,14 @@ void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec,
                            c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
     prof_mark(c, st);
     if (!fuse) {
-        launch_finalize_scales(c->wpart, new_scale, tb, c->n, st);
+        launch_finalize_scales(c->wpart, new_scale, tb, c->n, st, c->wsplit, c->wsums, c->wdone);
         prof_mark(c, st);
     }
     launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, c->mode,
                        fuse ? c->sscale : nullptr, c->sdone, st);
     prof_mark(c, st);
     if (!fuse) {
-        launch_finalize_scales(c->spart, c->sscale, tbs, 1, st);
+        launch_finalize_scales(c->spart, c->sscale, tbs, 1, st, c->ssplit, c->ssums, c->sdone);
         prof_mark(c, st);
     }
     launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, c->mode, st);
@@ -435,7 +454,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
-    cudaFree(c->wdone); cudaFree(c->sdone);
+    cudaFree(c->wdone); cudaFree(c->sdone); cudaFree(c->wsums); cudaFree(c->ssums);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
     drop_graphs(c);
     for (cudaGraphExec_t e : c->retired) cudaGraphExecDestroy(e);

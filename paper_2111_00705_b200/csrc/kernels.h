@@ -17,9 +17,12 @@ void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint3
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
                         int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
                         unsigned int *done, cudaStream_t st);
-// Correctly rounded scale of every (row, segment) from the partial sums.
+// Correctly rounded scale of every (row, segment) from the partial sums.  split > 1 (segments
+// of very many tiles): that many blocks share a segment; split_sums holds rows x q x split
+// sums, split_done rows x q zeroed counters (left zeroed).
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
-                            cudaStream_t st);
+                            cudaStream_t st, int split = 1, dd *split_sums = nullptr,
+                            unsigned int *split_done = nullptr);
 // Server pass A (lines 8-9): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
 // sign(w) into sbits and writes partial sums of |w| to spart.  sscale != NULL: the scales are
 // finished in the same launch (done: q zeroed counters), as in the worker pass.

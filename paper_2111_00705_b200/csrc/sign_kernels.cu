@@ -404,6 +404,45 @@ k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Table
     }
 }
 
+// The same for segments of very many tiles (a flat 1.5e9-coordinate buffer has 91,553):
+// gridDim.z blocks share a (row, segment), each adds a contiguous run of its tiles; the block
+// that finishes last (ticket) adds the gridDim.z sums in block order.  Same value whichever
+// block that is; no block waits.  grid = (q, rows, split); done: rows x q zeroed counters,
+// left zeroed; sums: rows x q x split.
+__global__ void __launch_bounds__(kFinBlock)
+k_finalize_scales_split(const dd *__restrict__ part, float *__restrict__ scales, Tables tb,
+                        dd *sums, unsigned int *done)
+{
+    __shared__ int is_last;
+    const int r = blockIdx.x, row = blockIdx.y, z = blockIdx.z, nz = gridDim.z;
+    const int64_t lo = tb.off[r], hi = tb.off[r + 1];
+    const int64_t T0 = lo / tb.tile, T1 = (hi - 1) / tb.tile;
+    const int64_t per = (T1 - T0 + nz) / nz;              // tiles per block, rounded up
+    const int64_t A = T0 + z * per, B = min(A + per, T1 + 1);
+    const dd *p = part + (int64_t)row * tb.nparts;
+    dd acc = {0.0, 0.0};
+    for (int64_t T = A + threadIdx.x; T < B; T += kFinBlock)
+        acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
+    acc = block_sum<kFinBlock>(acc);
+    const int64_t slot = (int64_t)row * tb.q + r;
+    if (threadIdx.x == 0) {
+        sums[slot * nz + z] = acc;
+        __threadfence();
+        is_last = atomicAdd(done + slot, 1u) == (unsigned int)(nz - 1);
+    }
+    __syncthreads();
+    if (!is_last || threadIdx.x != 0) return;
+    __threadfence();
+    dd tot = {0.0, 0.0};
+    for (int i = 0; i < nz; ++i) {
+        const double2 v = __ldcg(reinterpret_cast<const double2 *>(sums + slot * nz + i));
+        tot = dd_add(tot, dd{v.x, v.y});
+    }
+    const double l1 = __dadd_rn(tot.hi, tot.lo);
+    scales[slot] = __double2float_rn(__ddiv_rn(l1, (double)(hi - lo)));
+    done[slot] = 0u;
+}
+
 // ------------------------------------------------------------------------------------
 // Server pass A.  grid = (ntiles).
 //
@@ -743,8 +782,13 @@ void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint3
 }
 
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
-                            cudaStream_t st)
+                            cudaStream_t st, int split, dd *split_sums, unsigned int *split_done)
 {
+    if (split > 1) {
+        dim3 grid((unsigned)tb.q, (unsigned)rows, (unsigned)split);
+        k_finalize_scales_split<<<grid, kFinBlock, 0, st>>>(part, scales, tb, split_sums, split_done);
+        return;
+    }
     dim3 grid((unsigned)tb.q, (unsigned)rows);
     k_finalize_scales<<<grid, kFinBlock, 0, st>>>(part, scales, tb);
 }

@@ -161,6 +161,15 @@ def test_sign_worker_counts_cover_table_and_sequential_server_sums(n):
     run_free(synth.Workload("N", 5 * 4096, n, synth.SIGN, 3, offsets=off, seed=n), 3)
 
 
+def test_segment_of_more_than_4096_tiles_is_summed_by_several_blocks():
+    """Flat buffer of 8195 tiles of 4096 coordinates: three blocks of the scale kernel share
+    the segment and the last one to finish adds their sums; a second, short segment beside it
+    is summed by one block (the others find nothing to add)."""
+    d = 8195 * 4096 + 3
+    off = np.array([0, d - 5000, d])
+    run_free(synth.Workload("LS", d, 1, synth.SIGN, 2, offsets=off, seed=31), 2, tile=4096)
+
+
 @pytest.mark.parametrize("n,launches", [(4, 3), (5, 5)])
 @pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
 def test_scales_finished_in_the_passes_or_by_their_own_kernel(n, launches, mode):
