@@ -452,6 +452,17 @@ k_finalize_scales_split(const dd *__restrict__ part, float *__restrict__ scales,
 // shared-memory load; the per-worker scales of the tile's segment sit in shared memory too.
 // ------------------------------------------------------------------------------------
 constexpr int kNC = 16;     // workers staged per chunk
+constexpr int kTabWorkers = 8;   // workers whose sum is read from the pattern table
+
+// Transpose of an 8x8 bit matrix held in 64 bits: bit (8 i + j) <-> bit (8 j + i)
+// (three rounds of masked swaps of 1x1, 2x2 and 4x4 blocks).
+__device__ __forceinline__ uint64_t transpose8x8(uint64_t x)
+{
+    x = (x & 0xAA55AA55AA55AA55ull) | ((x & 0x00AA00AA00AA00AAull) << 7) | ((x >> 7) & 0x00AA00AA00AA00AAull);
+    x = (x & 0xCCCC3333CCCC3333ull) | ((x & 0x0000CCCC0000CCCCull) << 14) | ((x >> 14) & 0x0000CCCC0000CCCCull);
+    x = (x & 0xF0F0F0F00F0F0F0Full) | ((x & 0x00000000F0F0F0F0ull) << 28) | ((x >> 28) & 0x00000000F0F0F0F0ull);
+    return x;
+}
 
 template <int VPT, int MODE>
 __global__ void __launch_bounds__(kBlock)
@@ -464,6 +475,10 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
     constexpr bool EF = MODE != 0;
     __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
     __shared__ float ssm[kNC];
+    // tab[p]: the sequential sum over the first nt workers of +-s_i with the signs of pattern
+    // p (bit i = worker i's sign bit), formed by the same additions in the same order as
+    // adding worker by worker, hence the same bits
+    __shared__ float tab[1 << kTabWorkers];
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t base = T * tb.tile;
@@ -477,9 +492,19 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         constexpr int kIter = kSpan * (kBlock / 32);      // per block per iteration
         const bool multi = n > kNC;
         const int g = lane >> 3, sh = (lane & 7) * 4;
+        // the table serves the first nt workers (only in the 8-coordinates-per-thread layout)
+        const int nt = (multi || VPT != 2) ? 0 : min(n, kTabWorkers);
         if (!multi) {
             if (threadIdx.x < n) ssm[threadIdx.x] = wscale[(int64_t)threadIdx.x * tb.q + first];
             __syncthreads();
+            if (nt > 0) {
+                if (threadIdx.x < (1 << nt)) {
+                    float t = 0.0f;
+                    for (int i = 0; i < nt; ++i) t = __fadd_rn(t, signed_scale((threadIdx.x >> i) & 1u, ssm[i]));
+                    tab[threadIdx.x] = t;
+                }
+                __syncthreads();
+            }
         }
         dd acc = {0.0, 0.0};
         for (int it = 0; it < tb.tile / kIter; ++it) {
@@ -508,8 +533,29 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                     wsm[warp][i][wd & 3][wd >> 2] = ld_ro_u32(wbits + (int64_t)(i0 + i) * wp + (wb >> 5) + wd);
                 }
                 if (multi) __syncthreads(); else __syncwarp();
+                if constexpr (VPT == 2) {
+                    if (nt > 0) {
+                        // byte i = worker i's sign bits of this thread's 8 coordinates; after the
+                        // transpose byte j = the workers' sign bits (the pattern) of coordinate j
+                        uint32_t lo = 0u, hi = 0u;
+#pragma unroll
+                        for (int i = 0; i < kTabWorkers; ++i) {
+                            if (i < nt) {
+                                const uint2 q2 = *reinterpret_cast<const uint2 *>(&wsm[warp][i][g][0]);
+                                const uint32_t b8 = ((q2.x >> sh) & 0xFu) | (((q2.y >> sh) & 0xFu) << 4);
+                                if (i < 4) lo |= b8 << (8 * i); else hi |= b8 << (8 * (i - 4));
+                            }
+                        }
+                        const uint64_t pat = transpose8x8(((uint64_t)hi << 32) | lo);
+                        const uint32_t plo = (uint32_t)pat, phi = (uint32_t)(pat >> 32);
+                        a[0][0] = tab[plo & 0xFFu];         a[0][1] = tab[(plo >> 8) & 0xFFu];
+                        a[0][2] = tab[(plo >> 16) & 0xFFu]; a[0][3] = tab[plo >> 24];
+                        a[1][0] = tab[phi & 0xFFu];         a[1][1] = tab[(phi >> 8) & 0xFFu];
+                        a[1][2] = tab[(phi >> 16) & 0xFFu]; a[1][3] = tab[phi >> 24];
+                    }
+                }
 #pragma unroll 4
-                for (int i = 0; i < nc; ++i) {
+                for (int i = nt; i < nc; ++i) {
                     const float s = ssm[i];
                     uint32_t W[VPT];
                     if constexpr (VPT == 4) {
