@@ -39,7 +39,7 @@ FALLBACK_HBM_GBS = 6650.0
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
     # k_worker_sign_ring: 2.656 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "84a00272e92be4b7", "bytes_per_launch": 4 * (1.797453e+09 + 8.5803776e+08)},
+    "C4": {"hash": "2625ca31ec76df80", "bytes_per_launch": 4 * (1.797405e+09 + 8.57283072e+08)},
 }
 
 
