@@ -897,13 +897,15 @@ __device__ __forceinline__ int64_t lower_bound_u32(const uint32_t *p, int64_t co
 }
 
 constexpr int kAggChunk = 64;      // workers whose entry ranges are searched at once
+constexpr int kAggPre = 16;        // workers whose first 256 entries are fetched before they are added
 
 __global__ void __launch_bounds__(kBlock)
 k_topk_aggregate(const uint32_t *__restrict__ idx_all, const float *__restrict__ val_all,
                  const uint32_t *__restrict__ fin_off_all, int64_t nbt, int n, int64_t k, int64_t d,
-                 float *__restrict__ ghat_s, int n_pow2)
+                 float *__restrict__ ghat_s, int n_pow2, const uint32_t *__restrict__ hit,
+                 const uint32_t *__restrict__ tile_off_all, int64_t nt4k)
 {
-    __shared__ float acc[kAggSpan];
+    __shared__ __align__(16) float acc[kAggSpan];
     __shared__ int64_t range[kAggChunk][2];
     const int64_t base = (int64_t)blockIdx.x * kAggSpan;
     const int64_t end = min(base + (int64_t)kAggSpan, d);
@@ -917,35 +919,87 @@ k_topk_aggregate(const uint32_t *__restrict__ idx_all, const float *__restrict__
             // enclosing compaction tile, whose bounds are the scanned tile counts
             const int i = i0 + (threadIdx.x >> 1), side = threadIdx.x & 1;
             const uint32_t *idx = idx_all + (int64_t)i * k;
-            int64_t t_lo = 0, t_hi = k;       // without tile counts (rand-k): the whole payload
-            if (fin_off_all) {
-                t_lo = fin_off_all[(int64_t)i * nbt + tile];
-                t_hi = tile + 1 < nbt ? (int64_t)fin_off_all[(int64_t)i * nbt + tile + 1] : k;
+            int64_t pos;
+            if (fin_off_all && hit[i] && base + kAggSpan <= d) {
+                // rows selected from lists have the payload offset of every 4096-coordinate
+                // tile: the span's entries are known without a search
+                const int64_t t4 = (side == 0 ? base : end) / kSub;
+                pos = t4 < nt4k ? (int64_t)tile_off_all[(int64_t)i * nt4k + t4] : k;
+            } else {
+                int64_t t_lo = 0, t_hi = k;   // without tile counts (rand-k): the whole payload
+                if (fin_off_all) {
+                    t_lo = fin_off_all[(int64_t)i * nbt + tile];
+                    t_hi = tile + 1 < nbt ? (int64_t)fin_off_all[(int64_t)i * nbt + tile + 1] : k;
+                }
+                pos = t_hi;
+                if (!fin_off_all || side == 0 || end < (tile + 1) * (int64_t)(kTileWords * 32))
+                    pos = (side == 1 && end >= ((int64_t)1 << 32))
+                              ? min(t_hi, k)
+                              : t_lo + lower_bound_u32(idx + t_lo, min(t_hi, k) - t_lo, (uint32_t)(side == 0 ? base : end));
             }
-            int64_t pos = t_hi;
-            if (!fin_off_all || side == 0 || end < (tile + 1) * (int64_t)(kTileWords * 32))
-                pos = (side == 1 && end >= ((int64_t)1 << 32))
-                          ? min(t_hi, k)
-                          : t_lo + lower_bound_u32(idx + t_lo, min(t_hi, k) - t_lo, (uint32_t)(side == 0 ? base : end));
             range[threadIdx.x >> 1][side] = min(pos, k);
         }
         __syncthreads();
-        for (int c = 0; c < nc; ++c) {                      // workers in increasing order
-            const uint32_t *idx = idx_all + (int64_t)(i0 + c) * k;
-            const float *val = val_all + (int64_t)(i0 + c) * k;
-            const int64_t lo = range[c][0], hi = range[c][1];
-            for (int64_t t = lo + threadIdx.x; t < hi; t += kBlock) {
-                const uint32_t e = idx[t] - (uint32_t)base;
-                if (e < (uint32_t)kAggSpan) acc[e] = __fadd_rn(acc[e], val[t]);
+        // The additions are ordered by worker (a barrier after each), so their operands are
+        // fetched beforehand, kAggPre workers at a time: the loads of all of them are in
+        // flight together instead of one memory latency per worker.
+        for (int c0 = 0; c0 < nc; c0 += kAggPre) {
+            uint32_t pe[kAggPre];
+            float pv[kAggPre];
+#pragma unroll
+            for (int u = 0; u < kAggPre; ++u) {
+                pe[u] = 0xffffffffu;
+                pv[u] = 0.0f;
+                if (c0 + u < nc) {
+                    const int64_t t = range[c0 + u][0] + threadIdx.x;
+                    if (t < range[c0 + u][1]) {
+                        pe[u] = idx_all[(int64_t)(i0 + c0 + u) * k + t] - (uint32_t)base;
+                        pv[u] = val_all[(int64_t)(i0 + c0 + u) * k + t];
+                    }
+                }
             }
-            __syncthreads();
+#pragma unroll
+            for (int u = 0; u < kAggPre; ++u) {                 // workers in increasing order
+                if (c0 + u >= nc) break;                        // block-uniform
+                if (pe[u] < (uint32_t)kAggSpan) acc[pe[u]] = __fadd_rn(acc[pe[u]], pv[u]);
+                const uint32_t *idx = idx_all + (int64_t)(i0 + c0 + u) * k;
+                const float *val = val_all + (int64_t)(i0 + c0 + u) * k;
+                const int64_t hi = range[c0 + u][1];
+                for (int64_t t = range[c0 + u][0] + kBlock + threadIdx.x; t < hi; t += kBlock) {   // dense payloads
+                    const uint32_t e = idx[t] - (uint32_t)base;
+                    if (e < (uint32_t)kAggSpan) acc[e] = __fadd_rn(acc[e], val[t]);
+                }
+                __syncthreads();
+            }
         }
     }
     const float fn = (float)n, rn = 1.0f / fn;
+    auto mean = [&](float a) { return n_pow2 ? __fmul_rn(a, rn) : __fdiv_rn(a, fn); };
+    if (end - base == kAggSpan && ((uintptr_t)ghat_s & 15u) == 0) {
+        // all loads of the span first (independent), then the additions: a loop of
+        // read-modify-writes of one array would wait for each store before the next load
+        constexpr int kPer = kAggSpan / 4 / kBlock;
+        float4 G[kPer];
+#pragma unroll
+        for (int u = 0; u < kPer; ++u)
+            G[u] = *reinterpret_cast<const float4 *>(ghat_s + base + (int64_t)(u * kBlock + threadIdx.x) * 4);
+#pragma unroll
+        for (int u = 0; u < kPer; ++u) {
+            const int t = (u * kBlock + threadIdx.x) * 4;
+            const float4 a = *reinterpret_cast<const float4 *>(&acc[t]);
+            if (a.x != 0.0f || a.y != 0.0f || a.z != 0.0f || a.w != 0.0f) {     // adding an exact zero changes nothing
+                if (a.x != 0.0f) G[u].x = __fadd_rn(G[u].x, mean(a.x));
+                if (a.y != 0.0f) G[u].y = __fadd_rn(G[u].y, mean(a.y));
+                if (a.z != 0.0f) G[u].z = __fadd_rn(G[u].z, mean(a.z));
+                if (a.w != 0.0f) G[u].w = __fadd_rn(G[u].w, mean(a.w));
+                *reinterpret_cast<float4 *>(ghat_s + base + t) = G[u];
+            }
+        }
+        return;
+    }
     for (int t = threadIdx.x; t < (int)(end - base); t += kBlock) {
         const float a = acc[t];
-        if (a != 0.0f)                         // adding an exact zero changes nothing
-            ghat_s[base + t] = __fadd_rn(ghat_s[base + t], n_pow2 ? __fmul_rn(a, rn) : __fdiv_rn(a, fn));
+        if (a != 0.0f) ghat_s[base + t] = __fadd_rn(ghat_s[base + t], mean(a));
     }
 }
 
@@ -1059,7 +1113,8 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
 void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st)
 {
     const unsigned blocks = (unsigned)((ww->d + kAggSpan - 1) / kAggSpan);
-    k_topk_aggregate<<<blocks, kBlock, 0, st>>>(ww->idx, ww->val, ww->cnt_fin, ww->nbt, n, ww->k, ww->d, ghat_s, (n & (n - 1)) == 0);
+    k_topk_aggregate<<<blocks, kBlock, 0, st>>>(ww->idx, ww->val, ww->cnt_fin, ww->nbt, n, ww->k, ww->d, ghat_s, (n & (n - 1)) == 0,
+                                                ww->hit, ww->cnt_gt, ww->nt4k);
 }
 
 // ---- rand-k: the coordinate sets come from the caller -------------------------------------
