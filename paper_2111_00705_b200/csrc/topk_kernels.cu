@@ -15,8 +15,10 @@
 // keeps them per 4096-coordinate tile as a short list (position in the tile, value) in index
 // order.  Every later pass of such a row walks these lists, one warp per tile, with coalesced
 // reads; selection, ties and the ordered compaction follow from per-tile counts and two
-// scans, without bitmaps.  If fewer than k coordinates lie above the floor (or a tile cannot
-// keep its list) the classic two dense passes and the bitmap passes run instead.  The same file holds the sparse
+// scans, without bitmaps.  A tile with more coordinates above the floor than its list holds
+// (a selection concentrated in one tensor) is read again from the data by those passes.  If
+// fewer than k coordinates lie above the floor the classic two dense passes and the bitmap
+// passes run instead.  The same file holds the sparse
 // server aggregation and the rand-k path, which shares the payload kernels.
 #include "topk.h"
 
@@ -50,11 +52,11 @@ struct TopkWorkspace {
     uint32_t *bm_in, *bm_cand;        // rows x wp (rows whose guess failed)
     uint32_t *floor_bucket;           // rows: guessed level-1 bucket for the next selection
     uint32_t *hit;                    // rows: 1 if the guess held in the current selection
-    uint32_t *ovf;                    // rows: 1 if some tile had more than kStashCap values to keep
     // lists of the coordinates at or above the guessed bucket, per 4096-coordinate tile:
     float *stash;                     // rows x nt4k x kStashCap: values u, in index order
     uint16_t *stash_pos;              // rows x nt4k x kStashCap: positions inside the tile
-    uint32_t *stash_cnt;              // rows x nt4k: list lengths (may exceed kStashCap: ovf)
+    uint32_t *stash_cnt;              // rows x nt4k: list lengths; above kStashCap the tile kept no
+                                      // complete list and the later passes read it from a and b
     uint32_t *cnt_gt, *cnt_eq;        // rows x nt4k: per tile, keys above / equal to the threshold;
                                       // after the scans: payload offset / tie rank of the tile
     int64_t nt4k;                     // ceil(d / 4096)
@@ -281,7 +283,7 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
             float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
-            uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ ovf, int64_t d, int vec_ok)
+            uint32_t *__restrict__ stash_cnt_all, int64_t d, int vec_ok)
 {
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
@@ -347,10 +349,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if ((BG[v][3] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].w; spos[r] = (uint16_t)(p0 + 3); } }
             rank += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
         }
-        if (threadIdx.x == 0) {
-            stash_cnt_all[tile] = total;
-            if (total > (uint32_t)kStashCap) ovf[row] = 1u;
-        }
+        if (threadIdx.x == 0) stash_cnt_all[tile] = total;
     } else {
         const int64_t end = min(base + (int64_t)kSub, d);
         uint32_t run = 0;                             // coordinates kept so far, block-uniform
@@ -374,10 +373,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             run += total;
             __syncthreads();
         }
-        if (threadIdx.x == 0) {
-            stash_cnt_all[tile] = run;
-            if (run > (uint32_t)kStashCap) ovf[row] = 1u;
-        }
+        if (threadIdx.x == 0) stash_cnt_all[tile] = run;
     }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
@@ -385,13 +381,12 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
         if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
-// Did the guess hold?  It did if at least k coordinates lie at or above the floor (and every
-// tile could keep the values of its coordinates at or above the floor); then the
+// Did the guess hold?  It did if at least k coordinates lie at or above the floor; then the
 // level-1 bucket follows from the histogram of those coordinates.  Otherwise the row's
 // level-1 histogram is cleared for the full pass.  grid = (rows), one block.
 __global__ void __launch_bounds__(kBlock)
 k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
-                 const uint32_t *__restrict__ floor_bucket, const uint32_t *__restrict__ ovf,
+                 const uint32_t *__restrict__ floor_bucket,
                  uint32_t *__restrict__ hit)
 {
     __shared__ uint32_t tot[kBlock];
@@ -420,7 +415,7 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
         }
     }
     __syncthreads();
-    const uint32_t ok = found && !ovf[row];             // a tile that could not keep its values: redo
+    const uint32_t ok = found;
     if (threadIdx.x == 0) hit[row] = ok;
     if (!ok)
         for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
@@ -436,15 +431,21 @@ constexpr int kWarpTiles = 2;
 constexpr int kListTiles = kWarpTiles * (kBlock / 32);
 constexpr int kPre = 4;
 
+// A tile with more than kStashCap coordinates at or above the floor (the selection is
+// concentrated there) has no complete list: the passes walk its coordinates in a and b
+// instead ("dense" tile).  Every key a pass looks for is at or above the floor, so the
+// result is that of a complete list.
 struct WarpLists {
     const float *val[kWarpTiles];
     const uint16_t *pos[kWarpTiles];
-    uint32_t cnt[kWarpTiles];
+    uint32_t cnt[kWarpTiles];      // list length; 0 for a dense tile
+    uint32_t dense[kWarpTiles];    // coordinates of a dense tile, else 0
     int64_t tile[kWarpTiles];      // index of the tile inside its row (>= nt4k: none, cnt = 0)
 };
 
 __device__ __forceinline__ WarpLists warp_lists(const float *stash_all, const uint16_t *stash_pos_all,
-                                                const uint32_t *stash_cnt_all, int row, int64_t nt4k)
+                                                const uint32_t *stash_cnt_all, int row, int64_t nt4k,
+                                                int64_t d)
 {
     WarpLists w;
     const int64_t t0 = ((int64_t)blockIdx.x * (kBlock / 32) + (threadIdx.x >> 5)) * kWarpTiles;
@@ -455,14 +456,16 @@ __device__ __forceinline__ WarpLists warp_lists(const float *stash_all, const ui
         const int64_t g = (int64_t)row * nt4k + (any ? w.tile[m] : 0);
         w.val[m] = stash_all + g * kStashCap;
         w.pos[m] = stash_pos_all + g * kStashCap;
-        w.cnt[m] = any ? min(stash_cnt_all[g], (uint32_t)kStashCap) : 0u;
+        const uint32_t raw = any ? stash_cnt_all[g] : 0u;
+        w.cnt[m] = raw <= (uint32_t)kStashCap ? raw : 0u;
+        w.dense[m] = raw <= (uint32_t)kStashCap ? 0u : (uint32_t)min((int64_t)kSub, d - w.tile[m] * kSub);
     }
     return w;
 }
 
-// f(value) for every entry of the warp's lists.
-template <typename F>
-__device__ __forceinline__ void for_each_listed(const WarpLists &w, F f)
+// f(value) for every entry of the warp's lists (every coordinate of its dense tiles).
+template <bool HAS_B, typename F>
+__device__ __forceinline__ void for_each_listed(const WarpLists &w, const float *a, const float *b, F f)
 {
     const uint32_t lane = threadIdx.x & 31;
     float v[kWarpTiles][kPre];
@@ -476,6 +479,7 @@ __device__ __forceinline__ void for_each_listed(const WarpLists &w, F f)
         for (int i = 0; i < kPre; ++i)
             if (lane + 32 * i < w.cnt[m]) f(v[m][i]);
         for (uint32_t e = lane + 32 * kPre; e < w.cnt[m]; e += 32) f(w.val[m][e]);
+        for (uint32_t e = lane; e < w.dense[m]; e += 32) f(diff1<HAS_B>(a, b, w.tile[m] * kSub + e));
     }
 }
 
@@ -498,18 +502,22 @@ struct HistLevel3 {
 
 // After a successful guess: the level-2 histogram of the listed values that fall into the
 // threshold bucket (what the second dense pass would have produced).  grid = (nbt, rows).
+template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
-k_topk_split(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
+             const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
-             const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all, int64_t nt4k)
+             const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all, int64_t nt4k,
+             int64_t d)
 {
     __shared__ uint32_t h[kBins2];
     const int row = blockIdx.y;
     if (!hit[row] || (int64_t)blockIdx.x * kListTiles >= nt4k) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
-    for_each_listed(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k),
-                    HistLevel2{h, sel_all[row].b1});
+    for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
+                           a_all + (int64_t)row * d, HAS_B ? b_all + (int64_t)row * d : nullptr,
+                           HistLevel2{h, sel_all[row].b1});
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
     for (int t = threadIdx.x; t < kBins2; t += kBlock)
@@ -537,7 +545,9 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
     if (hit[row]) {                                   // the tiles' lists hold the values
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
-        for_each_listed(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k), HistLevel3{h, pre});
+        for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
+                               a_all + (int64_t)row * d, HAS_B ? b_all + (int64_t)row * d : nullptr,
+                               HistLevel3{h, pre});
     } else {                                          // classic path: gather a and b
         const float *a = a_all + (int64_t)row * d;
         const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
@@ -583,7 +593,9 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
     uint32_t nt = 0;
     if (hit[row]) {                                   // the tiles' lists hold the values
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
-        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
+        const float *a = a_all + (int64_t)row * d;
+        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
         const uint32_t lane = threadIdx.x & 31;
         float v[kWarpTiles][kPre];
 #pragma unroll
@@ -593,6 +605,11 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
 #pragma unroll
         for (int m = 0; m < kWarpTiles; ++m) {
             uint32_t gt = 0, eq = 0;
+            for (uint32_t e = lane; e < w.dense[m]; e += 32) {
+                const uint32_t key = key_of(diff1<HAS_B>(a, b, w.tile[m] * kSub + e));
+                gt += key > T;
+                eq += key == T;
+            }
 #pragma unroll
             for (int i = 0; i < kPre; ++i)
                 if (lane + 32 * i < w.cnt[m]) { gt += key_of(v[m][i]) > T; eq += key_of(v[m][i]) == T; }
@@ -755,20 +772,24 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
 // is written with the index.  Other rows: from the selection bitmap; a thread owns 4
 // consecutive bitmap words, ranks come from popcount scans, values follow in k_topk_gather.
 // ------------------------------------------------------------------------------------
+template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
-k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
+k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all,
+                const uint32_t *__restrict__ bm_in_all, const uint32_t *__restrict__ fin_off_all,
                 const uint32_t *__restrict__ hit, const Sel *__restrict__ sel_all,
                 const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
                 const uint32_t *__restrict__ stash_cnt_all, const uint32_t *__restrict__ cnt_gt_all,
                 const uint32_t *__restrict__ cnt_eq_all, uint32_t *__restrict__ idx_all,
-                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k)
+                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d)
 {
     const int row = blockIdx.y;
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
     if (hit[row]) {
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
-        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k);
+        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
+        const float *a = a_all + (int64_t)row * d;
+        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
         const Sel s = sel_all[row];
         const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
         const bool all_ties = s.k3 == s.c3;
@@ -793,8 +814,7 @@ k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restri
             const uint32_t base = (uint32_t)(w.tile[m] * kSub);
             // one chunk of 32 entries in index order: ballots give the tie ranks and the
             // payload positions
-            auto chunk = [&](uint32_t e, float val_e, uint32_t pos_e) {
-                const bool valid = e < w.cnt[m];
+            auto chunk = [&](bool valid, float val_e, uint32_t pos_e) {
                 const uint32_t key = key_of(val_e);
                 const bool eq = valid && key == T;
                 const uint32_t eqm = __ballot_sync(kFull, eq);
@@ -810,11 +830,16 @@ k_topk_emit_idx(const uint32_t *__restrict__ bm_in_all, const uint32_t *__restri
             };
 #pragma unroll
             for (int i = 0; i < kPre; ++i)
-                if (32u * i < w.cnt[m]) chunk(lane + 32 * i, v[m][i], ps[m][i]);       // warp-uniform
+                if (32u * i < w.cnt[m]) chunk(lane + 32 * i < w.cnt[m], v[m][i], ps[m][i]);       // warp-uniform
             for (uint32_t e0 = 32 * kPre; e0 < w.cnt[m]; e0 += 32) {
                 const uint32_t e = e0 + lane;
                 const bool valid = e < w.cnt[m];
-                chunk(e, valid ? w.val[m][e] : 0.0f, valid ? (uint32_t)w.pos[m][e] : 0u);
+                chunk(valid, valid ? w.val[m][e] : 0.0f, valid ? (uint32_t)w.pos[m][e] : 0u);
+            }
+            for (uint32_t e0 = 0; e0 < w.dense[m]; e0 += 32) {              // a tile without a list
+                const uint32_t e = e0 + lane;
+                const bool valid = e < w.dense[m];
+                chunk(valid, valid ? diff1<HAS_B>(a, b, w.tile[m] * kSub + e) : 0.0f, e);
             }
         }
         return;
@@ -1010,7 +1035,7 @@ static void free_ws(TopkWorkspace *w)
 {
     cudaFree(w->hist); cudaFree(w->sel); cudaFree(w->bm_in); cudaFree(w->bm_cand);
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
-    cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->ovf); cudaFree(w->stash);
+    cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->stash);
     cudaFree(w->stash_pos); cudaFree(w->stash_cnt); cudaFree(w->cnt_gt); cudaFree(w->cnt_eq);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
@@ -1039,7 +1064,6 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         get((void **)&w->bm_cand, (size_t)rows * w->wp * 4);
         get((void **)&w->floor_bucket, (size_t)rows * 4);
         get((void **)&w->hit, (size_t)rows * 4);
-        get((void **)&w->ovf, (size_t)rows * 4);
         w->nt4k = (d + kSub - 1) / kSub;
         get((void **)&w->stash, (size_t)rows * w->nt4k * kStashCap * 4);
         get((void **)&w->stash_pos, (size_t)rows * w->nt4k * kStashCap * 2);
@@ -1077,16 +1101,15 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
     const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
     cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
-    cudaMemsetAsync(w->ovf, 0, (size_t)w->rows * 4, st);
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
-    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->ovf, w->d, vec_ok);
-    k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->ovf, w->hit);
+    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok);
+    k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
     k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
     k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok);
-    k_topk_split<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k);
+    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k, w->d);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
     k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->bm_cand, w->hist, w->d, w->wp, w->nt4k);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
@@ -1095,7 +1118,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
     k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit);
-    k_topk_emit_idx<<<sparse, kBlock, 0, st>>>(w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
         k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);

@@ -390,6 +390,28 @@ def test_topk_threshold_guess_hits_and_misses():
     check_state(g, o, FINAL_TOL, exact=True)
 
 
+@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF])
+def test_topk_selection_concentrated_in_a_few_tiles(mode):
+    """One tensor with gradients 100x larger than the rest takes the whole selection: its
+    4096-coordinate tiles have far more candidates than a tile's list holds (512), so the list
+    passes read those tiles from the data again; the other tiles keep their (short) lists.
+    Steady state (the guess holds) over several steps, ragged d."""
+    rng = np.random.default_rng(5)
+    d, n, k = 40 * 4096 + 123, 3, 6000
+    big = slice(7 * 4096 + 100, 10 * 4096 + 50)             # 12238 coordinates, k of them kept
+    w = synth.Workload("CONC", d, n, synth.TOPK, 6, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d), mode=mode)
+    for t in range(6):
+        grads = rng.standard_normal((n, d)).astype(np.float32)
+        grads[:, big] *= 100.0
+        if t == 4:
+            grads[:, 20 * 4096:20 * 4096 + 700] = 1e4       # a second dense tile appears
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.close(); o.close()
+
+
 def test_topk_ties_lower_index_wins():
     """Few distinct magnitudes: most of the selection is decided by the tie rule."""
     rng = np.random.default_rng(0)
