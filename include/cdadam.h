@@ -7,11 +7,11 @@
  * model x, the moments m, v, vhat and all compression state.  One call of cdadam_step is one
  * iteration t of Algorithm 1:
  *
- *   worker i :  c^(i) = C(g^(i) - ghat^(i));  ghat^(i) += c^(i)            (lines 5-6)
- *   server   :  ghat += (1/n) sum_i c^(i);  c = C(ghat - gtil);  gtil += c  (lines 8-10)
+ *   worker i :  c^(i) = C(g^(i) - ghat^(i));  ghat^(i) += c^(i)
+ *   server   :  ghat += (1/n) sum_i c^(i);  c = C(ghat - gtil);  gtil += c
  *   worker   :  gtil += c (the same vector on every worker, kept once);
  *               m = b1 m + (1-b1) gtil;  v = b2 v + (1-b2) gtil^2;
- *               vhat = max(vhat, v);  x -= lr * m / sqrt(vhat + eps)       (lines 12-16)
+ *               vhat = max(vhat, v);  x -= lr * m / sqrt(vhat + eps)
  *
  * C is the scaled-sign compressor (||u||_1 / |segment| * sign(u), one bit per coordinate plus
  * one float per segment), the top-k compressor (k (index, value) pairs) or the identity
@@ -84,7 +84,7 @@ enum {
  *   k          entries kept by top-k / rand-k at the workers and at the server,
  *              1 <= k <= d; ignored for the other compressors
  * All state is allocated here, on the current device, and zero-initialised (Algorithm 1
- * line 1; x_1 = 0 until cdadam_set_params).  Scaled sign starts with one segment [0, d).
+ * initialisation; x_1 = 0 until cdadam_set_params).  Scaled sign starts with one segment [0, d).
  * Synchronous.  Returns NULL on failure (see cdadam_last_error).  The caller destroys the
  * context with cdadam_destroy.
  */
@@ -95,7 +95,7 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k,
 void cdadam_destroy(cdadam_ctx *ctx);
 
 /*
- * One iteration of Algorithm 1 (lines 4-16) on the n gradients g_t^(i).
+ * One iteration of Algorithm 1 (its whole loop body) on the n gradients g_t^(i).
  *   grads   device, n x d floats, row i = worker i, row-major, contiguous; borrowed until
  *           the work queued on `stream` has completed; never written.  A base address
  *           that is a multiple of 16 bytes together with d % 4 == 0 selects the

@@ -262,7 +262,7 @@ static void alloc_payloads(oracle_ctx *o)
 }
 
 /* Inputs of Algorithm 1: x_1 (set later, default 0), alpha, beta1, beta2, nu, C.
- * All state starts at zero (line 1 of the algorithm: C(0) = 0). */
+ * All state starts at zero (the initialisation of Algorithm 1: C(0) = 0). */
 oracle_ctx *oracle_create(int64_t d, int n, int compressor, int64_t k,
                           float beta1, float beta2, float lr, float nu)
 {
@@ -420,7 +420,7 @@ static void compress(oracle_ctx *o, const float *u, float *c, int who)
         memcpy(c, u, (size_t)o->d * sizeof(float));
 }
 
-/* AMSGrad update of Algorithm 1 (lines 13-16) with gradient estimate ge:
+/* AMSGrad update of Algorithm 1 (its last four assignments) with gradient estimate ge:
  *   m = beta1 m + (1-beta1) ge;  v = beta2 v + (1-beta2) ge^2;  vhat = max(vhat, v);
  *   x = x - alpha * m / sqrt(vhat + nu)          (nu inside the root, no bias correction) */
 static void amsgrad(oracle_ctx *o, const float *ge)

@@ -328,11 +328,11 @@ void enqueue_topk_step(cdadam_ctx *c, const void *grads_in, bool, bool vec, cuda
 {
     const float *grads = static_cast<const float *>(grads_in);
     const bool svec = c->d % 4 == 0;
-    topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // lines 5-6
+    topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // workers: compress, update ghat^(i)
     prof_mark(c, st);
-    topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
+    topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // server: ghat += mean
     prof_mark(c, st);
-    topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // lines 9-10, 12
+    topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // server: compress, update gtil
     prof_mark(c, st);
     launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
     prof_mark(c, st);
@@ -571,11 +571,11 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
         topk_payload(c->tk_w, 0, &widx, &wval);
         topk_payload(c->tk_s, 0, &sidx, &sval);
         if (!ef) {
-            randk_gather(c->tk_w, grads, c->ghat_w, true, st);                 // lines 5-6
+            randk_gather(c->tk_w, grads, c->ghat_w, true, st);                 // workers: compress, update ghat^(i)
             prof_mark(c, st);
-            topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // line 8
+            topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // server: ghat += mean
             prof_mark(c, st);
-            randk_gather(c->tk_s, c->ghat_s, c->gtil, true, st);               // lines 9-10, 12
+            randk_gather(c->tk_s, c->ghat_s, c->gtil, true, st);               // server: compress, update gtil
             prof_mark(c, st);
             launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
             prof_mark(c, st);

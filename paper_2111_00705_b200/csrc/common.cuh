@@ -209,7 +209,7 @@ __device__ __forceinline__ int find_segment(const int64_t *off, int lo, int hi, 
 }
 
 // ------------------------------------------------------------------------------------
-// AMSGrad update of one coordinate (Algorithm 1 lines 13-16): nu inside the root, no bias
+// AMSGrad update of one coordinate (the last four assignments of Algorithm 1): nu inside the root, no bias
 // correction, one rounding per operation, no fused multiply-add.  With a weight decay
 // lambda (Section 6; decoupled form) x also loses (alpha lambda) x_t.
 // ------------------------------------------------------------------------------------

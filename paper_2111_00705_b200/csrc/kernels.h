@@ -6,7 +6,7 @@
 namespace cdadam {
 
 // ---- scaled sign -------------------------------------------------------------------
-// Worker pass (Algorithm 1 lines 5-6) for all n workers: applies the previous payload
+// Worker pass (Algorithm 1: the workers' compression and state update) for all n workers: applies the previous payload
 // (bits in wbits, scales in scale_old) to ghat_w (grads: n x d binary32 or bfloat16), forms u = g - ghat_w, packs sign(u) into
 // wbits and writes per-tile double-double partial sums of |u| to wpart.  For large tiles the
 // variant with a TMA prefetch ring runs; it sets *error_flag (device) if a bounded wait on
@@ -23,7 +23,7 @@ void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint3
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
                             cudaStream_t st, int split = 1, dd *split_sums = nullptr,
                             unsigned int *split_done = nullptr);
-// Server pass A (lines 8-9): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
+// Server pass A (Algorithm 1: server aggregation and compression): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
 // sign(w) into sbits and writes partial sums of |w| to spart.  sscale != NULL: the scales are
 // finished in the same launch (done: q zeroed counters), as in the worker pass.
 // mode: 0 Algorithm 1, 1 error feedback, 2 naive compression (w = mean; gtil is not read).
@@ -31,7 +31,7 @@ void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_
                         const float *gtil, uint32_t *sbits, dd *spart, const Tables &tb,
                         int n, int64_t wp, bool vec_ok, int mode, float *sscale, unsigned int *done,
                         cudaStream_t st);
-// Server pass B and worker update (lines 10, 12-16): gtil += decode(c); AMSGrad.
+// Server pass B and worker update (Algorithm 1: state update of gtil, AMSGrad): gtil += decode(c); AMSGrad.
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
                         float *m, float *v, float *vhat, float *x, const Tables &tb, Hyper hp,
                         bool vec_ok, int mode, cudaStream_t st);

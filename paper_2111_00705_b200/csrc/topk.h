@@ -23,7 +23,7 @@ int topk_launches_per_step(int n);
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                  cudaStream_t st);
 
-// Sparse server aggregation (Algorithm 1 line 8) from the n payloads held in `ww`:
+// Sparse server aggregation (Algorithm 1: ghat += mean of the workers' messages) from the n payloads held in `ww`:
 //   ghat_s += (sum_i c_i) / n on the coordinates some worker sent, workers added in the
 //   order 0, 1, ..., n-1.
 void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st);

@@ -865,7 +865,7 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
 }
 
 // ------------------------------------------------------------------------------------
-// Payload values and the state update at the kept coordinates (Algorithm 1 lines 6 / 10):
+// Payload values and the state update at the kept coordinates (Algorithm 1: ghat^(i) += c^(i), gtil += c):
 // val = u_j = a_j - b_j, b_j += u_j.  One thread per payload entry.  grid = (ceil(k/256), rows).
 // Rows whose values were already written from the lists only update b.
 // ------------------------------------------------------------------------------------
@@ -901,7 +901,7 @@ k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
 }
 
 // ------------------------------------------------------------------------------------
-// Sparse server aggregation (Algorithm 1 line 8): ghat_s += (sum_i c_i) / n.
+// Sparse server aggregation (Algorithm 1): ghat_s += (sum_i c_i) / n.
 //
 // A block owns kAggSpan consecutive coordinates and keeps their sums in shared memory.
 // Every payload is sorted by index, so worker i's entries for the block are one contiguous
