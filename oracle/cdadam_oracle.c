@@ -198,6 +198,7 @@ void oracle_compress_randk(const float *x, int64_t d, int64_t k, const uint32_t 
 typedef struct oracle_ctx {
     int64_t d, k;
     int n, compressor, mode, q;
+    int64_t *kseg;           /* top-k applied per segment: entries kept in each (NULL: whole vector) */
     float wd;                /* decoupled weight decay lambda (0 = none) */
     float base_lr, gamma;    /* step-size milestones */
     int n_milestones;
@@ -240,7 +241,7 @@ void oracle_destroy(oracle_ctx *o)
     free(o->w_bits); free(o->w_scales); free(o->w_idx); free(o->w_val);
     free(o->s_bits); free(o->s_scales); free(o->s_idx); free(o->s_val);
     free(o->force_w_scales); free(o->force_s_scales);
-    free(o->rand_w); free(o->rand_s);
+    free(o->rand_w); free(o->rand_s); free(o->kseg);
     free(o);
 }
 
@@ -293,6 +294,32 @@ int oracle_set_segments(oracle_ctx *o, int q, const int64_t *off)
     memcpy(o->off, off, (size_t)(q + 1) * sizeof(int64_t));
     o->q = q;
     alloc_payloads(o);
+    return 0;
+}
+
+/* Top-k applied to every segment on its own (the per-tensor use of a compressor, as for the
+ * scaled sign): segment r keeps its kseg[r] coordinates of largest magnitude, ties to the
+ * lower index.  The message is the concatenation of the segments' (index, value) lists, so it
+ * is still listed by ascending index and has k = sum_r kseg[r] entries. */
+int oracle_set_topk_segments(oracle_ctx *o, int q, const int64_t *off, const int64_t *kseg)
+{
+    if (!o || o->compressor != ORC_TOPK || o->steps != 0) return -1;
+    if (q < 1 || off[0] != 0 || off[q] != o->d) return -1;
+    int64_t total = 0;
+    for (int r = 0; r < q; ++r) {
+        if (off[r + 1] <= off[r] || kseg[r] < 1 || kseg[r] > off[r + 1] - off[r]) return -1;
+        total += kseg[r];
+    }
+    if (oracle_set_segments(o, q, off) != 0) return -1;
+    free(o->kseg);
+    o->kseg = (int64_t *)malloc((size_t)q * sizeof(int64_t));
+    memcpy(o->kseg, kseg, (size_t)q * sizeof(int64_t));
+    o->k = total;
+    free(o->w_idx); free(o->w_val); free(o->s_idx); free(o->s_val);
+    o->w_idx = (uint32_t *)calloc((size_t)(o->n * total), sizeof(uint32_t));
+    o->w_val = zeros(o->n * total);
+    o->s_idx = (uint32_t *)calloc((size_t)total, sizeof(uint32_t));
+    o->s_val = zeros(total);
     return 0;
 }
 
@@ -410,7 +437,17 @@ static void compress(oracle_ctx *o, const float *u, float *c, int who)
     else if (o->compressor == ORC_SIGN)
         oracle_compress_sign(u, o->d, o->q, o->off, oracle_payload_bits(o, who),
                              oracle_payload_scales(o, who), c);
-    else if (o->compressor == ORC_TOPK)
+    else if (o->compressor == ORC_TOPK && o->kseg) {
+        uint32_t *idx = oracle_payload_idx(o, who);
+        float *val = oracle_payload_val(o, who);
+        for (int r = 0; r < o->q; ++r) {             /* C on every segment on its own */
+            const int64_t lo = o->off[r], len = o->off[r + 1] - lo;
+            oracle_compress_topk(u + lo, len, o->kseg[r], idx, val, c + lo);
+            for (int64_t t = 0; t < o->kseg[r]; ++t) idx[t] += (uint32_t)lo;   /* positions in the whole vector */
+            idx += o->kseg[r];
+            val += o->kseg[r];
+        }
+    } else if (o->compressor == ORC_TOPK)
         oracle_compress_topk(u, o->d, o->k, oracle_payload_idx(o, who),
                              oracle_payload_val(o, who), c);
     else if (o->compressor == ORC_RANDK)

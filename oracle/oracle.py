@@ -53,6 +53,8 @@ def _load():
     lib.oracle_destroy.argtypes = [c.c_void_p]
     lib.oracle_set_segments.restype = c.c_int
     lib.oracle_set_segments.argtypes = [c.c_void_p, c.c_int, ip]
+    lib.oracle_set_topk_segments.restype = c.c_int
+    lib.oracle_set_topk_segments.argtypes = [c.c_void_p, c.c_int, ip, ip]
     lib.oracle_set_mode.restype = c.c_int
     lib.oracle_set_mode.argtypes = [c.c_void_p, c.c_int]
     lib.oracle_set_lr.restype = c.c_int
@@ -173,6 +175,17 @@ class Oracle:
 
     def set_lr(self, lr):
         self._lib.oracle_set_lr(self._h, lr)
+
+    def set_topk_segments(self, offsets, k_per_segment):
+        """Top-k on every segment on its own; the payload has sum(k_per_segment) entries."""
+        off, op = _offsets(self.d, offsets)
+        ks = np.ascontiguousarray(k_per_segment, dtype=np.int64)
+        assert ks.size == off.size - 1
+        ip = ctypes.POINTER(ctypes.c_int64)
+        if self._lib.oracle_set_topk_segments(self._h, off.size - 1, op, ks.ctypes.data_as(ip)) != 0:
+            raise ValueError("bad top-k segments")
+        self.q = off.size - 1
+        self.k = int(ks.sum())
 
     def set_weight_decay(self, weight_decay):
         if self._lib.oracle_set_weight_decay(self._h, weight_decay) != 0:

@@ -572,3 +572,49 @@ def test_weight_decay_and_lr_milestones_against_independent_recursion(wd):
         o.set_lr_milestones(base, [2], 1.5)            # alpha_t must not increase
     with pytest.raises(ValueError):
         o.set_weight_decay(-1.0)
+
+
+# ------------------------------------------------------------------ top-k per segment
+
+def test_topk_per_segment_brute_force_and_reduction_to_whole_vector():
+    """Top-k on every segment on its own: against a Python sort of every segment (ties to the
+    lower index), against the whole-vector compressor on the slices, and with one segment
+    against the whole-vector step."""
+    rng = np.random.default_rng(77)
+    d, n = 97, 3
+    off = np.array([0, 5, 6, 40, 41, 97])
+    ks = np.array([2, 1, 7, 1, 20])
+    G = np.round(rng.standard_normal((3, n, d)) * 3).astype(np.float32) / 2        # many ties
+    o = orc.Oracle(d, n, orc.TOPK, k=1)
+    o.set_topk_segments(off, ks)
+    prev = np.zeros((n, d), np.float32)
+    for t in range(3):
+        o.step(G[t])
+        for i in range(n):
+            u = G[t, i] - prev[i]
+            idx, val = o.payload(i)
+            assert idx.size == ks.sum() and np.all(np.diff(idx.astype(np.int64)) > 0)
+            want = []
+            for r in range(len(ks)):
+                lo, hi = off[r], off[r + 1]
+                order = sorted(range(lo, hi), key=lambda j: (-abs(float(u[j])), j))[:ks[r]]
+                want += sorted(order)
+                # the whole-vector compressor on the slice gives the same entries
+                si, sv, _ = orc.compress_topk(u[lo:hi], int(ks[r]))
+                assert (si + lo).tolist() == sorted(order)
+            assert idx.tolist() == want
+            assert np.array_equal(val, u[idx])
+            dec = np.zeros(d, np.float32); dec[idx] = val
+            assert np.array_equal(o.state("ghat_w")[i], prev[i] + dec)          # Markov identity
+        prev = o.state("ghat_w").copy()
+    # one segment holding everything = the compressor of Appendix A on the whole vector
+    a = orc.Oracle(d, n, orc.TOPK, k=9); a.set_topk_segments([0, d], [9])
+    b = orc.Oracle(d, n, orc.TOPK, k=9)
+    for t in range(3):
+        a.step(G[t]); b.step(G[t])
+    for name in orc.STATE_NAMES:
+        assert np.array_equal(a.state(name), b.state(name)), name
+    with pytest.raises(ValueError):
+        orc.Oracle(d, n, orc.TOPK, k=1).set_topk_segments([0, 5, d], [6, 1])     # k_r > |S_r|
+    with pytest.raises(ValueError):
+        orc.Oracle(d, n, orc.SIGN).set_topk_segments([0, d], [1])
