@@ -150,6 +150,22 @@ int cdadam_set_params(cdadam_ctx *ctx, const float *x0, void *stream);
 int cdadam_set_segments(cdadam_ctx *ctx, int q, const int64_t *offsets);
 
 /*
+ * Apply the top-k compressor independently to q contiguous segments ("per tensor", as
+ * cdadam_set_segments does for the scaled sign; Appendix A defines top-k on a whole vector,
+ * here the vector is the segment): segment r = [offsets[r], offsets[r+1]) keeps its
+ * k_per_segment[r] coordinates of largest magnitude (ties: lower coordinate), at the workers
+ * and at the server.  offsets: host, q+1 values, strictly increasing from 0 to d;
+ * k_per_segment: host, q values, 1 <= k_per_segment[r] <= length of segment r.  A message is
+ * the concatenation of the segments' lists: sum_r k_per_segment[r] (coordinate, value) pairs,
+ * coordinates in the whole vector, increasing; that sum replaces the k given to
+ * cdadam_create.  The selection runs segment by segment, so this is meant for a moderate
+ * number of large segments.  Only CDADAM_TOPK in the mode CDADAM_MARKOV, only before the
+ * first step; synchronous (re-allocates the selection workspaces).
+ */
+int cdadam_set_topk_segments(cdadam_ctx *ctx, int q, const int64_t *offsets,
+                             const int64_t *k_per_segment);
+
+/*
  * Rand-k compressor (Appendix A: C(x) keeps x on k coordinates drawn uniformly at random).
  * The draws are inputs: before each step give the coordinate sets the n workers (device,
  * n x k uint32, row i = worker i) and the server (device, k uint32) use in that step.  Every

@@ -32,6 +32,7 @@ _SIGNATURES = {
     "cdadam_set_random_sets": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_mode": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_set_tile": (_c.c_int, [_c.c_void_p, _c.c_int]),
+    "cdadam_set_topk_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int64)]),
     "cdadam_set_lr": (_c.c_int, [_c.c_void_p, _c.c_float]),
     "cdadam_set_lr_milestones": (_c.c_int, [_c.c_void_p, _c.c_float, _c.c_int, _c.POINTER(_c.c_int64), _c.c_float]),
     "cdadam_set_weight_decay": (_c.c_int, [_c.c_void_p, _c.c_float]),
@@ -200,6 +201,16 @@ class CDAdam:
 
     def set_tile(self, tile):
         _check(lib().cdadam_set_tile(self._h, int(tile)))
+
+    def set_topk_segments(self, offsets, k_per_segment):
+        """Top-k on every segment on its own; the payload has sum(k_per_segment) entries."""
+        off = [int(a) for a in offsets]
+        ks = [int(a) for a in k_per_segment]
+        if len(ks) != len(off) - 1:
+            raise ValueError("one k per segment")
+        _check(lib().cdadam_set_topk_segments(self._h, len(ks), (ctypes.c_int64 * len(off))(*off),
+                                              (ctypes.c_int64 * len(ks))(*ks)))
+        self.k = sum(ks)
 
     def set_lr(self, lr):
         _check(lib().cdadam_set_lr(self._h, lr))

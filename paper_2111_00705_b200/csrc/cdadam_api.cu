@@ -155,6 +155,10 @@ struct cdadam_ctx {
     bool sets_given = false;   // rand-k: coordinate sets have been supplied
     // top-k
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
+    // top-k per segment: a selection workspace per segment (rows strided by d); tk_w / tk_s
+    // then hold only the concatenated payloads
+    std::vector<int64_t> seg_off, seg_k, seg_at;
+    std::vector<TopkWorkspace *> seg_w, seg_s;
     // host-gradient staging
     float *stage = nullptr;
     // Replay of a step as a CUDA graph where launches matter: scaled sign with grids of one
@@ -328,6 +332,28 @@ void enqueue_topk_step(cdadam_ctx *c, const void *grads_in, bool, bool vec, cuda
 {
     const float *grads = static_cast<const float *>(grads_in);
     const bool svec = c->d % 4 == 0;
+    if (!c->seg_w.empty()) {
+        // the compressor on every segment on its own; the payloads are concatenated (still
+        // listed by increasing coordinate) and the rest of the iteration is as without segments
+        const int q = (int)c->seg_w.size();
+        for (int r = 0; r < q; ++r) {
+            const int64_t lo = c->seg_off[r];
+            topk_select(c->seg_w[r], grads + lo, c->ghat_w + lo, true, vec && lo % 4 == 0, st);
+            topk_payload_concat(c->tk_w, c->seg_at[r], c->seg_w[r], lo, st);
+        }
+        prof_mark(c, st);
+        topk_aggregate(c->tk_w, c->ghat_s, c->n, st);
+        prof_mark(c, st);
+        for (int r = 0; r < q; ++r) {
+            const int64_t lo = c->seg_off[r];
+            topk_select(c->seg_s[r], c->ghat_s + lo, c->gtil + lo, true, svec && lo % 4 == 0, st);
+            topk_payload_concat(c->tk_s, c->seg_at[r], c->seg_s[r], lo, st);
+        }
+        prof_mark(c, st);
+        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+        prof_mark(c, st);
+        return;
+    }
     topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // workers: compress, update ghat^(i)
     prof_mark(c, st);
     topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // server: ghat += mean
@@ -456,6 +482,8 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     cudaFree(c->wdone); cudaFree(c->sdone); cudaFree(c->wsums); cudaFree(c->ssums);
     topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
+    for (TopkWorkspace *w : c->seg_w) topk_workspace_destroy(w);
+    for (TopkWorkspace *w : c->seg_s) topk_workspace_destroy(w);
     drop_graphs(c);
     for (cudaGraphExec_t e : c->retired) cudaGraphExecDestroy(e);
     if (c->cap_stream) cudaStreamDestroy(c->cap_stream);
@@ -632,6 +660,50 @@ int cdadam_set_params(cdadam_ctx *c, const float *x0, void *stream)
     return cdadam_set_state(c, CDADAM_STATE_X, x0, stream);
 }
 
+int cdadam_set_topk_segments(cdadam_ctx *c, int q, const int64_t *offsets, const int64_t *k_per_segment)
+{
+    if (!c || !offsets || !k_per_segment) return fail(CDADAM_ERR_ARG, "cdadam_set_topk_segments: NULL argument");
+    if (c->comp != CDADAM_TOPK) return fail(CDADAM_ERR_STATE, "top-k segments apply to the top-k compressor only");
+    if (c->mode != CDADAM_MARKOV) return fail(CDADAM_ERR_STATE, "top-k segments are available for Algorithm 1 only");
+    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
+    if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
+    if (offsets[0] != 0 || offsets[q] != c->d) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
+    int64_t total = 0;
+    for (int r = 0; r < q; ++r) {
+        if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
+        if (k_per_segment[r] < 1 || k_per_segment[r] > offsets[r + 1] - offsets[r])
+            return fail(CDADAM_ERR_ARG, "segment %d: k must be in [1, segment length]", r);
+        total += k_per_segment[r];
+    }
+    DeviceGuard guard(c->device);
+    CU_TRY(cudaDeviceSynchronize());
+    topk_workspace_destroy(c->tk_w); topk_workspace_destroy(c->tk_s);
+    c->tk_w = c->tk_s = nullptr;
+    for (TopkWorkspace *w : c->seg_w) topk_workspace_destroy(w);
+    for (TopkWorkspace *w : c->seg_s) topk_workspace_destroy(w);
+    c->seg_w.clear(); c->seg_s.clear(); c->seg_off.clear(); c->seg_k.clear(); c->seg_at.clear();
+    c->k = total;
+    int rc;
+    if ((rc = topk_workspace_create(&c->tk_w, c->d, total, c->n, nullptr, nullptr, false)) ||
+        (rc = topk_workspace_create(&c->tk_s, c->d, total, 1, nullptr, nullptr, false)))
+        return fail(rc, "top-k payload allocation failed");
+    int64_t at = 0;
+    for (int r = 0; r < q; ++r) {
+        const int64_t len = offsets[r + 1] - offsets[r];
+        TopkWorkspace *ww = nullptr, *ws = nullptr;
+        if ((rc = topk_workspace_create(&ww, len, k_per_segment[r], c->n, nullptr, nullptr, true, c->d)) ||
+            (rc = topk_workspace_create(&ws, len, k_per_segment[r], 1, nullptr, nullptr, true, c->d))) {
+            topk_workspace_destroy(ww);
+            return fail(rc, "top-k workspace allocation failed (segment %d)", r);
+        }
+        c->seg_w.push_back(ww); c->seg_s.push_back(ws);
+        c->seg_off.push_back(offsets[r]); c->seg_k.push_back(k_per_segment[r]); c->seg_at.push_back(at);
+        at += k_per_segment[r];
+    }
+    drop_graphs(c);
+    return CDADAM_OK;
+}
+
 int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
 {
     if (!c || !offsets) return fail(CDADAM_ERR_ARG, "cdadam_set_segments: NULL argument");
@@ -677,6 +749,7 @@ int cdadam_set_mode(cdadam_ctx *c, int mode)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_mode: NULL context");
     if (mode != CDADAM_MARKOV && mode != CDADAM_EF && mode != CDADAM_NAIVE) return fail(CDADAM_ERR_ARG, "unknown mode %d", mode);
+    if (mode != CDADAM_MARKOV && !c->seg_w.empty()) return fail(CDADAM_ERR_STATE, "top-k segments are available for Algorithm 1 only");
     if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the mode must be set before the first step");
     c->mode = mode;
     return CDADAM_OK;
@@ -782,6 +855,8 @@ int cdadam_launches_per_step(cdadam_ctx *c)
 {
     if (!c) return 0;
     if (c->comp == CDADAM_SIGN) return c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5;
+    if (c->comp == CDADAM_TOPK && !c->seg_w.empty())
+        return (int)c->seg_w.size() * (topk_launches_per_step(c->n) + 1) + 2;
     if (c->comp == CDADAM_TOPK)
         return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : c->mode == CDADAM_NAIVE ? 3 : 0);
     if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : c->mode == CDADAM_NAIVE ? 7 : 4;

@@ -9,10 +9,13 @@ namespace cdadam {
 struct TopkWorkspace;
 
 // Scratch and payload buffers for selecting k of d coordinates in each of `rows` vectors.
-// If idx/val are NULL the workspace owns the payload arrays (rows x k each).
+// If idx/val are NULL the workspace owns the payload arrays (rows x k each).  stride: elements
+// between consecutive rows of the vectors given to topk_select (0 = d; larger when the rows
+// are segments of longer vectors).
 // with_select = false allocates the payload arrays only (rand-k needs no selection scratch).
 int topk_workspace_create(TopkWorkspace **w, int64_t d, int64_t k, int rows,
-                          uint32_t *idx = nullptr, float *val = nullptr, bool with_select = true);
+                          uint32_t *idx = nullptr, float *val = nullptr, bool with_select = true,
+                          int64_t stride = 0);
 void topk_workspace_destroy(TopkWorkspace *w);
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
 int topk_launches_per_step(int n);
@@ -22,6 +25,11 @@ int topk_launches_per_step(int n);
 // payload; if update_b, b_r[j] += u_j at the kept coordinates.  a, b: rows x d.
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                  cudaStream_t st);
+
+// Top-k per segment: copies the payload of `seg` (a segment starting at coordinate `offset` of
+// the whole vector) into entries [at, at + seg.k) of every row of `whole`'s payload, indices
+// moved by `offset`.
+void topk_payload_concat(TopkWorkspace *whole, int64_t at, TopkWorkspace *seg, int64_t offset, cudaStream_t st);
 
 // Sparse server aggregation (Algorithm 1: ghat += mean of the workers' messages) from the n payloads held in `ww`:
 //   ghat_s += (sum_i c_i) / n on the coordinates some worker sent, workers added in the

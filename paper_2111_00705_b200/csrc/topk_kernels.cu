@@ -46,6 +46,7 @@ struct Sel {                          // outcome of the three levels for one row
 
 struct TopkWorkspace {
     int64_t d, k, wp, nbt;
+    int64_t stride;                   // elements between the rows of a and b (>= d)
     int rows;
     uint32_t *hist;                   // rows x kHistStride
     Sel *sel;                         // rows
@@ -105,15 +106,15 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
-             uint32_t *__restrict__ hist_all, const uint32_t *__restrict__ hit, int64_t d, int vec_ok)
+             uint32_t *__restrict__ hist_all, const uint32_t *__restrict__ hit, int64_t d, int vec_ok, int64_t stride)
 {
     __shared__ uint32_t h[kBins1];
     if (hit[blockIdx.y]) return;                      // the guessed bucket held: nothing to redo
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
     __syncthreads();
     const int row = blockIdx.y;
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // blocks loop over tiles: the grid is small, so rows whose guess held cost almost nothing
     for (int64_t base = (int64_t)blockIdx.x * kSub; base < d; base += (int64_t)gridDim.x * kSub) {
@@ -202,15 +203,15 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
             uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all,
-            const uint32_t *__restrict__ hit, int64_t d, int64_t wp, int vec_ok)
+            const uint32_t *__restrict__ hit, int64_t d, int64_t wp, int vec_ok, int64_t stride)
 {
     __shared__ uint32_t h[kBins2];
     if (hit[blockIdx.y]) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
     const int row = blockIdx.y;
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t b1 = sel_all[row].b1;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -283,7 +284,7 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
             float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
-            uint32_t *__restrict__ stash_cnt_all, int64_t d, int vec_ok)
+            uint32_t *__restrict__ stash_cnt_all, int64_t d, int vec_ok, int64_t stride)
 {
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
@@ -292,8 +293,8 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
     if (fl >= (uint32_t)kBins1) return;               // no guess for this row
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
     __syncthreads();
-    const float *a = a_all + (int64_t)row * d;
-    const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     const int64_t tile = (int64_t)row * gridDim.x + blockIdx.x;
     float *stash = stash_all + tile * kStashCap;
     uint16_t *spos = stash_pos_all + tile * kStashCap;
@@ -508,7 +509,7 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
              const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all, int64_t nt4k,
-             int64_t d)
+             int64_t d, int64_t stride)
 {
     __shared__ uint32_t h[kBins2];
     const int row = blockIdx.y;
@@ -516,7 +517,7 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
     __syncthreads();
     for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
-                           a_all + (int64_t)row * d, HAS_B ? b_all + (int64_t)row * d : nullptr,
+                           a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr,
                            HistLevel2{h, sel_all[row].b1});
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
@@ -535,7 +536,7 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
              const uint32_t *__restrict__ stash_cnt_all,
              const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
-             int64_t wp, int64_t nt4k)
+             int64_t wp, int64_t nt4k, int64_t stride)
 {
     __shared__ uint32_t h[kBins3];
     for (int t = threadIdx.x; t < kBins3; t += kBlock) h[t] = 0;
@@ -546,11 +547,11 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
     if (hit[row]) {                                   // the tiles' lists hold the values
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
         for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
-                               a_all + (int64_t)row * d, HAS_B ? b_all + (int64_t)row * d : nullptr,
+                               a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr,
                                HistLevel3{h, pre});
     } else {                                          // classic path: gather a and b
-        const float *a = a_all + (int64_t)row * d;
-        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const float *a = a_all + (int64_t)row * stride;
+        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
         const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
         for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
             uint32_t word = bm_cand[w0 + t];
@@ -583,7 +584,7 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
                const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ cnt_gt_all,
                uint32_t *__restrict__ cnt_eq_all,
                uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
-               uint32_t *__restrict__ cnt_tie_all, int64_t d, int64_t wp, int64_t nbt, int64_t nt4k)
+               uint32_t *__restrict__ cnt_tie_all, int64_t d, int64_t wp, int64_t nbt, int64_t nt4k, int64_t stride)
 {
     const int row = blockIdx.y;
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
@@ -594,8 +595,8 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
     if (hit[row]) {                                   // the tiles' lists hold the values
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
         const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
-        const float *a = a_all + (int64_t)row * d;
-        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const float *a = a_all + (int64_t)row * stride;
+        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
         const uint32_t lane = threadIdx.x & 31;
         float v[kWarpTiles][kPre];
 #pragma unroll
@@ -630,8 +631,8 @@ k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
         }
         return;
     } else {
-        const float *a = a_all + (int64_t)row * d;
-        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const float *a = a_all + (int64_t)row * stride;
+        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
         const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
         for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
             uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
@@ -780,7 +781,7 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
                 const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
                 const uint32_t *__restrict__ stash_cnt_all, const uint32_t *__restrict__ cnt_gt_all,
                 const uint32_t *__restrict__ cnt_eq_all, uint32_t *__restrict__ idx_all,
-                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d)
+                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d, int64_t stride)
 {
     const int row = blockIdx.y;
     uint32_t *idx = idx_all + (int64_t)row * k;
@@ -788,8 +789,8 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
     if (hit[row]) {
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
         const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
-        const float *a = a_all + (int64_t)row * d;
-        const float *b = HAS_B ? b_all + (int64_t)row * d : nullptr;
+        const float *a = a_all + (int64_t)row * stride;
+        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
         const Sel s = sel_all[row];
         const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
         const bool all_ties = s.k3 == s.c3;
@@ -873,24 +874,24 @@ template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
               const uint32_t *__restrict__ idx_all, float *__restrict__ val_all,
-              const uint32_t *__restrict__ have_val, int64_t d, int64_t k)
+              const uint32_t *__restrict__ have_val, int64_t d, int64_t k, int64_t stride)
 {
     const int row = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
     if (t >= k) return;
     const int64_t j = idx_all[(int64_t)row * k + t];
     if (j >= d) return;                       // caller-supplied sets are checked separately
-    const float *a = a_all + (int64_t)row * d;
+    const float *a = a_all + (int64_t)row * stride;
     if (have_val && have_val[row]) {          // the payload values were written with the indices
         if (HAS_B && UPDATE_B) {
-            float *b = b_all + (int64_t)row * d;
+            float *b = b_all + (int64_t)row * stride;
             b[j] = __fadd_rn(b[j], val_all[(int64_t)row * k + t]);
         }
         return;
     }
     float u;
     if (HAS_B) {
-        float *b = b_all + (int64_t)row * d;
+        float *b = b_all + (int64_t)row * stride;
         const float bj = b[j];
         u = __fsub_rn(a[j], bj);
         if (UPDATE_B) b[j] = __fadd_rn(bj, u);
@@ -1042,12 +1043,13 @@ static void free_ws(TopkWorkspace *w)
 }
 
 int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, uint32_t *idx,
-                          float *val, bool with_select)
+                          float *val, bool with_select, int64_t stride)
 {
     *out = nullptr;
     TopkWorkspace *w = new TopkWorkspace();
     memset(w, 0, sizeof *w);
     w->d = d; w->k = k; w->rows = rows;
+    w->stride = stride > 0 ? stride : d;
     w->wp = (d + 31) / 32;
     w->nbt = (w->wp + kTileWords - 1) / kTileWords;
     w->own_payload = idx == nullptr;
@@ -1104,26 +1106,26 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
-    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok);
+    k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok, w->stride);
     k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
-    k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok);
+    k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
-    k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok);
-    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k, w->d);
+    k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok, w->stride);
+    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k, w->d, w->stride);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
-    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->bm_cand, w->hist, w->d, w->wp, w->nt4k);
+    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->bm_cand, w->hist, w->d, w->wp, w->nt4k, w->stride);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
-    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k);
+    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k, w->stride);
     k_scan_lists<<<w->rows, kBlock, 0, st>>>(w->sel, w->hit, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
     k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit);
-    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
-        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);
+        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride);
     else
-        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k);
+        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride);
 }
 
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
@@ -1131,6 +1133,27 @@ void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool
 {
     if (b) select_impl<true>(w, a, b, update_b, vec_ok, st);
     else select_impl<false>(w, a, nullptr, false, vec_ok, st);
+}
+
+// Payload of a segment into the payload of the whole vector: entries [at, at + k_seg) of every
+// row, indices moved by the segment's offset.  grid = (ceil(k_seg/256), rows).
+__global__ void __launch_bounds__(kBlock)
+k_payload_concat(uint32_t *__restrict__ dst_idx, float *__restrict__ dst_val, int64_t k_all, int64_t at,
+                 const uint32_t *__restrict__ src_idx, const float *__restrict__ src_val, int64_t k_seg,
+                 uint32_t offset)
+{
+    const int row = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t >= k_seg) return;
+    dst_idx[(int64_t)row * k_all + at + t] = src_idx[(int64_t)row * k_seg + t] + offset;
+    dst_val[(int64_t)row * k_all + at + t] = src_val[(int64_t)row * k_seg + t];
+}
+
+void topk_payload_concat(TopkWorkspace *whole, int64_t at, TopkWorkspace *seg, int64_t offset, cudaStream_t st)
+{
+    const dim3 grid((unsigned)((seg->k + kBlock - 1) / kBlock), (unsigned)seg->rows);
+    k_payload_concat<<<grid, kBlock, 0, st>>>(whole->idx, whole->val, whole->k, at, seg->idx, seg->val, seg->k,
+                                              (uint32_t)offset);
 }
 
 void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st)
@@ -1162,9 +1185,9 @@ void randk_set(TopkWorkspace *w, const uint32_t *sets, int *error_flag, cudaStre
 void randk_gather(TopkWorkspace *w, const float *a, float *b, bool update_b, cudaStream_t st)
 {
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
-    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k);
-    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k);
-    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, nullptr, w->d, w->k);
+    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride);
+    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride);
+    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, nullptr, w->d, w->k, w->stride);
 }
 
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)

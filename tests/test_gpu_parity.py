@@ -412,6 +412,48 @@ def test_topk_selection_concentrated_in_a_few_tiles(mode):
     g.close(); o.close()
 
 
+@pytest.mark.parametrize("case", ["ragged", "aligned_large", "one_segment"])
+def test_topk_per_segment_matches_oracle(case):
+    """Top-k applied to every segment on its own (per tensor): concatenated payloads bit-exact,
+    all state exact, over several steps (so the per-segment threshold guesses are used)."""
+    if case == "ragged":
+        d, n = 30011, 3
+        off = [0, 5, 6, 4101, 4102, 20000, d]
+        ks = [2, 1, 300, 1, 77, 1000]
+    elif case == "aligned_large":
+        d, n = 3 * 40960, 4
+        off = [0, 40960, 2 * 40960, d]
+        ks = [400, 41, 4000]
+    else:
+        d, n = 50000, 2
+        off, ks = [0, d], [500]
+    w = synth.Workload("SEGK", d, n, synth.TOPK, 5, k=1, seed=41)
+    g, o = make_pair(w)
+    g.set_topk_segments(off, ks)
+    o.set_topk_segments(off, ks)
+    w.k = sum(ks)
+    rng = np.random.default_rng(7)
+    scale = np.repeat(10.0 ** rng.uniform(-2, 1, len(ks)), np.diff(off)).astype(np.float32)
+    for t_ in range(1, 6):
+        grads = w.grads(t_, "cpu") * torch.from_numpy(scale)        # tensors of different scales
+        g.step(grads.cuda()); o.step(grads.numpy())
+        check_payloads(g, o, w)
+        check_state(g, o, STEP_TOL, exact=True)
+    if case == "one_segment":                                   # = the whole-vector compressor
+        h = cd.CDAdam(d, n, cd.TOPK, k=500, x0=w.x0("cpu").cuda())
+        for t_ in range(1, 6):
+            h.step((w.grads(t_, "cpu") * torch.from_numpy(scale)).cuda())
+        assert torch.equal(h.params(), g.params())
+        h.close()
+    assert cd.lib().cdadam_set_topk_segments(g._h, 1, (ctypes.c_int64 * 2)(0, d), (ctypes.c_int64 * 1)(1)) == cd.ERR_STATE
+    g.close(); o.close()
+    f = cd.CDAdam(100, 2, cd.TOPK, k=3)
+    with pytest.raises(cd.CdadamError):
+        f.set_topk_segments([0, 10, 100], [11, 1])                  # k_r above the segment length
+    with pytest.raises(cd.CdadamError):
+        cd.CDAdam(100, 2, cd.SIGN).set_topk_segments([0, 100], [1])
+
+
 def test_topk_ties_lower_index_wins():
     """Few distinct magnitudes: most of the selection is decided by the tie rule."""
     rng = np.random.default_rng(0)
