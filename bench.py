@@ -191,6 +191,57 @@ def replicas_throughput(world, steps, total_ms):
     return world * steps / (total_ms * 1e-3)
 
 
+def run_distributed(args, w, dev, rank, world):
+    """The distributed deployment (one process per GPU, each with its share of the n workers,
+    messages over NCCL): device-timed K iterations, max over ranks.  Total work is fixed as N
+    grows, so scaling is "strong".  Rank 0 prints one JSON line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2111_00705_b200 import distributed as dd
+    from paper_2111_00705_b200 import synth
+    if w.compressor != synth.SIGN:
+        raise SystemExit("--layout %s: the distributed deployment takes the scaled-sign workloads" % args.layout)
+    if not dist.is_initialized():                      # a single process: a group of one
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", str(29000 + os.getpid() % 2000))
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
+    server_rank = 0 if args.layout == "server" else None
+    args.warmup = max(args.warmup, 3)
+    opt = dd.DistributedCDAdam(w.d, w.n, None, server_rank, beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps,
+                               offsets=w.offsets, x0=w.x0(dev), device=dev)
+    first, per = dd.partition(w.n, world, rank, server_rank)
+    grads = [w.grads(t + 1, dev).reshape(w.n, w.d)[first:first + per].contiguous().reshape(-1) if per else None
+             for t in range(2)]
+    stream = torch.cuda.current_stream()
+    for t in range(args.warmup):
+        opt.step(grads[t % 2])
+    dist.barrier(); torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index) if rank == 0 else None
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for t in range(args.steps):
+        opt.step(grads[t % 2])
+    b.record(stream)
+    dist.barrier(); torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    total_ms = max_over_ranks_ms(a.elapsed_time(b), dev)
+    opt.shard.device_status()
+    value = args.steps / (total_ms * 1e-3)
+    words = (w.d + 31) // 32
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "layout": args.layout, "workers_per_rank": per,
+                       "l2": "inputs larger than L2" if per * w.d * 4 >= 2 * 126e6 else "not flushed"},
+            "params_per_s": value * w.d,
+            "message_bytes_per_worker": words * 4 + 4 * w.q,
+            "gpu_launches": 5 * args.steps, "clocks": clocks}))
+    opt.close()
+    dist.destroy_process_group()
+
+
 def describe(w):
     from paper_2111_00705_b200 import synth
     comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity",
@@ -215,6 +266,11 @@ def main():
                     help="markov = Algorithm 1 (default); ef = classical error feedback, naive = naive "
                          "compression (the comparison schemes of Section 4; their bytes differ, so the "
                          "roofline figures of such a run are not the headline's)")
+    ap.add_argument("--layout", default="replicas", choices=["replicas", "sharded", "server"],
+                    help="replicas (default): every rank runs the whole n-worker problem on its own.  "
+                         "sharded: the distributed deployment, n/N workers per rank, worker messages "
+                         "all-gathered over NCCL, server stage computed on every rank (scaled sign only; "
+                         "strong scaling).  server: rank 0 is the server and holds no worker (N >= 2)")
     ap.add_argument("--tile", type=int, default=0,
                     help="force the kernels' tile size (profiler captures of scaled-down cases)")
     ap.add_argument("--scale", type=float, default=1.0,
@@ -247,6 +303,9 @@ def main():
         torch.cuda.synchronize()
 
     w = synth.workload(args.workload, scale=args.scale)
+    if args.layout != "replicas":
+        run_distributed(args, w, dev, rank, world)
+        return
     if args.compressor == "randk":
         w.compressor, w.k, w.offsets = synth.RANDK, max(1, w.d // 100), None
     if args.warmup < 3:
@@ -267,7 +326,9 @@ def main():
     if args.grads == "bf16":
         grads = [g.to(torch.bfloat16) for g in grads]
         opt.step = opt.step_bf16
-    small = w.n * w.d * 4 < 512e6
+    # L2 holds 126 MB.  A step whose gradients alone are at least twice that (and whose worker
+    # state is as large again) cannot find its inputs there; smaller workloads get the flush.
+    small = w.n * w.d * 4 < 2 * 126e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
     stream = torch.cuda.current_stream()
 

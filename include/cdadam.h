@@ -131,6 +131,58 @@ int cdadam_step_bf16(cdadam_ctx *ctx, const void *grads_bf16, void *stream);
 int cdadam_step_host(cdadam_ctx *ctx, const float *grads_host, float *x_out_host,
                      void *stream);
 
+/*
+ * Distributed deployment of Algorithm 1 (Section 5: the workers send c^(i) to the server, the
+ * server sends c to all workers, and every worker keeps gtil, m, v, vhat and x and updates the
+ * model itself).  A process creates a context for the workers it holds and runs an iteration
+ * in its three stages; between the stages the caller moves the messages (d sign bits and q
+ * scales each, the paper's 32 + d bits for q = 1) with whatever transport it has - the
+ * library makes no network call.  The result is that of one context holding all n workers,
+ * bit for bit, because every stage computes the same binary32 operations in the same order.
+ *
+ * cdadam_create_shard: as cdadam_create with the scaled-sign compressor, for the workers
+ *   [first_worker, first_worker + n_local) of n.  n_local may be 0 (a process that is only
+ *   the server).  The worker state ghat^(i) is allocated for the n_local workers only;
+ *   CDADAM_STATE_GHAT_W is n_local x d.  The message buffers hold all n worker messages.
+ *   cdadam_step, cdadam_step_bf16 and cdadam_step_host are refused (CDADAM_ERR_STATE) when
+ *   n_local < n.  Segments, mode, step size, weight decay as for any context, set alike on
+ *   every process.
+ *
+ * cdadam_step_workers: worker stage for the context's own workers (Algorithm 1, the workers'
+ *   compression and state update).  grads: device, n_local x d floats, row r is worker
+ *   first_worker + r (may be NULL when n_local = 0).  Writes rows [first_worker,
+ *   first_worker + n_local) of the worker message buffers.
+ * cdadam_step_server: server stage (aggregation, compression, Algorithm 1) from all n worker
+ *   messages in the buffers; writes the server message.  Only a process that acts as the
+ *   server calls it; calling it on every process, after all n messages have been gathered
+ *   everywhere, replaces the server's broadcast by redundant computation.
+ * cdadam_step_update: gtil += c and the AMSGrad update from the server message in the
+ *   buffers (Algorithm 1, the state update of the server and of every worker).  Completes
+ *   the iteration.
+ * Order per iteration: workers, [server], update; anything else is CDADAM_ERR_STATE.  All
+ * three are asynchronous on `stream`, allocate nothing, and must not be under stream capture.
+ * The caller orders its transfers with the stream (the messages are written by the work
+ * queued by cdadam_step_workers / cdadam_step_server and read by the next stage).
+ *
+ * cdadam_exchange_buffers: device pointers, owned by the context, of the message buffers:
+ *   worker_bits    n x words uint32, row i = the sign words of worker i (bit layout as in
+ *                  cdadam_last_payload)
+ *   worker_scales  n x q floats, row i = the scales of worker i.  This buffer ALTERNATES
+ *                  between two arrays from one iteration to the next: ask again after every
+ *                  cdadam_step_workers
+ *   server_bits    words uint32;  server_scales  q floats
+ *   words = ceil(d / 32).  Any output pointer may be NULL.  A context that holds all n
+ *   workers may use the staged calls too.
+ */
+cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local,
+                                float beta1, float beta2, float lr, float eps);
+int cdadam_step_workers(cdadam_ctx *ctx, const float *grads, void *stream);
+int cdadam_step_server(cdadam_ctx *ctx, void *stream);
+int cdadam_step_update(cdadam_ctx *ctx, void *stream);
+int cdadam_exchange_buffers(cdadam_ctx *ctx, uint32_t **worker_bits, float **worker_scales,
+                            uint32_t **server_bits, float **server_scales, int64_t *words,
+                            int *q);
+
 /* Device pointer to the model x (d floats), owned by the context, valid until destroy.
  * Its contents are x_{t+1} once the stream of the last step has completed.  NULL if ctx
  * is NULL. */

@@ -26,6 +26,14 @@ _SIGNATURES = {
     "cdadam_step": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_bf16": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_host": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_create_shard": (_c.c_void_p, [_c.c_int64, _c.c_int, _c.c_int, _c.c_int,
+                                          _c.c_float, _c.c_float, _c.c_float, _c.c_float]),
+    "cdadam_step_workers": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_step_server": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
+    "cdadam_step_update": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
+    "cdadam_exchange_buffers": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
+                                           _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
+                                           _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int)]),
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
@@ -130,9 +138,9 @@ class CDAdam:
         self.d, self.n, self.compressor, self.k = int(d), int(n), int(compressor), int(k)
         self.q = 1
         self.mode = int(mode)
+        self.first_worker, self.n_local = 0, self.n
         with torch.cuda.device(self.device):
-            self._h = lib().cdadam_create(self.d, self.n, self.compressor, self.k,
-                                          beta1, beta2, lr, eps)
+            self._h = self._create(beta1, beta2, lr, eps)
         if not self._h:
             raise CdadamError(ERR_ARG, last_error())
         if mode != MARKOV:
@@ -141,6 +149,9 @@ class CDAdam:
             self.set_segments(offsets)
         if x0 is not None:
             self.set_params(x0)
+
+    def _create(self, beta1, beta2, lr, eps):
+        return lib().cdadam_create(self.d, self.n, self.compressor, self.k, beta1, beta2, lr, eps)
 
     def close(self):
         if self._h:
@@ -224,14 +235,14 @@ class CDAdam:
         _check(lib().cdadam_set_weight_decay(self._h, weight_decay))
 
     def get_state(self, name, stream=None):
-        count = self.n * self.d if name == "ghat_w" else self.d
+        count = self.n_local * self.d if name == "ghat_w" else self.d
         out = torch.empty(count, dtype=torch.float32, device=self.device)
         _check(lib().cdadam_get_state(self._h, STATE_NAMES.index(name), ctypes.c_void_p(out.data_ptr()),
                                       _stream(stream)))
-        return out.view(self.n, self.d) if name == "ghat_w" else out
+        return out.view(self.n_local, self.d) if name == "ghat_w" else out
 
     def set_state(self, name, value, stream=None):
-        count = self.n * self.d if name == "ghat_w" else self.d
+        count = self.n_local * self.d if name == "ghat_w" else self.d
         _check(lib().cdadam_set_state(self._h, STATE_NAMES.index(name), _dev_f32(value, count, name),
                                       _stream(stream)))
 
@@ -271,6 +282,48 @@ class CDAdam:
 
     def launches_per_step(self):
         return lib().cdadam_launches_per_step(self._h)
+
+
+class CDAdamShard(CDAdam):
+    """A context for the workers [first_worker, first_worker + n_local) of n (scaled sign):
+    one process of a distributed deployment.  An iteration runs in its stages with the
+    messages moved by the caller in between (see ``distributed.py``)."""
+
+    def __init__(self, d, n, first_worker, n_local, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
+                 offsets=None, x0=None, device=None, mode=MARKOV):
+        self._shard = (int(first_worker), int(n_local))
+        super().__init__(d, n, SIGN, 0, beta1, beta2, lr, eps, offsets, x0, device, mode)
+        self.first_worker, self.n_local = self._shard
+
+    def _create(self, beta1, beta2, lr, eps):
+        return lib().cdadam_create_shard(self.d, self.n, self._shard[0], self._shard[1], beta1, beta2, lr, eps)
+
+    def step_workers(self, grads, stream=None):
+        """Worker stage on the n_local x d device gradients of this context's workers."""
+        g = None if self.n_local == 0 else _dev_f32(grads, self.n_local * self.d, "grads")
+        _check(lib().cdadam_step_workers(self._h, g, _stream(stream)))
+
+    def step_server(self, stream=None):
+        """Server stage from the n worker messages in the exchange buffers."""
+        _check(lib().cdadam_step_server(self._h, _stream(stream)))
+
+    def step_update(self, stream=None):
+        """gtil += c and the AMSGrad update from the server message in the exchange buffers."""
+        _check(lib().cdadam_step_update(self._h, _stream(stream)))
+
+    def exchange_buffers(self):
+        """Torch views (no copy) of the message buffers: worker_bits int32[n, words],
+        worker_scales float32[n, q], server_bits int32[words], server_scales float32[q].
+        worker_scales alternates between two arrays: ask again after every step_workers."""
+        wb, ws, sb, ss = (ctypes.c_void_p() for _ in range(4))
+        words, q = ctypes.c_int64(), ctypes.c_int()
+        _check(lib().cdadam_exchange_buffers(self._h, ctypes.byref(wb), ctypes.byref(ws), ctypes.byref(sb),
+                                             ctypes.byref(ss), ctypes.byref(words), ctypes.byref(q)))
+        w, q = words.value, q.value
+        return {"worker_bits": _view(wb.value, self.n * w, torch.int32, self.device).view(self.n, w),
+                "worker_scales": _view(ws.value, self.n * q, torch.float32, self.device).view(self.n, q),
+                "server_bits": _view(sb.value, w, torch.int32, self.device),
+                "server_scales": _view(ss.value, q, torch.float32, self.device)}
 
 
 def compress_sign(x, offsets=None, stream=None):

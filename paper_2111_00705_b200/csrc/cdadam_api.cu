@@ -131,6 +131,11 @@ constexpr int64_t kFuseMaxBlocks = 4 * 148;   // one wave of 256-thread blocks a
 struct cdadam_ctx {
     int64_t d = 0, k = 0, wp = 0, steps = 0;
     int n = 0, comp = 0, device = 0;
+    // Distributed deployment: this context holds the workers [first, first + nloc) of the n.
+    // An ordinary context holds all of them (first = 0, nloc = n).  The worker state and the
+    // worker pass's scratch have nloc rows; the message buffers (wbits, wscale) have n rows.
+    int first = 0, nloc = 0;
+    int phase = 0;          // split step: 0 = between iterations, 1 = worker stage queued, 2 = server stage queued
     int tile_override = 0;  // 0 = choose from d and q
     int mode = CDADAM_MARKOV;
     Hyper hp{};
@@ -219,18 +224,18 @@ int alloc_sign_buffers(cdadam_ctx *c)
     if ((rc = dev_zalloc(&c->wscale[1], (size_t)c->n * q))) return rc;
     if ((rc = dev_zalloc(&c->zero_scale, (size_t)c->n * q))) return rc;
     if ((rc = dev_zalloc(&c->sscale, (size_t)q))) return rc;
-    if ((rc = dev_zalloc(&c->wpart, (size_t)c->n * c->ts.tb.nparts))) return rc;
+    if ((rc = dev_zalloc(&c->wpart, (size_t)c->nloc * c->ts.tb.nparts))) return rc;
     if ((rc = dev_zalloc(&c->spart, (size_t)c->ts_s.tb.nparts))) return rc;
-    if ((rc = dev_zalloc(&c->wdone, (size_t)c->n * q))) return rc;
+    if ((rc = dev_zalloc(&c->wdone, (size_t)c->nloc * q))) return rc;
     if ((rc = dev_zalloc(&c->sdone, (size_t)q))) return rc;
     // Finishing the scales inside the passes saves two launches but lengthens every block by
     // a fence and an atomic round trip: measured 12 % faster when all blocks of a pass are
     // resident at once (d = 65,536, n = 4) and 4 to 13 % slower on grids of many waves.
-    c->fuse_finish = (int64_t)c->n * c->ts.tb.ntiles <= kFuseMaxBlocks && c->ts_s.tb.ntiles <= kFuseMaxBlocks;
+    c->fuse_finish = (int64_t)c->nloc * c->ts.tb.ntiles <= kFuseMaxBlocks && c->ts_s.tb.ntiles <= kFuseMaxBlocks;
     // a segment of more than 4096 tiles is shared by several blocks of the scale kernel
     c->wsplit = finalize_split(c->ts);
     c->ssplit = finalize_split(c->ts_s);
-    if (c->wsplit > 1 && (rc = dev_zalloc(&c->wsums, (size_t)c->n * q * c->wsplit))) return rc;
+    if (c->wsplit > 1 && (rc = dev_zalloc(&c->wsums, (size_t)c->nloc * q * c->wsplit))) return rc;
     if (c->ssplit > 1 && (rc = dev_zalloc(&c->ssums, (size_t)q * c->ssplit))) return rc;
     return CDADAM_OK;
 }
@@ -296,35 +301,59 @@ void drop_graphs(cdadam_ctx *c)
     for (auto &g : c->graphs) retire_graph(c, g);
 }
 
-// The three to five launches of one scaled-sign step, queued on st.  Changes no host state.
-void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
+// The stages of one scaled-sign step, queued on st; none changes host state.  `new_scale`
+// is the n x q array that receives (workers) or holds (server) the scales of this iteration's
+// worker messages.  The worker stage covers the context's own workers: rows
+// [first, first + nloc) of the message buffers.
+void enqueue_sign_workers(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, float *new_scale, cudaStream_t st)
 {
-    const Tables &tb = c->ts.tb, &tbs = c->ts_s.tb;
-    const bool ef = c->mode == CDADAM_EF;
-    const bool svec = c->d % 4 == 0;
-    const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
-    float *new_scale = c->wscale[c->cur ^ 1];
+    const Tables &tb = c->ts.tb;
     const bool naive = c->mode == CDADAM_NAIVE;
     const bool fuse = c->fuse_finish && !naive;
-    if (naive)      // the payload is C(g) itself: no worker state is read or written
-        launch_pack_sign(static_cast<const float *>(grads_in), c->wbits, c->wpart, tb, c->n, c->wp, vec, st);
-    else
-        launch_worker_sign(grads_in, bf16, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, ef,
-                           c->error_flag, fuse ? new_scale : nullptr, c->wdone, st);
+    const int64_t so = (int64_t)c->first * tb.q;
+    const float *old_scale = (c->pending ? c->wscale[c->cur] : c->zero_scale) + so;
+    uint32_t *bits = c->wbits + (int64_t)c->first * c->wp;
+    if (c->nloc > 0) {
+        if (naive)      // the payload is C(g) itself: no worker state is read or written
+            launch_pack_sign(static_cast<const float *>(grads_in), bits, c->wpart, tb, c->nloc, c->wp, vec, st);
+        else
+            launch_worker_sign(grads_in, bf16, c->ghat_w, bits, old_scale, c->wpart, tb, c->nloc, c->wp, vec,
+                               c->mode == CDADAM_EF, c->error_flag, fuse ? new_scale + so : nullptr, c->wdone, st);
+    }
     prof_mark(c, st);
     if (!fuse) {
-        launch_finalize_scales(c->wpart, new_scale, tb, c->n, st, c->wsplit, c->wsums, c->wdone);
+        if (c->nloc > 0) launch_finalize_scales(c->wpart, new_scale + so, tb, c->nloc, st, c->wsplit, c->wsums, c->wdone);
         prof_mark(c, st);
     }
-    launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, svec, c->mode,
+}
+
+void enqueue_sign_server(cdadam_ctx *c, const float *new_scale, cudaStream_t st)
+{
+    const Tables &tbs = c->ts_s.tb;
+    const bool fuse = c->fuse_finish && c->mode != CDADAM_NAIVE;
+    launch_server_sign(c->wbits, new_scale, c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, c->d % 4 == 0, c->mode,
                        fuse ? c->sscale : nullptr, c->sdone, st);
     prof_mark(c, st);
     if (!fuse) {
         launch_finalize_scales(c->spart, c->sscale, tbs, 1, st, c->ssplit, c->ssums, c->sdone);
         prof_mark(c, st);
     }
-    launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, tbs, c->hp, svec, c->mode, st);
+}
+
+void enqueue_sign_update(cdadam_ctx *c, cudaStream_t st)
+{
+    launch_update_sign(c->sbits, c->sscale, c->ghat_s, c->gtil, c->m, c->v, c->vhat, c->x, c->ts_s.tb, c->hp, c->d % 4 == 0,
+                       c->mode, st);
     prof_mark(c, st);
+}
+
+// The three to five launches of one scaled-sign step, queued on st.  Changes no host state.
+void enqueue_sign_step(cdadam_ctx *c, const void *grads_in, bool bf16, bool vec, cudaStream_t st)
+{
+    float *new_scale = c->wscale[c->cur ^ 1];
+    enqueue_sign_workers(c, grads_in, bf16, vec, new_scale, st);
+    enqueue_sign_server(c, new_scale, st);
+    enqueue_sign_update(c, st);
 }
 
 // One iteration of Algorithm 1 with the top-k compressor, queued on st.  No host state changes.
@@ -427,16 +456,19 @@ extern "C" {
 
 const char *cdadam_last_error(void) { return g_err; }
 
-cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float beta1, float beta2,
-                          float lr, float eps)
+static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compressor, int64_t k, float beta1,
+                               float beta2, float lr, float eps)
 {
     if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
     if (n < 1 || n > 65535) { fail(CDADAM_ERR_ARG, "n must be in [1, 65535]"); return nullptr; }
+    if (first < 0 || nloc < 0 || first + nloc > n) { fail(CDADAM_ERR_ARG, "the context's workers [first, first + n_local) must lie in [0, n)"); return nullptr; }
+    if (nloc != n && compressor != CDADAM_SIGN) { fail(CDADAM_ERR_ARG, "a context that holds a part of the workers needs the scaled-sign compressor"); return nullptr; }
     if (compressor < CDADAM_SIGN || compressor > CDADAM_RANDK) { fail(CDADAM_ERR_ARG, "unknown compressor %d", compressor); return nullptr; }
     if ((compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k and rand-k need 1 <= k <= d"); return nullptr; }
     cdadam_ctx *c = new (std::nothrow) cdadam_ctx;
     if (!c) { fail(CDADAM_ERR_ALLOC, "out of host memory"); return nullptr; }
-    c->d = d; c->n = n; c->comp = compressor; c->k = (compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) ? k : 0;
+    c->d = d; c->n = n; c->first = first; c->nloc = nloc;
+    c->comp = compressor; c->k = (compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) ? k : 0;
     c->wp = (d + 31) / 32;
     c->hp.beta1 = beta1; c->hp.beta2 = beta2; c->hp.lr = lr; c->hp.nu = eps;
     c->hp.omb1 = 1.0f - beta1; c->hp.omb2 = 1.0f - beta2;
@@ -444,7 +476,7 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
     int rc = CDADAM_OK;
     const int64_t flat[2] = {0, d};
     do {
-        if ((rc = dev_zalloc(&c->ghat_w, (size_t)n * d))) break;
+        if ((rc = dev_zalloc(&c->ghat_w, (size_t)nloc * d))) break;
         if ((rc = dev_zalloc(&c->ghat_s, (size_t)d))) break;
         if ((rc = dev_zalloc(&c->gtil, (size_t)d))) break;
         if ((rc = dev_zalloc(&c->m, (size_t)d))) break;
@@ -468,6 +500,18 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
     } while (0);
     if (rc != CDADAM_OK || cudaDeviceSynchronize() != cudaSuccess) { cdadam_destroy(c); return nullptr; }
     return c;
+}
+
+cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float beta1, float beta2,
+                          float lr, float eps)
+{
+    return create_impl(d, n, 0, n, compressor, k, beta1, beta2, lr, eps);
+}
+
+cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local, float beta1, float beta2,
+                                float lr, float eps)
+{
+    return create_impl(d, n, first_worker, n_local, CDADAM_SIGN, 0, beta1, beta2, lr, eps);
 }
 
 void cdadam_destroy(cdadam_ctx *c)
@@ -497,25 +541,41 @@ void cdadam_destroy(cdadam_ctx *c)
 static int ensure_stage(cdadam_ctx *c)
 {
     if (c->stage) return CDADAM_OK;
-    const size_t bytes = (size_t)c->n * c->d * sizeof(float);
+    const size_t bytes = (size_t)(c->nloc ? c->nloc : 1) * c->d * sizeof(float);
     cudaError_t e = cudaMalloc((void **)&c->stage, bytes);
     if (e != cudaSuccess) { c->stage = nullptr; return fail(CDADAM_ERR_ALLOC, "staging buffer: %s", cudaGetErrorString(e)); }
     return CDADAM_OK;
 }
 
+// Launch arguments alternate from step to step (double-buffered scales, the deferred
+// payload), so a step recorded into a caller's graph would replay wrongly.
+static int refuse_capture(cudaStream_t st)
+{
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) cudaGetLastError();
+    else if (cs != cudaStreamCaptureStatusNone)
+        return fail(CDADAM_ERR_STATE, "cdadam_step: the stream is being captured; a step cannot be part of a caller's graph");
+    return CDADAM_OK;
+}
+
+// alpha_t = base * gamma^(milestones already passed), by repeated binary32 products
+static void step_size_of_this_step(cdadam_ctx *c)
+{
+    if (c->milestones.empty()) return;
+    float lr = c->base_lr;
+    for (int64_t after : c->milestones)
+        if (after <= c->steps) lr = lr * c->gamma;
+    apply_lr(c, lr);
+}
+
 static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *stream)
 {
     if (!c || !grads_in) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
+    if (c->nloc != c->n) return fail(CDADAM_ERR_STATE, "cdadam_step: this context holds a part of the workers; use the staged calls");
+    if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_step: a staged iteration is under way");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
-    {
-        // Launch arguments alternate from step to step (double-buffered scales, the deferred
-        // payload), so a step recorded into a caller's graph would replay wrongly.
-        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
-        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) cudaGetLastError();
-        else if (cs != cudaStreamCaptureStatusNone)
-            return fail(CDADAM_ERR_STATE, "cdadam_step: the stream is being captured; a step cannot be part of a caller's graph");
-    }
+    if (int rc = refuse_capture(st)) return rc;
     const float *grads = static_cast<const float *>(grads_in);
     if (bf16 && (c->comp != CDADAM_SIGN || c->mode == CDADAM_NAIVE)) {
         // only the scaled-sign worker pass reads bfloat16 directly; the other compressors
@@ -527,13 +587,7 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
         bf16 = false;
     }
     const bool vec = aligned16(grads) && c->d % (bf16 ? 8 : 4) == 0;
-    if (!c->milestones.empty()) {
-        // alpha_t = base * gamma^(milestones already passed), by repeated binary32 products
-        float lr = c->base_lr;
-        for (int64_t after : c->milestones)
-            if (after <= c->steps) lr = lr * c->gamma;
-        apply_lr(c, lr);
-    }
+    step_size_of_this_step(c);
     prof_mark(c, st);
     const bool ef = c->mode == CDADAM_EF;
     const bool naive = c->mode == CDADAM_NAIVE;
@@ -634,6 +688,73 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
 
 int cdadam_step(cdadam_ctx *c, const float *grads, void *stream) { return step_impl(c, grads, false, stream); }
 
+// ---- one iteration in its three stages (distributed deployment of Algorithm 1) ---------------
+
+static int staged_ok(cdadam_ctx *c, const char *what)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "%s: NULL context", what);
+    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "%s: the staged calls take the scaled-sign compressor", what);
+    if (c->prof_on) return fail(CDADAM_ERR_STATE, "%s: per-stage timing covers cdadam_step only", what);
+    return CDADAM_OK;
+}
+
+int cdadam_step_workers(cdadam_ctx *c, const float *grads, void *stream)
+{
+    if (int rc = staged_ok(c, "cdadam_step_workers")) return rc;
+    if (c->nloc > 0 && !grads) return fail(CDADAM_ERR_ARG, "cdadam_step_workers: NULL gradients");
+    if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_step_workers: the previous iteration has not been completed by cdadam_step_update");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    step_size_of_this_step(c);
+    enqueue_sign_workers(c, grads, false, aligned16(grads) && c->d % 4 == 0, c->wscale[c->cur ^ 1], st);
+    if (int rc = check_launch("cdadam_step_workers")) return rc;
+    c->cur ^= 1;                              // wscale[cur] now holds this iteration's scales
+    c->pending = c->mode != CDADAM_NAIVE;
+    c->phase = 1;
+    return CDADAM_OK;
+}
+
+int cdadam_step_server(cdadam_ctx *c, void *stream)
+{
+    if (int rc = staged_ok(c, "cdadam_step_server")) return rc;
+    if (c->phase != 1) return fail(CDADAM_ERR_STATE, "cdadam_step_server: call cdadam_step_workers first (once per iteration)");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    enqueue_sign_server(c, c->wscale[c->cur], st);
+    if (int rc = check_launch("cdadam_step_server")) return rc;
+    c->phase = 2;
+    return CDADAM_OK;
+}
+
+int cdadam_step_update(cdadam_ctx *c, void *stream)
+{
+    if (int rc = staged_ok(c, "cdadam_step_update")) return rc;
+    if (c->phase == 0) return fail(CDADAM_ERR_STATE, "cdadam_step_update: call cdadam_step_workers first");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    enqueue_sign_update(c, st);
+    if (int rc = check_launch("cdadam_step_update")) return rc;
+    c->phase = 0;
+    c->steps += 1;
+    return CDADAM_OK;
+}
+
+int cdadam_exchange_buffers(cdadam_ctx *c, uint32_t **worker_bits, float **worker_scales, uint32_t **server_bits,
+                            float **server_scales, int64_t *words, int *q)
+{
+    if (int rc = staged_ok(c, "cdadam_exchange_buffers")) return rc;
+    if (worker_bits) *worker_bits = c->wbits;
+    if (worker_scales) *worker_scales = c->wscale[c->cur];
+    if (server_bits) *server_bits = c->sbits;
+    if (server_scales) *server_scales = c->sscale;
+    if (words) *words = c->wp;
+    if (q) *q = c->ts.tb.q;
+    return CDADAM_OK;
+}
+
 int cdadam_step_bf16(cdadam_ctx *c, const void *grads, void *stream) { return step_impl(c, grads, true, stream); }
 
 int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, void *stream)
@@ -641,6 +762,7 @@ int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, 
     if (!c || !grads_host) return fail(CDADAM_ERR_ARG, "cdadam_step_host: NULL argument");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
+    if (c->nloc != c->n) return fail(CDADAM_ERR_STATE, "cdadam_step_host: this context holds a part of the workers; use the staged calls");
     const size_t bytes = (size_t)c->n * c->d * sizeof(float);
     int rc0 = ensure_stage(c);
     if (rc0) return rc0;
@@ -665,7 +787,7 @@ int cdadam_set_topk_segments(cdadam_ctx *c, int q, const int64_t *offsets, const
     if (!c || !offsets || !k_per_segment) return fail(CDADAM_ERR_ARG, "cdadam_set_topk_segments: NULL argument");
     if (c->comp != CDADAM_TOPK) return fail(CDADAM_ERR_STATE, "top-k segments apply to the top-k compressor only");
     if (c->mode != CDADAM_MARKOV) return fail(CDADAM_ERR_STATE, "top-k segments are available for Algorithm 1 only");
-    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
+    if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
     if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
     if (offsets[0] != 0 || offsets[q] != c->d) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
     int64_t total = 0;
@@ -708,7 +830,7 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
 {
     if (!c || !offsets) return fail(CDADAM_ERR_ARG, "cdadam_set_segments: NULL argument");
     if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "segments apply to the scaled-sign compressor only");
-    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
+    if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
     if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
     if (offsets[0] != 0 || offsets[q] != c->d) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
     for (int r = 0; r < q; ++r)
@@ -726,7 +848,7 @@ int cdadam_set_tile(cdadam_ctx *c, int tile)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_tile: NULL context");
     if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "tiles apply to the scaled-sign compressor only");
-    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the tile size must be set before the first step");
+    if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "the tile size must be set before the first step");
     if (tile != 0 && (tile < kSub || tile % kSub != 0 || tile > 64 * kSub))
         return fail(CDADAM_ERR_ARG, "tile must be 0 or a multiple of %d up to %d", kSub, 64 * kSub);
     c->tile_override = tile;
@@ -750,7 +872,7 @@ int cdadam_set_mode(cdadam_ctx *c, int mode)
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_mode: NULL context");
     if (mode != CDADAM_MARKOV && mode != CDADAM_EF && mode != CDADAM_NAIVE) return fail(CDADAM_ERR_ARG, "unknown mode %d", mode);
     if (mode != CDADAM_MARKOV && !c->seg_w.empty()) return fail(CDADAM_ERR_STATE, "top-k segments are available for Algorithm 1 only");
-    if (c->steps != 0) return fail(CDADAM_ERR_STATE, "the mode must be set before the first step");
+    if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "the mode must be set before the first step");
     c->mode = mode;
     return CDADAM_OK;
 }
@@ -795,12 +917,14 @@ int cdadam_get_state(cdadam_ctx *c, int name, float *dst, void *stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (name == CDADAM_STATE_GHAT_W && c->comp == CDADAM_SIGN && c->pending) {
-        launch_apply_sign(c->ghat_w, c->wbits, c->wscale[c->cur], c->ts.tb, c->n, c->wp, c->mode == CDADAM_EF, st);
+        if (c->nloc > 0)
+            launch_apply_sign(c->ghat_w, c->wbits + (int64_t)c->first * c->wp, c->wscale[c->cur] + (int64_t)c->first * c->ts.tb.q,
+                              c->ts.tb, c->nloc, c->wp, c->mode == CDADAM_EF, st);
         int rc = check_launch("apply deferred payload");
         if (rc) return rc;
         c->pending = false;
     }
-    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->n * c->d : (size_t)c->d;
+    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->nloc * c->d : (size_t)c->d;
     CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, st));
     return CDADAM_OK;
 }
@@ -811,7 +935,7 @@ int cdadam_set_state(cdadam_ctx *c, int name, const float *src, void *stream)
     float *dst = state_ptr(c, name);
     if (!dst) return fail(CDADAM_ERR_ARG, "unknown state name %d", name);
     DeviceGuard guard(c->device);
-    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->n * c->d : (size_t)c->d;
+    const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->nloc * c->d : (size_t)c->d;
     CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     if (name == CDADAM_STATE_GHAT_W) c->pending = false;   // the given values are final
     return CDADAM_OK;
