@@ -46,15 +46,14 @@ k_step_identity(const float *__restrict__ grads, float *__restrict__ ghat_w,
     }
 }
 
-__global__ void __launch_bounds__(kBlock)
+// One float4 of each of the five vectors per thread, no loop: short blocks at full occupancy
+// keep the most loads in flight for 5 read and 4 written streams.  grid = ceil(d / 1024).
+__global__ void __launch_bounds__(kBlock, 5)
 k_amsgrad(const float *__restrict__ gtil, float *__restrict__ m, float *__restrict__ v,
           float *__restrict__ vhat, float *__restrict__ x, int64_t d, Hyper hp, int vec_ok)
 {
-    const int64_t nvec = vec_ok ? d / 4 : 0;
-    const int64_t stride = (int64_t)gridDim.x * kBlock;
-    const int64_t t0 = (int64_t)blockIdx.x * kBlock + threadIdx.x;
-    for (int64_t q = t0; q < nvec; q += stride) {
-        const int64_t j = q * 4;
+    const int64_t j = ((int64_t)blockIdx.x * kBlock + threadIdx.x) * 4;
+    if (vec_ok && j + 4 <= d) {
         const float4 G = ld_ro4(gtil + j);
         float4 M = ld_rw4(m + j), V = ld_rw4(v + j), Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
         amsgrad1(G.x, M.x, V.x, Vh.x, X.x, hp);
@@ -62,11 +61,13 @@ k_amsgrad(const float *__restrict__ gtil, float *__restrict__ m, float *__restri
         amsgrad1(G.z, M.z, V.z, Vh.z, X.z, hp);
         amsgrad1(G.w, M.w, V.w, Vh.w, X.w, hp);
         st_rw4(m + j, M); st_rw4(v + j, V); st_rw4(vhat + j, Vh); st_rw4(x + j, X);
+        return;
     }
-    for (int64_t j = nvec * 4 + t0; j < d; j += stride) {
-        float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
-        amsgrad1(gtil[j], mm, vv, vh, xx, hp);
-        m[j] = mm; v[j] = vv; vhat[j] = vh; x[j] = xx;
+    const int64_t end = j + 4 < d ? j + 4 : d;
+    for (int64_t i = j; i < end; ++i) {
+        float mm = m[i], vv = v[i], vh = vhat[i], xx = x[i];
+        amsgrad1(gtil[i], mm, vv, vh, xx, hp);
+        m[i] = mm; v[i] = vv; vhat[i] = vh; x[i] = xx;
     }
 }
 
@@ -154,7 +155,7 @@ void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
                     Hyper hp, bool vec_ok, cudaStream_t st)
 {
-    k_amsgrad<<<grid_for(vec_ok ? d / 4 : d), kBlock, 0, st>>>(gtil, m, v, vhat, x, d, hp, vec_ok);
+    k_amsgrad<<<(unsigned)((d + 4 * kBlock - 1) / (4 * kBlock)), kBlock, 0, st>>>(gtil, m, v, vhat, x, d, hp, vec_ok);
 }
 
 }  // namespace cdadam

@@ -676,41 +676,74 @@ k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__rest
 // tile, the rank of its first tie among the row's ties (cnt_eq) and the payload offset of its
 // first kept coordinate (cnt_gt); a tile keeps its keys above T and those of its ties whose
 // rank is below k3.  Every eighth tile's offset is also the offset of its 32768-coordinate
-// span (cnt_fin), which the server aggregation uses.  A thread owns a contiguous run of
-// tiles.  grid = (rows).
+// span (cnt_fin), which the server aggregation uses.  The counts pass through shared memory
+// in chunks of 4096 tiles (coalesced loads and stores); inside a chunk a thread owns 16
+// consecutive tiles (padded rows, no bank conflicts).  grid = (rows).
+constexpr int kScanPer = 16;
+constexpr int kScanChunk = kBlock * kScanPer;
+__device__ __forceinline__ int scan_slot(int i) { return i + i / kScanPer; }
+
 __global__ void __launch_bounds__(kBlock)
 k_scan_lists(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all,
              uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt)
 {
+    __shared__ uint32_t s_eq[kScanChunk + kBlock], s_gt[kScanChunk + kBlock];
     const int row = blockIdx.x;
     if (!hit[row]) return;
     const Sel s = sel_all[row];
     const bool all_ties = s.k3 == s.c3;
     uint32_t *gt = cnt_gt_all + (int64_t)row * nt4k, *eq = cnt_eq_all + (int64_t)row * nt4k;
     uint32_t *fin = cnt_fin_all + (int64_t)row * nbt;
-    const int64_t per = (nt4k + kBlock - 1) / kBlock;
-    const int64_t t0 = min((int64_t)threadIdx.x * per, nt4k), t1 = min(t0 + per, nt4k);
-    uint32_t sum_eq = 0;
-    for (int64_t t = t0; t < t1; ++t) sum_eq += eq[t];
-    uint32_t total;
-    uint32_t tie_rank = block_excl_scan(sum_eq, total);
-    uint32_t sum_keep = 0;
-    for (int64_t t = t0; t < t1; ++t) {
-        const uint32_t e = eq[t];
-        const uint32_t take = all_ties ? e : (tie_rank >= s.k3 ? 0u : min(e, s.k3 - tie_rank));
-        eq[t] = tie_rank;
-        tie_rank += e;
-        const uint32_t keep = gt[t] + take;
-        gt[t] = keep;
-        sum_keep += keep;
-    }
-    uint32_t off = block_excl_scan(sum_keep, total);
-    for (int64_t t = t0; t < t1; ++t) {
-        const uint32_t keep = gt[t];
-        gt[t] = off;
-        if (t % kTilesPerBlock == 0) fin[t / kTilesPerBlock] = off;
-        off += keep;
+    uint32_t carry_eq = 0, carry_keep = 0;             // block-uniform
+    for (int64_t c0 = 0; c0 < nt4k; c0 += kScanChunk) {
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) {
+            const int i = m * kBlock + threadIdx.x;
+            const int64_t t = c0 + i;
+            s_eq[scan_slot(i)] = t < nt4k ? eq[t] : 0u;
+            s_gt[scan_slot(i)] = t < nt4k ? gt[t] : 0u;
+        }
+        __syncthreads();
+        const int mine = threadIdx.x * (kScanPer + 1);  // first slot of this thread's 16 tiles
+        uint32_t sum_eq = 0;
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) sum_eq += s_eq[mine + m];
+        uint32_t total_eq, total_keep;
+        uint32_t tie_rank = carry_eq + block_excl_scan(sum_eq, total_eq);
+        uint32_t sum_keep = 0;
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) {
+            const uint32_t e = s_eq[mine + m];
+            const uint32_t take = all_ties ? e : (tie_rank >= s.k3 ? 0u : min(e, s.k3 - tie_rank));
+            s_eq[mine + m] = tie_rank;
+            tie_rank += e;
+            const uint32_t keep = s_gt[mine + m] + take;
+            s_gt[mine + m] = keep;
+            sum_keep += keep;
+        }
+        uint32_t off = carry_keep + block_excl_scan(sum_keep, total_keep);
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) {
+            const uint32_t keep = s_gt[mine + m];
+            s_gt[mine + m] = off;
+            off += keep;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) {
+            const int i = m * kBlock + threadIdx.x;
+            const int64_t t = c0 + i;
+            if (t < nt4k) {
+                const uint32_t o = s_gt[scan_slot(i)];
+                eq[t] = s_eq[scan_slot(i)];
+                gt[t] = o;
+                if (t % kTilesPerBlock == 0) fin[t / kTilesPerBlock] = o;
+            }
+        }
+        carry_eq += total_eq;
+        carry_keep += total_keep;
+        __syncthreads();
     }
 }
 
@@ -1105,7 +1138,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
-    const dim3 fallback(std::min(dense.x, 148u * 4u), (unsigned)w->rows);
+    const dim3 fallback(std::min(dense.x, std::max(148u, 148u * 4u / (unsigned)w->rows)), (unsigned)w->rows);
     k_topk_spec<HAS_B><<<dense, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok, w->stride);
     k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
     k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride);
