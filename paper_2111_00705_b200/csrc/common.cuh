@@ -99,6 +99,32 @@ __device__ __forceinline__ dd block_sum(dd a)
 }
 
 // ------------------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel queued with launch_after() may be scheduled while
+// the kernel before it in the stream is still running: its blocks start, run up to
+// grid_dep_wait() and stop there until the earlier kernel has finished and its writes are
+// visible.  Everything a kernel reads that an earlier kernel of the same step writes must
+// therefore be read after grid_dep_wait(); what precedes it (table look-ups, loads of
+// vectors no earlier kernel of the step writes) overlaps the earlier kernel's tail and the
+// launch latency.  grid_dep_launch() in the earlier kernel lets the next one be scheduled as
+// soon as all of its own blocks have started.  Both are no-ops in a kernel launched the
+// ordinary way.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... P, typename... A>
+inline cudaError_t launch_after(void (*kernel)(P...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, A... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<P>(args)...);
+}
+
+// ------------------------------------------------------------------------------------
 // 128-bit global memory accesses.  Read-only streams (gradients, payload bits) use the
 // non-coherent path without L1 allocation; read-modify-write state uses streaming
 // (evict-first) loads and stores: every vector is touched once per kernel.

@@ -254,6 +254,7 @@ k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
               dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok,
               float *__restrict__ scale_new, unsigned int *__restrict__ done)
 {
+    grid_dep_launch();
     const int i = blockIdx.y;
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
@@ -308,6 +309,7 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
 {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) uint64_t full[kRingStages];
+    grid_dep_launch();
     const int i = blockIdx.y;
     const int64_t T = tb.order[blockIdx.x];
     const int first = tb.tile_first[T], last = tb.tile_last[T];
@@ -390,11 +392,13 @@ constexpr int kFinBlock = 512;
 __global__ void __launch_bounds__(kFinBlock)
 k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Tables tb)
 {
+    grid_dep_launch();
     const int r = blockIdx.x, row = blockIdx.y;
     const int64_t lo = tb.off[r], hi = tb.off[r + 1];
     const int64_t T0 = lo / tb.tile, T1 = (hi - 1) / tb.tile;
     const dd *p = part + (int64_t)row * tb.nparts;
     dd acc = {0.0, 0.0};
+    grid_dep_wait();                                   // the partial sums come from the pass before
     for (int64_t T = T0 + threadIdx.x; T <= T1; T += kFinBlock)
         acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
     acc = block_sum<kFinBlock>(acc);
@@ -421,6 +425,8 @@ k_finalize_scales_split(const dd *__restrict__ part, float *__restrict__ scales,
     const int64_t A = T0 + z * per, B = min(A + per, T1 + 1);
     const dd *p = part + (int64_t)row * tb.nparts;
     dd acc = {0.0, 0.0};
+    grid_dep_launch();
+    grid_dep_wait();                                   // the partial sums come from the pass before
     for (int64_t T = A + threadIdx.x; T < B; T += kFinBlock)
         acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
     acc = block_sum<kFinBlock>(acc);
@@ -486,6 +492,8 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float fn = (float)n;
     const float rn = 1.0f / fn;               // exact when n is a power of two
+    grid_dep_launch();
+    grid_dep_wait();                          // worker sign words and scales come from the kernels before
 
     if (vec_ok && first == last && base + tb.tile <= tb.d) {
         constexpr int kSpan = 128 * VPT;                  // coordinates per warp per iteration
@@ -665,9 +673,12 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
         const int64_t j = base + threadIdx.x * 4;
         // error feedback reads the server's compressor input p (ghat buffer), not the old error;
         // naive compression reads and writes no compression state
-        float4 Gt = MODE == 2 ? make_float4(0.0f, 0.0f, 0.0f, 0.0f) : EF ? ld_ro4(ghat_s + j) : ld_rw4(gtil + j);
+        float4 Gt = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (MODE == 0) Gt = ld_rw4(gtil + j);           // no earlier kernel of the step writes gtil, m, v, vhat, x
         float4 M = ld_rw4(m + j), V = ld_rw4(v + j);
         float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
+        grid_dep_wait();                                // server sign words, scales (and p) come from the kernels before
+        if (EF) Gt = ld_ro4(ghat_s + j);
         const uint32_t nib = ld_ro_u32(sbits + (j >> 5)) >> (j & 31);
         const int first = tb.tile_first[T], last = tb.tile_last[T];
         float s0, s1, s2, s3;
@@ -698,6 +709,7 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
 
     const int first = tb.tile_first[T], last = tb.tile_last[T];
     const int64_t end = min(base + (int64_t)kUpdSpan, tb.d);
+    grid_dep_wait();
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
         const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
@@ -832,11 +844,11 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
 {
     if (split > 1) {
         dim3 grid((unsigned)tb.q, (unsigned)rows, (unsigned)split);
-        k_finalize_scales_split<<<grid, kFinBlock, 0, st>>>(part, scales, tb, split_sums, split_done);
+        launch_after(k_finalize_scales_split, grid, dim3(kFinBlock), 0, st, part, scales, tb, split_sums, split_done);
         return;
     }
     dim3 grid((unsigned)tb.q, (unsigned)rows);
-    k_finalize_scales<<<grid, kFinBlock, 0, st>>>(part, scales, tb);
+    launch_after(k_finalize_scales, grid, dim3(kFinBlock), 0, st, part, scales, tb);
 }
 
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,
@@ -845,15 +857,9 @@ void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_
                         cudaStream_t st)
 {
     const int pow2 = (n & (n - 1)) == 0;
-    if (mode == 2)
-        k_server_sign<2, 2><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                                    spart, tb, n, wp, vec_ok, pow2, sscale, done);
-    else if (mode == 1)
-        k_server_sign<2, 1><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                                       spart, tb, n, wp, vec_ok, pow2, sscale, done);
-    else
-        k_server_sign<2, 0><<<(unsigned)tb.ntiles, kBlock, 0, st>>>(wbits, wscale, ghat_s, gtil, sbits,
-                                                                        spart, tb, n, wp, vec_ok, pow2, sscale, done);
+    auto kern = mode == 2 ? k_server_sign<2, 2> : mode == 1 ? k_server_sign<2, 1> : k_server_sign<2, 0>;
+    launch_after(kern, dim3((unsigned)tb.ntiles), dim3(kBlock), 0, st, wbits, wscale, ghat_s, gtil, sbits, spart, tb, n, wp,
+                 (int)vec_ok, pow2, sscale, done);
 }
 
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
@@ -861,12 +867,8 @@ void launch_update_sign(const uint32_t *sbits, const float *sscale, const float 
                         bool vec_ok, int mode, cudaStream_t st)
 {
     const unsigned blocks = (unsigned)((tb.d + kUpdSpan - 1) / kUpdSpan);
-    if (mode == 2)
-        k_update_sign<2><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
-    else if (mode == 1)
-        k_update_sign<1><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
-    else
-        k_update_sign<0><<<blocks, kBlock, 0, st>>>(sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, vec_ok);
+    auto kern = mode == 2 ? k_update_sign<2> : mode == 1 ? k_update_sign<1> : k_update_sign<0>;
+    launch_after(kern, dim3(blocks), dim3(kBlock), 0, st, sbits, sscale, ghat_s, gtil, m, v, vhat, x, tb, hp, (int)vec_ok);
 }
 
 void launch_apply_sign(float *ghat_w, const uint32_t *wbits, const float *scales,
