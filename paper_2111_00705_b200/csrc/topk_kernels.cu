@@ -41,7 +41,8 @@ struct Sel {                          // outcome of the three levels for one row
     uint32_t b1, k1, c1;              // bucket, entries still to take inside it, its size
     uint32_t b2, k2, c2;
     uint32_t b3, k3, c3;              // T = b1<<20 | b2<<9 | b3; take k3 of the c3 ties
-    uint32_t pad[3];
+    uint32_t pre;                     // rows whose guess held: key bits 30..11 of T (bits 10..0 zero)
+    uint32_t pad[2];
 };
 
 struct TopkWorkspace {
@@ -161,7 +162,8 @@ k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, in
 {
     __shared__ uint32_t tot[kBlock];
     const int row = blockIdx.x;
-    if (level == 0 && hit[row]) return;               // level 1 was settled by the guess
+    const bool listed = hit[row] != 0u;               // the guess held: two levels, 20 + 11 key bits
+    if (listed && level != 1) return;
     Sel *sel = sel_all + row;
     const int nb = level == 2 ? kBins3 : kBins1;
     const uint32_t *hist = hist_all + (int64_t)row * kHistStride +
@@ -180,12 +182,18 @@ k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, in
         if (above < want && above + c >= want) {
             const uint32_t bucket = lo + t, rem = want - above;
             if (level == 0) { sel->b1 = bucket; sel->k1 = rem; sel->c1 = c; }
-            else if (level == 1) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
+            else if (level == 1 && !listed) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
             else {
-                sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
+                if (listed) {                        // T = prefix | bits 10..0, in the three-level layout
+                    const uint32_t T = sel->pre | bucket;
+                    sel->b1 = T >> 20; sel->b2 = (T >> 9) & (kBins2 - 1); sel->b3 = T & (kBins3 - 1);
+                    sel->k3 = rem; sel->c3 = c;
+                } else {
+                    sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
+                }
                 // guess for the next selection of this row: a little below this threshold,
                 // one bucket more after a guess that failed
-                const uint32_t margin = hit[row] ? kGuessMargin : kGuessMargin + 1u;
+                const uint32_t margin = listed ? kGuessMargin : kGuessMargin + 1u;
                 floor_bucket[row] = sel->b1 > margin ? sel->b1 - margin : 1u;
             }
         }
@@ -270,6 +278,13 @@ k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
         if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
+// Bin of a key at or above the floor key fk in the speculative pass: 2^11 keys per bin
+// counted from the floor, so the 2047 regular bins span four level-1 buckets (half an
+// octave) and bin 2047 takes everything above.  A threshold that falls into a regular bin
+// is then known down to key bit 11, and one more pass over the lists (bits 10..0) gives it
+// exactly: two levels instead of three.
+__device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t fk) { return min((key - fk) >> 11, (uint32_t)kBins1 - 1u); }
+
 // ------------------------------------------------------------------------------------
 // Speculative single dense pass.  The threshold moves little from one iteration to the
 // next, so the level-1 bucket of the previous selection, lowered by a margin, is taken as a
@@ -291,6 +306,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const int row = blockIdx.y;
     const uint32_t fl = floor_bucket[row];
     if (fl >= (uint32_t)kBins1) return;               // no guess for this row
+    const uint32_t fk = fl << 20;                     // lowest key at or above the floor
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
     __syncthreads();
     const float *a = a_all + (int64_t)row * stride;
@@ -318,16 +334,15 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
                 A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
                 A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
             }
-            const uint32_t hx = key_of(A[v].x) >> 20, hy = key_of(A[v].y) >> 20;
-            const uint32_t hz = key_of(A[v].z) >> 20, hw = key_of(A[v].w) >> 20;
-            BG[v][0] = __ballot_sync(kFull, hx >= fl);
-            BG[v][1] = __ballot_sync(kFull, hy >= fl);
-            BG[v][2] = __ballot_sync(kFull, hz >= fl);
-            BG[v][3] = __ballot_sync(kFull, hw >= fl);
-            if (hx >= fl) atomicAdd(&h[hx], 1u);
-            if (hy >= fl) atomicAdd(&h[hy], 1u);
-            if (hz >= fl) atomicAdd(&h[hz], 1u);
-            if (hw >= fl) atomicAdd(&h[hw], 1u);
+            const uint32_t kx = key_of(A[v].x), ky = key_of(A[v].y), kz = key_of(A[v].z), kw = key_of(A[v].w);
+            BG[v][0] = __ballot_sync(kFull, kx >= fk);
+            BG[v][1] = __ballot_sync(kFull, ky >= fk);
+            BG[v][2] = __ballot_sync(kFull, kz >= fk);
+            BG[v][3] = __ballot_sync(kFull, kw >= fk);
+            if (kx >= fk) atomicAdd(&h[fine_bin(kx, fk)], 1u);
+            if (ky >= fk) atomicAdd(&h[fine_bin(ky, fk)], 1u);
+            if (kz >= fk) atomicAdd(&h[fine_bin(kz, fk)], 1u);
+            if (kw >= fk) atomicAdd(&h[fine_bin(kw, fk)], 1u);
             mine += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
         }
         if (lane == 0) wcnt[warp] = mine;             // the same in every lane
@@ -358,10 +373,10 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const int64_t j = j0 + threadIdx.x;
             const bool valid = j < end;
             const float u = valid ? diff1<HAS_B>(a, b, j) : 0.0f;
-            const uint32_t hi = key_of(u) >> 20;
-            const bool ge = valid && hi >= fl;
+            const uint32_t key = key_of(u);
+            const bool ge = valid && key >= fk;
             const uint32_t wg = __ballot_sync(kFull, ge);
-            if (ge) atomicAdd(&h[hi], 1u);
+            if (ge) atomicAdd(&h[fine_bin(key, fk)], 1u);
             if (lane == 0) wcnt[warp] = __popc(wg);
             __syncthreads();
             uint32_t r = run + __popc(wg & lt), total = 0;
@@ -382,9 +397,10 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
         if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
-// Did the guess hold?  It did if at least k coordinates lie at or above the floor; then the
-// level-1 bucket follows from the histogram of those coordinates.  Otherwise the row's
-// level-1 histogram is cleared for the full pass.  grid = (rows), one block.
+// Did the guess hold?  It did if the k-th largest key lies in one of the regular fine bins
+// above the floor; then key bits 30..11 of the threshold follow from the histogram of those
+// coordinates.  Otherwise the row's level-1 histogram is cleared for the full pass.
+// grid = (rows), one block.
 __global__ void __launch_bounds__(kBlock)
 k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
                  const uint32_t *__restrict__ floor_bucket,
@@ -408,8 +424,9 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
     if (fl < (uint32_t)kBins1) {
         for (int t = per - 1; t >= 0; --t) {
             const uint32_t c = hist[lo + t];
-            if (above < k && above + c >= k) {
-                sel->b1 = lo + t; sel->k1 = k - above; sel->c1 = c;
+            if (above < k && above + c >= k && lo + t < kBins1 - 1) {    // the last bin is open-ended: no threshold from it
+                sel->pre = (fl << 20) + ((uint32_t)(lo + t) << 11);
+                sel->b1 = sel->pre >> 20; sel->k1 = k - above; sel->c1 = c;
                 found = 1u;
             }
             above += c;
@@ -484,25 +501,18 @@ __device__ __forceinline__ void for_each_listed(const WarpLists &w, const float 
     }
 }
 
-struct HistLevel2 {
-    uint32_t *h, b1;
+struct HistLow11 {                    // keys that share bits 30..11 with the threshold, by bits 10..0
+    uint32_t *h, pre11;
     __device__ __forceinline__ void operator()(float v) const
     {
         const uint32_t key = key_of(v);
-        if ((key >> 20) == b1) atomicAdd(&h[(key >> 9) & (kBins2 - 1)], 1u);
-    }
-};
-struct HistLevel3 {
-    uint32_t *h, pre;
-    __device__ __forceinline__ void operator()(float v) const
-    {
-        const uint32_t key = key_of(v);
-        if ((key >> 9) == pre) atomicAdd(&h[key & (kBins3 - 1)], 1u);
+        if ((key >> 11) == pre11) atomicAdd(&h[key & (kBins2 - 1)], 1u);
     }
 };
 
-// After a successful guess: the level-2 histogram of the listed values that fall into the
-// threshold bucket (what the second dense pass would have produced).  grid = (nbt, rows).
+// After a successful guess: the histogram of key bits 10..0 over the listed values that share
+// the threshold's bits 30..11; the pick that follows gives the exact threshold.
+// grid = (nbt, rows).
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
@@ -518,7 +528,7 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
     __syncthreads();
     for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
                            a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr,
-                           HistLevel2{h, sel_all[row].b1});
+                           HistLow11{h, sel_all[row].pre >> 11});
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
     for (int t = threadIdx.x; t < kBins2; t += kBlock)
@@ -526,33 +536,28 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
 }
 
 // ------------------------------------------------------------------------------------
-// Level 3: histogram of key & 511 over the candidates whose upper 22 key bits match.
-// grid = (nbt, rows); a thread walks the set bits of its bitmap words.
+// Level 3 (rows whose guess failed): histogram of key & 511 over the candidates whose upper
+// 22 key bits match.  grid = (blocks, rows), blocks loop over the 32768-coordinate spans; a
+// thread walks the set bits of its bitmap words.
 // ------------------------------------------------------------------------------------
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-             const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
-             const uint32_t *__restrict__ stash_cnt_all,
-             const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all, int64_t d,
-             int64_t wp, int64_t nt4k, int64_t stride)
+             const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all,
+             int64_t wp, int64_t nbt, int64_t stride)
 {
     __shared__ uint32_t h[kBins3];
+    const int row = blockIdx.y;
+    if (hit[row]) return;                             // rows with lists have their threshold already
     for (int t = threadIdx.x; t < kBins3; t += kBlock) h[t] = 0;
     __syncthreads();
-    const int row = blockIdx.y;
     const uint32_t *bm_cand = bm_cand_all + (int64_t)row * wp;
     const uint32_t pre = (sel_all[row].b1 << 11) | sel_all[row].b2;
-    if (hit[row]) {                                   // the tiles' lists hold the values
-        if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
-        for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
-                               a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr,
-                               HistLevel3{h, pre});
-    } else {                                          // classic path: gather a and b
-        const float *a = a_all + (int64_t)row * stride;
-        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
-        const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
+    for (int64_t bx = blockIdx.x; bx < nbt; bx += gridDim.x) {
+        const int64_t w0 = bx * kTileWords;
         for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
             uint32_t word = bm_cand[w0 + t];
             while (word) {
@@ -761,7 +766,7 @@ __device__ __forceinline__ uint32_t lowest_set_bits(uint32_t word, uint32_t coun
 // ------------------------------------------------------------------------------------
 // Ties (rows whose guess failed): keep those of global rank < k3 in index order (only if
 // not all are kept), then count the kept coordinates of every tile.  A thread owns 4
-// consecutive bitmap words.  grid = (nbt, rows).
+// consecutive bitmap words.  grid = (blocks, rows), blocks loop over the spans.
 // ------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kBlock)
 k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
@@ -774,7 +779,8 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp;
     const uint32_t *bm_tie = bm_cand_all + (int64_t)row * wp;
     const Sel s = sel_all[row];
-    const int64_t w0 = (int64_t)blockIdx.x * kTileWords + threadIdx.x * 4;
+    for (int64_t bx = blockIdx.x; bx < nbt; bx += gridDim.x) {       // block-uniform
+    const int64_t w0 = bx * kTileWords + threadIdx.x * 4;
     uint32_t keep[4], tie[4];
 #pragma unroll
     for (int m = 0; m < 4; ++m) {
@@ -784,7 +790,7 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
     if (s.k3 != s.c3) {                               // block-uniform
         const uint32_t mine = __popc(tie[0]) + __popc(tie[1]) + __popc(tie[2]) + __popc(tie[3]);
         uint32_t total;
-        uint32_t rank = block_excl_scan(mine, total) + tie_off_all[(int64_t)row * nbt + blockIdx.x];
+        uint32_t rank = block_excl_scan(mine, total) + tie_off_all[(int64_t)row * nbt + bx];
 #pragma unroll
         for (int m = 0; m < 4; ++m) {
             if (tie[m] && rank < s.k3) {
@@ -796,7 +802,8 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
     }
     uint32_t total;
     block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total);
-    if (threadIdx.x == 0) cnt_fin_all[(int64_t)row * nbt + blockIdx.x] = total;
+    if (threadIdx.x == 0) cnt_fin_all[(int64_t)row * nbt + bx] = total;
+    }
 }
 
 // ------------------------------------------------------------------------------------
@@ -1146,12 +1153,13 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok, w->stride);
     k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k, w->d, w->stride);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
-    k_topk_hist3<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->bm_cand, w->hist, w->d, w->wp, w->nt4k, w->stride);
+    const dim3 fallback_sparse(std::min(sparse.x, fallback.x), (unsigned)w->rows);
+    k_topk_hist3<HAS_B><<<fallback_sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_cand, w->hist, w->wp, w->nbt, w->stride);
     k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
     k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k, w->stride);
     k_scan_lists<<<w->rows, kBlock, 0, st>>>(w->sel, w->hit, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
-    k_topk_ties<<<sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
+    k_topk_ties<<<fallback_sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
     k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit);
     k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
