@@ -39,8 +39,8 @@ FALLBACK_HBM_GBS = 6650.0
 # keyed by workload, with the hash of the kernel sources at capture time.  A changed source
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
-    # k_worker_sign_ring: 2.656 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "a88fbf5f92bd194e", "bytes_per_launch": 4 * (1.797405e+09 + 8.57283072e+08)},
+    # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
+    "C4": {"hash": "7f8da041b7e2dc41", "bytes_per_launch": 4 * (1.797478e+09 + 8.56346624e+08)},
 }
 
 

@@ -11,14 +11,16 @@
 // atomics: the result does not depend on the order of execution.
 //
 // Normally ONE dense pass suffices: the level-1 bucket of the previous selection, lowered by
-// a margin, serves as a floor; the pass histograms only the coordinates at or above it and
+// a margin, serves as a floor; the pass histograms only the coordinates at or above it, in
+// bins of 2^11 keys counted from the floor (four level-1 buckets wide, the last bin open), and
 // keeps them per 4096-coordinate tile as a short list (position in the tile, value) in index
-// order.  Every later pass of such a row walks these lists, one warp per tile, with coalesced
-// reads; selection, ties and the ordered compaction follow from per-tile counts and two
-// scans, without bitmaps.  A tile with more coordinates above the floor than its list holds
+// order.  The histogram fixes key bits 30..11 of the threshold; one pass over the lists
+// (bits 10..0) fixes the rest: two levels instead of three.  Every later pass of such a row
+// walks these lists, one warp per tile, with coalesced reads; selection, ties and the ordered
+// compaction follow from per-tile counts and two scans, without bitmaps.  A tile with more coordinates above the floor than its list holds
 // (a selection concentrated in one tensor) is read again from the data by those passes.  If
-// fewer than k coordinates lie above the floor the classic two dense passes and the bitmap
-// passes run instead.  The same file holds the sparse
+// fewer than k coordinates lie above the floor, or the threshold lies above the fine bins,
+// the classic two dense passes and the bitmap passes run instead.  The same file holds the sparse
 // server aggregation and the rand-k path, which shares the payload kernels.
 #include "topk.h"
 
@@ -318,7 +320,15 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     if (vec_ok && base + kSub <= d) {
+        // Few coordinates lie at or above the floor (a percent or two), so the per-coordinate
+        // work is kept out of the dense loop: a thread only tests each of its four float4
+        // groups as a whole (one vote per group), flagged groups are moved to a small list in
+        // shared memory in index order, and the warp then works on that list densely - keys,
+        // histogram, ranks and the writes of the tile's (position, value) list.
+        __shared__ float4 s_u[kBlock / 32][kWarpSpan / 4];
+        __shared__ uint16_t s_p[kBlock / 32][kWarpSpan / 4];
         const int64_t wb = base + warp * kWarpSpan;
+        const float fkf = __uint_as_float(fk);
         float4 A[4], Bv[4];
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
@@ -326,24 +336,45 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             A[v] = ld_ro4(a + j);
             if (HAS_B) Bv[v] = ld_ro4(b + j);
         }
-        uint32_t BG[4][4];
-        uint32_t mine = 0;
+        uint32_t FB[4];
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
             if (HAS_B) {
                 A[v].x = __fsub_rn(A[v].x, Bv[v].x); A[v].y = __fsub_rn(A[v].y, Bv[v].y);
                 A[v].z = __fsub_rn(A[v].z, Bv[v].z); A[v].w = __fsub_rn(A[v].w, Bv[v].w);
             }
-            const uint32_t kx = key_of(A[v].x), ky = key_of(A[v].y), kz = key_of(A[v].z), kw = key_of(A[v].w);
-            BG[v][0] = __ballot_sync(kFull, kx >= fk);
-            BG[v][1] = __ballot_sync(kFull, ky >= fk);
-            BG[v][2] = __ballot_sync(kFull, kz >= fk);
-            BG[v][3] = __ballot_sync(kFull, kw >= fk);
-            if (kx >= fk) atomicAdd(&h[fine_bin(kx, fk)], 1u);
-            if (ky >= fk) atomicAdd(&h[fine_bin(ky, fk)], 1u);
-            if (kz >= fk) atomicAdd(&h[fine_bin(kz, fk)], 1u);
-            if (kw >= fk) atomicAdd(&h[fine_bin(kw, fk)], 1u);
-            mine += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
+            // |u| >= floor for a finite u; true for a NaN as well, like the comparison of the key bits
+            const bool f = !(fabsf(A[v].x) < fkf) || !(fabsf(A[v].y) < fkf) || !(fabsf(A[v].z) < fkf) ||
+                           !(fabsf(A[v].w) < fkf);
+            FB[v] = __ballot_sync(kFull, f);
+        }
+        uint32_t nsl = 0;                             // flagged groups of this warp, in index order
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            if ((FB[v] >> lane) & 1u) {
+                const uint32_t sl = nsl + __popc(FB[v] & lt);
+                s_u[warp][sl] = A[v];
+                s_p[warp][sl] = (uint16_t)(warp * kWarpSpan + v * 128 + lane * 4);
+            }
+            nsl += __popc(FB[v]);
+        }
+        __syncwarp();
+        // which of the four coordinates of list entry sl are at or above the floor (bit c = component c)
+        auto kept_of = [&](uint32_t sl, float4 &U) -> uint32_t {
+            if (sl >= nsl) return 0u;
+            U = s_u[warp][sl];
+            return (key_of(U.x) >= fk ? 1u : 0u) | (key_of(U.y) >= fk ? 2u : 0u) | (key_of(U.z) >= fk ? 4u : 0u) |
+                   (key_of(U.w) >= fk ? 8u : 0u);
+        };
+        uint32_t mine = 0;
+        for (uint32_t s0 = 0; s0 < nsl; s0 += 32) {   // warp-uniform
+            float4 U;
+            const uint32_t pm = kept_of(s0 + lane, U);
+            if (pm & 1u) atomicAdd(&h[fine_bin(key_of(U.x), fk)], 1u);
+            if (pm & 2u) atomicAdd(&h[fine_bin(key_of(U.y), fk)], 1u);
+            if (pm & 4u) atomicAdd(&h[fine_bin(key_of(U.z), fk)], 1u);
+            if (pm & 8u) atomicAdd(&h[fine_bin(key_of(U.w), fk)], 1u);
+            mine += __reduce_add_sync(kFull, (uint32_t)__popc(pm));
         }
         if (lane == 0) wcnt[warp] = mine;             // the same in every lane
         __syncthreads();
@@ -353,17 +384,26 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
             if (w8 < warp) rank += wcnt[w8];
             total += wcnt[w8];
         }
-        // index order: coordinate = warp * 512 + v * 128 + lane * 4 + component
+        // index order: coordinate = warp * 512 + v * 128 + lane * 4 + component = list order, then component
+        for (uint32_t s0 = 0; s0 < nsl; s0 += 32) {
+            float4 U;
+            const uint32_t pm = kept_of(s0 + lane, U);
+            const uint32_t cnt = __popc(pm);
+            uint32_t inc = cnt;
 #pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            uint32_t r = rank + __popc(BG[v][0] & lt) + __popc(BG[v][1] & lt) + __popc(BG[v][2] & lt) +
-                         __popc(BG[v][3] & lt);
-            const uint32_t p0 = (uint32_t)(warp * kWarpSpan + v * 128 + lane * 4);
-            if ((BG[v][0] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].x; spos[r] = (uint16_t)p0; } ++r; }
-            if ((BG[v][1] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].y; spos[r] = (uint16_t)(p0 + 1); } ++r; }
-            if ((BG[v][2] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].z; spos[r] = (uint16_t)(p0 + 2); } ++r; }
-            if ((BG[v][3] >> lane) & 1u) { if (r < kStashCap) { stash[r] = A[v].w; spos[r] = (uint16_t)(p0 + 3); } }
-            rank += __popc(BG[v][0]) + __popc(BG[v][1]) + __popc(BG[v][2]) + __popc(BG[v][3]);
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t t = __shfl_up_sync(kFull, inc, o);
+                if (lane >= o) inc += t;
+            }
+            uint32_t r = rank + inc - cnt;
+            if (pm) {
+                const uint32_t p0 = s_p[warp][s0 + lane];
+                if (pm & 1u) { if (r < kStashCap) { stash[r] = U.x; spos[r] = (uint16_t)p0; } ++r; }
+                if (pm & 2u) { if (r < kStashCap) { stash[r] = U.y; spos[r] = (uint16_t)(p0 + 1); } ++r; }
+                if (pm & 4u) { if (r < kStashCap) { stash[r] = U.z; spos[r] = (uint16_t)(p0 + 2); } ++r; }
+                if (pm & 8u) { if (r < kStashCap) { stash[r] = U.w; spos[r] = (uint16_t)(p0 + 3); } }
+            }
+            rank += __shfl_sync(kFull, inc, 31);
         }
         if (threadIdx.x == 0) stash_cnt_all[tile] = total;
     } else {
