@@ -199,8 +199,8 @@ def run_distributed(args, w, dev, rank, world):
     import torch.distributed as dist
     from paper_2111_00705_b200 import distributed as dd
     from paper_2111_00705_b200 import synth
-    if w.compressor != synth.SIGN:
-        raise SystemExit("--layout %s: the distributed deployment takes the scaled-sign workloads" % args.layout)
+    if w.compressor not in (synth.SIGN, synth.TOPK):
+        raise SystemExit("--layout %s: the distributed deployment takes the scaled-sign and top-k workloads" % args.layout)
     if not dist.is_initialized():                      # a single process: a group of one
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", str(29000 + os.getpid() % 2000))
@@ -208,7 +208,7 @@ def run_distributed(args, w, dev, rank, world):
     server_rank = 0 if args.layout == "server" else None
     args.warmup = max(args.warmup, 3)
     opt = dd.DistributedCDAdam(w.d, w.n, None, server_rank, beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps,
-                               offsets=w.offsets, x0=w.x0(dev), device=dev)
+                               offsets=w.offsets, x0=w.x0(dev), device=dev, compressor=w.compressor, k=w.k)
     first, per = dd.partition(w.n, world, rank, server_rank)
     grads = [w.grads(t + 1, dev).reshape(w.n, w.d)[first:first + per].contiguous().reshape(-1) if per else None
              for t in range(2)]
@@ -236,8 +236,8 @@ def run_distributed(args, w, dev, rank, world):
             "config": {"workload": describe(w), "layout": args.layout, "workers_per_rank": per,
                        "l2": "inputs larger than L2" if per * w.d * 4 >= 2 * 126e6 else "not flushed"},
             "params_per_s": value * w.d,
-            "message_bytes_per_worker": words * 4 + 4 * w.q,
-            "gpu_launches": 5 * args.steps, "clocks": clocks}))
+            "message_bytes_per_worker": words * 4 + 4 * w.q if w.compressor == synth.SIGN else 8 * w.k,
+            "gpu_launches": opt.shard.launches_per_step() * args.steps, "clocks": clocks}))
     opt.close()
     dist.destroy_process_group()
 

@@ -140,7 +140,7 @@ int cdadam_step_host(cdadam_ctx *ctx, const float *grads_host, float *x_out_host
  * library makes no network call.  The result is that of one context holding all n workers,
  * bit for bit, because every stage computes the same binary32 operations in the same order.
  *
- * cdadam_create_shard: as cdadam_create with the scaled-sign compressor, for the workers
+ * cdadam_create_shard: as cdadam_create, with CDADAM_SIGN or CDADAM_TOPK, for the workers
  *   [first_worker, first_worker + n_local) of n.  n_local may be 0 (a process that is only
  *   the server).  The worker state ghat^(i) is allocated for the n_local workers only;
  *   CDADAM_STATE_GHAT_W is n_local x d.  The message buffers hold all n worker messages.
@@ -173,8 +173,17 @@ int cdadam_step_host(cdadam_ctx *ctx, const float *grads_host, float *x_out_host
  *   server_bits    words uint32;  server_scales  q floats
  *   words = ceil(d / 32).  Any output pointer may be NULL.  A context that holds all n
  *   workers may use the staged calls too.
+ *   With CDADAM_TOPK (Algorithm 1 on the whole vector; not the comparison modes, not per
+ *   segment) the same four pointers are the messages' coordinates and values: worker_bits =
+ *   n x k uint32 coordinates (increasing in every row), worker_scales = n x k float values,
+ *   server_bits / server_scales = the server's k coordinates and values; words = q = k.
+ *   A process that skips cdadam_step_server adds the server message it was given to its gtil
+ *   in cdadam_step_update.  Messages that arrive from other processes carry no per-tile
+ *   offsets, so the server aggregation of such a context searches the sorted coordinates
+ *   (slower than the one-context path, same sums in the same order).
  */
 cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local,
+                                int compressor, int64_t k,
                                 float beta1, float beta2, float lr, float eps);
 int cdadam_step_workers(cdadam_ctx *ctx, const float *grads, void *stream);
 int cdadam_step_server(cdadam_ctx *ctx, void *stream);

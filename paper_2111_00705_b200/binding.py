@@ -26,7 +26,7 @@ _SIGNATURES = {
     "cdadam_step": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_bf16": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_host": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p, _c.c_void_p]),
-    "cdadam_create_shard": (_c.c_void_p, [_c.c_int64, _c.c_int, _c.c_int, _c.c_int,
+    "cdadam_create_shard": (_c.c_void_p, [_c.c_int64, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int64,
                                           _c.c_float, _c.c_float, _c.c_float, _c.c_float]),
     "cdadam_step_workers": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_step_server": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
@@ -285,18 +285,19 @@ class CDAdam:
 
 
 class CDAdamShard(CDAdam):
-    """A context for the workers [first_worker, first_worker + n_local) of n (scaled sign):
-    one process of a distributed deployment.  An iteration runs in its stages with the
-    messages moved by the caller in between (see ``distributed.py``)."""
+    """A context for the workers [first_worker, first_worker + n_local) of n (scaled sign or
+    top-k): one process of a distributed deployment.  An iteration runs in its stages with
+    the messages moved by the caller in between (see ``distributed.py``)."""
 
     def __init__(self, d, n, first_worker, n_local, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
-                 offsets=None, x0=None, device=None, mode=MARKOV):
+                 offsets=None, x0=None, device=None, mode=MARKOV, compressor=SIGN, k=0):
         self._shard = (int(first_worker), int(n_local))
-        super().__init__(d, n, SIGN, 0, beta1, beta2, lr, eps, offsets, x0, device, mode)
+        super().__init__(d, n, compressor, k, beta1, beta2, lr, eps, offsets, x0, device, mode)
         self.first_worker, self.n_local = self._shard
 
     def _create(self, beta1, beta2, lr, eps):
-        return lib().cdadam_create_shard(self.d, self.n, self._shard[0], self._shard[1], beta1, beta2, lr, eps)
+        return lib().cdadam_create_shard(self.d, self.n, self._shard[0], self._shard[1], self.compressor, self.k,
+                                         beta1, beta2, lr, eps)
 
     def step_workers(self, grads, stream=None):
         """Worker stage on the n_local x d device gradients of this context's workers."""
@@ -314,7 +315,9 @@ class CDAdamShard(CDAdam):
     def exchange_buffers(self):
         """Torch views (no copy) of the message buffers: worker_bits int32[n, words],
         worker_scales float32[n, q], server_bits int32[words], server_scales float32[q].
-        worker_scales alternates between two arrays: ask again after every step_workers."""
+        worker_scales alternates between two arrays: ask again after every step_workers.
+        With top-k the same keys hold the coordinates (int32[n, k], int32[k]) and the values
+        (float32[n, k], float32[k]) of the messages."""
         wb, ws, sb, ss = (ctypes.c_void_p() for _ in range(4))
         words, q = ctypes.c_int64(), ctypes.c_int()
         _check(lib().cdadam_exchange_buffers(self._h, ctypes.byref(wb), ctypes.byref(ws), ctypes.byref(sb),

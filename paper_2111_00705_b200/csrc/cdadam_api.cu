@@ -160,6 +160,10 @@ struct cdadam_ctx {
     bool sets_given = false;   // rand-k: coordinate sets have been supplied
     // top-k
     TopkWorkspace *tk_w = nullptr, *tk_s = nullptr;
+    // a top-k context that holds a part of the workers: the messages of all n workers
+    // (n x k coordinates and values); tk_w then selects into the rows of its own workers
+    uint32_t *pay_idx = nullptr;
+    float *pay_val = nullptr;
     // top-k per segment: a selection workspace per segment (rows strided by d); tk_w / tk_s
     // then hold only the concatenated payloads
     std::vector<int64_t> seg_off, seg_k, seg_at;
@@ -462,7 +466,7 @@ static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compre
     if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
     if (n < 1 || n > 65535) { fail(CDADAM_ERR_ARG, "n must be in [1, 65535]"); return nullptr; }
     if (first < 0 || nloc < 0 || first + nloc > n) { fail(CDADAM_ERR_ARG, "the context's workers [first, first + n_local) must lie in [0, n)"); return nullptr; }
-    if (nloc != n && compressor != CDADAM_SIGN) { fail(CDADAM_ERR_ARG, "a context that holds a part of the workers needs the scaled-sign compressor"); return nullptr; }
+    if (nloc != n && compressor != CDADAM_SIGN && compressor != CDADAM_TOPK) { fail(CDADAM_ERR_ARG, "a context that holds a part of the workers needs the scaled-sign or the top-k compressor"); return nullptr; }
     if (compressor < CDADAM_SIGN || compressor > CDADAM_RANDK) { fail(CDADAM_ERR_ARG, "unknown compressor %d", compressor); return nullptr; }
     if ((compressor == CDADAM_TOPK || compressor == CDADAM_RANDK) && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k and rand-k need 1 <= k <= d"); return nullptr; }
     cdadam_ctx *c = new (std::nothrow) cdadam_ctx;
@@ -493,6 +497,12 @@ static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compre
         } else if (compressor == CDADAM_RANDK) {
             if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n, nullptr, nullptr, false))) { fail(rc, "rand-k payload allocation failed"); break; }
             if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1, nullptr, nullptr, false))) { fail(rc, "rand-k payload allocation failed"); break; }
+        } else if (compressor == CDADAM_TOPK && nloc != n) {
+            if ((rc = dev_zalloc(&c->pay_idx, (size_t)n * c->k))) break;
+            if ((rc = dev_zalloc(&c->pay_val, (size_t)n * c->k))) break;
+            if ((rc = topk_workspace_create(&c->tk_w, d, c->k, nloc > 0 ? nloc : 1, c->pay_idx + (int64_t)first * c->k,
+                                            c->pay_val + (int64_t)first * c->k))) { fail(rc, "top-k workspace allocation failed"); break; }
+            if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1))) { fail(rc, "top-k workspace allocation failed"); break; }
         } else if (compressor == CDADAM_TOPK) {
             if ((rc = topk_workspace_create(&c->tk_w, d, c->k, n))) { fail(rc, "top-k workspace allocation failed"); break; }
             if ((rc = topk_workspace_create(&c->tk_s, d, c->k, 1))) { fail(rc, "top-k workspace allocation failed"); break; }
@@ -508,10 +518,14 @@ cdadam_ctx *cdadam_create(int64_t d, int n, int compressor, int64_t k, float bet
     return create_impl(d, n, 0, n, compressor, k, beta1, beta2, lr, eps);
 }
 
-cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local, float beta1, float beta2,
-                                float lr, float eps)
+cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local, int compressor, int64_t k,
+                                float beta1, float beta2, float lr, float eps)
 {
-    return create_impl(d, n, first_worker, n_local, CDADAM_SIGN, 0, beta1, beta2, lr, eps);
+    if (compressor != CDADAM_SIGN && compressor != CDADAM_TOPK) {
+        fail(CDADAM_ERR_ARG, "the staged iteration takes the scaled-sign or the top-k compressor");
+        return nullptr;
+    }
+    return create_impl(d, n, first_worker, n_local, compressor, k, beta1, beta2, lr, eps);
 }
 
 void cdadam_destroy(cdadam_ctx *c)
@@ -522,6 +536,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->ghat_w); cudaFree(c->ghat_s); cudaFree(c->gtil);
     cudaFree(c->m); cudaFree(c->v); cudaFree(c->vhat); cudaFree(c->x);
     cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
+    cudaFree(c->pay_idx); cudaFree(c->pay_val);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     cudaFree(c->wdone); cudaFree(c->sdone); cudaFree(c->wsums); cudaFree(c->ssums);
@@ -693,7 +708,10 @@ int cdadam_step(cdadam_ctx *c, const float *grads, void *stream) { return step_i
 static int staged_ok(cdadam_ctx *c, const char *what)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "%s: NULL context", what);
-    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "%s: the staged calls take the scaled-sign compressor", what);
+    if (c->comp != CDADAM_SIGN && c->comp != CDADAM_TOPK)
+        return fail(CDADAM_ERR_STATE, "%s: the staged calls take the scaled-sign or the top-k compressor", what);
+    if (c->comp == CDADAM_TOPK && (c->mode != CDADAM_MARKOV || !c->seg_w.empty()))
+        return fail(CDADAM_ERR_STATE, "%s: with top-k the staged calls run Algorithm 1 on the whole vector only", what);
     if (c->prof_on) return fail(CDADAM_ERR_STATE, "%s: per-stage timing covers cdadam_step only", what);
     return CDADAM_OK;
 }
@@ -707,7 +725,14 @@ int cdadam_step_workers(cdadam_ctx *c, const float *grads, void *stream)
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
     step_size_of_this_step(c);
-    enqueue_sign_workers(c, grads, false, aligned16(grads) && c->d % 4 == 0, c->wscale[c->cur ^ 1], st);
+    const bool vec = aligned16(grads) && c->d % 4 == 0;
+    if (c->comp == CDADAM_TOPK) {
+        if (c->nloc > 0) topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);   // workers: compress, update ghat^(i)
+        if (int rc = check_launch("cdadam_step_workers")) return rc;
+        c->phase = 1;
+        return CDADAM_OK;
+    }
+    enqueue_sign_workers(c, grads, false, vec, c->wscale[c->cur ^ 1], st);
     if (int rc = check_launch("cdadam_step_workers")) return rc;
     c->cur ^= 1;                              // wscale[cur] now holds this iteration's scales
     c->pending = c->mode != CDADAM_NAIVE;
@@ -722,7 +747,15 @@ int cdadam_step_server(cdadam_ctx *c, void *stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
-    enqueue_sign_server(c, c->wscale[c->cur], st);
+    if (c->comp == CDADAM_TOPK) {
+        // messages gathered from other processes come without the selecting side's per-tile
+        // offsets: their entries are found by searching the sorted coordinates
+        if (c->pay_idx) topk_aggregate_rows(c->pay_idx, c->pay_val, c->k, c->d, c->n, c->ghat_s, st);
+        else topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                       // server: ghat += mean
+        topk_select(c->tk_s, c->ghat_s, c->gtil, true, c->d % 4 == 0, st);       // server: compress, update gtil
+    } else {
+        enqueue_sign_server(c, c->wscale[c->cur], st);
+    }
     if (int rc = check_launch("cdadam_step_server")) return rc;
     c->phase = 2;
     return CDADAM_OK;
@@ -735,7 +768,18 @@ int cdadam_step_update(cdadam_ctx *c, void *stream)
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
-    enqueue_sign_update(c, st);
+    if (c->comp == CDADAM_TOPK) {
+        // a process that did not run the server stage holds the server's message (k coordinates
+        // and values) in the buffers: gtil += c there, as the server did on its own copy
+        if (c->phase == 1) {
+            const uint32_t *sidx; const float *sval;
+            topk_payload(c->tk_s, 0, &sidx, &sval);
+            launch_scatter_add(c->gtil, sidx, sval, c->k, c->d, st);
+        }
+        launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, c->d % 4 == 0, st);
+    } else {
+        enqueue_sign_update(c, st);
+    }
     if (int rc = check_launch("cdadam_step_update")) return rc;
     c->phase = 0;
     c->steps += 1;
@@ -746,6 +790,19 @@ int cdadam_exchange_buffers(cdadam_ctx *c, uint32_t **worker_bits, float **worke
                             float **server_scales, int64_t *words, int *q)
 {
     if (int rc = staged_ok(c, "cdadam_exchange_buffers")) return rc;
+    if (c->comp == CDADAM_TOPK) {
+        const uint32_t *widx, *sidx;
+        const float *wval, *sval;
+        topk_payload(c->tk_w, 0, &widx, &wval);
+        topk_payload(c->tk_s, 0, &sidx, &sval);
+        if (worker_bits) *worker_bits = c->pay_idx ? c->pay_idx : const_cast<uint32_t *>(widx);
+        if (worker_scales) *worker_scales = c->pay_val ? c->pay_val : const_cast<float *>(wval);
+        if (server_bits) *server_bits = const_cast<uint32_t *>(sidx);
+        if (server_scales) *server_scales = const_cast<float *>(sval);
+        if (words) *words = c->k;
+        if (q) *q = (int)std::min<int64_t>(c->k, 0x7fffffff);
+        return CDADAM_OK;
+    }
     if (worker_bits) *worker_bits = c->wbits;
     if (worker_scales) *worker_scales = c->wscale[c->cur];
     if (server_bits) *server_bits = c->sbits;
@@ -953,8 +1010,12 @@ int cdadam_last_payload(cdadam_ctx *c, int who, const void **a, const float **b,
         return CDADAM_OK;
     }
     if (c->comp == CDADAM_TOPK || c->comp == CDADAM_RANDK) {
-        TopkWorkspace *w = who == CDADAM_SERVER ? c->tk_s : c->tk_w;
-        topk_payload(w, who == CDADAM_SERVER ? 0 : who, (const uint32_t **)a, b);
+        if (who != CDADAM_SERVER && c->pay_idx) {
+            *a = c->pay_idx + (int64_t)who * c->k; *b = c->pay_val + (int64_t)who * c->k;
+        } else {
+            TopkWorkspace *w = who == CDADAM_SERVER ? c->tk_s : c->tk_w;
+            topk_payload(w, who == CDADAM_SERVER ? 0 : who, (const uint32_t **)a, b);
+        }
         *count = c->k;
         return CDADAM_OK;
     }

@@ -152,6 +152,23 @@ void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64
     k_scatter_set<<<grid, kBlock, 0, st>>>(dst, idx, val, k, d);
 }
 
+// dst[idx[t]] += val[t] for one message of k distinct coordinates (a worker applying the
+// server's top-k message to its copy of gtil); coordinates >= d are skipped.
+__global__ void __launch_bounds__(kBlock)
+k_scatter_add(float *__restrict__ dst, const uint32_t *__restrict__ idx, const float *__restrict__ val,
+              int64_t k, int64_t d)
+{
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t >= k) return;
+    const int64_t j = idx[t];
+    if (j < d) dst[j] = __fadd_rn(dst[j], val[t]);
+}
+
+void launch_scatter_add(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d, cudaStream_t st)
+{
+    k_scatter_add<<<(unsigned)((k + kBlock - 1) / kBlock), kBlock, 0, st>>>(dst, idx, val, k, d);
+}
+
 void launch_amsgrad(const float *gtil, float *m, float *v, float *vhat, float *x, int64_t d,
                     Hyper hp, bool vec_ok, cudaStream_t st)
 {

@@ -58,6 +58,7 @@ void launch_add_into(float *dst, const float *src, int64_t count, bool vec_ok, c
 void launch_scatter_set(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d,
                         int rows, cudaStream_t st);
 // dst[idx[t]] = 0 for t < rows * k: one vector, the coordinate sets of all rows.
+void launch_scatter_add(float *dst, const uint32_t *idx, const float *val, int64_t k, int64_t d, cudaStream_t st);
 void launch_scatter_zero_shared(float *dst, const uint32_t *idx, int64_t k, int rows, cudaStream_t st);
 
 // ---- AMSGrad alone on a dense gradient estimate (top-k path) ------------------------------

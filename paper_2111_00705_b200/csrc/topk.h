@@ -36,6 +36,12 @@ void topk_payload_concat(TopkWorkspace *whole, int64_t at, TopkWorkspace *seg, i
 //   order 0, 1, ..., n-1.
 void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st);
 
+// The same from n messages laid out as n x k arrays (coordinates increasing in every row)
+// that come without the selecting side's per-tile offsets: every block finds its entries by
+// binary search.
+void topk_aggregate_rows(const uint32_t *idx, const float *val, int64_t k, int64_t d, int n, float *ghat_s,
+                         cudaStream_t st);
+
 // Rand-k (Appendix A): the k coordinates of every row are given by the caller.
 // randk_set copies rows x k device indices into the payload and checks them (strictly
 // increasing, below d; *error_flag = 2 otherwise).  randk_gather fills the payload values

@@ -1244,6 +1244,13 @@ void topk_aggregate(TopkWorkspace *ww, float *ghat_s, int n, cudaStream_t st)
                                                 ww->hit, ww->cnt_gt, ww->nt4k);
 }
 
+void topk_aggregate_rows(const uint32_t *idx, const float *val, int64_t k, int64_t d, int n, float *ghat_s,
+                         cudaStream_t st)
+{
+    const unsigned blocks = (unsigned)((d + kAggSpan - 1) / kAggSpan);
+    k_topk_aggregate<<<blocks, kBlock, 0, st>>>(idx, val, nullptr, 0, n, k, d, ghat_s, (n & (n - 1)) == 0, nullptr, nullptr, 0);
+}
+
 // ---- rand-k: the coordinate sets come from the caller -------------------------------------
 // Every row's set must be strictly increasing and below d; a violation sets *error_flag.
 __global__ void __launch_bounds__(kBlock)

@@ -23,7 +23,7 @@ def make_shards(w, world, server_rank, x0, mode=cd.MARKOV):
     for r in range(world):
         first, per = dd.partition(w.n, world, r, server_rank)
         out.append(cd.CDAdamShard(w.d, w.n, first, per, beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps,
-                                  offsets=w.offsets, x0=x0.cuda(), mode=mode))
+                                  offsets=w.offsets, x0=x0.cuda(), mode=mode, compressor=w.compressor, k=w.k))
     return out
 
 
@@ -55,8 +55,8 @@ def run_case(w, world, server_rank, steps, mode=cd.MARKOV):
     x0 = w.x0("cpu")
     shards = make_shards(w, world, server_rank, x0, mode)
     args = dict(beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps)
-    full = cd.CDAdam(w.d, w.n, cd.SIGN, offsets=w.offsets, x0=x0.cuda(), mode=mode, **args)
-    o = orc.Oracle(w.d, w.n, orc.SIGN, offsets=w.offsets, x0=x0.numpy(), mode=mode, **args)
+    full = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.cuda(), mode=mode, **args)
+    o = orc.Oracle(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.numpy(), mode=mode, **args)
     for t in range(1, steps + 1):
         grads = w.grads(t, "cpu")
         gd = grads.cuda().reshape(w.n, w.d)
@@ -123,6 +123,35 @@ def test_sharded_error_feedback_mode():
     run_case(w, 2, None, 3, mode=cd.EF)
 
 
+@pytest.mark.parametrize("world,server_rank", [(2, None), (4, None), (3, 0), (5, 2)])
+def test_sharded_top_k_equals_the_single_context_and_the_oracle(world, server_rank):
+    w = synth.workload("C3", scale=0.004, steps=4)      # d = 102,400, n = 16, k = 1,024
+    run_case(w, world, server_rank, 4)
+
+
+def test_sharded_top_k_ties_and_ragged_dimension():
+    w = synth.workload("C3", scale=0.001, steps=3)
+    w.d -= 7
+    w.n, w.k = 4, 300
+    w.grads = lambda t, device="cpu", d=w.d, n=w.n: torch.randint(-3, 4, (n, d), generator=torch.Generator().manual_seed(t)).float().to(device)
+    run_case(w, 2, None, 3)
+    run_case(w, 3, 1, 3)
+
+
+def test_staged_top_k_on_a_context_with_all_workers():
+    w = synth.workload("C3", scale=0.002, steps=3)
+    x0 = w.x0("cpu")
+    s = cd.CDAdamShard(w.d, w.n, 0, w.n, x0=x0.cuda(), compressor=cd.TOPK, k=w.k)
+    o = orc.Oracle(w.d, w.n, orc.TOPK, k=w.k, x0=x0.numpy())
+    for t in range(1, 4):
+        grads = w.grads(t, "cpu")
+        s.step_workers(grads.cuda().reshape(-1)); s.step_server(); s.step_update()
+        o.step(grads.numpy())
+        for name in ("x", "gtil", "ghat_s", "ghat_w"):
+            assert np.array_equal(s.get_state(name).cpu().numpy().ravel(), o.state(name).ravel()), (t, name)
+    s.close(); o.close()
+
+
 def test_staged_calls_on_a_context_with_all_workers_and_call_order():
     w = synth.workload("C1", scale=0.25, steps=3)
     x0 = w.x0("cpu")
@@ -155,8 +184,10 @@ def test_staged_calls_on_a_context_with_all_workers_and_call_order():
         part.step(w.grads(1, "cuda").reshape(-1))        # a part of the workers: staged calls only
     part.close()
     lib = cd.lib()
-    assert not lib.cdadam_create_shard(100, 4, 3, 2, 0.9, 0.999, 1e-3, 1e-8)     # workers 3, 4 of 4
-    assert not lib.cdadam_create_shard(100, 4, -1, 2, 0.9, 0.999, 1e-3, 1e-8)
+    assert not lib.cdadam_create_shard(100, 4, 3, 2, cd.SIGN, 0, 0.9, 0.999, 1e-3, 1e-8)     # workers 3, 4 of 4
+    assert not lib.cdadam_create_shard(100, 4, -1, 2, cd.SIGN, 0, 0.9, 0.999, 1e-3, 1e-8)
+    assert not lib.cdadam_create_shard(100, 4, 0, 2, cd.IDENTITY, 0, 0.9, 0.999, 1e-3, 1e-8)
+    assert not lib.cdadam_create_shard(100, 4, 0, 2, cd.TOPK, 0, 0.9, 0.999, 1e-3, 1e-8)     # k out of range
 
 
 def test_distributed_class_over_a_one_rank_nccl_group(tmp_path):
