@@ -258,6 +258,10 @@ int cdadam_set_mode(cdadam_ctx *ctx, int mode);
  * the worker pass and for the server side, the default).
  * Results do not depend on it.  Tiles of 16384 coordinates or more select the worker kernel
  * with the asynchronous-copy prefetch ring.  Only before the first step; synchronous.
+ * With CDADAM_TOPK the selection always works on 4096-coordinate tiles and the value only
+ * picks the kernel of its dense pass: 16384 or more = the prefetch-ring kernel wherever rows
+ * are 16-byte aligned, a smaller non-zero value = the plain kernel, 0 = chosen from the size
+ * (call it after cdadam_set_topk_segments, if that is used).
  */
 int cdadam_set_tile(cdadam_ctx *ctx, int tile);
 

@@ -509,6 +509,8 @@ static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compre
         }
     } while (0);
     if (rc != CDADAM_OK || cudaDeviceSynchronize() != cudaSuccess) { cdadam_destroy(c); return nullptr; }
+    topk_workspace_set_error_flag(c->tk_w, c->error_flag);
+    topk_workspace_set_error_flag(c->tk_s, c->error_flag);
     return c;
 }
 
@@ -875,6 +877,8 @@ int cdadam_set_topk_segments(cdadam_ctx *c, int q, const int64_t *offsets, const
             topk_workspace_destroy(ww);
             return fail(rc, "top-k workspace allocation failed (segment %d)", r);
         }
+        topk_workspace_set_error_flag(ww, c->error_flag);
+        topk_workspace_set_error_flag(ws, c->error_flag);
         c->seg_w.push_back(ww); c->seg_s.push_back(ws);
         c->seg_off.push_back(offsets[r]); c->seg_k.push_back(k_per_segment[r]); c->seg_at.push_back(at);
         at += k_per_segment[r];
@@ -904,10 +908,21 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
 int cdadam_set_tile(cdadam_ctx *c, int tile)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_tile: NULL context");
-    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "tiles apply to the scaled-sign compressor only");
+    if (c->comp != CDADAM_SIGN && c->comp != CDADAM_TOPK)
+        return fail(CDADAM_ERR_STATE, "tiles apply to the scaled-sign and top-k compressors only");
     if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "the tile size must be set before the first step");
     if (tile != 0 && (tile < kSub || tile % kSub != 0 || tile > 64 * kSub))
         return fail(CDADAM_ERR_ARG, "tile must be 0 or a multiple of %d up to %d", kSub, 64 * kSub);
+    if (c->comp == CDADAM_TOPK) {
+        // the selection works on 4096-coordinate tiles throughout; the knob only picks the
+        // kernel of the dense pass
+        const int ring = tile == 0 ? 0 : tile >= 4 * kSub ? 1 : -1;
+        topk_workspace_set_ring(c->tk_w, ring);
+        topk_workspace_set_ring(c->tk_s, ring);
+        for (TopkWorkspace *w : c->seg_w) topk_workspace_set_ring(w, ring);
+        for (TopkWorkspace *w : c->seg_s) topk_workspace_set_ring(w, ring);
+        return CDADAM_OK;
+    }
     c->tile_override = tile;
     std::vector<int64_t> off = c->ts.off;         // rebuild the tables for the current segments
     return cdadam_set_segments(c, (int)off.size() - 1, off.data());

@@ -17,6 +17,12 @@ int topk_workspace_create(TopkWorkspace **w, int64_t d, int64_t k, int rows,
                           uint32_t *idx = nullptr, float *val = nullptr, bool with_select = true,
                           int64_t stride = 0);
 void topk_workspace_destroy(TopkWorkspace *w);
+// Device word that a selection kernel sets to 1 when a bounded wait on an asynchronous copy
+// runs out (NULL: not reported).
+void topk_workspace_set_error_flag(TopkWorkspace *w, int *error_flag);
+// Which kernel makes the dense pass: 0 = chosen from the size (the default), 1 = the
+// prefetch-ring kernel wherever rows are 16-byte aligned, -1 = the plain kernel.
+void topk_workspace_set_ring(TopkWorkspace *w, int ring);
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
 int topk_launches_per_step(int n);
 

@@ -412,6 +412,37 @@ def test_topk_selection_concentrated_in_a_few_tiles(mode):
     g.close(); o.close()
 
 
+@pytest.mark.parametrize("mode", [cd.MARKOV, cd.EF, cd.NAIVE])
+def test_topk_dense_pass_with_the_prefetch_ring_at_small_sizes(mode):
+    """Large problems make their dense pass with the prefetch-ring kernel; set_tile(16384)
+    selects it at sizes the oracle finishes quickly.  Whole tiles go through the ring, the
+    ragged last tile through the plain kernel; both with and without the state operand."""
+    w = synth.workload("C3", scale=0.01)                    # d = 256,000 = 62.5 tiles, n = 16
+    run_free(w, 5, tile=16384, mode=mode)
+    w = synth.Workload("RING1", 9 * 4096, 2, synth.TOPK, 4, k=999, seed=5)       # whole tiles only, odd count
+    run_free(w, 4, tile=16384, mode=mode)
+
+
+def test_topk_prefetch_ring_with_failed_guesses_and_dense_tiles():
+    rng = np.random.default_rng(11)
+    d, n, k = 40 * 4096 + 2048, 3, 6000                     # rows stay 16-byte aligned, last tile ragged
+    big = slice(7 * 4096 + 100, 10 * 4096 + 50)
+    w = synth.Workload("RINGCONC", d, n, synth.TOPK, 8, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d))
+    g.set_tile(16384)
+    for t, scale in enumerate((1.0, 1.0, 0.05, 0.05, 3.0, 3.0, 1.0, 1.0)):
+        grads = (rng.standard_normal((n, d)) * scale).astype(np.float32)
+        if t >= 4:
+            grads[:, big] *= 100.0                          # one tensor takes the whole selection: tiles without lists
+        if t == 6:
+            grads[:, 20 * 4096:20 * 4096 + 700] = 1e4
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.device_status()
+    g.close(); o.close()
+
+
 @pytest.mark.parametrize("case", ["ragged", "aligned_large", "one_segment"])
 def test_topk_per_segment_matches_oracle(case):
     """Top-k applied to every segment on its own (per tensor): concatenated payloads bit-exact,
@@ -431,6 +462,8 @@ def test_topk_per_segment_matches_oracle(case):
     g, o = make_pair(w)
     g.set_topk_segments(off, ks)
     o.set_topk_segments(off, ks)
+    if case == "aligned_large":
+        g.set_tile(16384)                                       # dense passes through the prefetch ring, rows strided by d
     w.k = sum(ks)
     rng = np.random.default_rng(7)
     scale = np.repeat(10.0 ** rng.uniform(-2, 1, len(ks)), np.diff(off)).astype(np.float32)
@@ -641,9 +674,10 @@ def test_stage_timing_and_late_configuration_calls():
     with pytest.raises(cd.CdadamError):
         g.set_tile(8192)                                  # after the first step
     assert cd.lib().cdadam_set_mode(g._h, cd.EF) == cd.ERR_STATE
-    h = cd.CDAdam(100, 2, cd.TOPK, k=3)
+    h = cd.CDAdam(100, 2, cd.IDENTITY)
     with pytest.raises(cd.CdadamError):
-        h.set_tile(4096)                                  # tiles belong to scaled sign
+        h.set_tile(4096)                                  # the identity compressor has no tiles
+    cd.CDAdam(100, 2, cd.TOPK, k=3).set_tile(4096)        # top-k: picks the kernel of the dense pass
     f = cd.CDAdam(100, 2, cd.SIGN)
     with pytest.raises(cd.CdadamError):
         f.set_tile(1000)                                  # not a multiple of 4096
