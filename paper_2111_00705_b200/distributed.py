@@ -4,7 +4,8 @@ workers, the messages moved with ``torch.distributed`` (NCCL between GPUs).
 This module is plumbing: which process holds which workers, and which message rows go where.
 All arithmetic of the method runs in the library's kernels through ``binding.CDAdamShard``;
 the messages are the d sign bits and q scales per worker that Algorithm 1 sends (Section 5),
-taken from and delivered into the library's own buffers without a copy.
+or the k coordinates and values of top-k, taken from and delivered into the library's own
+buffers without a copy.
 
 Two layouts:
 
@@ -83,7 +84,8 @@ def broadcast_server_message(bits, scales, group=None, server_rank=0):
 
 
 class DistributedCDAdam:
-    """Algorithm 1 across the processes of a ``torch.distributed`` group, scaled sign.
+    """Algorithm 1 across the processes of a ``torch.distributed`` group, scaled sign (the
+    default) or top-k (``compressor=binding.TOPK, k=...``).
 
     Every process calls ``step(grads_local)`` with the gradients of its own workers
     (n_local x d, CUDA float32; ``None`` on a server that holds none); afterwards
