@@ -314,6 +314,20 @@ int cdadam_last_payload(cdadam_ctx *ctx, int who, const void **a, const float **
 int64_t cdadam_step_count(cdadam_ctx *ctx);
 
 /*
+ * Resuming from a checkpoint.  The iterate of Algorithm 1 is the seven state vectors plus the
+ * iteration counter t (it selects the step size when milestones are set).  To save: read every
+ * vector with cdadam_get_state (for scaled sign this first applies the last worker messages to
+ * ghat^(i), so the saved vectors are final) and t with cdadam_step_count.  To resume: create a
+ * context with the same arguments, segments, mode, step-size schedule and weight decay, load
+ * the vectors with cdadam_set_state and t with cdadam_set_step_count; the iterations that
+ * follow are those of the uninterrupted run, bit for bit (top-k starts its first selection
+ * without a threshold guess, which costs time, not accuracy).  t >= 0; not between the stages
+ * of an iteration (CDADAM_ERR_STATE).  Configuration calls that are allowed only before the
+ * first step stay allowed while t is 0.
+ */
+int cdadam_set_step_count(cdadam_ctx *ctx, int64_t t);
+
+/*
  * Waits for `stream` and reports whether any kernel of this context has given up a bounded
  * wait (the large-tile worker kernel waits, with an iteration limit, for its bulk
  * asynchronous copies; it never spins without bound).  CDADAM_ERR_TIMEOUT means the state

@@ -49,6 +49,7 @@ _SIGNATURES = {
     "cdadam_last_payload": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_void_p),
                                        _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_int64)]),
     "cdadam_step_count": (_c.c_int64, [_c.c_void_p]),
+    "cdadam_set_step_count": (_c.c_int, [_c.c_void_p, _c.c_int64]),
     "cdadam_device_status": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "cdadam_launches_per_step": (_c.c_int, [_c.c_void_p]),
     "cdadam_compress_sign": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int,
@@ -279,6 +280,22 @@ class CDAdam:
 
     def step_count(self):
         return lib().cdadam_step_count(self._h)
+
+    def set_step_count(self, t):
+        """The iteration counter of a run resumed from saved state (see state_dict)."""
+        _check(lib().cdadam_set_step_count(self._h, int(t)))
+
+    def state_dict(self, stream=None):
+        """Everything a resumed run needs: copies of the seven state vectors and the counter."""
+        out = {name: self.get_state(name, stream) for name in STATE_NAMES}
+        out["step_count"] = self.step_count()
+        return out
+
+    def load_state_dict(self, state, stream=None):
+        """Load what state_dict returned into a context created with the same configuration."""
+        for name in STATE_NAMES:
+            self.set_state(name, state[name].reshape(-1), stream)
+        self.set_step_count(state["step_count"])
 
     def launches_per_step(self):
         return lib().cdadam_launches_per_step(self._h)

@@ -1039,6 +1039,15 @@ int cdadam_last_payload(cdadam_ctx *c, int who, const void **a, const float **b,
 
 int64_t cdadam_step_count(cdadam_ctx *c) { return c ? c->steps : 0; }
 
+int cdadam_set_step_count(cdadam_ctx *c, int64_t t)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_step_count: NULL context");
+    if (t < 0) return fail(CDADAM_ERR_ARG, "the iteration counter cannot be negative");
+    if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_set_step_count: a staged iteration is under way");
+    c->steps = t;
+    return CDADAM_OK;
+}
+
 int cdadam_device_status(cdadam_ctx *c, void *stream)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "cdadam_device_status: NULL context");

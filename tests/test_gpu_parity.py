@@ -712,3 +712,45 @@ def test_argument_errors_are_reported_not_fatal():
     with pytest.raises(cd.CdadamError):
         g.last_payload(5)
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("name,scale,mode", [("C2", 0.01, cd.MARKOV), ("C2", 0.005, cd.EF), ("C3", 0.004, cd.MARKOV),
+                                             ("C1", 0.25, cd.NAIVE)])
+def test_checkpoint_and_resume_continue_the_run_bit_for_bit(name, scale, mode):
+    """Save after 3 iterations (state vectors + counter), load into a fresh context, run 3 more
+    on both: same messages and state as the uninterrupted run and as the oracle.  The step-size
+    milestones make the counter matter."""
+    w = synth.workload(name, scale=scale)
+    x0 = w.x0("cpu")
+
+    def fresh():
+        g = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.cuda(), mode=mode)
+        g.set_lr_milestones(1e-3, [2, 4], 0.5)
+        g.set_weight_decay(1e-2)
+        return g
+
+    a = fresh()
+    o = orc.Oracle(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=x0.numpy(), mode=mode)
+    o.set_lr_milestones(1e-3, [2, 4], 0.5)
+    o.set_weight_decay(1e-2)
+    for t in range(1, 4):
+        grads = w.grads(t, "cpu")
+        a.step(grads.cuda()); o.step(grads.numpy())
+    saved = a.state_dict()
+    assert saved["step_count"] == 3
+    b = fresh()
+    b.load_state_dict(saved)
+    assert b.step_count() == 3
+    for t in range(4, 7):
+        grads = w.grads(t, "cpu")
+        a.step(grads.cuda()); b.step(grads.cuda()); o.step(grads.numpy())
+        check_payloads(b, o, w)
+        for who in list(range(w.n)) + [cd.SERVER]:
+            pa, pb = a.last_payload(who), b.last_payload(who)
+            assert torch.equal(pa[0], pb[0]) and torch.equal(pa[1].view(torch.int32), pb[1].view(torch.int32))
+    check_state(b, o, FINAL_TOL, exact=True)
+    for nm in orc.STATE_NAMES:
+        assert torch.equal(a.get_state(nm), b.get_state(nm)), nm
+    with pytest.raises(cd.CdadamError):
+        b.set_step_count(-1)
+    a.close(); b.close(); o.close()
