@@ -637,7 +637,7 @@ k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uin
 // before any is used.  Blocks beyond the last tile return (the grid is sized for the
 // bitmap passes of the rows whose guess failed).
 constexpr int kTilesPerBlock = kTileWords * 32 / kSub;      // tiles per 32768-coordinate span
-constexpr int kWarpTiles = 2;
+constexpr int kWarpTiles = 1;
 constexpr int kListTiles = kWarpTiles * (kBlock / 32);
 constexpr int kPre = 4;
 
