@@ -338,6 +338,27 @@ def test_sign_every_small_and_ragged_size(d):
     run_free(w, 3)
 
 
+@pytest.mark.parametrize("lo", [70, 400, 730])
+def test_sign_and_topk_every_size_up_to_1025(lo):
+    """Every d from 70 to 1025 (the smaller ones are above), two iterations each, scaled sign
+    with a segment boundary at a position that moves with d, and top-k with k moving with d:
+    messages bit-exact, x exact."""
+    for d in range(lo, min(lo + 330, 1026)):
+        grads = [torch.randn(2, d, generator=torch.Generator().manual_seed(1000 * t + d)) for t in (1, 2)]
+        off = np.array([0, 1 + (d * 7) % (d - 1), d])
+        for comp, kw in ((cd.SIGN, dict(offsets=off)), (cd.TOPK, dict(k=1 + (d * 13) % d))):
+            g = cd.CDAdam(d, 2, comp, **kw)
+            o = orc.Oracle(d, 2, comp, **kw)
+            for gr in grads:
+                g.step(gr.cuda().reshape(-1)); o.step(gr.numpy())
+            for who in (0, 1, cd.SERVER):
+                a, b = g.last_payload(who)
+                oa, ob = o.payload(who)
+                assert np.array_equal(u32(a), oa) and np.array_equal(u32(b), ob.view(np.uint32)), (d, comp, who)
+            assert np.array_equal(g.params().cpu().numpy(), o.state("x")), (d, comp)
+            g.close(); o.close()
+
+
 @pytest.mark.parametrize("shift", range(0, 32, 3))
 def test_sign_segment_boundaries_at_every_residue(shift):
     d = 3 * 4096 + 77
