@@ -196,8 +196,11 @@ def test_distributed_class_over_a_one_rank_nccl_group(tmp_path):
     import torch.distributed as dist
     w = synth.workload("C2", scale=0.01, steps=3)
     x0 = w.x0("cpu")
-    dist.init_process_group("nccl", init_method="file://" + str(tmp_path / "rendezvous"), rank=0, world_size=1,
-                            device_id=torch.device("cuda", torch.cuda.current_device()))
+    try:
+        dist.init_process_group("nccl", init_method="file://" + str(tmp_path / "rendezvous"), rank=0, world_size=1,
+                                device_id=torch.device("cuda", torch.cuda.current_device()))
+    except Exception as exc:                       # no usable NCCL on this machine: nothing of ours to test
+        pytest.skip("NCCL process group could not be created: %s" % exc)
     try:
         opt = dd.DistributedCDAdam(w.d, w.n, offsets=w.offsets, x0=x0.cuda())
         o = orc.Oracle(w.d, w.n, orc.SIGN, offsets=w.offsets, x0=x0.numpy())
