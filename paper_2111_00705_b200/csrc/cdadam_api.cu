@@ -1066,8 +1066,9 @@ int cdadam_launches_per_step(cdadam_ctx *c)
     if (c->comp == CDADAM_SIGN) return c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5;
     if (c->comp == CDADAM_TOPK && !c->seg_w.empty())
         return (int)c->seg_w.size() * (topk_launches_per_step(c->n) + 1) + 2;
-    if (c->comp == CDADAM_TOPK)
-        return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : c->mode == CDADAM_NAIVE ? 3 : 0);
+    if (c->comp == CDADAM_TOPK)     // (for gradient rows that are 16-byte aligned)
+        return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : c->mode == CDADAM_NAIVE ? 3 : 0) +
+               topk_dense_launches(c->tk_w, c->d % 4 == 0) - 1 + topk_dense_launches(c->tk_s, c->d % 4 == 0) - 1;
     if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : c->mode == CDADAM_NAIVE ? 7 : 4;
     return 1;
 }

@@ -25,6 +25,8 @@ void topk_workspace_set_error_flag(TopkWorkspace *w, int *error_flag);
 void topk_workspace_set_ring(TopkWorkspace *w, int ring);
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
 int topk_launches_per_step(int n);
+// 1 or 2: kernels that make the dense pass of one selection in this workspace (rows aligned or not).
+int topk_dense_launches(const TopkWorkspace *w, bool vec_ok);
 
 // For every row r: u = a_r - b_r (b may be NULL: u = a_r); keep the k coordinates of
 // largest |u| (ties: lower index); write their indices (increasing) and values u_j to the

@@ -1332,6 +1332,22 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
 constexpr int kSelectLaunches = 16;
 int topk_launches_per_step(int) { return 2 * kSelectLaunches + 1; }
 
+// Whole tiles per row that the dense pass takes through the prefetch ring (0: none).
+static int64_t ring_tiles(const TopkWorkspace *w, bool vec_ok)
+{
+    const bool ring_ok = vec_ok && w->stride % 4 == 0 && w->ring >= 0 &&
+                         (w->ring > 0 || (int64_t)w->rows * (w->d / kSub) >= 32768);
+    return ring_ok ? w->d / kSub : 0;
+}
+
+// Kernels of the dense pass: the ring kernel and the plain one share it when the ring takes
+// the whole tiles and a ragged last tile remains.
+int topk_dense_launches(const TopkWorkspace *w, bool vec_ok)
+{
+    const int64_t full = ring_tiles(w, vec_ok);
+    return full > 0 && full < w->nt4k ? 2 : 1;
+}
+
 template <bool HAS_B>
 static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                         cudaStream_t st)
@@ -1346,9 +1362,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // tiles enough to fill the device several times over with its three blocks of eight tiles
     // per SM (measured: 16 x 6250 tiles 0.50 -> 0.47 ms, 1 x 6250 tiles 0.039 -> 0.047 ms);
     // the ragged last tile, or everything else, through the plain kernel
-    const bool ring_ok = vec_ok && w->stride % 4 == 0 && w->ring >= 0 &&
-                         (w->ring > 0 || (int64_t)w->rows * (w->d / kSub) >= 32768);
-    const int64_t full_tiles = ring_ok ? w->d / kSub : 0;
+    const int64_t full_tiles = ring_tiles(w, vec_ok);
     if (full_tiles > 0) {
         constexpr int kBytes = kSpecStages * (HAS_B ? 2 : 1) * kSub * (int)sizeof(float);
         cudaFuncSetAttribute(k_topk_spec_ring<HAS_B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
