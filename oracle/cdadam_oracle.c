@@ -24,7 +24,10 @@
  * vanilla AMSGrad for the identity compressor; for the naive-compression mode a second
  * hand-worked step and its statelessness; for the decoupled weight decay and the step-size
  * milestones the closed form x_t = x_1 prod (1 - alpha_t lambda) at zero gradients and an
- * independently written recursion.  No function here is "parity unpinned".
+ * independently written recursion; for the error-feedback mode a hand-worked three-iteration
+ * run and the server recursion rebuilt from the messages; for the given-scales branch of the
+ * sampled checks the bit-for-bit repeat of a computed run and planted hand-over mistakes.
+ * No function here is "parity unpinned".
  */
 #include <stdint.h>
 #include <stdlib.h>

@@ -618,3 +618,231 @@ def test_topk_per_segment_brute_force_and_reduction_to_whole_vector():
         orc.Oracle(d, n, orc.TOPK, k=1).set_topk_segments([0, 5, d], [6, 1])     # k_r > |S_r|
     with pytest.raises(ValueError):
         orc.Oracle(d, n, orc.SIGN).set_topk_segments([0, d], [1])
+
+
+# ------------------------------------------------------------------ error feedback, server half
+
+def run_ef_example(o, gold, steps=(1, 2, 3)):
+    """Drive the oracle through the hand-worked error-feedback example; returns the list of
+    (key, got, want) triples that differ, so a planted mistake can be shown to be noticed."""
+    n = int(gold["n"][0])
+    bad = []
+
+    def chk(key, got, atol=0.0):
+        want = gold[key]
+        got = np.atleast_1d(np.asarray(got, dtype=np.float64))
+        if got.shape != (len(want),) or np.any(np.abs(got - np.asarray(want)) > atol):
+            bad.append((key, got.tolist(), want))
+
+    for t in steps:
+        p = "t%d." % t
+        o.step(np.array([gold[p + "g0"], gold[p + "g1"]], dtype=np.float32))
+        for i in range(n):
+            bits, scales = o.payload(i)
+            chk(p + "w%d.scale" % i, scales[0])
+            chk(p + "w%d.word" % i, bits[0])
+            chk(p + "w%d.delta" % i, o.state("ghat_w")[i])
+        bits, scales = o.payload(-1)
+        chk(p + "s.scale", scales[0])
+        chk(p + "s.word", bits[0])
+        chk(p + "s.delta", o.state("gtil"))
+        # delta + c gives back what the server compressed: mean plus the old error
+        c = decode_sign(bits, scales, np.array([0, 4]), 4)
+        chk(p + "s.p", o.state("gtil") + c)
+        for name in ("m", "v", "vhat"):
+            chk(p + name, o.state(name))
+        chk(p + "x", o.state("x"), atol=0.0 if t == 1 else 1.5e-7)   # 7 digits in the fixture
+    return bad
+
+
+def ef_example_oracle(gold):
+    return orc.Oracle(int(gold["d"][0]), int(gold["n"][0]), orc.SIGN, beta1=gold["beta1"][0],
+                      beta2=gold["beta2"][0], lr=gold["alpha"][0], eps=gold["nu"][0],
+                      x0=gold["x1"], mode=orc.EF)
+
+
+def test_error_feedback_worked_example_three_iterations():
+    """Section 4, error feedback, both directions, scaled sign: the hand-worked run."""
+    gold = read_golden("worked_example_ef.txt")
+    o = ef_example_oracle(gold)
+    assert run_ef_example(o, gold) == []
+    assert not o.state("ghat_s").any()         # this mode keeps one error vector at the server
+    # x_4 to binary32 accuracy from the exact expression (x_3 is rounded once on the way)
+    r = 0.5 / math.sqrt(223 / 128)
+    x3 = [0.75 - r, 1.25 + r, 0.75 - r, 1.25 + r]
+    want = [a - b * r for a, b in zip(x3, gold["t3.m"])]
+    np.testing.assert_allclose(o.state("x"), want, rtol=0, atol=2.5e-7)
+
+
+def test_error_feedback_example_notices_a_lost_server_error():
+    """The example must be able to fail on the server half: lose the server's error before
+    iteration 3 (what dropping the '+ delta' term of the server's input would do) and both the
+    server's scale and its sign word leave the hand-worked values; lose it before iteration 2
+    and the new error does.  Same for a worker's error."""
+    gold = read_golden("worked_example_ef.txt")
+    o = ef_example_oracle(gold)
+    assert run_ef_example(o, gold, (1, 2)) == []
+    o.state("gtil")[:] = 0
+    keys = {k for k, _, _ in run_ef_example(o, gold, (3,))}
+    assert {"t3.s.scale", "t3.s.word", "t3.s.delta", "t3.s.p", "t3.m", "t3.x"} <= keys
+    assert not any(k.startswith("t3.w") for k in keys)      # the workers are untouched by it
+    o = ef_example_oracle(gold)
+    assert run_ef_example(o, gold, (1,)) == []
+    o.state("gtil")[:] = 0
+    keys = {k for k, _, _ in run_ef_example(o, gold, (2,))}
+    assert "t2.s.delta" in keys and "t2.s.p" in keys
+    o = ef_example_oracle(gold)
+    assert run_ef_example(o, gold, (1,)) == []
+    o.state("ghat_w")[1][:] = 0
+    keys = {k for k, _, _ in run_ef_example(o, gold, (2,))}
+    assert {"t2.w1.scale", "t2.w1.delta"} <= keys and "t2.w0.scale" not in keys
+
+
+@pytest.mark.parametrize("comp", [orc.TOPK, orc.SIGN, orc.IDENTITY])
+def test_error_feedback_server_recursion(comp):
+    """Server half of the error-feedback scheme (Section 4), from the messages alone:
+    p = (sum_i c^(i), i ascending) / n + delta_old;  c = C(p);  delta_new = p - c;  the
+    moments are driven by c, not by p or by a running estimate."""
+    rng = np.random.default_rng(29)
+    d, n, k = 240, 3, 9
+    off = np.array([0, 70, 101, d])
+    kw = dict(k=k) if comp == orc.TOPK else (dict(offsets=off) if comp == orc.SIGN else {})
+    b1, b2 = np.float32(0.9), np.float32(0.999)
+    o = orc.Oracle(d, n, comp, mode=orc.EF, beta1=float(b1), beta2=float(b2), **kw)
+    m_prev = np.zeros(d, np.float32); v_prev = np.zeros(d, np.float32)
+    for t in range(5):
+        d_old = o.state("gtil").copy()
+        dw_old = o.state("ghat_w").copy()
+        g = (rng.standard_normal((n, d)) * (1 + 3 * (rng.random((n, d)) < 0.05))).astype(np.float32)
+        o.step(g)
+        acc = np.zeros(d, np.float32)
+        for i in range(n):                         # decode the n messages, add them in order
+            if comp == orc.TOPK:
+                idx, val = o.payload(i)
+                c_i = np.zeros(d, np.float32); c_i[idx] = val
+            elif comp == orc.SIGN:
+                c_i = decode_sign(*o.payload(i), off, d)
+            else:
+                c_i = g[i] + dw_old[i]
+            acc = acc + c_i
+        p = acc / np.float32(n) + d_old
+        if comp == orc.TOPK:
+            idx, val = o.payload(-1)
+            order = sorted(range(d), key=lambda j: (-abs(float(p[j])), j))[:k]
+            assert idx.tolist() == sorted(order)
+            assert np.array_equal(val, p[idx])
+            c = np.zeros(d, np.float32); c[idx] = val
+            assert np.array_equal(o.state("gtil") + c, p)            # exact: c is p where kept
+            assert not o.state("gtil")[idx].any()
+        elif comp == orc.SIGN:
+            bits, scales = o.payload(-1)
+            for r in range(3):
+                seg = p[off[r]:off[r + 1]]
+                assert scales[r] == np.float32(math.fsum(abs(float(z)) for z in seg) / seg.size)
+            c = decode_sign(bits, scales, off, d)
+            assert np.array_equal(c >= 0, p >= 0)
+        else:
+            c = p
+        assert np.array_equal(o.state("gtil"), p - c)
+        m = b1 * m_prev + (np.float32(1) - b1) * c
+        v = b2 * v_prev + (np.float32(1) - b2) * (c * c)
+        assert np.array_equal(o.state("m"), m) and np.array_equal(o.state("v"), v)
+        m_prev, v_prev = m, v
+    assert not o.state("ghat_s").any()
+
+
+# ------------------------------------------------------------------ scales given from outside
+
+def forced_pair(rng, n=3, d=333, off=(0, 50, 81, 200, 333), mode=orc.MARKOV):
+    off = np.array(off)
+    x0 = (rng.standard_normal(d) * 0.02).astype(np.float32)
+    free = orc.Oracle(d, n, orc.SIGN, offsets=off, x0=x0, mode=mode)
+    given = orc.Oracle(d, n, orc.SIGN, offsets=off, x0=x0, mode=mode)
+    return off, free, given
+
+
+def test_given_scales_reproduce_the_computed_run():
+    """An oracle handed the scales another one computed (the sampled full-size checks use this
+    branch) repeats that run bit for bit: every sign word, scale and state vector, and each
+    decoded coordinate is plus or minus the given scale of its segment."""
+    rng = np.random.default_rng(41)
+    n, d = 3, 333
+    off, free, given = forced_pair(rng)
+    q = off.size - 1
+    for t in range(3):
+        g = (rng.standard_normal((n, d)) * np.repeat([1.0, 1e-2, 30.0, 0.3], np.diff(off))).astype(np.float32)
+        prev_w = given.state("ghat_w").copy(); prev_t = given.state("gtil").copy()
+        free.step(g)
+        ws = np.stack([free.payload(i)[1] for i in range(n)])        # n x q, row i = worker i
+        ss = free.payload(-1)[1]
+        given.force_scales(ws, ss)
+        given.step(g)
+        for who in list(range(n)) + [-1]:
+            for a, b in zip(free.payload(who), given.payload(who)):
+                assert np.array_equal(a, b)
+        for name in orc.STATE_NAMES:
+            assert np.array_equal(free.state(name), given.state(name)), name
+        for i in range(n):                      # c_j = +-given[i][r] by segment, written out
+            u = g[i] - prev_w[i]
+            for r in range(q):
+                sl = slice(off[r], off[r + 1])
+                want = np.where(u[sl] >= 0, ws[i, r], -ws[i, r]).astype(np.float32)
+                assert np.array_equal(prev_w[i][sl] + want, given.state("ghat_w")[i][sl])
+        w = given.state("ghat_s") - prev_t
+        for r in range(q):
+            sl = slice(off[r], off[r + 1])
+            want = np.where(w[sl] >= 0, ss[r], -ss[r]).astype(np.float32)
+            assert np.array_equal(prev_t[sl] + want, given.state("gtil")[sl])
+    # a sample of the coordinates with the full problem's scales follows the full run there
+    pick = np.sort(rng.choice(d, 60, replace=False))
+    seg_of = np.searchsorted(off, pick, side="right") - 1
+    sub_off = np.concatenate([[0], np.cumsum(np.bincount(seg_of, minlength=q))])
+    assert np.all(np.diff(sub_off) > 0)
+    full = orc.Oracle(d, n, orc.SIGN, offsets=off)
+    sub = orc.Oracle(pick.size, n, orc.SIGN, offsets=sub_off)
+    for t in range(3):
+        g = rng.standard_normal((n, d)).astype(np.float32)
+        full.step(g)
+        sub.force_scales(np.stack([full.payload(i)[1] for i in range(n)]), full.payload(-1)[1])
+        sub.step(g[:, pick])
+        for name in orc.STATE_NAMES:
+            assert np.array_equal(full.state(name)[..., pick], sub.state(name)), name
+    # back to computed scales
+    sub.force_scales(None, None)
+    sub.step(g[:, pick])
+    assert not np.array_equal(sub.payload(-1)[1], full.payload(-1)[1])
+
+
+@pytest.mark.parametrize("mistake", ["rows_swapped", "server_for_worker", "one_doubled",
+                                     "segments_reversed"])
+def test_given_scales_planted_mistakes_change_the_state(mistake):
+    """Hand the scales over wrongly, the way a slip in that branch would use them (worker rows
+    exchanged, the server's scales used for a worker, one scale doubled, segment order
+    reversed): the worker states or the second Markov state must leave the computed run."""
+    rng = np.random.default_rng(43)
+    n, d = 3, 333
+    off, free, given = forced_pair(rng)
+    sig = np.repeat([1.0, 1e-2, 30.0, 0.3], np.diff(off))
+    for t in range(2):
+        g = (rng.standard_normal((n, d)) * sig * (1 + np.arange(n))[:, None]).astype(np.float32)
+        free.step(g)
+        ws = np.stack([free.payload(i)[1] for i in range(n)]); ss = free.payload(-1)[1]
+        if t == 1:
+            if mistake == "rows_swapped":
+                ws = ws[[1, 0, 2]]
+            elif mistake == "server_for_worker":
+                ws = ws.copy(); ws[2] = ss
+            elif mistake == "one_doubled":
+                ss = ss.copy(); ss[1] *= 2
+            else:
+                ws = ws[:, ::-1]; ss = ss[::-1]
+        given.force_scales(ws, ss)
+        given.step(g)
+    if mistake == "one_doubled":
+        assert np.array_equal(free.state("ghat_w"), given.state("ghat_w"))
+        sl = slice(off[1], off[2])
+        assert not np.array_equal(free.state("gtil")[sl], given.state("gtil")[sl])
+        assert np.array_equal(free.state("gtil")[:off[1]], given.state("gtil")[:off[1]])
+    else:
+        assert not np.array_equal(free.state("ghat_w"), given.state("ghat_w"))
+        assert not np.array_equal(free.state("gtil"), given.state("gtil"))
