@@ -12,8 +12,12 @@ independent replica of the same problem ("replicas only"), value is the sum over
 Prints one JSON line (rank 0).  `value` is steps/s with the gradients already resident in
 device memory; `e2e` is the same through cdadam_step_host with pinned HOST gradients, the
 host->device copy of n*d floats and the device->host copy of x inside the timed region.
+The timed region is R blocks of exactly K steps (R >= 5 and enough for about a second in
+all); `ms_per_step` and `value` come from the median block, `repeats` gives the spread.
 `roofline` is for the dominant kernel (the worker pass), timed with CUDA events recorded by
-the library on the launching stream in a separate pass of the same K steps.
+the library on the launching stream in a separate pass of the same K steps.  The default
+run (C4, one GPU) then times C5, C3 and C2 the same way and reports them in
+`other_workloads`; C4 stays the headline.
 `--impl reference` times the CPU oracle (tests/-only code, as it stands, one core) on a
 bounded sample of the same workload.
 """
@@ -40,7 +44,9 @@ FALLBACK_HBM_GBS = 6650.0
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
     # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "7f8da041b7e2dc41", "bytes_per_launch": 4 * (1.797478e+09 + 8.56346624e+08)},
+    "C4": {"hash": "7f8da041b7e2dc41", "bytes_per_launch": 4 * (1.797478e+09 + 8.56346624e+08),
+           "note": "extrapolated from an ncu capture of the same kernel on the workload scaled by 0.25 "
+                   "(same tile and kernel variant), multiplied by 4: traffic is proportional to n*d"},
 }
 
 
@@ -168,7 +174,7 @@ def run_reference(args, rank):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec_full * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic", "params_per_s": value * w.d,
-            "config": {"workload": describe(w), "replicas": 1},
+            "config": {"workload": describe(w), "replicas": 1, "l2": l2_note(w)},
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
@@ -242,11 +248,181 @@ def run_distributed(args, w, dev, rank, world):
     dist.destroy_process_group()
 
 
+def l2_small(w):
+    return w.n * w.d * 4 < 2 * 126e6
+
+
+def l2_note(w):
+    """How the timed steps are kept from finding their inputs in L2 (the GPU arm's protocol)."""
+    return ("flushed between steps" if l2_small(w) else
+            "inputs larger than L2 (%.2f GB of gradients per step)" % (w.n * w.d * 4 / 1e9))
+
+
 def describe(w):
     from paper_2111_00705_b200 import synth
     comp = {synth.SIGN: "scaled-sign", synth.TOPK: "top-k k=%d" % w.k, synth.IDENTITY: "identity",
             synth.RANDK: "rand-k k=%d" % w.k}[w.compressor]
     return "%s d=%d n=%d %s q=%d %s fp32" % (w.name, w.d, w.n, comp, w.q, w.dist)
+
+
+def run_workload(args, w, dev, rank, world, barrier, headline):
+    """Times one workload on this rank's GPU: W warm-up steps, then R repeats of a block of
+    exactly K steps (device time per block, max over ranks; R >= 5 and enough for the timed
+    region to last about a second), the clock sampler running from before the warm-up to
+    after the last repeat; then a per-kernel pass for the roofline of the dominant kernel.
+    The headline workload also gets the end-to-end leg through the host-buffer entry point."""
+    import torch
+    from paper_2111_00705_b200 import binding as cd
+    from paper_2111_00705_b200 import synth
+
+    opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
+                    beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev,
+                    mode={"markov": cd.MARKOV, "ef": cd.EF, "naive": cd.NAIVE}[args.mode])
+    if args.tile:
+        opt.set_tile(args.tile)
+    if w.compressor == synth.RANDK:      # the draws are inputs; one set of draws serves all steps
+        import numpy as np
+        opt.set_random_sets(torch.from_numpy(synth.random_sets(w.d, w.k, w.n, w.seed, 1).view(np.int32)).to(dev),
+                            torch.from_numpy(synth.random_sets(w.d, w.k, 1, w.seed + 1, 1)[0].view(np.int32)).to(dev))
+    # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
+    # flushed between steps instead
+    nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1
+    grads = [w.grads(t + 1, dev).reshape(-1) for t in range(nbuf)]
+    bf16 = headline and args.grads == "bf16"
+    step = opt.step
+    if bf16:
+        grads = [g.to(torch.bfloat16) for g in grads]
+        step = opt.step_bf16
+    # L2 holds 126 MB.  A step whose gradients alone are at least twice that (and whose worker
+    # state is as large again) cannot find its inputs there; smaller workloads get the flush.
+    small = l2_small(w)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
+    stream = torch.cuda.current_stream()
+    K = args.steps
+
+    def block():
+        """K steps; returns the device milliseconds spent in the steps (flushes not counted)."""
+        if flush is None:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for t in range(K):
+                step(grads[t % nbuf], stream)
+            b.record(stream)
+            return [(a, b)]
+        pairs = []
+        for t in range(K):              # time each step alone so that the L2 flush is not counted
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream); step(grads[t % nbuf], stream); b.record(stream)
+            pairs.append((a, b))
+        return pairs
+
+    barrier()
+    sampler = ClockSampler(dev.index) if rank == 0 else None     # runs from here to the last repeat
+    for t in range(args.warmup):
+        if flush is not None:
+            flush.zero_()
+        step(grads[t % nbuf], stream)
+    barrier()
+    probe = block()                      # one untimed block sizes the number of repeats
+    barrier()
+    est_ms = max(sum(a.elapsed_time(b) for a, b in probe), 1e-3)
+    repeats = args.repeats if args.repeats > 0 else int(min(400, max(5, -(-args.region_ms // est_ms))))
+
+    # ---- timed region: R blocks of K steps, device time per block, max over ranks --------
+    blocks = []
+    barrier()
+    for r in range(repeats):
+        blocks.append(block())
+        if flush is not None or r % 8 == 7:
+            barrier()                    # bound the queue depth (events, flushes)
+    barrier()
+    block_ms = [sum(a.elapsed_time(b) for a, b in pairs) for pairs in blocks]
+    block_ms = max_over_ranks_list(block_ms, dev)
+    clocks = sampler.stop() if sampler else None
+    med = statistics.median(block_ms)
+    ms_per_step = med / K
+    if clocks and clocks.get("sm_mhz"):
+        clocks["ms_per_step_x_sm_mhz"] = ms_per_step * clocks["sm_mhz"]
+
+    # ---- per-kernel pass for the roofline ------------------------------------------------
+    opt.profile_enable(True)
+    for t in range(K):
+        if flush is not None:
+            flush.zero_()
+        step(grads[t % nbuf], stream)
+    stage_ms, psteps = opt.profile_read()
+    opt.profile_enable(False)
+    stage_ms = {k: v / max(psteps, 1) for k, v in stage_ms.items()}
+    step_bytes, dom_bytes = algorithmic_bytes(w, bf16)
+    dom_name = max(stage_ms, key=stage_ms.get)
+    peak, peak_kind = measured_peak()
+    achieved = dom_bytes / (stage_ms[dom_name] * 1e-3) / 1e9 if stage_ms[dom_name] > 0 else 0.0
+    traffic = traffic_note = None
+    cap = NCU_TRAFFIC.get(w.name)
+    if cap and cap.get("hash") == kernel_source_hash() and not bf16 and args.mode == "markov":
+        traffic = cap["bytes_per_launch"]
+        traffic_note = cap["note"]
+    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
+                "traffic": traffic, "traffic_source": traffic_note,
+                "algorithmic_bytes_per_launch": dom_bytes,
+                "ms_per_launch": stage_ms[dom_name],
+                "timed": "separate pass of the same %d steps with events around every kernel" % K}
+
+    # ---- end to end: host gradients in, x out, copies inside the timed region ------------
+    e2e = None
+    if headline:
+        try:
+            if args.e2e_steps < 1:
+                raise RuntimeError("skipped (--e2e-steps 0)")
+            if bf16:
+                raise RuntimeError("skipped (host path takes binary32 gradients)")
+            gh = [g.cpu().pin_memory() for g in grads[:1]]
+            xh = torch.empty(w.d, dtype=torch.float32).pin_memory()
+            opt.step_host(gh[0], xh, stream)                       # allocates the staging buffer
+            barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for t in range(args.e2e_steps):
+                opt.step_host(gh[0], xh, stream)
+            b.record(stream)
+            barrier()
+            e_ms = max_over_ranks_ms(a.elapsed_time(b), dev)
+            e2e = {"value": replicas_throughput(world, args.e2e_steps, e_ms), "unit": UNIT,
+                   "h2d_bytes_per_step": w.n * w.d * 4, "d2h_bytes_per_step": w.d * 4,
+                   "steps": args.e2e_steps}
+            del gh, xh
+        except Exception as exc:                                   # e.g. not enough pinned memory
+            e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
+
+    launches = opt.launches_per_step() * K * repeats
+    opt.device_status()          # raises if a kernel reported a bounded wait that ran out
+    opt.close()
+    del grads, flush
+    torch.cuda.empty_cache()
+    gbs = step_bytes / (ms_per_step * 1e-3) / 1e9
+    return {"workload": describe(w), "ms_per_step": ms_per_step,
+            "value": replicas_throughput(world, K, med),
+            "repeats": {"count": repeats, "steps_per_repeat": K, "statistic": "median",
+                        "ms_per_step_min": min(block_ms) / K, "ms_per_step_max": max(block_ms) / K,
+                        "timed_region_ms": sum(block_ms)},
+            "l2": l2_note(w),
+            "step_hbm": {"algorithmic_bytes": step_bytes, "gbs": gbs, "frac_of_8tbs": gbs / 8e3,
+                         "frac_of_measured": gbs / peak},
+            "stage_ms": stage_ms, "roofline": roofline, "e2e": e2e, "gpu_launches": launches,
+            "clocks": clocks}
+
+
+def max_over_ranks_list(ms_list, device):
+    """Per-block device times of this rank -> elementwise maximum over all ranks."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1):
+        return list(ms_list)
+    t = torch.tensor(ms_list, dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
 
 
 def main():
@@ -256,7 +432,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="C4")
     ap.add_argument("--impl", default="cdadam", choices=["cdadam", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=10)
+    ap.add_argument("--repeats", type=int, default=0,
+                    help="blocks of --steps steps that are timed (the median is reported); 0 = at least 5 "
+                         "and enough for the timed region to last --region-ms")
+    ap.add_argument("--region-ms", type=float, default=1200.0,
+                    help="minimum total length of the timed region when --repeats is 0")
+    ap.add_argument("--others", default="auto", choices=["auto", "on", "off"],
+                    help="after the headline workload, also time C5, C3 and C2 and report them in "
+                         "`other_workloads` (auto: on for the default C4 run on one GPU)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--compressor", default=None, choices=[None, "randk"],
                     help="randk: run the workload's shapes with the rand-k compressor (k as in C3: d/100)")
@@ -286,7 +470,6 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2111_00705_b200 import binding as cd
     from paper_2111_00705_b200 import synth
 
     if not torch.cuda.is_available():
@@ -310,113 +493,32 @@ def main():
         w.compressor, w.k, w.offsets = synth.RANDK, max(1, w.d // 100), None
     if args.warmup < 3:
         args.warmup = 3
-    opt = cd.CDAdam(w.d, w.n, w.compressor, k=w.k, offsets=w.offsets, x0=w.x0(dev),
-                    beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev,
-                    mode={"markov": cd.MARKOV, "ef": cd.EF, "naive": cd.NAIVE}[args.mode])
-    if args.tile:
-        opt.set_tile(args.tile)
-    if w.compressor == synth.RANDK:      # the draws are inputs; one set of draws serves all steps
-        import numpy as np
-        opt.set_random_sets(torch.from_numpy(synth.random_sets(w.d, w.k, w.n, w.seed, 1).view(np.int32)).to(dev),
-                            torch.from_numpy(synth.random_sets(w.d, w.k, 1, w.seed + 1, 1)[0].view(np.int32)).to(dev))
-    # two gradient sets, alternated; each is far larger than L2 except for C1, where L2 is
-    # flushed between steps instead
-    nbuf = 2 if w.n * w.d * 4 * 2 < 60e9 else 1
-    grads = [w.grads(t + 1, dev).reshape(-1) for t in range(nbuf)]
-    if args.grads == "bf16":
-        grads = [g.to(torch.bfloat16) for g in grads]
-        opt.step = opt.step_bf16
-    # L2 holds 126 MB.  A step whose gradients alone are at least twice that (and whose worker
-    # state is as large again) cannot find its inputs there; smaller workloads get the flush.
-    small = w.n * w.d * 4 < 2 * 126e6
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if small else None
-    stream = torch.cuda.current_stream()
+    head = run_workload(args, w, dev, rank, world, barrier, True)
 
-    def one_step(t):
-        if flush is not None:
-            flush.zero_()
-        opt.step(grads[t % nbuf], stream)
-
-    for t in range(args.warmup):
-        one_step(t)
-    barrier()
-
-    # ---- timed region: K steps, device time, max over ranks -----------------------------
-    sampler = ClockSampler(local_rank) if rank == 0 else None
-    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-    barrier()
-    if flush is None:
-        evs[0].record(stream)
-        for t in range(args.steps):
-            opt.step(grads[t % nbuf], stream)
-        evs[1].record(stream)
-        barrier()
-        total_ms = evs[0].elapsed_time(evs[1])
-    else:                       # time each step alone so that the L2 flush is not counted
-        pairs = []
-        for t in range(args.steps):
-            flush.zero_()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(stream); opt.step(grads[t % nbuf], stream); b.record(stream)
-            pairs.append((a, b))
-        barrier()
-        total_ms = sum(a.elapsed_time(b) for a, b in pairs)
-    clocks = sampler.stop() if sampler else None
-    total_ms = max_over_ranks_ms(total_ms, dev)
-    ms_per_step = total_ms / args.steps
-    value = replicas_throughput(world, args.steps, total_ms)
-
-    # ---- per-kernel pass for the roofline ------------------------------------------------
-    opt.profile_enable(True)
-    for t in range(args.steps):
-        one_step(t)
-    stage_ms, psteps = opt.profile_read()
-    opt.profile_enable(False)
-    stage_ms = {k: v / max(psteps, 1) for k, v in stage_ms.items()}
-    step_bytes, dom_bytes = algorithmic_bytes(w, args.grads == "bf16")
-    dom_name = max(stage_ms, key=stage_ms.get)
-    peak, peak_kind = measured_peak()
-    achieved = dom_bytes / (stage_ms[dom_name] * 1e-3) / 1e9 if stage_ms[dom_name] > 0 else 0.0
-    traffic = None
-    cap = NCU_TRAFFIC.get(w.name)
-    if cap and cap.get("hash") == kernel_source_hash():
-        traffic = cap["bytes_per_launch"]
-    roofline = {"bound": "hbm", "kernel": dom_name, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "peak_source": "%s copy bandwidth" % peak_kind,
-                "traffic": traffic, "algorithmic_bytes_per_launch": dom_bytes,
-                "ms_per_launch": stage_ms[dom_name],
-                "timed": "separate pass of the same %d steps with events around every kernel" % args.steps}
-
-    # ---- end to end: host gradients in, x out, copies inside the timed region ------------
-    e2e = None
-    try:
-        if args.e2e_steps < 1:
-            raise RuntimeError("skipped (--e2e-steps 0)")
-        if args.grads != "f32":
-            raise RuntimeError("skipped (host path takes binary32 gradients)")
-        gh = [g.cpu().pin_memory() for g in grads[:1]]
-        xh = torch.empty(w.d, dtype=torch.float32).pin_memory()
-        opt.step_host(gh[0], xh, stream)                       # allocates the staging buffer
-        barrier()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(stream)
-        for t in range(args.e2e_steps):
-            opt.step_host(gh[0], xh, stream)
-        b.record(stream)
-        barrier()
-        e_ms = max_over_ranks_ms(a.elapsed_time(b), dev)
-        e2e = {"value": replicas_throughput(world, args.e2e_steps, e_ms), "unit": UNIT,
-               "h2d_bytes_per_step": w.n * w.d * 4, "d2h_bytes_per_step": w.d * 4,
-               "steps": args.e2e_steps}
-        del gh, xh
-    except Exception as exc:                                   # e.g. not enough pinned memory
-        e2e = {"value": None, "unit": UNIT, "error": str(exc)[:200]}
-
-    launches = opt.launches_per_step() * args.steps
-    opt.device_status()          # raises if a kernel reported a bounded wait that ran out
-    opt.close()
-    del grads
-    torch.cuda.empty_cache()
+    # the other full-size configurations, same protocol, shorter record
+    others = None
+    plain = (args.scale == 1.0 and args.mode == "markov" and args.grads == "f32" and not args.compressor
+             and not args.tile)
+    if args.others == "on" or (args.others == "auto" and world == 1 and w.name == "C4" and plain):
+        others = {}
+        for name in ("C5", "C3", "C2"):
+            if name == w.name:
+                continue
+            try:
+                r = run_workload(args, synth.workload(name), dev, rank, world, barrier, False)
+                rf = r["roofline"]
+                others[name] = {"workload": r["workload"], "ms_per_step": r["ms_per_step"],
+                                "steps_per_s": r["value"], "repeats": r["repeats"], "l2": r["l2"],
+                                "algorithmic_gbs": r["step_hbm"]["gbs"],
+                                "frac_of_8tbs": r["step_hbm"]["frac_of_8tbs"],
+                                "frac_of_measured": r["step_hbm"]["frac_of_measured"],
+                                "stage_ms": r["stage_ms"],
+                                "dominant": {"kernel": rf["kernel"], "ms_per_launch": rf["ms_per_launch"],
+                                             "achieved_gbs": rf["achieved"], "frac_of_measured": rf["frac"]},
+                                "gpu_launches": r["gpu_launches"], "clocks": r["clocks"]}
+            except Exception as exc:                               # e.g. the device is too small for C5
+                others[name] = {"error": str(exc)[:200]}
+                torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and not args.no_cpu_baseline:
@@ -428,23 +530,19 @@ def main():
                          "seconds per step scaled by 1/%g" % (frac, ws.d, ws.n, sample_steps, frac)}
 
     if rank == 0:
-        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-                "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        line = {"metric": METRIC, "value": head["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": args.warmup, "ms_per_step": head["ms_per_step"], "higher_is_better": True,
                 "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": {"workload": describe(w) + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale)
+                "config": {"workload": head["workload"] + ("" if args.scale == 1.0 else " (scaled by %g)" % args.scale)
                            + {"markov": "", "ef": " [error-feedback mode]", "naive": " [naive-compression mode]"}[args.mode]
                            + ("" if args.grads == "f32" else " [bf16 gradients]"),
-                           "replicas": world,
-                           "l2": "flushed between steps" if flush is not None else
-                                 "inputs larger than L2 (%.2f GB of gradients per step)" % (w.n * w.d * 4 / 1e9)},
-                "params_per_s": value * w.d,
-                "step_hbm": {"algorithmic_bytes": step_bytes,
-                             "gbs": step_bytes / (ms_per_step * 1e-3) / 1e9,
-                             "frac_of_8tbs": step_bytes / (ms_per_step * 1e-3) / 8e12,
-                             "frac_of_measured": step_bytes / (ms_per_step * 1e-3) / 1e9 / peak},
-                "stage_ms": stage_ms,
-                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-                "clocks": clocks}
+                           "replicas": world, "l2": head["l2"]},
+                "repeats": head["repeats"],
+                "params_per_s": head["value"] * w.d,
+                "step_hbm": head["step_hbm"], "stage_ms": head["stage_ms"],
+                "roofline": head["roofline"], "cpu_baseline": cpu, "e2e": head["e2e"],
+                "gpu_launches": head["gpu_launches"], "clocks": head["clocks"],
+                "other_workloads": others}
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

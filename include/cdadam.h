@@ -192,6 +192,65 @@ int cdadam_exchange_buffers(cdadam_ctx *ctx, uint32_t **worker_bits, float **wor
                             uint32_t **server_bits, float **server_scales, int64_t *words,
                             int *q);
 
+/*
+ * Coordinate-sharded deployment of Algorithm 1: a context owns the coordinates [lo, hi) of
+ * every vector - the n workers' gradients and states ghat^(i), the server's ghat and gtil,
+ * and m, v, vhat, x - and several contexts (one per GPU) cover [0, d) between them.  Every
+ * assignment of Algorithm 1 acts coordinate by coordinate, except the l1 norms inside the
+ * scaled-sign compressor (Appendix A, "Scaled sign": ||x||_1 is a sum over all coordinates of
+ * a segment).  So an iteration runs in three stages with two small exchanges in between:
+ *
+ *   cdadam_range_workers  worker pass on the range: u = g - ghat^(i), its sign words, and this
+ *                         range's part of sum |u_j| for every (worker, segment), each part one
+ *                         double-double (two binary64 numbers: value and rounding error)
+ *   -- exchange 1: every context receives the parts of all ranges: n * q pairs per range --
+ *   cdadam_range_server   adds the parts range by range (range 0 first), rounds to binary64,
+ *                         divides by the WHOLE segment's length, rounds to binary32: the
+ *                         workers' scales, the same on every context.  Then the server pass on
+ *                         the range and this range's parts of sum |w_j|, q pairs
+ *   -- exchange 2: q pairs per range --
+ *   cdadam_range_update   the server's scales likewise; gtil += c and AMSGrad on the range
+ *
+ * The parts are added in a fixed order and carry about 104 significant bits, so the scales,
+ * and with them every bit of the payloads and of the state, are those of one context that
+ * holds the whole problem (an all-reduce that adds in an order of the library's choosing
+ * would not guarantee that).  The library makes no network call: the caller moves the sums.
+ *
+ * cdadam_create_range: d, n and the hyper-parameters as in cdadam_create, for the coordinates
+ *   lo <= j < hi (0 <= lo < hi <= d), as range number `range` of `ranges` (ranges ordered by
+ *   lo; the number only fixes the slot in the exchange buffers and the order of the sums).
+ *   CDADAM_SIGN only (k is ignored).  All vectors of this context have hi - lo coordinates:
+ *   gradients are n x (hi - lo), cdadam_get_state / cdadam_set_state / cdadam_params move
+ *   (hi - lo)-vectors, cdadam_last_payload gives the hi - lo sign bits (bit 0 = coordinate lo)
+ *   and one scale per segment that meets the range.  cdadam_set_segments takes the segments
+ *   of the WHOLE problem (offsets from 0 to d), the same on every context; cdadam_set_mode
+ *   takes CDADAM_MARKOV or CDADAM_EF.  cdadam_step and the cdadam_step_* calls are refused.
+ * cdadam_range_workers: grads device, n x (hi - lo) floats, row i = worker i's coordinates
+ *   lo..hi-1.  cdadam_range_server, cdadam_range_update: as described above.  Order per
+ *   iteration: workers, server, update (anything else: CDADAM_ERR_STATE).  Asynchronous on
+ *   `stream`; nothing is allocated; not under stream capture.
+ * cdadam_range_buffers: the exchange buffers, device memory owned by the context.
+ *   worker_sums: ranges x n x q x 2 doubles; slot [r][i][s] is range r's (value, error) pair for
+ *   worker i and segment s of the whole problem (zero where the segment misses the range).
+ *   cdadam_range_workers writes slot [range]; before cdadam_range_server the caller fills
+ *   the other slots with the other contexts' slot (an in-place all-gather of
+ *   *worker_doubles = 2 n q doubles per range).  server_sums: ranges x q x 2 doubles,
+ *   written by cdadam_range_server, gathered before cdadam_range_update
+ *   (*server_doubles = 2 q per range).  *q_local: segments that meet the range;
+ *   *segment_of_local: device, q_local numbers: which segment of the whole problem each
+ *   local one is.  The pointers change when cdadam_set_segments or cdadam_set_tile is called.
+ *   Any output pointer may be NULL.
+ */
+cdadam_ctx *cdadam_create_range(int64_t d, int n, int64_t lo, int64_t hi, int range, int ranges,
+                                int compressor, int64_t k,
+                                float beta1, float beta2, float lr, float eps);
+int cdadam_range_workers(cdadam_ctx *ctx, const float *grads, void *stream);
+int cdadam_range_server(cdadam_ctx *ctx, void *stream);
+int cdadam_range_update(cdadam_ctx *ctx, void *stream);
+int cdadam_range_buffers(cdadam_ctx *ctx, double **worker_sums, double **server_sums,
+                         int64_t *worker_doubles, int64_t *server_doubles, int *q_local,
+                         const int32_t **segment_of_local);
+
 /* Device pointer to the model x (d floats), owned by the context, valid until destroy.
  * Its contents are x_{t+1} once the stream of the last step has completed.  NULL if ctx
  * is NULL. */

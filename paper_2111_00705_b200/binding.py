@@ -34,6 +34,14 @@ _SIGNATURES = {
     "cdadam_exchange_buffers": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
                                            _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
                                            _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int)]),
+    "cdadam_create_range": (_c.c_void_p, [_c.c_int64, _c.c_int, _c.c_int64, _c.c_int64, _c.c_int, _c.c_int, _c.c_int,
+                                          _c.c_int64, _c.c_float, _c.c_float, _c.c_float, _c.c_float]),
+    "cdadam_range_workers": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
+    "cdadam_range_server": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
+    "cdadam_range_update": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
+    "cdadam_range_buffers": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
+                                        _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int),
+                                        _c.POINTER(_c.c_void_p)]),
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
@@ -122,7 +130,7 @@ class _DevView:
 
 
 def _view(ptr, count, dtype, device):
-    typestr = {torch.float32: "<f4", torch.int32: "<i4"}[dtype]
+    typestr = {torch.float32: "<f4", torch.int32: "<i4", torch.float64: "<f8"}[dtype]
     if count == 0:
         return torch.empty(0, dtype=dtype, device=device)
     return torch.as_tensor(_DevView(ptr, count, typestr), device=device)
@@ -344,6 +352,56 @@ class CDAdamShard(CDAdam):
                 "worker_scales": _view(ws.value, self.n * q, torch.float32, self.device).view(self.n, q),
                 "server_bits": _view(sb.value, w, torch.int32, self.device),
                 "server_scales": _view(ss.value, q, torch.float32, self.device)}
+
+
+class CDAdamRange(CDAdam):
+    """A context for the coordinates [lo, hi) of a d-dimensional problem with n workers
+    (scaled sign): one process of a coordinate-sharded deployment.  Every vector of the
+    context has hi - lo coordinates; `offsets` are the segments of the WHOLE problem.  An
+    iteration runs in three stages, the l1 sums of the ranges moved by the caller in between
+    (see ``distributed.py``)."""
+
+    def __init__(self, d, n, lo, hi, rank, ranks, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
+                 offsets=None, x0=None, device=None, mode=MARKOV):
+        self._range = (int(d), int(lo), int(hi), int(rank), int(ranks))
+        self.dim, self.lo, self.hi, self.rank, self.ranks = self._range
+        self.q_all = 1 if offsets is None else len(offsets) - 1
+        super().__init__(hi - lo, n, SIGN, 0, beta1, beta2, lr, eps, offsets, x0, device, mode)
+
+    def _create(self, beta1, beta2, lr, eps):
+        d, lo, hi, rank, ranks = self._range
+        return lib().cdadam_create_range(d, self.n, lo, hi, rank, ranks, SIGN, 0, beta1, beta2, lr, eps)
+
+    def set_segments(self, offsets):
+        super().set_segments(offsets)
+        self.q_all = len(offsets) - 1
+        self.q = self.range_buffers()["q_local"]
+
+    def range_workers(self, grads, stream=None):
+        """Worker pass on the n x (hi - lo) device gradients; writes this range's l1 parts."""
+        _check(lib().cdadam_range_workers(self._h, _dev_f32(grads, self.n * self.d, "grads"), _stream(stream)))
+
+    def range_server(self, stream=None):
+        """Workers' scales from the gathered parts, server pass on the range, its l1 parts."""
+        _check(lib().cdadam_range_server(self._h, _stream(stream)))
+
+    def range_update(self, stream=None):
+        """Server's scales from the gathered parts; gtil += c and AMSGrad on the range."""
+        _check(lib().cdadam_range_update(self._h, _stream(stream)))
+
+    def range_buffers(self):
+        """Torch views (no copy) of the exchange buffers: worker_sums float64[ranks, n, q, 2],
+        server_sums float64[ranks, q, 2] (value and rounding error of each range's part of the
+        l1 sums; slot [rank] is this context's), q_local and segment_of_local int32[q_local]."""
+        ws, ss, seg = ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_void_p()
+        wd, sd, ql = ctypes.c_int64(), ctypes.c_int64(), ctypes.c_int()
+        _check(lib().cdadam_range_buffers(self._h, ctypes.byref(ws), ctypes.byref(ss), ctypes.byref(wd),
+                                          ctypes.byref(sd), ctypes.byref(ql), ctypes.byref(seg)))
+        q = sd.value // 2
+        return {"worker_sums": _view(ws.value, self.ranks * wd.value, torch.float64, self.device).view(self.ranks, self.n, q, 2),
+                "server_sums": _view(ss.value, self.ranks * sd.value, torch.float64, self.device).view(self.ranks, q, 2),
+                "q_local": ql.value,
+                "segment_of_local": _view(seg.value, ql.value, torch.int32, self.device)}
 
 
 def compress_sign(x, offsets=None, stream=None):

@@ -136,6 +136,17 @@ struct cdadam_ctx {
     // worker pass's scratch have nloc rows; the message buffers (wbits, wscale) have n rows.
     int first = 0, nloc = 0;
     int phase = 0;          // split step: 0 = between iterations, 1 = worker stage queued, 2 = server stage queued
+    // Coordinate-sharded iteration: this context owns the coordinates [range_lo, range_lo + d)
+    // of all n workers' vectors and of the server's, in a problem of dimension range_dim, as
+    // range number range_rank of range_count.  Segments are those of the whole problem cut to
+    // the range: local segment r is segment rs_gidx[r] of q_all, of whole length rs_glen[r].
+    bool is_range = false;
+    int64_t range_lo = 0, range_dim = 0;
+    int range_rank = 0, range_count = 1, q_all = 1;
+    dd *rs_w = nullptr, *rs_s = nullptr;      // l1 sums of all ranges: range_count x n x q_all, range_count x q_all
+    int32_t *rs_gidx = nullptr;               // q_loc (device)
+    int64_t *rs_glen = nullptr;               // q_loc (device)
+    std::vector<int64_t> range_off_all;       // the whole problem's q_all + 1 segment offsets
     int tile_override = 0;  // 0 = choose from d and q
     int mode = CDADAM_MARKOV;
     Hyper hp{};
@@ -241,6 +252,40 @@ int alloc_sign_buffers(cdadam_ctx *c)
     c->ssplit = finalize_split(c->ts_s);
     if (c->wsplit > 1 && (rc = dev_zalloc(&c->wsums, (size_t)c->nloc * q * c->wsplit))) return rc;
     if (c->ssplit > 1 && (rc = dev_zalloc(&c->ssums, (size_t)q * c->ssplit))) return rc;
+    return CDADAM_OK;
+}
+
+// Segments of the whole problem cut to the context's coordinate range: local offsets (from 0
+// to d), and for every local segment its number and length in the whole problem.
+void cut_segments(const cdadam_ctx *c, int q_all, const int64_t *off_all, std::vector<int64_t> &off_loc,
+                  std::vector<int32_t> &gidx, std::vector<int64_t> &glen)
+{
+    const int64_t lo = c->range_lo, hi = c->range_lo + c->d;
+    off_loc.assign(1, 0);
+    gidx.clear(); glen.clear();
+    for (int r = 0; r < q_all; ++r) {
+        const int64_t a = std::max(off_all[r], lo), b = std::min(off_all[r + 1], hi);
+        if (a >= b) continue;
+        off_loc.push_back(b - lo);
+        gidx.push_back(r);
+        glen.push_back(off_all[r + 1] - off_all[r]);
+    }
+}
+
+// Buffers of the coordinate-sharded iteration for the current segments (tables already built).
+int alloc_range_buffers(cdadam_ctx *c, int q_all, const std::vector<int32_t> &gidx, const std::vector<int64_t> &glen)
+{
+    cudaFree(c->rs_w); cudaFree(c->rs_s); cudaFree(c->rs_gidx); cudaFree(c->rs_glen);
+    c->rs_w = c->rs_s = nullptr; c->rs_gidx = nullptr; c->rs_glen = nullptr;
+    c->q_all = q_all;
+    int rc;
+    if ((rc = dev_zalloc(&c->rs_w, (size_t)c->range_count * c->n * q_all))) return rc;
+    if ((rc = dev_zalloc(&c->rs_s, (size_t)c->range_count * q_all))) return rc;
+    if ((rc = dev_zalloc(&c->rs_gidx, gidx.size()))) return rc;
+    if ((rc = dev_zalloc(&c->rs_glen, glen.size()))) return rc;
+    CU_TRY(cudaMemcpy(c->rs_gidx, gidx.data(), gidx.size() * sizeof(int32_t), cudaMemcpyHostToDevice));
+    CU_TRY(cudaMemcpy(c->rs_glen, glen.data(), glen.size() * sizeof(int64_t), cudaMemcpyHostToDevice));
+    c->fuse_finish = false;      // a scale needs the other ranges' sums: never finished inside a pass
     return CDADAM_OK;
 }
 
@@ -530,6 +575,26 @@ cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local,
     return create_impl(d, n, first_worker, n_local, compressor, k, beta1, beta2, lr, eps);
 }
 
+cdadam_ctx *cdadam_create_range(int64_t d, int n, int64_t lo, int64_t hi, int range, int ranges, int compressor,
+                                int64_t k, float beta1, float beta2, float lr, float eps)
+{
+    (void)k;
+    if (compressor != CDADAM_SIGN) {
+        fail(CDADAM_ERR_ARG, "the coordinate-sharded iteration takes the scaled-sign compressor");
+        return nullptr;
+    }
+    if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
+    if (lo < 0 || hi <= lo || hi > d) { fail(CDADAM_ERR_ARG, "the range [lo, hi) must be non-empty and lie in [0, d)"); return nullptr; }
+    if (ranges < 1 || ranges > 4096 || range < 0 || range >= ranges) { fail(CDADAM_ERR_ARG, "range number must be in [0, ranges), ranges in [1, 4096]"); return nullptr; }
+    cdadam_ctx *c = create_impl(hi - lo, n, 0, n, compressor, 0, beta1, beta2, lr, eps);
+    if (!c) return nullptr;
+    c->is_range = true;
+    c->range_lo = lo; c->range_dim = d; c->range_rank = range; c->range_count = ranges;
+    const int64_t flat[2] = {0, d};
+    if (cdadam_set_segments(c, 1, flat) != CDADAM_OK) { cdadam_destroy(c); return nullptr; }
+    return c;
+}
+
 void cdadam_destroy(cdadam_ctx *c)
 {
     if (!c) return;
@@ -539,6 +604,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->m); cudaFree(c->v); cudaFree(c->vhat); cudaFree(c->x);
     cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
     cudaFree(c->pay_idx); cudaFree(c->pay_val);
+    cudaFree(c->rs_w); cudaFree(c->rs_s); cudaFree(c->rs_gidx); cudaFree(c->rs_glen);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     cudaFree(c->wdone); cudaFree(c->sdone); cudaFree(c->wsums); cudaFree(c->ssums);
@@ -589,6 +655,7 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
 {
     if (!c || !grads_in) return fail(CDADAM_ERR_ARG, "cdadam_step: NULL argument");
     if (c->nloc != c->n) return fail(CDADAM_ERR_STATE, "cdadam_step: this context holds a part of the workers; use the staged calls");
+    if (c->is_range) return fail(CDADAM_ERR_STATE, "cdadam_step: this context holds a part of the coordinates; use the cdadam_range_* calls");
     if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_step: a staged iteration is under way");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
@@ -715,6 +782,7 @@ static int staged_ok(cdadam_ctx *c, const char *what)
     if (c->comp == CDADAM_TOPK && (c->mode != CDADAM_MARKOV || !c->seg_w.empty()))
         return fail(CDADAM_ERR_STATE, "%s: with top-k the staged calls run Algorithm 1 on the whole vector only", what);
     if (c->prof_on) return fail(CDADAM_ERR_STATE, "%s: per-stage timing covers cdadam_step only", what);
+    if (c->is_range) return fail(CDADAM_ERR_STATE, "%s: this context holds a part of the coordinates; use the cdadam_range_* calls", what);
     return CDADAM_OK;
 }
 
@@ -814,6 +882,85 @@ int cdadam_exchange_buffers(cdadam_ctx *c, uint32_t **worker_bits, float **worke
     return CDADAM_OK;
 }
 
+// ---- one iteration on a coordinate range (coordinate-sharded deployment) ----------------------
+
+static int range_ok(cdadam_ctx *c, const char *what)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "%s: NULL context", what);
+    if (!c->is_range) return fail(CDADAM_ERR_STATE, "%s: the context was not made by cdadam_create_range", what);
+    if (c->mode == CDADAM_NAIVE) return fail(CDADAM_ERR_STATE, "%s: Algorithm 1 and the error-feedback mode only", what);
+    if (c->prof_on) return fail(CDADAM_ERR_STATE, "%s: per-stage timing covers cdadam_step only", what);
+    return CDADAM_OK;
+}
+
+int cdadam_range_workers(cdadam_ctx *c, const float *grads, void *stream)
+{
+    if (int rc = range_ok(c, "cdadam_range_workers")) return rc;
+    if (!grads) return fail(CDADAM_ERR_ARG, "cdadam_range_workers: NULL gradients");
+    if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_range_workers: the previous iteration has not been completed by cdadam_range_update");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    step_size_of_this_step(c);
+    const Tables &tb = c->ts.tb;
+    const bool vec = aligned16(grads) && c->d % 4 == 0;
+    const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
+    launch_worker_sign(grads, false, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, c->mode == CDADAM_EF,
+                       c->error_flag, nullptr, c->wdone, st);
+    launch_range_sums(c->wpart, c->rs_w + (int64_t)c->range_rank * c->n * c->q_all, tb, c->n, c->rs_gidx, c->q_all, st);
+    if (int rc = check_launch("cdadam_range_workers")) return rc;
+    c->cur ^= 1;                              // wscale[cur] receives this iteration's scales in the server stage
+    c->pending = true;
+    c->phase = 1;
+    return CDADAM_OK;
+}
+
+int cdadam_range_server(cdadam_ctx *c, void *stream)
+{
+    if (int rc = range_ok(c, "cdadam_range_server")) return rc;
+    if (c->phase != 1) return fail(CDADAM_ERR_STATE, "cdadam_range_server: call cdadam_range_workers first (once per iteration)");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    const Tables &tbs = c->ts_s.tb;
+    launch_range_scales(c->rs_w, c->range_count, c->n, c->q_all, c->rs_gidx, c->rs_glen, c->wscale[c->cur], tbs.q, st);
+    launch_server_sign(c->wbits, c->wscale[c->cur], c->ghat_s, c->gtil, c->sbits, c->spart, tbs, c->n, c->wp, c->d % 4 == 0,
+                       c->mode, nullptr, c->sdone, st);
+    launch_range_sums(c->spart, c->rs_s + (int64_t)c->range_rank * c->q_all, tbs, 1, c->rs_gidx, c->q_all, st);
+    if (int rc = check_launch("cdadam_range_server")) return rc;
+    c->phase = 2;
+    return CDADAM_OK;
+}
+
+int cdadam_range_update(cdadam_ctx *c, void *stream)
+{
+    if (int rc = range_ok(c, "cdadam_range_update")) return rc;
+    if (c->phase != 2) return fail(CDADAM_ERR_STATE, "cdadam_range_update: call cdadam_range_server first");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    launch_range_scales(c->rs_s, c->range_count, 1, c->q_all, c->rs_gidx, c->rs_glen, c->sscale, c->ts_s.tb.q, st);
+    enqueue_sign_update(c, st);
+    if (int rc = check_launch("cdadam_range_update")) return rc;
+    c->phase = 0;
+    c->steps += 1;
+    return CDADAM_OK;
+}
+
+int cdadam_range_buffers(cdadam_ctx *c, double **worker_sums, double **server_sums, int64_t *worker_doubles,
+                         int64_t *server_doubles, int *q_local, const int32_t **segment_of_local)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_range_buffers: NULL context");
+    if (!c->is_range) return fail(CDADAM_ERR_STATE, "cdadam_range_buffers: the context was not made by cdadam_create_range");
+    if (worker_sums) *worker_sums = reinterpret_cast<double *>(c->rs_w);
+    if (server_sums) *server_sums = reinterpret_cast<double *>(c->rs_s);
+    if (worker_doubles) *worker_doubles = 2 * (int64_t)c->n * c->q_all;
+    if (server_doubles) *server_doubles = 2 * (int64_t)c->q_all;
+    if (q_local) *q_local = c->ts.tb.q;
+    if (segment_of_local) *segment_of_local = c->rs_gidx;
+    return CDADAM_OK;
+}
+
 int cdadam_step_bf16(cdadam_ctx *c, const void *grads, void *stream) { return step_impl(c, grads, true, stream); }
 
 int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, void *stream)
@@ -821,7 +968,7 @@ int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, 
     if (!c || !grads_host) return fail(CDADAM_ERR_ARG, "cdadam_step_host: NULL argument");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
-    if (c->nloc != c->n) return fail(CDADAM_ERR_STATE, "cdadam_step_host: this context holds a part of the workers; use the staged calls");
+    if (c->nloc != c->n || c->is_range) return fail(CDADAM_ERR_STATE, "cdadam_step_host: this context holds a part of the workers or coordinates; use the staged calls");
     const size_t bytes = (size_t)c->n * c->d * sizeof(float);
     int rc0 = ensure_stage(c);
     if (rc0) return rc0;
@@ -892,17 +1039,29 @@ int cdadam_set_segments(cdadam_ctx *c, int q, const int64_t *offsets)
     if (!c || !offsets) return fail(CDADAM_ERR_ARG, "cdadam_set_segments: NULL argument");
     if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "segments apply to the scaled-sign compressor only");
     if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
-    if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
-    if (offsets[0] != 0 || offsets[q] != c->d) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
+    const int64_t dim = c->is_range ? c->range_dim : c->d;
+    if (q < 1 || (int64_t)q > dim) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
+    if (offsets[0] != 0 || offsets[q] != dim) return fail(CDADAM_ERR_ARG, "offsets must start at 0 and end at d");
     for (int r = 0; r < q; ++r)
         if (offsets[r + 1] <= offsets[r]) return fail(CDADAM_ERR_ARG, "offsets must be strictly increasing (segment %d)", r);
     DeviceGuard guard(c->device);
     CU_TRY(cudaDeviceSynchronize());
+    std::vector<int64_t> local;
+    std::vector<int32_t> gidx;
+    std::vector<int64_t> glen;
+    const int q_all = q;
+    if (c->is_range) {             // the whole problem's segments, cut to this context's coordinates
+        c->range_off_all.assign(offsets, offsets + q + 1);
+        cut_segments(c, q, offsets, local, gidx, glen);
+        q = (int)gidx.size();
+        offsets = local.data();
+    }
     int rc = c->ts.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q, false), nullptr, false);
     if (rc) return rc;
     rc = c->ts_s.build(c->d, q, offsets, c->tile_override ? c->tile_override : choose_tile(c->d, q, true), nullptr, false);
     if (rc) return rc;
-    return alloc_sign_buffers(c);
+    if ((rc = alloc_sign_buffers(c))) return rc;
+    return c->is_range ? alloc_range_buffers(c, q_all, gidx, glen) : CDADAM_OK;
 }
 
 int cdadam_set_tile(cdadam_ctx *c, int tile)
@@ -924,7 +1083,7 @@ int cdadam_set_tile(cdadam_ctx *c, int tile)
         return CDADAM_OK;
     }
     c->tile_override = tile;
-    std::vector<int64_t> off = c->ts.off;         // rebuild the tables for the current segments
+    std::vector<int64_t> off = c->is_range ? c->range_off_all : c->ts.off;   // rebuild the tables for the current segments
     return cdadam_set_segments(c, (int)off.size() - 1, off.data());
 }
 
@@ -988,6 +1147,8 @@ int cdadam_get_state(cdadam_ctx *c, int name, float *dst, void *stream)
     if (!src) return fail(CDADAM_ERR_ARG, "unknown state name %d", name);
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
+    if (name == CDADAM_STATE_GHAT_W && c->is_range && c->phase == 1)
+        return fail(CDADAM_ERR_STATE, "cdadam_get_state: the scales of this iteration's worker messages are known after cdadam_range_server");
     if (name == CDADAM_STATE_GHAT_W && c->comp == CDADAM_SIGN && c->pending) {
         if (c->nloc > 0)
             launch_apply_sign(c->ghat_w, c->wbits + (int64_t)c->first * c->wp, c->wscale[c->cur] + (int64_t)c->first * c->ts.tb.q,
@@ -1063,6 +1224,7 @@ int cdadam_device_status(cdadam_ctx *c, void *stream)
 int cdadam_launches_per_step(cdadam_ctx *c)
 {
     if (!c) return 0;
+    if (c->is_range) return 7;      // worker pass, sums | scales, server pass, sums | scales, update
     if (c->comp == CDADAM_SIGN) return c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5;
     if (c->comp == CDADAM_TOPK && !c->seg_w.empty())
         return (int)c->seg_w.size() * (topk_launches_per_step(c->n) + 1) + 2;

@@ -23,6 +23,16 @@ void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint3
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,
                             cudaStream_t st, int split = 1, dd *split_sums = nullptr,
                             unsigned int *split_done = nullptr);
+// Coordinate-sharded iteration (the l1 norm of Appendix A's scaled sign is a sum over the
+// coordinates, which several contexts may share).  launch_range_sums: this context's part of
+// the l1 sum of every (row, local segment), one double-double each, into slot gidx[r] of the
+// row's q_all slots.  launch_range_scales: the sums of all ranges (ranges x rows x q_all),
+// added in the order of the ranges, rounded and divided by the whole segment's length glen[r]
+// -> scales (rows x q_loc).
+void launch_range_sums(const dd *part, dd *sums, const Tables &tb, int rows, const int32_t *gidx, int q_all,
+                       cudaStream_t st);
+void launch_range_scales(const dd *all, int ranges, int rows, int q_all, const int32_t *gidx, const int64_t *glen,
+                         float *scales, int q_loc, cudaStream_t st);
 // Server pass A (Algorithm 1: server aggregation and compression): ghat_s += mean_i decode(c_i); w = ghat_s - gtil; packs
 // sign(w) into sbits and writes partial sums of |w| to spart.  sscale != NULL: the scales are
 // finished in the same launch (done: q zeroed counters), as in the worker pass.

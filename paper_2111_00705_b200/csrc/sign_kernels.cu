@@ -450,6 +450,47 @@ k_finalize_scales_split(const dd *__restrict__ part, float *__restrict__ scales,
 }
 
 // ------------------------------------------------------------------------------------
+// Coordinate-sharded iteration.  A context that owns the coordinates [lo, hi) of every vector
+// cannot finish a scale: the l1 norm of a segment is a sum over all coordinates of the
+// segment, whoever owns them.  It reduces its own part of every (row, segment) to one
+// double-double (k_range_sums, the tiles in the fixed order of k_finalize_scales), the
+// owners' sums are brought together by the caller, and every context adds them in the order
+// of the ranges and rounds (k_range_scales): binary64 nearest, divided by the length of the
+// WHOLE segment, rounded to binary32.  A double-double carries about 104 bits, so the value
+// that is rounded, and with it the scale, is the one a single context computes.
+//   sums:   rows x q_all double-doubles of this context; a local segment r goes to slot
+//           gidx[r], the slots of segments that do not meet the range stay zero
+//   all:    ranges x rows x q_all, slot by slot the sums of every range
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kFinBlock)
+k_range_sums(const dd *__restrict__ part, dd *__restrict__ sums, Tables tb,
+             const int32_t *__restrict__ gidx, int q_all)
+{
+    const int r = blockIdx.x, row = blockIdx.y;
+    const int64_t lo = tb.off[r], hi = tb.off[r + 1];
+    const int64_t T0 = lo / tb.tile, T1 = (hi - 1) / tb.tile;
+    const dd *p = part + (int64_t)row * tb.nparts;
+    dd acc = {0.0, 0.0};
+    for (int64_t T = T0 + threadIdx.x; T <= T1; T += kFinBlock)
+        acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
+    acc = block_sum<kFinBlock>(acc);
+    if (threadIdx.x == 0) sums[(int64_t)row * q_all + gidx[r]] = acc;
+}
+
+__global__ void __launch_bounds__(kBlock)
+k_range_scales(const dd *__restrict__ all, int ranges, int q_all, const int32_t *__restrict__ gidx,
+               const int64_t *__restrict__ glen, float *__restrict__ scales, int q_loc)
+{
+    const int r = blockIdx.x * kBlock + threadIdx.x, row = blockIdx.y, rows = gridDim.y;
+    if (r >= q_loc) return;
+    dd tot = {0.0, 0.0};
+    for (int z = 0; z < ranges; ++z)                   // the ranges in increasing order
+        tot = dd_add(tot, all[((int64_t)z * rows + row) * q_all + gidx[r]]);
+    const double l1 = __dadd_rn(tot.hi, tot.lo);
+    scales[(int64_t)row * q_loc + r] = __double2float_rn(__ddiv_rn(l1, (double)glen[r]));
+}
+
+// ------------------------------------------------------------------------------------
 // Server pass A.  grid = (ntiles).
 //
 // Vector path: a warp owns 128*VPT consecutive coordinates per iteration.  The sign words
@@ -849,6 +890,19 @@ void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int
     }
     dim3 grid((unsigned)tb.q, (unsigned)rows);
     launch_after(k_finalize_scales, grid, dim3(kFinBlock), 0, st, part, scales, tb);
+}
+
+void launch_range_sums(const dd *part, dd *sums, const Tables &tb, int rows, const int32_t *gidx, int q_all,
+                       cudaStream_t st)
+{
+    k_range_sums<<<dim3((unsigned)tb.q, (unsigned)rows), kFinBlock, 0, st>>>(part, sums, tb, gidx, q_all);
+}
+
+void launch_range_scales(const dd *all, int ranges, int rows, int q_all, const int32_t *gidx, const int64_t *glen,
+                         float *scales, int q_loc, cudaStream_t st)
+{
+    k_range_scales<<<dim3((unsigned)((q_loc + kBlock - 1) / kBlock), (unsigned)rows), kBlock, 0, st>>>(
+        all, ranges, q_all, gidx, glen, scales, q_loc);
 }
 
 void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_s,

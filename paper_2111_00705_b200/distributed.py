@@ -117,3 +117,65 @@ class DistributedCDAdam:
 
     def close(self):
         self.shard.close()
+
+
+# ---------------------------------------------------------------------------------------------
+# Coordinate-sharded deployment: every process owns a coordinate range of all n workers' vectors
+# and of the server's.  The one thing that crosses ranges is the l1 norm inside the scaled-sign
+# compressor (Appendix A): each process reduces its part of every (worker, segment) sum to a
+# double-double, the parts are all-gathered and every process adds them in rank order.  An
+# all-reduce is NOT used: its order of additions is the library's choice, and the scale has to
+# be the same bits everywhere and equal to the one-process value.
+# ---------------------------------------------------------------------------------------------
+
+def range_partition(d, world, rank, align=16384):
+    """[lo, hi) of `rank`: [0, d) cut into `world` contiguous ranges whose inner boundaries are
+    multiples of `align` (the largest tile of the kernels, so that full tiles stay full); the
+    last range takes the ragged end.  Ranges may differ by one `align` unit in length."""
+    if not (0 <= rank < world):
+        raise ValueError("rank out of range")
+    units = -(-d // align)
+    if units < world:
+        raise ValueError("d = %d is too small for %d ranges aligned to %d" % (d, world, align))
+    base, extra = divmod(units, world)
+    start = rank * base + min(rank, extra)
+    stop = start + base + (1 if rank < extra else 0)
+    return start * align, min(d, stop * align)
+
+
+def gather_range_sums(sums, group=None):
+    """In-place all-gather of the l1 parts: `sums` is the [ranks, ...] exchange buffer of this
+    process with its own slot [rank] filled in; on return every slot holds its owner's parts,
+    slot r from the process of rank r.  No arithmetic happens here."""
+    rank = dist.get_rank(group)
+    flat = sums.view(sums.shape[0], -1)
+    dist.all_gather_into_tensor(flat.view(-1), flat[rank].clone(), group=group)
+
+
+class RangeShardedCDAdam:
+    """Algorithm 1 with scaled sign, coordinate-sharded across the processes of a
+    ``torch.distributed`` group: process r owns coordinates range_partition(d, world, r) of every
+    vector.  ``step(grads_local)`` takes the n x (hi - lo) gradients of the owned coordinates;
+    ``params()`` is the owned slice of x_{t+1}.  Two all-gathers of a few hundred bytes per
+    iteration (2 n q and 2 q doubles per process); no vector ever crosses a process."""
+
+    def __init__(self, d, n, group=None, align=16384, **kwargs):
+        self.group = group
+        self.world = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+        self.lo, self.hi = range_partition(d, self.world, self.rank, align)
+        self.range = binding.CDAdamRange(d, n, self.lo, self.hi, self.rank, self.world, **kwargs)
+
+    def step(self, grads_local):
+        r = self.range
+        r.range_workers(grads_local)
+        gather_range_sums(r.range_buffers()["worker_sums"], self.group)
+        r.range_server()
+        gather_range_sums(r.range_buffers()["server_sums"], self.group)
+        r.range_update()
+
+    def params(self):
+        return self.range.params()
+
+    def close(self):
+        self.range.close()

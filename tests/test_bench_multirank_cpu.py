@@ -50,3 +50,24 @@ def test_reference_arm_prints_on_rank_zero_only():
     line = json.loads(r.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["value"] > 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["unit"] == "steps/s"
+
+
+def _rank_blocks(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank),
+                      WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    mine = [10.0, 11.0, 9.0] if rank == 0 else [10.5, 10.0, 12.0]
+    got = bench.max_over_ranks_list(mine, "cpu")
+    dist.barrier()
+    if rank == 0:
+        with open(out, "w") as f:
+            json.dump(got, f)
+    dist.destroy_process_group()
+
+
+def test_repeat_blocks_take_the_max_over_ranks_block_by_block(tmp_path):
+    out = str(tmp_path / "blocks.json")
+    port = 31500 + os.getpid() % 2000
+    mp.spawn(_rank_blocks, args=(2, port, out), nprocs=2, join=True)
+    assert json.load(open(out)) == [10.5, 11.0, 12.0]

@@ -87,3 +87,57 @@ def test_three_ranks_with_a_server_gather_then_broadcast(tmp_path):
         assert (res[r]["bits"][others] == -1).all()
     for got in res:                        # the server message reaches everyone
         assert torch.equal(got["sbits"], _row_bits(99)) and torch.equal(got["sscales"], _row_scales(99))
+
+
+# ---- coordinate-sharded deployment: the ranges and the exchange of the l1 parts ---------------
+
+def test_range_partition_covers_the_coordinates_with_aligned_cuts():
+    for d, world, align in ((112000, 3, 4096), (110_000_000, 8, 16384), (65536, 4, 16384), (1_500_000_000, 8, 16384),
+                            (100, 2, 64)):
+        cuts = [dd.range_partition(d, world, r, align) for r in range(world)]
+        assert cuts[0][0] == 0 and cuts[-1][1] == d
+        for (a, b), (c, e) in zip(cuts, cuts[1:]):
+            assert b == c and b % align == 0 and a < b
+        sizes = [b - a for a, b in cuts[:-1]]
+        assert max(sizes) - min(sizes) <= align
+    with pytest.raises(ValueError):
+        dd.range_partition(100, 4, 0, 64)               # fewer aligned units than ranges
+    with pytest.raises(ValueError):
+        dd.range_partition(1000, 2, 2, 64)
+
+
+def _sums_main(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    n, q = 3, 4
+    # the exchange buffer as the library lays it out: [ranks, n, q, 2] doubles, own slot filled
+    sums = torch.full((world, n, q, 2), float("nan"), dtype=torch.float64)
+    sums[rank] = _own_sums(rank, n, q)
+    dd.gather_range_sums(sums)
+    # what every process then does with them (in the library's kernel): add range by range
+    total = torch.zeros(n, q, dtype=torch.float64)
+    for r in range(world):
+        total = total + sums[r, :, :, 0]
+    torch.save({"sums": sums, "total": total}, os.path.join(out_dir, "s%d.pt" % rank))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def _own_sums(rank, n, q):
+    # values whose sum depends on the order of the additions in binary64
+    base = torch.tensor([1e16, 1.0, -1e16, 3.0], dtype=torch.float64)[rank % 4]
+    t = torch.zeros(n, q, 2, dtype=torch.float64)
+    t[:, :, 0] = base + torch.arange(n * q, dtype=torch.float64).view(n, q)
+    t[:, :, 1] = 2.0 ** -60 * (rank + 1)
+    return t
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_l1_parts_are_gathered_slot_by_slot_and_added_in_rank_order(world, tmp_path):
+    port = 27000 + (os.getpid() * 11 + world * 17) % 3000
+    mp.spawn(_sums_main, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    res = [torch.load(os.path.join(str(tmp_path), "s%d.pt" % r)) for r in range(world)]
+    want = torch.stack([_own_sums(r, 3, 4) for r in range(world)])
+    for got in res:
+        assert torch.equal(got["sums"], want)           # slot r holds rank r's parts, bit for bit
+        assert torch.equal(got["total"], res[0]["total"])   # the same additions everywhere

@@ -113,6 +113,16 @@ def test_c1_full_free_run():
     run_free(synth.workload("C1"), 10)
 
 
+@pytest.mark.parametrize("name,scale", [("C2", 0.01), ("C3", 0.004), ("C4", 0.002), ("C5", 0.0001)])
+def test_configurations_run_their_own_number_of_steps(name, scale):
+    """Free runs of the configurations' own lengths (C2 100, C3 50, C4 50, C5 20 steps) at a
+    scaled-down d: payloads bit for bit after every step, every state vector within 1e-5
+    after every step and within 1e-4 (and bit for bit) after the last one."""
+    w = synth.workload(name, scale=scale)
+    assert w.steps == {"C2": 100, "C3": 50, "C4": 50, "C5": 20}[name]
+    run_free(w, w.steps)
+
+
 def test_c1_teacher_forced():
     run_teacher_forced(synth.workload("C1"), 4)
 
