@@ -394,6 +394,19 @@ int cdadam_set_step_count(cdadam_ctx *ctx, int64_t t);
  */
 int cdadam_device_status(cdadam_ctx *ctx, void *stream);
 
+/*
+ * Polls after which a kernel's wait on one of its bulk asynchronous copies gives up (the
+ * prefetch-ring kernels of the scaled-sign worker pass and of the top-k dense pass poll an
+ * mbarrier; the default is 2^22 polls, seconds of waiting, never reached by a copy that is
+ * merely slow).  polls < 0 restores the default.  0 makes every such wait give up at once:
+ * the kernels then report through cdadam_device_status and leave in order, the blocks having
+ * first waited, with the default limit, for their copies in flight - which is how the error
+ * path can be exercised without anything going wrong on the device.  Applies to the
+ * following iterations.  After cdadam_device_status has returned CDADAM_ERR_TIMEOUT the
+ * context accepts no further iterations (CDADAM_ERR_STATE): its state is not valid.
+ */
+int cdadam_set_wait_limit(cdadam_ctx *ctx, int polls);
+
 /* Number of kernels one cdadam_step launches in the context's current configuration. */
 int cdadam_launches_per_step(cdadam_ctx *ctx);
 

@@ -60,6 +60,7 @@ _SIGNATURES = {
     "cdadam_set_step_count": (_c.c_int, [_c.c_void_p, _c.c_int64]),
     "cdadam_device_status": (_c.c_int, [_c.c_void_p, _c.c_void_p]),
     "cdadam_launches_per_step": (_c.c_int, [_c.c_void_p]),
+    "cdadam_set_wait_limit": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "cdadam_compress_sign": (_c.c_int, [_c.c_void_p, _c.c_int64, _c.c_int,
                                         _c.POINTER(_c.c_int64), _c.c_void_p, _c.c_void_p,
                                         _c.c_void_p]),
@@ -285,6 +286,10 @@ class CDAdam:
     def device_status(self, stream=None):
         """Wait for the stream; raise if a kernel reported that a bounded wait ran out."""
         _check(lib().cdadam_device_status(self._h, _stream(stream)))
+
+    def set_wait_limit(self, polls):
+        """Polls before a kernel's wait on an asynchronous copy gives up (< 0: the default)."""
+        _check(lib().cdadam_set_wait_limit(self._h, int(polls)))
 
     def step_count(self):
         return lib().cdadam_step_count(self._h)

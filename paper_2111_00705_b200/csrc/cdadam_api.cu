@@ -166,6 +166,8 @@ struct cdadam_ctx {
     dd *wsums = nullptr, *ssums = nullptr;
     bool fuse_finish = false;    // scales finished inside the worker / server pass
     int *error_flag = nullptr;   // device word set by a kernel whose bounded wait ran out
+    int wait_limit = -1;         // polls before such a wait gives up (< 0: the kernels' default)
+    bool void_state = false;     // a wait ran out (seen by cdadam_device_status): no further iterations
     int cur = 0;            // wscale[cur] holds the scales of the last worker payloads
     bool pending = false;   // the last worker payloads are not yet added to ghat_w
     bool sets_given = false;   // rand-k: coordinate sets have been supplied
@@ -367,7 +369,8 @@ void enqueue_sign_workers(cdadam_ctx *c, const void *grads_in, bool bf16, bool v
             launch_pack_sign(static_cast<const float *>(grads_in), bits, c->wpart, tb, c->nloc, c->wp, vec, st);
         else
             launch_worker_sign(grads_in, bf16, c->ghat_w, bits, old_scale, c->wpart, tb, c->nloc, c->wp, vec,
-                               c->mode == CDADAM_EF, c->error_flag, fuse ? new_scale + so : nullptr, c->wdone, st);
+                               c->mode == CDADAM_EF, c->error_flag, fuse ? new_scale + so : nullptr, c->wdone, st,
+                               c->wait_limit);
     }
     prof_mark(c, st);
     if (!fuse) {
@@ -556,6 +559,9 @@ static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compre
     if (rc != CDADAM_OK || cudaDeviceSynchronize() != cudaSuccess) { cdadam_destroy(c); return nullptr; }
     topk_workspace_set_error_flag(c->tk_w, c->error_flag);
     topk_workspace_set_error_flag(c->tk_s, c->error_flag);
+    // Algorithm 1 with top-k: ghat^(i) += c^(i) at the kept coordinates is left to the next
+    // iteration's dense pass (cdadam_get_state applies what is pending)
+    if (compressor == CDADAM_TOPK) topk_workspace_set_defer(c->tk_w, true);
     return c;
 }
 
@@ -657,6 +663,7 @@ static int step_impl(cdadam_ctx *c, const void *grads_in, bool bf16, void *strea
     if (c->nloc != c->n) return fail(CDADAM_ERR_STATE, "cdadam_step: this context holds a part of the workers; use the staged calls");
     if (c->is_range) return fail(CDADAM_ERR_STATE, "cdadam_step: this context holds a part of the coordinates; use the cdadam_range_* calls");
     if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_step: a staged iteration is under way");
+    if (c->void_state) return fail(CDADAM_ERR_STATE, "cdadam_step: a kernel's wait ran out in an earlier iteration; the state is not valid");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
@@ -791,6 +798,7 @@ int cdadam_step_workers(cdadam_ctx *c, const float *grads, void *stream)
     if (int rc = staged_ok(c, "cdadam_step_workers")) return rc;
     if (c->nloc > 0 && !grads) return fail(CDADAM_ERR_ARG, "cdadam_step_workers: NULL gradients");
     if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_step_workers: the previous iteration has not been completed by cdadam_step_update");
+    if (c->void_state) return fail(CDADAM_ERR_STATE, "cdadam_step_workers: a kernel's wait ran out in an earlier iteration; the state is not valid");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
@@ -898,6 +906,7 @@ int cdadam_range_workers(cdadam_ctx *c, const float *grads, void *stream)
     if (int rc = range_ok(c, "cdadam_range_workers")) return rc;
     if (!grads) return fail(CDADAM_ERR_ARG, "cdadam_range_workers: NULL gradients");
     if (c->phase != 0) return fail(CDADAM_ERR_STATE, "cdadam_range_workers: the previous iteration has not been completed by cdadam_range_update");
+    if (c->void_state) return fail(CDADAM_ERR_STATE, "cdadam_range_workers: a kernel's wait ran out in an earlier iteration; the state is not valid");
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
     if (int rc = refuse_capture(st)) return rc;
@@ -906,7 +915,7 @@ int cdadam_range_workers(cdadam_ctx *c, const float *grads, void *stream)
     const bool vec = aligned16(grads) && c->d % 4 == 0;
     const float *old_scale = c->pending ? c->wscale[c->cur] : c->zero_scale;
     launch_worker_sign(grads, false, c->ghat_w, c->wbits, old_scale, c->wpart, tb, c->n, c->wp, vec, c->mode == CDADAM_EF,
-                       c->error_flag, nullptr, c->wdone, st);
+                       c->error_flag, nullptr, c->wdone, st, c->wait_limit);
     launch_range_sums(c->wpart, c->rs_w + (int64_t)c->range_rank * c->n * c->q_all, tb, c->n, c->rs_gidx, c->q_all, st);
     if (int rc = check_launch("cdadam_range_workers")) return rc;
     c->cur ^= 1;                              // wscale[cur] receives this iteration's scales in the server stage
@@ -1087,6 +1096,18 @@ int cdadam_set_tile(cdadam_ctx *c, int tile)
     return cdadam_set_segments(c, (int)off.size() - 1, off.data());
 }
 
+int cdadam_set_wait_limit(cdadam_ctx *c, int polls)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_set_wait_limit: NULL context");
+    c->wait_limit = polls < 0 ? -1 : polls;
+    topk_workspace_set_wait_limit(c->tk_w, polls);
+    topk_workspace_set_wait_limit(c->tk_s, polls);
+    for (TopkWorkspace *w : c->seg_w) topk_workspace_set_wait_limit(w, polls);
+    for (TopkWorkspace *w : c->seg_s) topk_workspace_set_wait_limit(w, polls);
+    drop_graphs(c);                            // the limit is a launch argument
+    return CDADAM_OK;
+}
+
 int cdadam_set_random_sets(cdadam_ctx *c, const uint32_t *workers, const uint32_t *server, void *stream)
 {
     if (!c || !workers || !server) return fail(CDADAM_ERR_ARG, "cdadam_set_random_sets: NULL argument");
@@ -1157,6 +1178,11 @@ int cdadam_get_state(cdadam_ctx *c, int name, float *dst, void *stream)
         if (rc) return rc;
         c->pending = false;
     }
+    if (name == CDADAM_STATE_GHAT_W && c->comp == CDADAM_TOPK && c->tk_w && c->nloc > 0) {
+        topk_flush(c->tk_w, c->ghat_w, st);              // the last worker messages, if still to be applied
+        int rc = check_launch("apply deferred payload");
+        if (rc) return rc;
+    }
     const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->nloc * c->d : (size_t)c->d;
     CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, st));
     return CDADAM_OK;
@@ -1170,7 +1196,10 @@ int cdadam_set_state(cdadam_ctx *c, int name, const float *src, void *stream)
     DeviceGuard guard(c->device);
     const size_t count = name == CDADAM_STATE_GHAT_W ? (size_t)c->nloc * c->d : (size_t)c->d;
     CU_TRY(cudaMemcpyAsync(dst, src, count * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
-    if (name == CDADAM_STATE_GHAT_W) c->pending = false;   // the given values are final
+    if (name == CDADAM_STATE_GHAT_W) {                     // the given values are final
+        c->pending = false;
+        if (c->comp == CDADAM_TOPK) topk_forget_pending(c->tk_w, (cudaStream_t)stream);
+    }
     return CDADAM_OK;
 }
 
@@ -1217,7 +1246,10 @@ int cdadam_device_status(cdadam_ctx *c, void *stream)
     CU_TRY(cudaMemcpyAsync(&flag, c->error_flag, sizeof flag, cudaMemcpyDeviceToHost, (cudaStream_t)stream));
     CU_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     if (flag == 2) return fail(CDADAM_ERR_ARG, "a rand-k coordinate set was not strictly increasing or had a coordinate >= d; the state is not valid");
-    if (flag) return fail(CDADAM_ERR_TIMEOUT, "a kernel gave up waiting for an asynchronous copy; the state is not valid");
+    if (flag) {
+        c->void_state = true;
+        return fail(CDADAM_ERR_TIMEOUT, "a kernel gave up waiting for an asynchronous copy; the state is not valid");
+    }
     return CDADAM_OK;
 }
 

@@ -145,6 +145,12 @@ __device__ __forceinline__ void st_rw4(float *p, float4 v)
     __stcs(reinterpret_cast<float4 *>(p), v);
 }
 __device__ __forceinline__ uint32_t ld_ro_u32(const uint32_t *p) { return __ldg(p); }
+// Coherent (L2) loads for what the kernel queued just before wrote: under programmatic
+// dependent launch this grid is already resident while that kernel runs, so such data is not
+// read-only for this grid's lifetime and must not go through the non-coherent path.
+__device__ __forceinline__ uint32_t ld_cg_u32(const uint32_t *p) { return __ldcg(p); }
+__device__ __forceinline__ float ld_cg_f32(const float *p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ld_cg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
 
 // ------------------------------------------------------------------------------------
 // Bulk asynchronous copies (TMA, one-dimensional, no multicast) global -> shared, completed
@@ -177,10 +183,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
                  : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
     return done != 0;
 }
-constexpr int kWaitLimit = 1 << 22;     // try_wait attempts before a wait gives up
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity)
+constexpr int kWaitLimit = 1 << 22;     // try_wait attempts before a wait gives up (default)
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, int limit = kWaitLimit)
 {
-    for (int spin = 0; spin < kWaitLimit; ++spin)
+    for (int spin = 0; spin < limit; ++spin)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }

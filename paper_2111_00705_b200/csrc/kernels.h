@@ -9,14 +9,14 @@ namespace cdadam {
 // Worker pass (Algorithm 1: the workers' compression and state update) for all n workers: applies the previous payload
 // (bits in wbits, scales in scale_old) to ghat_w (grads: n x d binary32 or bfloat16), forms u = g - ghat_w, packs sign(u) into
 // wbits and writes per-tile double-double partial sums of |u| to wpart.  For large tiles the
-// variant with a TMA prefetch ring runs; it sets *error_flag (device) if a bounded wait on
-// a copy ran out.  With scale_new != NULL the block that completes a (worker, segment) also
+// variant with a prefetch ring of bulk asynchronous copies runs; it sets *error_flag (device)
+// if a bounded wait on a copy ran out (wait_limit polls; < 0 = the default).  With scale_new != NULL the block that completes a (worker, segment) also
 // turns its partial sums into the scale (done: n x q zeroed counters, left zeroed), and no
 // launch_finalize_scales is needed.
 void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
                         int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
-                        unsigned int *done, cudaStream_t st);
+                        unsigned int *done, cudaStream_t st, int wait_limit = -1);
 // Correctly rounded scale of every (row, segment) from the partial sums.  split > 1 (segments
 // of very many tiles): that many blocks share a segment; split_sums holds rows x q x split
 // sums, split_done rows x q zeroed counters (left zeroed).

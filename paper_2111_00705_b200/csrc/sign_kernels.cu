@@ -305,7 +305,7 @@ __global__ void __launch_bounds__(kBlock, 3)
 k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
                    uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
                    dd *__restrict__ wpart, Tables tb, int64_t wp, int *__restrict__ error_flag,
-                   float *__restrict__ scale_new, unsigned int *__restrict__ done)
+                   float *__restrict__ scale_new, unsigned int *__restrict__ done, int wait_limit)
 {
     extern __shared__ __align__(128) unsigned char ring[];
     __shared__ __align__(8) uint64_t full[kRingStages];
@@ -347,10 +347,10 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
     const float s = so[first];
     dd acc = {0.0, 0.0};
     bool arrived = true;
-    for (int it = 0; it < iters; ++it) {
+    int it = 0;
+    for (; it < iters; ++it) {
         const int st = it % kRingStages;
-        arrived = mbar_wait_bounded(&full[st], (uint32_t)(it / kRingStages) & 1u);
-        if (!arrived) break;
+        const bool mine = mbar_wait_bounded(&full[st], (uint32_t)(it / kRingStages) & 1u, wait_limit);
         const float *src = reinterpret_cast<const float *>(ring + st * kRingStageBytes);
         const int64_t wb = base + (int64_t)it * kSub + warp * kWarpSpan;
         WorkerRegs r;
@@ -361,19 +361,23 @@ k_worker_sign_ring(const G *__restrict__ grads, float *__restrict__ ghat_w,
             r.G[v] = grad_lds4(reinterpret_cast<const G *>(src + kSub) + e);
             r.ow[v] = bw[(wb >> 5) + v * 4 + (lane >> 3)];
         }
-        __syncthreads();                                       // the stage has been read by all
+        // the stage has been read by all; the same barrier makes the outcome of the waits one
+        // decision of the whole block (a thread whose wait ran out has read a stage that may
+        // be incomplete: nothing of it is used)
+        arrived = !__syncthreads_or(!mine);
+        if (!arrived) break;
         if (threadIdx.x == 0 && it + kRingStages < iters) refill(it + kRingStages, st);
         worker_compute<EF>(r, gh, bw, wb, lane, s, acc);
     }
     if (!arrived) {
-        // A copy did not complete in time: report it, give the copies still in flight a
-        // bounded chance to land before this block's shared memory is released, and leave
-        // (the step's results are void; the scale of this segment is not finished).
+        // A copy did not complete in time: report it, give the copies still in flight (those
+        // of sub-tiles it .. it + kRingStages - 1, issued and not yet consumed) a bounded
+        // chance, the full default limit, to land before this block's shared memory is
+        // released, and leave: all threads of the block together.  The step's results are
+        // void; the scale of this segment is not finished.
         if (threadIdx.x == 0) atomicExch(error_flag, 1);
-        for (int st = 0; st < kRingStages; ++st) {
-            mbar_wait_bounded(&full[st], 0u);
-            mbar_wait_bounded(&full[st], 1u);
-        }
+        for (int j = it; j < iters && j < it + kRingStages; ++j)
+            mbar_wait_bounded(&full[j % kRingStages], (uint32_t)(j / kRingStages) & 1u);
         return;
     }
     acc = block_sum<kBlock>(acc);
@@ -399,8 +403,10 @@ k_finalize_scales(const dd *__restrict__ part, float *__restrict__ scales, Table
     const dd *p = part + (int64_t)row * tb.nparts;
     dd acc = {0.0, 0.0};
     grid_dep_wait();                                   // the partial sums come from the pass before
-    for (int64_t T = T0 + threadIdx.x; T <= T1; T += kFinBlock)
-        acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
+    for (int64_t T = T0 + threadIdx.x; T <= T1; T += kFinBlock) {
+        const double2 v = __ldcg(reinterpret_cast<const double2 *>(p + tb.pbase[T] + (r - tb.tile_first[T])));
+        acc = dd_add(acc, dd{v.x, v.y});
+    }
     acc = block_sum<kFinBlock>(acc);
     if (threadIdx.x == 0) {
         const double l1 = __dadd_rn(acc.hi, acc.lo);
@@ -427,8 +433,10 @@ k_finalize_scales_split(const dd *__restrict__ part, float *__restrict__ scales,
     dd acc = {0.0, 0.0};
     grid_dep_launch();
     grid_dep_wait();                                   // the partial sums come from the pass before
-    for (int64_t T = A + threadIdx.x; T < B; T += kFinBlock)
-        acc = dd_add(acc, p[tb.pbase[T] + (r - tb.tile_first[T])]);
+    for (int64_t T = A + threadIdx.x; T < B; T += kFinBlock) {
+        const double2 v = __ldcg(reinterpret_cast<const double2 *>(p + tb.pbase[T] + (r - tb.tile_first[T])));
+        acc = dd_add(acc, dd{v.x, v.y});
+    }
     acc = block_sum<kFinBlock>(acc);
     const int64_t slot = (int64_t)row * tb.q + r;
     if (threadIdx.x == 0) {
@@ -544,7 +552,7 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         // the table serves the first nt workers (only in the 8-coordinates-per-thread layout)
         const int nt = (multi || VPT != 2) ? 0 : min(n, kTabWorkers);
         if (!multi) {
-            if (threadIdx.x < n) ssm[threadIdx.x] = wscale[(int64_t)threadIdx.x * tb.q + first];
+            if (threadIdx.x < n) ssm[threadIdx.x] = ld_cg_f32(wscale + (int64_t)threadIdx.x * tb.q + first);
             __syncthreads();
             if (nt > 0) {
                 if (threadIdx.x < (1 << nt)) {
@@ -573,13 +581,13 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
                 const int nc = min(kNC, n - i0);
                 if (multi) {
                     __syncthreads();
-                    if (threadIdx.x < nc) ssm[threadIdx.x] = wscale[(int64_t)(i0 + threadIdx.x) * tb.q + first];
+                    if (threadIdx.x < nc) ssm[threadIdx.x] = ld_cg_f32(wscale + (int64_t)(i0 + threadIdx.x) * tb.q + first);
                 } else {
                     __syncwarp();
                 }
                 for (int idx = lane; idx < nc * 4 * VPT; idx += 32) {
                     const int i = idx / (4 * VPT), wd = idx % (4 * VPT);
-                    wsm[warp][i][wd & 3][wd >> 2] = ld_ro_u32(wbits + (int64_t)(i0 + i) * wp + (wb >> 5) + wd);
+                    wsm[warp][i][wd & 3][wd >> 2] = ld_cg_u32(wbits + (int64_t)(i0 + i) * wp + (wb >> 5) + wd);
                 }
                 if (multi) __syncthreads(); else __syncwarp();
                 if constexpr (VPT == 2) {
@@ -669,8 +677,8 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
             const int r = find_segment(tb.off, first, last, j);
             float a = 0.0f;
             for (int i = 0; i < n; ++i) {
-                const uint32_t bit = (wbits[(int64_t)i * wp + (j >> 5)] >> (j & 31)) & 1u;
-                a = __fadd_rn(a, signed_scale(bit, wscale[(int64_t)i * tb.q + r]));
+                const uint32_t bit = (ld_cg_u32(wbits + (int64_t)i * wp + (j >> 5)) >> (j & 31)) & 1u;
+                a = __fadd_rn(a, signed_scale(bit, ld_cg_f32(wscale + (int64_t)i * tb.q + r)));
             }
             float hn;
             w = server_step<EF>(__fdiv_rn(a, fn), EF ? 0.0f : ghat_s[j], MODE == 2 ? 0.0f : gtil[j], hn);
@@ -719,20 +727,20 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
         float4 M = ld_rw4(m + j), V = ld_rw4(v + j);
         float4 Vh = ld_rw4(vhat + j), X = ld_rw4(x + j);
         grid_dep_wait();                                // server sign words, scales (and p) come from the kernels before
-        if (EF) Gt = ld_ro4(ghat_s + j);
-        const uint32_t nib = ld_ro_u32(sbits + (j >> 5)) >> (j & 31);
+        if (EF) Gt = ld_cg4(ghat_s + j);
+        const uint32_t nib = ld_cg_u32(sbits + (j >> 5)) >> (j & 31);
         const int first = tb.tile_first[T], last = tb.tile_last[T];
         float s0, s1, s2, s3;
-        s0 = s1 = s2 = s3 = __ldg(sscale + first);
+        s0 = s1 = s2 = s3 = ld_cg_f32(sscale + first);
         if (first != last) {                            // the tile spans several segments
             int r = find_segment(tb.off, first, last, j);
-            s0 = __ldg(sscale + r);
+            s0 = ld_cg_f32(sscale + r);
             while (r < last && j + 1 >= tb.off[r + 1]) ++r;
-            s1 = __ldg(sscale + r);
+            s1 = ld_cg_f32(sscale + r);
             while (r < last && j + 2 >= tb.off[r + 1]) ++r;
-            s2 = __ldg(sscale + r);
+            s2 = ld_cg_f32(sscale + r);
             while (r < last && j + 3 >= tb.off[r + 1]) ++r;
-            s3 = __ldg(sscale + r);
+            s3 = ld_cg_f32(sscale + r);
         }
         const float ex = update_step<MODE != 0>(Gt.x, Gt.x, signed_scale(nib & 1u, s0), Gt.x);
         const float ey = update_step<MODE != 0>(Gt.y, Gt.y, signed_scale(nib & 2u, s1), Gt.y);
@@ -753,10 +761,10 @@ k_update_sign(const uint32_t *__restrict__ sbits, const float *__restrict__ ssca
     grid_dep_wait();
     for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
         const int r = find_segment(tb.off, first, last, j);
-        const uint32_t bit = (sbits[j >> 5] >> (j & 31)) & 1u;
-        const float stored = MODE == 2 ? 0.0f : EF ? ghat_s[j] : gtil[j];
+        const uint32_t bit = (ld_cg_u32(sbits + (j >> 5)) >> (j & 31)) & 1u;
+        const float stored = MODE == 2 ? 0.0f : EF ? ld_cg_f32(ghat_s + j) : gtil[j];
         float gt;
-        const float est = update_step<MODE != 0>(stored, stored, signed_scale(bit, sscale[r]), gt);
+        const float est = update_step<MODE != 0>(stored, stored, signed_scale(bit, ld_cg_f32(sscale + r)), gt);
         if (MODE != 2) gtil[j] = gt;
         float mm = m[j], vv = v[j], vh = vhat[j], xx = x[j];
         amsgrad1(est, mm, vv, vh, xx, hp);
@@ -850,14 +858,14 @@ template <typename G>
 static void launch_worker_sign_t(const G *grads, float *ghat_w, uint32_t *wbits,
                                  const float *scale_old, dd *wpart, const Tables &tb, int n,
                                  int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
-                                 unsigned int *done, cudaStream_t st)
+                                 unsigned int *done, cudaStream_t st, int wait_limit)
 {
     dim3 grid((unsigned)tb.ntiles, (unsigned)n);
     if (vec_ok && tb.tile >= 4 * kSub) {
         auto kern = ef ? k_worker_sign_ring<true, G> : k_worker_sign_ring<false, G>;
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
         kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag,
-                                                   scale_new, done);
+                                                   scale_new, done, wait_limit);
     } else if (ef) {
         k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
                                                         scale_new, done);
@@ -870,14 +878,15 @@ static void launch_worker_sign_t(const G *grads, float *ghat_w, uint32_t *wbits,
 void launch_worker_sign(const void *grads, bool grads_bf16, float *ghat_w, uint32_t *wbits,
                         const float *scale_old, dd *wpart, const Tables &tb, int n,
                         int64_t wp, bool vec_ok, bool ef, int *error_flag, float *scale_new,
-                        unsigned int *done, cudaStream_t st)
+                        unsigned int *done, cudaStream_t st, int wait_limit)
 {
+    if (wait_limit < 0) wait_limit = kWaitLimit;
     if (grads_bf16)
         launch_worker_sign_t(static_cast<const bf16_t *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
-                             vec_ok, ef, error_flag, scale_new, done, st);
+                             vec_ok, ef, error_flag, scale_new, done, st, wait_limit);
     else
         launch_worker_sign_t(static_cast<const float *>(grads), ghat_w, wbits, scale_old, wpart, tb, n, wp,
-                             vec_ok, ef, error_flag, scale_new, done, st);
+                             vec_ok, ef, error_flag, scale_new, done, st, wait_limit);
 }
 
 void launch_finalize_scales(const dd *part, float *scales, const Tables &tb, int rows,

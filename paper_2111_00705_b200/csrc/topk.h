@@ -23,6 +23,17 @@ void topk_workspace_set_error_flag(TopkWorkspace *w, int *error_flag);
 // Which kernel makes the dense pass: 0 = chosen from the size (the default), 1 = the
 // prefetch-ring kernel wherever rows are 16-byte aligned, -1 = the plain kernel.
 void topk_workspace_set_ring(TopkWorkspace *w, int ring);
+// Deferred state update for topk_select(..., update_b = true): a row selected from the dense
+// pass's lists keeps b += u for the next selection, whose dense pass has the tiles of b in hand
+// and applies the previous payload first (one pass over b instead of k random read-modify-
+// writes per row).  Between selections b then lacks the last payload at those rows;
+// topk_flush(w, b) applies what is pending (before b is read by anyone else), and
+// topk_forget_pending drops it (when b is replaced from outside).
+void topk_workspace_set_defer(TopkWorkspace *w, bool on);
+void topk_flush(TopkWorkspace *w, float *b, cudaStream_t st);
+void topk_forget_pending(TopkWorkspace *w, cudaStream_t st);
+// Polls after which a bounded wait on an asynchronous copy gives up (< 0: the default).
+void topk_workspace_set_wait_limit(TopkWorkspace *w, int polls);
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val);
 int topk_launches_per_step(int n);
 // 1 or 2: kernels that make the dense pass of one selection in this workspace (rows aligned or not).

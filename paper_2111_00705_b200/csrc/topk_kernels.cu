@@ -70,6 +70,13 @@ struct TopkWorkspace {
     bool own_payload;
     int *error_flag;                  // device word set by a kernel whose bounded wait ran out (may be NULL)
     int ring;                         // dense pass with the prefetch ring: 0 = by size, 1 = wherever rows are aligned, -1 = never
+    int wait_limit;                   // polls before a wait on an asynchronous copy gives up
+    // Deferred state update (topk_workspace_set_defer): rows selected from lists do not get
+    // b += u at the kept coordinates at once; the next selection's dense pass, which has the
+    // tile of b in hand anyway, applies the previous payload first (pending[row] = 1 until
+    // then).  topk_flush applies what is pending.
+    bool defer;
+    uint32_t *pending;                // rows
 };
 
 __device__ __forceinline__ uint32_t key_of(float u) { return __float_as_uint(u) & 0x7fffffffu; }
@@ -298,25 +305,46 @@ __device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t fk) { return
 // from this histogram and the second dense pass is not needed; otherwise the two classic
 // passes run.  grid = (tiles, rows) for the tiles tile0, tile0 + 1, ... of every row.
 // ------------------------------------------------------------------------------------
-template <bool HAS_B>
+// The payload of the previous selection that is still to be applied to a row's tile
+// (deferred state update): entries [begin, end) of the row's payload arrays.
+struct Pending {
+    const uint32_t *pending;          // rows: 1 = the row's last payload is not in b yet
+    const uint32_t *idx;              // rows x k
+    const float *val;                 // rows x k
+    const uint32_t *tile_off;         // rows x nt4k: payload offset of every tile's first entry
+    int64_t k;
+};
+
+// APPLY: first add the previous payload's values to b at this tile's kept coordinates
+// (Algorithm 1: ghat^(i) += c^(i), deferred from the previous iteration), then read b through
+// the coherent path, since this block has just written to it.
+template <bool HAS_B, bool APPLY>
 __global__ void __launch_bounds__(kBlock)
-k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
+k_topk_spec(const float *__restrict__ a_all, float *b_all,
             const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
             float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
             uint32_t *__restrict__ stash_cnt_all, int64_t d, int vec_ok, int64_t stride, int64_t tile0,
-            int64_t nt4k)
+            int64_t nt4k, Pending pd)
 {
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
     const int row = blockIdx.y;
     const uint32_t fl = floor_bucket[row];
-    if (fl >= (uint32_t)kBins1) return;               // no guess for this row
+    if (fl >= (uint32_t)kBins1) return;               // no guess for this row (and then nothing pending)
     const uint32_t fk = fl << 20;                     // lowest key at or above the floor
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
-    __syncthreads();
     const float *a = a_all + (int64_t)row * stride;
-    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
+    float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     const int64_t tile = (int64_t)row * nt4k + tile0 + blockIdx.x;      // tiles tile0.. of the row
+    if (APPLY && pd.pending[row]) {
+        const int64_t t = tile0 + blockIdx.x;
+        const int64_t begin = pd.tile_off[tile], end = t + 1 < nt4k ? (int64_t)pd.tile_off[tile + 1] : pd.k;
+        for (int64_t e = begin + threadIdx.x; e < end; e += kBlock) {
+            const uint32_t j = pd.idx[(int64_t)row * pd.k + e];
+            if ((int64_t)j < d) b[j] = __fadd_rn(__ldcg(b + j), pd.val[(int64_t)row * pd.k + e]);
+        }
+    }
+    __syncthreads();
     float *stash = stash_all + tile * kStashCap;
     uint16_t *spos = stash_pos_all + tile * kStashCap;
     const int64_t base = (tile0 + blockIdx.x) * kSub;
@@ -337,7 +365,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
         for (int v = 0; v < 4; ++v) {
             const int64_t j = wb + v * 128 + lane * 4;
             A[v] = ld_ro4(a + j);
-            if (HAS_B) Bv[v] = ld_ro4(b + j);
+            if (HAS_B) Bv[v] = APPLY ? ld_cg4(b + j) : ld_ro4(b + j);
         }
         uint32_t FB[4];
 #pragma unroll
@@ -415,7 +443,7 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
         for (int64_t j0 = base; j0 < end; j0 += kBlock) {
             const int64_t j = j0 + threadIdx.x;
             const bool valid = j < end;
-            const float u = valid ? diff1<HAS_B>(a, b, j) : 0.0f;
+            const float u = !valid ? 0.0f : !HAS_B ? a[j] : __fsub_rn(a[j], APPLY ? __ldcg(b + j) : b[j]);
             const uint32_t key = key_of(u);
             const bool ge = valid && key >= fk;
             const uint32_t wg = __ballot_sync(kFull, ge);
@@ -453,13 +481,13 @@ k_topk_spec(const float *__restrict__ a_all, const float *__restrict__ b_all,
 constexpr int kSpecTiles = 8;
 constexpr int kSpecStages = 2;
 
-template <bool HAS_B>
+template <bool HAS_B, bool APPLY>
 __global__ void __launch_bounds__(kBlock, 3)
-k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_all,
+k_topk_spec_ring(const float *__restrict__ a_all, float *b_all,
                  const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
                  float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
                  uint32_t *__restrict__ stash_cnt_all, int64_t full_tiles, int64_t stride, int64_t nt4k,
-                 int *__restrict__ error_flag)
+                 int *__restrict__ error_flag, int wait_limit, Pending pd)
 {
     constexpr int kStageFloats = (HAS_B ? 2 : 1) * kSub;
     extern __shared__ __align__(128) unsigned char spec_ring[];
@@ -467,9 +495,10 @@ k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_al
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
     __shared__ uint16_t s_p[kBlock / 32][kWarpSpan / 4];
+    __shared__ uint32_t s_off[kSpecTiles + 1];        // APPLY: payload offsets of the block's tiles
     const int row = blockIdx.y;
     const uint32_t fl = floor_bucket[row];
-    if (fl >= (uint32_t)kBins1) return;               // no guess for this row
+    if (fl >= (uint32_t)kBins1) return;               // no guess for this row (and then nothing pending)
     const uint32_t fk = fl << 20;
     const float fkf = __uint_as_float(fk);
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
@@ -477,14 +506,31 @@ k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_al
         for (int st = 0; st < kSpecStages; ++st) mbar_init(&full[st], 1);
         mbar_fence_init();
     }
-    __syncthreads();
-    const float *a = a_all + (int64_t)row * stride;
-    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     const int64_t t0 = (int64_t)blockIdx.x * kSpecTiles;
     const int iters = (int)min((int64_t)kSpecTiles, full_tiles - t0);
+    const bool apply = APPLY && pd.pending[row] != 0u;                 // block-uniform
+    if (apply && threadIdx.x <= iters) {
+        const int64_t t = t0 + threadIdx.x;
+        s_off[threadIdx.x] = t < nt4k ? pd.tile_off[(int64_t)row * nt4k + t] : (uint32_t)pd.k;
+    }
+    __syncthreads();
+    const float *a = a_all + (int64_t)row * stride;
+    float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
+    const uint32_t *pidx = APPLY ? pd.idx + (int64_t)row * pd.k : nullptr;
+    const float *pval = APPLY ? pd.val + (int64_t)row * pd.k : nullptr;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
     float *ring = reinterpret_cast<float *>(spec_ring);
+    // the first payload entry of this thread in the coming tile, fetched one tile ahead
+    uint32_t nx_idx = 0u;
+    float nx_val = 0.0f;
+    auto prefetch_entry = [&](int it) {
+        if (apply && it < iters) {
+            const uint32_t e = s_off[it] + threadIdx.x;
+            if (e < s_off[it + 1]) { nx_idx = pidx[e]; nx_val = pval[e]; }
+        }
+    };
+    prefetch_entry(0);
     auto refill = [&](int it, int st) {                        // one thread
         float *dst = ring + (size_t)st * kStageFloats;
         mbar_arrive_expect_tx(&full[st], (uint32_t)(kStageFloats * sizeof(float)));
@@ -494,12 +540,41 @@ k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_al
     if (threadIdx.x == 0)
         for (int st = 0; st < kSpecStages && st < iters; ++st) refill(st, st);
     bool arrived = true;
-    for (int it = 0; it < iters; ++it) {
+    int it = 0;
+    for (; it < iters; ++it) {
         const int st = it % kSpecStages;
-        arrived = mbar_wait_bounded(&full[st], (uint32_t)(it / kSpecStages) & 1u);
-        if (!arrived) break;
+        const bool landed = mbar_wait_bounded(&full[st], (uint32_t)(it / kSpecStages) & 1u, wait_limit);
         const float *sa = ring + (size_t)st * kStageFloats;
-        const float *sb = sa + kSub;
+        float *sb = ring + (size_t)st * kStageFloats + kSub;
+        if (apply) {
+            // Deferred state update: the previous payload's entries of this tile are added to
+            // the copy of b in the stage, and every 32-byte sector that holds one is written
+            // back whole (all eight floats are at hand, so the store needs no read).
+            const uint32_t tbase = (uint32_t)((t0 + it) * kSub);
+            const uint32_t e0 = s_off[it], e1 = s_off[it + 1];
+            const uint32_t my_pos = nx_idx - tbase;
+            const bool mine = e0 + threadIdx.x < e1 && my_pos < (uint32_t)kSub;   // (a valid payload never fails the second test)
+            if (mine && landed) sb[my_pos] = __fadd_rn(sb[my_pos], nx_val);
+            for (uint32_t e = e0 + kBlock + threadIdx.x; e < e1 && landed; e += kBlock) {      // tiles that kept many
+                const uint32_t pos = pidx[e] - tbase;
+                if (pos < (uint32_t)kSub) sb[pos] = __fadd_rn(sb[pos], pval[e]);
+            }
+            __syncthreads();
+            float *bt = b + (int64_t)tbase;
+            if (mine && landed) {
+                const uint32_t sec = my_pos & ~7u;
+                st_rw4(bt + sec, *reinterpret_cast<const float4 *>(sb + sec));
+                st_rw4(bt + sec + 4, *reinterpret_cast<const float4 *>(sb + sec + 4));
+            }
+            for (uint32_t e = e0 + kBlock + threadIdx.x; e < e1 && landed; e += kBlock) {
+                const uint32_t sec = (pidx[e] - tbase) & ~7u;
+                if (sec < (uint32_t)kSub) {
+                    st_rw4(bt + sec, *reinterpret_cast<const float4 *>(sb + sec));
+                    st_rw4(bt + sec + 4, *reinterpret_cast<const float4 *>(sb + sec + 4));
+                }
+            }
+            prefetch_entry(it + 1);
+        }
         // u of the group of four coordinates at tile position p
         auto group = [&](uint32_t p) -> float4 {
             float4 U = *reinterpret_cast<const float4 *>(sa + p);
@@ -547,7 +622,11 @@ k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_al
             mine += __reduce_add_sync(kFull, (uint32_t)__popc(pm));
         }
         if (lane == 0) wcnt[warp] = mine;
-        __syncthreads();
+        // the barrier also makes the outcome of the waits one decision of the whole block (a
+        // thread whose wait ran out has worked on a stage that may be incomplete; everything
+        // it touched so far is indexed by positions, not by data, and the results are void)
+        arrived = !__syncthreads_or(!landed);
+        if (!arrived) break;
         uint32_t rank = 0, total = 0;
 #pragma unroll
         for (int w8 = 0; w8 < kBlock / 32; ++w8) {
@@ -574,14 +653,19 @@ k_topk_spec_ring(const float *__restrict__ a_all, const float *__restrict__ b_al
         }
         if (threadIdx.x == 0) stash_cnt_all[tile] = total;
         __syncthreads();                              // the stage and wcnt have been read by all
-        if (threadIdx.x == 0 && it + kSpecStages < iters) refill(it + kSpecStages, st);
+        if (threadIdx.x == 0 && it + kSpecStages < iters) {
+            // the stage was also written by this block (deferred update): order those writes
+            // before the asynchronous copy that refills it
+            if (APPLY) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            refill(it + kSpecStages, st);
+        }
     }
     if (!arrived) {
+        // report, let the copies in flight (tiles it .. it + kSpecStages - 1 of this block) land
+        // within the default limit before the shared memory is released, and leave together
         if (threadIdx.x == 0 && error_flag) atomicExch(error_flag, 1);
-        for (int st = 0; st < kSpecStages; ++st) {
-            mbar_wait_bounded(&full[st], 0u);
-            mbar_wait_bounded(&full[st], 1u);
-        }
+        for (int j = it; j < iters && j < it + kSpecStages; ++j)
+            mbar_wait_bounded(&full[j % kSpecStages], (uint32_t)(j / kSpecStages) & 1u);
         return;
     }
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
@@ -1106,11 +1190,16 @@ template <bool HAS_B, bool UPDATE_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
               const uint32_t *__restrict__ idx_all, float *__restrict__ val_all,
-              const uint32_t *__restrict__ have_val, int64_t d, int64_t k, int64_t stride)
+              const uint32_t *__restrict__ have_val, int64_t d, int64_t k, int64_t stride,
+              uint32_t *__restrict__ pending)
 {
     const int row = blockIdx.y;
     const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
-    if (t >= k) return;
+    // deferred state update: a row selected from lists (values already in the payload) keeps
+    // its update for the next selection's dense pass
+    const bool deferred = pending && have_val[row];
+    if (pending && t == 0) pending[row] = deferred ? 1u : 0u;
+    if (t >= k || deferred) return;
     const int64_t j = idx_all[(int64_t)row * k + t];
     if (j >= d) return;                       // caller-supplied sets are checked separately
     const float *a = a_all + (int64_t)row * stride;
@@ -1131,6 +1220,23 @@ k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
         u = a[j];
     }
     val_all[(int64_t)row * k + t] = u;
+}
+
+// Applies the payloads whose state update is still pending: b_j += u_j at the kept
+// coordinates of every row with pending[row] != 0.  grid = (ceil(k/256), rows).  The flags are
+// cleared by the caller afterwards.
+__global__ void __launch_bounds__(kBlock)
+k_topk_apply_pending(float *__restrict__ b_all, const uint32_t *__restrict__ idx_all,
+                     const float *__restrict__ val_all, const uint32_t *__restrict__ pending, int64_t d,
+                     int64_t k, int64_t stride)
+{
+    const int row = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t >= k || !pending[row]) return;
+    const int64_t j = idx_all[(int64_t)row * k + t];
+    if (j >= d) return;
+    float *b = b_all + (int64_t)row * stride;
+    b[j] = __fadd_rn(b[j], val_all[(int64_t)row * k + t]);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1270,6 +1376,7 @@ static void free_ws(TopkWorkspace *w)
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
     cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->stash);
     cudaFree(w->stash_pos); cudaFree(w->stash_cnt); cudaFree(w->cnt_gt); cudaFree(w->cnt_eq);
+    cudaFree(w->pending);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
 }
@@ -1286,6 +1393,7 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
     w->nbt = (w->wp + kTileWords - 1) / kTileWords;
     w->own_payload = idx == nullptr;
     w->idx = idx; w->val = val;
+    w->wait_limit = kWaitLimit;
     bool ok = true;
     auto get = [&](void **p, size_t bytes) {
         *p = nullptr;
@@ -1307,6 +1415,7 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         if (ok && cudaMemset(w->floor_bucket, 0xff, (size_t)rows * 4) != cudaSuccess) ok = false;   // no guess yet
         get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
         get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
+        get((void **)&w->pending, (size_t)rows * 4);
     }
     if (w->own_payload) {
         get((void **)&w->idx, (size_t)rows * k * 4);
@@ -1322,6 +1431,23 @@ void topk_workspace_destroy(TopkWorkspace *w) { if (w) free_ws(w); }
 void topk_workspace_set_error_flag(TopkWorkspace *w, int *error_flag) { if (w) w->error_flag = error_flag; }
 
 void topk_workspace_set_ring(TopkWorkspace *w, int ring) { if (w) w->ring = ring; }
+
+void topk_workspace_set_defer(TopkWorkspace *w, bool on) { if (w && w->pending) w->defer = on; }
+
+void topk_flush(TopkWorkspace *w, float *b, cudaStream_t st)
+{
+    if (!w || !w->defer) return;
+    const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+    k_topk_apply_pending<<<entries, kBlock, 0, st>>>(b, w->idx, w->val, w->pending, w->d, w->k, w->stride);
+    cudaMemsetAsync(w->pending, 0, (size_t)w->rows * 4, st);
+}
+
+void topk_forget_pending(TopkWorkspace *w, cudaStream_t st)
+{
+    if (w && w->defer) cudaMemsetAsync(w->pending, 0, (size_t)w->rows * 4, st);
+}
+
+void topk_workspace_set_wait_limit(TopkWorkspace *w, int polls) { if (w) w->wait_limit = polls < 0 ? kWaitLimit : polls; }
 
 void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float **val)
 {
@@ -1363,17 +1489,22 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // per SM (measured: 16 x 6250 tiles 0.50 -> 0.47 ms, 1 x 6250 tiles 0.039 -> 0.047 ms);
     // the ragged last tile, or everything else, through the plain kernel
     const int64_t full_tiles = ring_tiles(w, vec_ok);
+    // deferred state update: the dense pass first applies the previous selection's payload
+    const bool defer = HAS_B && update_b && w->defer;
+    const Pending pd = {w->pending, w->idx, w->val, w->cnt_gt, w->k};
     if (full_tiles > 0) {
         constexpr int kBytes = kSpecStages * (HAS_B ? 2 : 1) * kSub * (int)sizeof(float);
-        cudaFuncSetAttribute(k_topk_spec_ring<HAS_B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
+        auto kern = defer ? k_topk_spec_ring<HAS_B, HAS_B> : k_topk_spec_ring<HAS_B, false>;
+        cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kBytes);
         const dim3 groups((unsigned)((full_tiles + kSpecTiles - 1) / kSpecTiles), (unsigned)w->rows);
-        k_topk_spec_ring<HAS_B><<<groups, kBlock, kBytes, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt,
-                                                               full_tiles, w->stride, w->nt4k, w->error_flag);
+        kern<<<groups, kBlock, kBytes, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt,
+                                            full_tiles, w->stride, w->nt4k, w->error_flag, w->wait_limit, pd);
     }
     if (full_tiles < w->nt4k) {
         const dim3 rest((unsigned)(w->nt4k - full_tiles), (unsigned)w->rows);
-        k_topk_spec<HAS_B><<<rest, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok,
-                                                    w->stride, full_tiles, w->nt4k);
+        auto kern = defer ? k_topk_spec<HAS_B, HAS_B> : k_topk_spec<HAS_B, false>;
+        kern<<<rest, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok,
+                                     w->stride, full_tiles, w->nt4k, pd);
     }
     k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
     k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride);
@@ -1392,9 +1523,10 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride);
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
     if (HAS_B && update_b)
-        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride);
+        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride,
+                                                               defer ? w->pending : nullptr);
     else
-        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride);
+        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);
 }
 
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
@@ -1461,9 +1593,9 @@ void randk_set(TopkWorkspace *w, const uint32_t *sets, int *error_flag, cudaStre
 void randk_gather(TopkWorkspace *w, const float *a, float *b, bool update_b, cudaStream_t st)
 {
     const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
-    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride);
-    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride);
-    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, nullptr, w->d, w->k, w->stride);
+    if (b && update_b) k_topk_gather<true, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride, nullptr);
+    else if (b) k_topk_gather<true, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, nullptr, w->d, w->k, w->stride, nullptr);
+    else k_topk_gather<false, false><<<entries, kBlock, 0, st>>>(a, nullptr, w->idx, w->val, nullptr, w->d, w->k, w->stride, nullptr);
 }
 
 int topk_compress(const float *x, int64_t d, int64_t k, uint32_t *idx, float *val, cudaStream_t st)
