@@ -219,7 +219,8 @@ int cdadam_exchange_buffers(cdadam_ctx *ctx, uint32_t **worker_bits, float **wor
  * cdadam_create_range: d, n and the hyper-parameters as in cdadam_create, for the coordinates
  *   lo <= j < hi (0 <= lo < hi <= d), as range number `range` of `ranges` (ranges ordered by
  *   lo; the number only fixes the slot in the exchange buffers and the order of the sums).
- *   CDADAM_SIGN only (k is ignored).  All vectors of this context have hi - lo coordinates:
+ *   CDADAM_SIGN (k is ignored; described here) or CDADAM_TOPK (described below).  All vectors
+ *   of this context have hi - lo coordinates:
  *   gradients are n x (hi - lo), cdadam_get_state / cdadam_set_state / cdadam_params move
  *   (hi - lo)-vectors, cdadam_last_payload gives the hi - lo sign bits (bit 0 = coordinate lo)
  *   and one scale per segment that meets the range.  cdadam_set_segments takes the segments
@@ -241,6 +242,35 @@ int cdadam_exchange_buffers(cdadam_ctx *ctx, uint32_t **worker_bits, float **wor
  *   local one is.  The pointers change when cdadam_set_segments or cdadam_set_tile is called.
  *   Any output pointer may be NULL.
  */
+/*
+ * With CDADAM_TOPK (Appendix A, "Top-k": the k coordinates of largest magnitude of the WHOLE
+ * vector) the one thing that crosses the ranges is the threshold: the k-th largest magnitude
+ * and, among the coordinates equal to it, which are kept (the lower coordinates first, i.e.
+ * the ranges in their order).  The selection is the exact three-level radix select of the
+ * one-GPU path without its threshold guess, cut at every point where it needs a sum over the
+ * whole vector: the histogram of each level is summed over the ranges (integer sums: order
+ * does not matter) before the bucket is picked, and the ties are given out in range order.
+ *
+ * cdadam_create_range(..., CDADAM_TOPK, k, ...): k = entries kept in the whole vector,
+ *   1 <= k <= d, at the workers and at the server (Algorithm 1 only).
+ * cdadam_range_topk(ctx, stage, grads, stream): stages 0..9 of one iteration, in order:
+ *   0..4 the workers' selection on g^(i) - ghat^(i) restricted to the range and
+ *        ghat^(i) += c^(i) (grads: device, n x (hi - lo), needed by all five);
+ *   5..9 the server: ghat += mean of the workers' messages (stage 5), the selection on
+ *        ghat - gtil, gtil += c, and AMSGrad on the range (stage 9).  grads may be NULL.
+ * cdadam_range_topk_buffer(ctx, stage, &buffer, &words): after every stage except 4 and 9
+ *   the caller gathers the stage's exchange buffer: `ranges` slots of `words` uint32 each
+ *   (n x 2048 after stages 0..3, 2048 after stages 5..8); the stage wrote slot `range`,
+ *   the next stage reads all slots (an in-place all-gather, as for the l1 parts).  After
+ *   stages 4 and 9 *buffer is NULL and *words 0.
+ * cdadam_last_payload on such a context: *count = min(k, hi - lo) entries per message, of
+ *   which the range's own kept coordinates come first (increasing, relative to lo) and the
+ *   rest carry the coordinate 0xffffffff and the value 0; over all ranges the entries that
+ *   are not so marked are the k of the whole vector.
+ */
+int cdadam_range_topk(cdadam_ctx *ctx, int stage, const float *grads, void *stream);
+int cdadam_range_topk_buffer(cdadam_ctx *ctx, int stage, uint32_t **buffer, int64_t *words_per_range);
+
 cdadam_ctx *cdadam_create_range(int64_t d, int n, int64_t lo, int64_t hi, int range, int ranges,
                                 int compressor, int64_t k,
                                 float beta1, float beta2, float lr, float eps);

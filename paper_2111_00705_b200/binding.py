@@ -42,6 +42,8 @@ _SIGNATURES = {
     "cdadam_range_buffers": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p),
                                         _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int64), _c.POINTER(_c.c_int),
                                         _c.POINTER(_c.c_void_p)]),
+    "cdadam_range_topk": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_void_p]),
+    "cdadam_range_topk_buffer": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_int64)]),
     "cdadam_params": (_c.c_void_p, [_c.c_void_p]),
     "cdadam_set_params": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_void_p]),
     "cdadam_set_segments": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64)]),
@@ -367,15 +369,32 @@ class CDAdamRange(CDAdam):
     (see ``distributed.py``)."""
 
     def __init__(self, d, n, lo, hi, rank, ranks, beta1=0.9, beta2=0.999, lr=1e-3, eps=1e-8,
-                 offsets=None, x0=None, device=None, mode=MARKOV):
+                 offsets=None, x0=None, device=None, mode=MARKOV, compressor=SIGN, k=0):
         self._range = (int(d), int(lo), int(hi), int(rank), int(ranks))
         self.dim, self.lo, self.hi, self.rank, self.ranks = self._range
         self.q_all = 1 if offsets is None else len(offsets) - 1
-        super().__init__(hi - lo, n, SIGN, 0, beta1, beta2, lr, eps, offsets, x0, device, mode)
+        self.k_all = int(k)                 # top-k: entries kept in the whole vector
+        super().__init__(hi - lo, n, compressor, min(int(k), hi - lo), beta1, beta2, lr, eps, offsets, x0, device, mode)
 
     def _create(self, beta1, beta2, lr, eps):
         d, lo, hi, rank, ranks = self._range
-        return lib().cdadam_create_range(d, self.n, lo, hi, rank, ranks, SIGN, 0, beta1, beta2, lr, eps)
+        return lib().cdadam_create_range(d, self.n, lo, hi, rank, ranks, self.compressor, self.k_all,
+                                         beta1, beta2, lr, eps)
+
+    TOPK_STAGES = 10
+
+    def range_topk(self, stage, grads=None, stream=None):
+        """Stage 0..9 of a top-k iteration on the range (0..4 take the n x (hi - lo) gradients)."""
+        g = None if grads is None else _dev_f32(grads, self.n * self.d, "grads")
+        _check(lib().cdadam_range_topk(self._h, int(stage), g, _stream(stream)))
+
+    def range_topk_buffer(self, stage):
+        """The exchange buffer to gather after `stage` as an int32[ranks, words] view, or None."""
+        buf, words = ctypes.c_void_p(), ctypes.c_int64()
+        _check(lib().cdadam_range_topk_buffer(self._h, int(stage), ctypes.byref(buf), ctypes.byref(words)))
+        if not buf.value:
+            return None
+        return _view(buf.value, self.ranks * words.value, torch.int32, self.device).view(self.ranks, words.value)
 
     def set_segments(self, offsets):
         super().set_segments(offsets)

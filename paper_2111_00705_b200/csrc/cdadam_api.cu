@@ -147,6 +147,8 @@ struct cdadam_ctx {
     int32_t *rs_gidx = nullptr;               // q_loc (device)
     int64_t *rs_glen = nullptr;               // q_loc (device)
     std::vector<int64_t> range_off_all;       // the whole problem's q_all + 1 segment offsets
+    int64_t range_k = 0;                      // top-k: entries kept in the WHOLE vector
+    uint32_t *rx_w = nullptr, *rx_s = nullptr;   // top-k exchange buffers: range_count x (n | 1) x 2048 words
     int tile_override = 0;  // 0 = choose from d and q
     int mode = CDADAM_MARKOV;
     Hyper hp{};
@@ -437,9 +439,8 @@ void enqueue_topk_step(cdadam_ctx *c, const void *grads_in, bool, bool vec, cuda
     }
     topk_select(c->tk_w, grads, c->ghat_w, true, vec, st);            // workers: compress, update ghat^(i)
     prof_mark(c, st);
-    topk_aggregate(c->tk_w, c->ghat_s, c->n, st);                      // server: ghat += mean
-    prof_mark(c, st);
-    topk_select(c->tk_s, c->ghat_s, c->gtil, true, svec, st);          // server: compress, update gtil
+    prof_mark(c, st);                                                  // (the aggregation runs inside the server's dense pass)
+    topk_select_aggregated(c->tk_s, c->tk_w, c->ghat_s, c->gtil, c->n, svec, st);   // server: ghat += mean; compress, update gtil
     prof_mark(c, st);
     launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
     prof_mark(c, st);
@@ -584,20 +585,32 @@ cdadam_ctx *cdadam_create_shard(int64_t d, int n, int first_worker, int n_local,
 cdadam_ctx *cdadam_create_range(int64_t d, int n, int64_t lo, int64_t hi, int range, int ranges, int compressor,
                                 int64_t k, float beta1, float beta2, float lr, float eps)
 {
-    (void)k;
-    if (compressor != CDADAM_SIGN) {
-        fail(CDADAM_ERR_ARG, "the coordinate-sharded iteration takes the scaled-sign compressor");
+    if (compressor != CDADAM_SIGN && compressor != CDADAM_TOPK) {
+        fail(CDADAM_ERR_ARG, "the coordinate-sharded iteration takes the scaled-sign or the top-k compressor");
         return nullptr;
     }
     if (d < 1 || d >= ((int64_t)1 << 32)) { fail(CDADAM_ERR_ARG, "d must be in [1, 2^32)"); return nullptr; }
     if (lo < 0 || hi <= lo || hi > d) { fail(CDADAM_ERR_ARG, "the range [lo, hi) must be non-empty and lie in [0, d)"); return nullptr; }
     if (ranges < 1 || ranges > 4096 || range < 0 || range >= ranges) { fail(CDADAM_ERR_ARG, "range number must be in [0, ranges), ranges in [1, 4096]"); return nullptr; }
-    cdadam_ctx *c = create_impl(hi - lo, n, 0, n, compressor, 0, beta1, beta2, lr, eps);
+    if (compressor == CDADAM_TOPK && (k < 1 || k > d)) { fail(CDADAM_ERR_ARG, "top-k needs 1 <= k <= d"); return nullptr; }
+    // a payload row of this range holds at most min(k, hi - lo) entries
+    cdadam_ctx *c = create_impl(hi - lo, n, 0, n, compressor, compressor == CDADAM_TOPK ? std::min(k, hi - lo) : 0,
+                                beta1, beta2, lr, eps);
     if (!c) return nullptr;
     c->is_range = true;
     c->range_lo = lo; c->range_dim = d; c->range_rank = range; c->range_count = ranges;
-    const int64_t flat[2] = {0, d};
-    if (cdadam_set_segments(c, 1, flat) != CDADAM_OK) { cdadam_destroy(c); return nullptr; }
+    if (compressor == CDADAM_SIGN) {
+        const int64_t flat[2] = {0, d};
+        if (cdadam_set_segments(c, 1, flat) != CDADAM_OK) { cdadam_destroy(c); return nullptr; }
+        return c;
+    }
+    c->range_k = k;
+    topk_workspace_set_defer(c->tk_w, false);          // the staged selection updates ghat^(i) at once
+    const size_t per = (size_t)topk_range_exchange_words(c->tk_s);
+    if (dev_zalloc(&c->rx_w, (size_t)ranges * n * per) || dev_zalloc(&c->rx_s, (size_t)ranges * per)) {
+        cdadam_destroy(c);
+        return nullptr;
+    }
     return c;
 }
 
@@ -611,6 +624,7 @@ void cdadam_destroy(cdadam_ctx *c)
     cudaFree(c->wbits); cudaFree(c->sbits); cudaFree(c->error_flag);
     cudaFree(c->pay_idx); cudaFree(c->pay_val);
     cudaFree(c->rs_w); cudaFree(c->rs_s); cudaFree(c->rs_gidx); cudaFree(c->rs_glen);
+    cudaFree(c->rx_w); cudaFree(c->rx_s);
     cudaFree(c->wscale[0]); cudaFree(c->wscale[1]); cudaFree(c->sscale); cudaFree(c->zero_scale);
     cudaFree(c->wpart); cudaFree(c->spart); cudaFree(c->stage);
     cudaFree(c->wdone); cudaFree(c->sdone); cudaFree(c->wsums); cudaFree(c->ssums);
@@ -896,6 +910,7 @@ static int range_ok(cdadam_ctx *c, const char *what)
 {
     if (!c) return fail(CDADAM_ERR_ARG, "%s: NULL context", what);
     if (!c->is_range) return fail(CDADAM_ERR_STATE, "%s: the context was not made by cdadam_create_range", what);
+    if (c->comp != CDADAM_SIGN) return fail(CDADAM_ERR_STATE, "%s: scaled sign only; a top-k range context runs cdadam_range_topk", what);
     if (c->mode == CDADAM_NAIVE) return fail(CDADAM_ERR_STATE, "%s: Algorithm 1 and the error-feedback mode only", what);
     if (c->prof_on) return fail(CDADAM_ERR_STATE, "%s: per-stage timing covers cdadam_step only", what);
     return CDADAM_OK;
@@ -970,6 +985,51 @@ int cdadam_range_buffers(cdadam_ctx *c, double **worker_sums, double **server_su
     return CDADAM_OK;
 }
 
+int cdadam_range_topk(cdadam_ctx *c, int stage, const float *grads, void *stream)
+{
+    if (!c) return fail(CDADAM_ERR_ARG, "cdadam_range_topk: NULL context");
+    if (!c->is_range || c->comp != CDADAM_TOPK) return fail(CDADAM_ERR_STATE, "cdadam_range_topk: the context was not made by cdadam_create_range with CDADAM_TOPK");
+    if (c->mode != CDADAM_MARKOV) return fail(CDADAM_ERR_STATE, "cdadam_range_topk: Algorithm 1 only");
+    if (stage < 0 || stage > 9) return fail(CDADAM_ERR_ARG, "cdadam_range_topk: stages are 0..9");
+    if (stage != c->phase) return fail(CDADAM_ERR_STATE, "cdadam_range_topk: stage %d is next", c->phase);
+    if (stage <= 4 && !grads) return fail(CDADAM_ERR_ARG, "cdadam_range_topk: the worker stages 0..4 take the gradients");
+    if (c->prof_on) return fail(CDADAM_ERR_STATE, "cdadam_range_topk: per-stage timing covers cdadam_step only");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (int rc = refuse_capture(st)) return rc;
+    if (stage == 0) step_size_of_this_step(c);
+    const bool svec = c->d % 4 == 0;
+    if (stage <= 4) {                                  // workers: c^(i) = C(g^(i) - ghat^(i)); ghat^(i) += c^(i)
+        topk_range_stage(c->tk_w, stage, grads, c->ghat_w, aligned16(grads) && svec, c->range_k, c->rx_w,
+                         c->range_rank, c->range_count, st);
+    } else {                                           // server: ghat += mean; c = C(ghat - gtil); gtil += c
+        if (stage == 5) {
+            const uint32_t *widx; const float *wval;
+            topk_payload(c->tk_w, 0, &widx, &wval);
+            topk_aggregate_rows(widx, wval, c->k, c->d, c->n, c->ghat_s, st);
+        }
+        topk_range_stage(c->tk_s, stage - 5, c->ghat_s, c->gtil, svec, c->range_k, c->rx_s, c->range_rank,
+                         c->range_count, st);
+        if (stage == 9) launch_amsgrad(c->gtil, c->m, c->v, c->vhat, c->x, c->d, c->hp, svec, st);
+    }
+    if (int rc = check_launch("cdadam_range_topk")) return rc;
+    c->phase = stage == 9 ? 0 : stage + 1;
+    if (stage == 9) c->steps += 1;
+    return CDADAM_OK;
+}
+
+int cdadam_range_topk_buffer(cdadam_ctx *c, int stage, uint32_t **buffer, int64_t *words_per_range)
+{
+    if (!c || !buffer || !words_per_range) return fail(CDADAM_ERR_ARG, "cdadam_range_topk_buffer: NULL argument");
+    if (!c->is_range || c->comp != CDADAM_TOPK) return fail(CDADAM_ERR_STATE, "cdadam_range_topk_buffer: the context was not made by cdadam_create_range with CDADAM_TOPK");
+    if (stage < 0 || stage > 9) return fail(CDADAM_ERR_ARG, "cdadam_range_topk_buffer: stages are 0..9");
+    const int64_t per = topk_range_exchange_words(c->tk_s);
+    if (stage == 4 || stage == 9) { *buffer = nullptr; *words_per_range = 0; }      // nothing to exchange after these
+    else if (stage < 4) { *buffer = c->rx_w; *words_per_range = (int64_t)c->n * per; }
+    else { *buffer = c->rx_s; *words_per_range = per; }
+    return CDADAM_OK;
+}
+
 int cdadam_step_bf16(cdadam_ctx *c, const void *grads, void *stream) { return step_impl(c, grads, true, stream); }
 
 int cdadam_step_host(cdadam_ctx *c, const float *grads_host, float *x_out_host, void *stream)
@@ -1001,6 +1061,7 @@ int cdadam_set_topk_segments(cdadam_ctx *c, int q, const int64_t *offsets, const
 {
     if (!c || !offsets || !k_per_segment) return fail(CDADAM_ERR_ARG, "cdadam_set_topk_segments: NULL argument");
     if (c->comp != CDADAM_TOPK) return fail(CDADAM_ERR_STATE, "top-k segments apply to the top-k compressor only");
+    if (c->is_range) return fail(CDADAM_ERR_STATE, "top-k segments are not available on a coordinate range");
     if (c->mode != CDADAM_MARKOV) return fail(CDADAM_ERR_STATE, "top-k segments are available for Algorithm 1 only");
     if (c->steps != 0 || c->phase != 0) return fail(CDADAM_ERR_STATE, "segments must be set before the first step");
     if (q < 1 || (int64_t)q > c->d) return fail(CDADAM_ERR_ARG, "q must be in [1, d]");
@@ -1256,13 +1317,20 @@ int cdadam_device_status(cdadam_ctx *c, void *stream)
 int cdadam_launches_per_step(cdadam_ctx *c)
 {
     if (!c) return 0;
+    if (c->is_range && c->comp == CDADAM_TOPK) return 46;    // two staged selections of 22, aggregation, AMSGrad
     if (c->is_range) return 7;      // worker pass, sums | scales, server pass, sums | scales, update
     if (c->comp == CDADAM_SIGN) return c->fuse_finish && c->mode != CDADAM_NAIVE ? 3 : 5;
-    if (c->comp == CDADAM_TOPK && !c->seg_w.empty())
-        return (int)c->seg_w.size() * (topk_launches_per_step(c->n) + 1) + 2;
-    if (c->comp == CDADAM_TOPK)     // (for gradient rows that are 16-byte aligned)
-        return topk_launches_per_step(c->n) + 1 + (c->mode == CDADAM_EF ? 5 : c->mode == CDADAM_NAIVE ? 3 : 0) +
-               topk_dense_launches(c->tk_w, c->d % 4 == 0) - 1 + topk_dense_launches(c->tk_s, c->d % 4 == 0) - 1;
+    if (c->comp == CDADAM_TOPK && !c->seg_w.empty())     // per segment: two selections and two payload copies
+        return (int)c->seg_w.size() * (topk_launches_per_step(c->n) + 2) + 2;
+    if (c->comp == CDADAM_TOPK) {   // (for gradient rows that are 16-byte aligned)
+        // Algorithm 1: two selections (the server's with the aggregation inside its dense pass,
+        // which is then one plain kernel) and AMSGrad; the comparison modes: a separate
+        // aggregation kernel and their dense helpers
+        const int workers_dense = topk_dense_launches(c->tk_w, c->d % 4 == 0) - 1;
+        if (c->mode == CDADAM_MARKOV) return topk_launches_per_step(c->n) + 1 + workers_dense;
+        return topk_launches_per_step(c->n) + 2 + (c->mode == CDADAM_EF ? 5 : 3) + workers_dense +
+               topk_dense_launches(c->tk_s, c->d % 4 == 0) - 1;
+    }
     if (c->comp == CDADAM_RANDK) return c->mode == CDADAM_EF ? 9 : c->mode == CDADAM_NAIVE ? 7 : 4;
     return 1;
 }

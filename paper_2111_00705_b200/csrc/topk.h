@@ -45,6 +45,27 @@ int topk_dense_launches(const TopkWorkspace *w, bool vec_ok);
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                  cudaStream_t st);
 
+// The server stage of Algorithm 1 in one selection: ghat_s += mean of the n payloads held in
+// `ww` (workers added in the order 0..n-1, as topk_aggregate does), then the selection of
+// ws (one row) on ghat_s - gtil with gtil updated at the kept coordinates.  The aggregation
+// runs inside the dense pass of the selection, tile by tile.  ww and ws: same d, ws->rows == 1,
+// ww selected by topk_select (its per-tile payload offsets are used where a row has them).
+void topk_select_aggregated(TopkWorkspace *ws, TopkWorkspace *ww, float *ghat_s, float *gtil, int n, bool vec_ok,
+                            cudaStream_t st);
+
+// Coordinate-sharded selection: the workspace holds the coordinates of one range of every
+// row; `ranges` such workspaces select the k_all largest of the whole rows between them.  One
+// selection is the stages 0..4 in order; after each of the stages 0..3 the caller gathers
+// the slots of all ranges in the exchange buffer (ranges x topk_range_exchange_words(w)
+// uint32; stage s writes slot `range`, stage s + 1 reads all slots).  After stage 4 the
+// payload rows hold this range's kept coordinates (increasing, relative to the range) and
+// values, the rest of each row marked with the coordinate 0xffffffff; b (if given) is
+// updated at the kept coordinates.  The workspace's k is the capacity of a payload row
+// (min(k_all, d) is enough).  No threshold guess is used: two dense passes per selection.
+void topk_range_stage(TopkWorkspace *w, int stage, const float *a, float *b, bool vec_ok, int64_t k_all,
+                      uint32_t *exchange, int range, int ranges, cudaStream_t st);
+int64_t topk_range_exchange_words(const TopkWorkspace *w);
+
 // Top-k per segment: copies the payload of `seg` (a segment starting at coordinate `offset` of
 // the whole vector) into entries [at, at + seg.k) of every row of `whole`'s payload, indices
 // moved by `offset`.

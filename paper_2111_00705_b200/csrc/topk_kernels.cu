@@ -61,6 +61,7 @@ struct TopkWorkspace {
     uint16_t *stash_pos;              // rows x nt4k x kStashCap: positions inside the tile
     uint32_t *stash_cnt;              // rows x nt4k: list lengths; above kStashCap the tile kept no
                                       // complete list and the later passes read it from a and b
+    uint16_t *cand;                   // rows x nt4k x 4: low key bits of a tile's first candidates (k_topk_split)
     uint32_t *cnt_gt, *cnt_eq;        // rows x nt4k: per tile, keys above / equal to the threshold;
                                       // after the scans: payload offset / tie rank of the tile
     int64_t nt4k;                     // ceil(d / 4096)
@@ -77,6 +78,11 @@ struct TopkWorkspace {
     // then).  topk_flush applies what is pending.
     bool defer;
     uint32_t *pending;                // rows
+    // the chain of kernels for the rows whose guess failed runs beside the chain for the rows
+    // selected from lists: a second stream, forked and joined with events inside topk_select
+    cudaStream_t side;
+    cudaEvent_t ev_fork, ev_join;
+    unsigned int *tick;               // 5 x rows ticket counters of that chain's passes (zero between uses)
 };
 
 __device__ __forceinline__ uint32_t key_of(float u) { return __float_as_uint(u) & 0x7fffffffu; }
@@ -113,12 +119,97 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
 }
 
 // ------------------------------------------------------------------------------------
+// Pick the bucket that holds the `want`-th largest entry of a row's histogram: the bucket b
+// with count(bins > b) < want <= count(bins >= b).  Run by one whole block for the row.
+// level 0/1/2 selects which histogram and which fields of Sel are read and written.
+// ------------------------------------------------------------------------------------
+__device__ __forceinline__ void pick_row(const uint32_t *hist_row, Sel *sel, int level, uint32_t k,
+                                         uint32_t *floor_bucket_row)
+{
+    __shared__ uint32_t tot[kBlock];
+    const int nb = level == 2 ? kBins3 : kBins1;
+    const uint32_t *hist = hist_row + (level == 0 ? 0 : level == 1 ? kBins1 : kBins1 + kBins2);
+    const uint32_t want = level == 0 ? k : level == 1 ? sel->k1 : sel->k2;
+    const int per = nb / kBlock;                    // 8 or 2 contiguous bins per thread
+    const int lo = threadIdx.x * per;
+    uint32_t mine = 0;
+    for (int t = 0; t < per; ++t) mine += __ldcg(hist + lo + t);
+    __syncthreads();                                // tot may still be read by an earlier call
+    tot[threadIdx.x] = mine;
+    __syncthreads();
+    uint32_t above = 0;                             // entries in bins owned by later threads
+    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+    for (int t = per - 1; t >= 0; --t) {
+        const uint32_t c = __ldcg(hist + lo + t);
+        if (above < want && above + c >= want) {
+            const uint32_t bucket = lo + t, rem = want - above;
+            if (level == 0) { sel->b1 = bucket; sel->k1 = rem; sel->c1 = c; }
+            else if (level == 1) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
+            else {
+                sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
+                // guess for the next selection of this row: below this threshold, one bucket
+                // more than after a guess that held
+                *floor_bucket_row = sel->b1 > kGuessMargin + 1u ? sel->b1 - (kGuessMargin + 1u) : 1u;
+            }
+        }
+        above += c;
+    }
+}
+
+// True, for all threads of the block, in the block that is the last of `count` blocks to get
+// here (the others' global writes before their call are then visible to it).  The counter
+// goes back to zero.  No block waits for another.  Used by the passes of the rows whose guess
+// failed, so that a row's pick or scan needs no launch of its own; those passes are rare and
+// short of memory traffic, so the fence costs nothing that matters (in the dense pass of the
+// common path it did: see pick_spec_row).
+__device__ __forceinline__ bool last_block_of_row(unsigned int *counter, unsigned int count)
+{
+    __shared__ int s_is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s_is_last = atomicAdd(counter, 1u) == count - 1u;
+        if (s_is_last) *counter = 0u;
+    }
+    __syncthreads();
+    const bool last = s_is_last != 0;
+    if (last) __threadfence();
+    return last;
+}
+
+// Exclusive scan of a row's nbt counts (in place, or only the total), by one whole block.
+__device__ __forceinline__ void scan_row(uint32_t *cnt, int64_t nbt, uint32_t *total_out, bool in_place)
+{
+    uint32_t carry = 0;
+    for (int64_t c = 0; c < nbt; c += kBlock) {
+        const int64_t t = c + threadIdx.x;
+        const uint32_t v = t < nbt ? __ldcg(cnt + t) : 0u;
+        uint32_t total;
+        const uint32_t ex = block_excl_scan(v, total);
+        if (in_place && t < nbt) cnt[t] = carry + ex;
+        carry += total;
+    }
+    if (total_out && threadIdx.x == 0) *total_out = carry;           // the row's sum (block-uniform)
+}
+
+// Tail of the classic passes when they run as one chain of launches (topk_select): what a
+// row needs next is done by the block that finishes the row last.  tick == NULL: no tail
+// (the coordinate-sharded selection picks after the histograms have been exchanged).
+struct RowTail {
+    unsigned int *tick;               // rows counters of this pass, or NULL
+    Sel *sel;
+    uint32_t *floor_bucket;
+    uint32_t k;
+};
+
+// ------------------------------------------------------------------------------------
 // Level 1: histogram of key >> 20 over all coordinates.  grid = (ceil(d/4096), rows).
 // ------------------------------------------------------------------------------------
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
-             uint32_t *__restrict__ hist_all, const uint32_t *__restrict__ hit, int64_t d, int vec_ok, int64_t stride)
+             uint32_t *__restrict__ hist_all, const uint32_t *__restrict__ hit, int64_t d, int vec_ok, int64_t stride,
+             RowTail tail)
 {
     __shared__ uint32_t h[kBins1];
     if (hit[blockIdx.y]) return;                      // the guessed bucket held: nothing to redo
@@ -160,6 +251,8 @@ k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
     uint32_t *hist = hist_all + (int64_t)row * kHistStride;
     for (int t = threadIdx.x; t < kBins1; t += kBlock)
         if (h[t]) atomicAdd(&hist[t], h[t]);
+    if (tail.tick && last_block_of_row(tail.tick + row, gridDim.x))
+        pick_row(hist, tail.sel + row, 0, tail.k, tail.floor_bucket + row);
 }
 
 // ------------------------------------------------------------------------------------
@@ -167,49 +260,18 @@ k_topk_hist1(const float *__restrict__ a_all, const float *__restrict__ b_all,
 // count(bins > b) < want <= count(bins >= b).  grid = (rows), one block.
 // level 0/1/2 selects which histogram and which fields of Sel are read and written.
 // ------------------------------------------------------------------------------------
+// Which rows a launch of the ordered compaction takes: the rows selected from the dense pass's
+// lists (the guess held) and the rows that go through the classic passes are handled by two
+// chains of kernels that run side by side.
+enum { kRowsListed = 1, kRowsClassic = 2 };
+
 __global__ void __launch_bounds__(kBlock)
 k_topk_pick(const uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, int level,
             uint32_t k, const uint32_t *__restrict__ hit, uint32_t *__restrict__ floor_bucket)
 {
-    __shared__ uint32_t tot[kBlock];
     const int row = blockIdx.x;
-    const bool listed = hit[row] != 0u;               // the guess held: two levels, 20 + 11 key bits
-    if (listed && level != 1) return;
-    Sel *sel = sel_all + row;
-    const int nb = level == 2 ? kBins3 : kBins1;
-    const uint32_t *hist = hist_all + (int64_t)row * kHistStride +
-                           (level == 0 ? 0 : level == 1 ? kBins1 : kBins1 + kBins2);
-    const uint32_t want = level == 0 ? k : level == 1 ? sel->k1 : sel->k2;
-    const int per = nb / kBlock;                    // 8 or 2 contiguous bins per thread
-    const int lo = threadIdx.x * per;
-    uint32_t mine = 0;
-    for (int t = 0; t < per; ++t) mine += hist[lo + t];
-    tot[threadIdx.x] = mine;
-    __syncthreads();
-    uint32_t above = 0;                             // entries in bins owned by later threads
-    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
-    for (int t = per - 1; t >= 0; --t) {
-        const uint32_t c = hist[lo + t];
-        if (above < want && above + c >= want) {
-            const uint32_t bucket = lo + t, rem = want - above;
-            if (level == 0) { sel->b1 = bucket; sel->k1 = rem; sel->c1 = c; }
-            else if (level == 1 && !listed) { sel->b2 = bucket; sel->k2 = rem; sel->c2 = c; }
-            else {
-                if (listed) {                        // T = prefix | bits 10..0, in the three-level layout
-                    const uint32_t T = sel->pre | bucket;
-                    sel->b1 = T >> 20; sel->b2 = (T >> 9) & (kBins2 - 1); sel->b3 = T & (kBins3 - 1);
-                    sel->k3 = rem; sel->c3 = c;
-                } else {
-                    sel->b3 = bucket; sel->k3 = rem; sel->c3 = c;
-                }
-                // guess for the next selection of this row: a little below this threshold,
-                // one bucket more after a guess that failed
-                const uint32_t margin = listed ? kGuessMargin : kGuessMargin + 1u;
-                floor_bucket[row] = sel->b1 > margin ? sel->b1 - margin : 1u;
-            }
-        }
-        above += c;
-    }
+    if (hit[row]) return;                             // rows selected from lists pick inside k_scan_lists
+    pick_row(hist_all + (int64_t)row * kHistStride, sel_all + row, level, k, floor_bucket + row);
 }
 
 // ------------------------------------------------------------------------------------
@@ -222,7 +284,7 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
             const Sel *__restrict__ sel_all, uint32_t *__restrict__ bm_in_all,
             uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all,
-            const uint32_t *__restrict__ hit, int64_t d, int64_t wp, int vec_ok, int64_t stride)
+            const uint32_t *__restrict__ hit, int64_t d, int64_t wp, int vec_ok, int64_t stride, RowTail tail)
 {
     __shared__ uint32_t h[kBins2];
     if (hit[blockIdx.y]) return;
@@ -287,6 +349,8 @@ k_topk_mark(const float *__restrict__ a_all, const float *__restrict__ b_all,
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
     for (int t = threadIdx.x; t < kBins2; t += kBlock)
         if (h[t]) atomicAdd(&hist[t], h[t]);
+    if (tail.tick && last_block_of_row(tail.tick + row, gridDim.x))
+        pick_row(hist_all + (int64_t)row * kHistStride, const_cast<Sel *>(sel_all) + row, 1, 0u, tail.floor_bucket + row);
 }
 
 // Bin of a key at or above the floor key fk in the speculative pass: 2^11 keys per bin
@@ -305,6 +369,81 @@ __device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t fk) { return
 // from this histogram and the second dense pass is not needed; otherwise the two classic
 // passes run.  grid = (tiles, rows) for the tiles tile0, tile0 + 1, ... of every row.
 // ------------------------------------------------------------------------------------
+// Did the guess hold?  It did if the k-th largest key lies in one of the regular fine bins
+// above the floor; then key bits 30..11 of the threshold follow from the histogram of those
+// coordinates.  Otherwise the row's level-1 histogram is cleared for the full pass.  Run by
+// one whole block for the row.  (Folding this into the dense pass - the block that finishes a
+// row last takes it over - was measured: the memory fence every block then needs before its
+// ticket drains the block's outstanding writes and cost the bandwidth-bound pass 0.2 ms.)
+__device__ __forceinline__ void pick_spec_row(uint32_t *hist, Sel *sel, uint32_t k, uint32_t fl, uint32_t *hit_row)
+{
+    __shared__ uint32_t tot[kBlock];
+    __shared__ uint32_t found;
+    if (threadIdx.x == 0) found = 0u;
+    const int per = kBins1 / kBlock, lo = threadIdx.x * per;
+    uint32_t own[kBins1 / kBlock];
+    uint32_t mine = 0;
+#pragma unroll
+    for (int t = 0; t < per; ++t) {
+        own[t] = fl < (uint32_t)kBins1 ? __ldcg(hist + lo + t) : 0u;
+        mine += own[t];
+    }
+    tot[threadIdx.x] = mine;
+    __syncthreads();
+    uint32_t above = 0;
+    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+    if (fl < (uint32_t)kBins1) {
+#pragma unroll
+        for (int t = per - 1; t >= 0; --t) {
+            const uint32_t c = own[t];
+            if (above < k && above + c >= k && lo + t < kBins1 - 1) {    // the last bin is open-ended: no threshold from it
+                sel->pre = (fl << 20) + ((uint32_t)(lo + t) << 11);
+                sel->b1 = sel->pre >> 20; sel->k1 = k - above; sel->c1 = c;
+                found = 1u;
+            }
+            above += c;
+        }
+    }
+    __syncthreads();
+    const uint32_t ok = found;
+    if (threadIdx.x == 0) *hit_row = ok;
+    if (!ok)
+        for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
+}
+
+// grid = (rows), one block each.
+__global__ void __launch_bounds__(kBlock)
+k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
+                 const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hit)
+{
+    const int row = blockIdx.x;
+    pick_spec_row(hist_all + (int64_t)row * kHistStride, sel_all + row, k, floor_bucket[row], hit + row);
+}
+
+// Server aggregation fused into the server's dense pass (Algorithm 1: ghat += mean of the
+// workers' messages, then c = C(ghat - gtil)): the n payloads whose entries a tile needs.
+struct Agg {
+    const uint32_t *idx;              // n x k coordinates, increasing in every row
+    const float *val;                 // n x k values
+    const uint32_t *tile_off;         // n x nt4k: payload offset of every 4096-coordinate tile (rows with hit)
+    const uint32_t *hit;              // n: 1 = the row has tile offsets; 0 = search its coordinates
+    int64_t k;
+    int n, n_pow2;
+};
+constexpr int kAggStageWorkers = 16;  // workers whose tile entries are staged in shared memory at once
+constexpr int kAggStageCap = 64;      // entries per worker and tile that the staged path holds
+
+__device__ __forceinline__ int64_t lower_bound_idx(const uint32_t *p, int64_t count, int64_t key)
+{
+    if (key >= ((int64_t)1 << 32)) return count;
+    int64_t lo = 0, hi = count;
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)p[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
 // The payload of the previous selection that is still to be applied to a row's tile
 // (deferred state update): entries [begin, end) of the row's payload arrays.
 struct Pending {
@@ -318,19 +457,34 @@ struct Pending {
 // APPLY: first add the previous payload's values to b at this tile's kept coordinates
 // (Algorithm 1: ghat^(i) += c^(i), deferred from the previous iteration), then read b through
 // the coherent path, since this block has just written to it.
-template <bool HAS_B, bool APPLY>
+// AGG (one row, the server's): a is the server aggregate ghat, read AND written.  Before
+// anything else the block adds the mean of the n workers' messages to its tile of a: the
+// entries of every worker inside the tile (a contiguous run of its payload) are summed per
+// coordinate in the order 0, 1, ..., n-1 in shared memory, then a_j += sum_j / n where the
+// sum is not zero.  The dense pass proper then works on the updated tile, which is still in
+// registers: the separate aggregation kernel's pass over ghat, and its launch, are saved.
+// With up to kAggStageWorkers workers and kAggStageCap entries each in the tile, the entries
+// are held in registers and added in rounds by their place among the coordinate's senders;
+// otherwise the block adds worker by worker with a barrier after each.  A row without a guess
+// still gets the aggregation.
+template <bool HAS_B, bool APPLY, bool AGG>
 __global__ void __launch_bounds__(kBlock)
 k_topk_spec(const float *__restrict__ a_all, float *b_all,
             const uint32_t *__restrict__ floor_bucket, uint32_t *__restrict__ hist_all,
             float *__restrict__ stash_all, uint16_t *__restrict__ stash_pos_all,
             uint32_t *__restrict__ stash_cnt_all, int64_t d, int vec_ok, int64_t stride, int64_t tile0,
-            int64_t nt4k, Pending pd)
+            int64_t nt4k, Pending pd, Agg ag, float *a_rw)
 {
     __shared__ uint32_t h[kBins1];
     __shared__ uint32_t wcnt[kBlock / 32];
+    // flagged groups of a warp in the dense loop; with AGG, first the per-coordinate sums of the
+    // warp's 512 coordinates (each warp's part is used by that warp alone, one use after the other)
+    __shared__ float4 s_u[kBlock / 32][kWarpSpan / 4];
+    __shared__ uint16_t s_p[kBlock / 32][kWarpSpan / 4];
     const int row = blockIdx.y;
     const uint32_t fl = floor_bucket[row];
-    if (fl >= (uint32_t)kBins1) return;               // no guess for this row (and then nothing pending)
+    const bool guess = fl < (uint32_t)kBins1;
+    if (!guess && !AGG) return;                       // no guess for this row (and then nothing pending)
     const uint32_t fk = fl << 20;                     // lowest key at or above the floor
     for (int t = threadIdx.x; t < kBins1; t += kBlock) h[t] = 0;
     const float *a = a_all + (int64_t)row * stride;
@@ -350,23 +504,126 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
     const int64_t base = (tile0 + blockIdx.x) * kSub;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const uint32_t lt = (1u << lane) - 1u;
-    if (vec_ok && base + kSub <= d) {
+    const bool vec_tile = vec_ok && base + kSub <= d;
+    float *acc = reinterpret_cast<float *>(&s_u[0][0]);           // AGG: kSub sums, warp w owns [512 w, 512 w + 512)
+    float4 A[4], Bv[4];
+    if (vec_tile) {                                   // issued first: in flight during the aggregation
+#pragma unroll
+        for (int v = 0; v < 4; ++v) {
+            const int64_t j = base + warp * kWarpSpan + v * 128 + lane * 4;
+            A[v] = AGG ? ld_rw4(a + j) : ld_ro4(a + j);
+            if (HAS_B) Bv[v] = APPLY ? ld_cg4(b + j) : ld_ro4(b + j);
+        }
+    }
+    if constexpr (AGG) {
+        __shared__ uint32_t s_rng[2];
+        __shared__ uint32_t s_mask[kSub / 2];         // per coordinate: which of up to 16 workers sent it
+        const int64_t t = tile0 + blockIdx.x;
+        for (int e = threadIdx.x; e < kSub; e += kBlock) acc[e] = 0.0f;
+        for (int e = threadIdx.x; e < kSub / 2; e += kBlock) s_mask[e] = 0u;
+        // entries of worker i inside [base, base + kSub): from the row's tile offsets, or by search
+        auto range_of = [&](int i, int side) -> uint32_t {
+            if (ag.hit[i]) return t + side < nt4k ? ag.tile_off[(int64_t)i * nt4k + t + side] : (uint32_t)ag.k;
+            return (uint32_t)lower_bound_idx(ag.idx + (int64_t)i * ag.k, ag.k, base + (int64_t)side * kSub);
+        };
+        // Staged path (up to 16 workers, all with tile offsets, up to kAggStageCap entries each in
+        // this tile): sixteen threads hold the entries of one worker, four slots each.
+        const int wi = threadIdx.x >> 4;
+        uint32_t beg = 0u, cnt = 0u;
+        bool staged = ag.n <= kAggStageWorkers;
+        if (staged && wi < ag.n) {
+            const uint32_t has = ag.hit[wi];
+            beg = ag.tile_off[(int64_t)wi * nt4k + t];
+            const uint32_t end = t + 1 < nt4k ? ag.tile_off[(int64_t)wi * nt4k + t + 1] : (uint32_t)ag.k;
+            cnt = end - beg;
+            staged = has != 0u && end >= beg && cnt <= (uint32_t)kAggStageCap;
+        }
+        if (!__syncthreads_or(!staged)) {             // (the barrier also orders the zeroing above)
+            // The sum of a coordinate runs over the workers in increasing order.  Every entry
+            // learns its place in that order from a bit mask of the coordinate's senders
+            // (integer atomics: order-free), and the additions are made in rounds, place by
+            // place with a barrier between: as many rounds as the most-sent coordinate has
+            // senders, each touching only the entries whose turn it is.
+            uint32_t pos[4], place[4];
+            float val[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                const uint32_t u = (threadIdx.x & 15) + 16 * r;
+                pos[r] = 0xffffffffu;
+                val[r] = 0.0f;
+                if (u < cnt) {
+                    pos[r] = ag.idx[(int64_t)wi * ag.k + beg + u] - (uint32_t)base;
+                    val[r] = ag.val[(int64_t)wi * ag.k + beg + u];
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (pos[r] < (uint32_t)kSub) atomicOr(&s_mask[pos[r] >> 1], 1u << (((pos[r] & 1u) << 4) + wi));
+            __syncthreads();
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                place[r] = 0xffffffffu;
+                if (pos[r] < (uint32_t)kSub) {
+                    const uint32_t senders = (s_mask[pos[r] >> 1] >> ((pos[r] & 1u) << 4)) & 0xffffu;
+                    place[r] = __popc(senders & ((1u << wi) - 1u));
+                    if (place[r] == 0u) acc[pos[r]] = val[r];            // 0 + v
+                }
+            }
+            for (uint32_t round = 1;; ++round) {
+                bool more = false;
+#pragma unroll
+                for (int r = 0; r < 4; ++r) more = more || (place[r] != 0xffffffffu && place[r] >= round);
+                if (!__syncthreads_or(more)) break;    // orders the rounds; after the last one, the sums are complete
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    if (place[r] == round) acc[pos[r]] = __fadd_rn(acc[pos[r]], val[r]);
+            }
+        } else {
+            // general case: worker after worker over the whole block, a barrier after each
+            for (int i = 0; i < ag.n; ++i) {
+                if (threadIdx.x < 2) s_rng[threadIdx.x] = range_of(i, threadIdx.x);
+                __syncthreads();
+                const uint32_t lo = s_rng[0], hi = s_rng[1];
+                for (uint32_t at = lo + threadIdx.x; at < hi; at += kBlock) {
+                    const uint32_t q = ag.idx[(int64_t)i * ag.k + at] - (uint32_t)base;
+                    if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], ag.val[(int64_t)i * ag.k + at]);
+                }
+                __syncthreads();
+            }
+        }
+        const float fn = (float)ag.n, rn = 1.0f / fn;
+        auto mean = [&](float v) { return ag.n_pow2 ? __fmul_rn(v, rn) : __fdiv_rn(v, fn); };
+        if (vec_tile) {
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const int p = warp * kWarpSpan + v * 128 + lane * 4;
+                const float4 c = *reinterpret_cast<const float4 *>(acc + p);
+                if (c.x != 0.0f || c.y != 0.0f || c.z != 0.0f || c.w != 0.0f) {   // adding an exact zero changes nothing
+                    if (c.x != 0.0f) A[v].x = __fadd_rn(A[v].x, mean(c.x));
+                    if (c.y != 0.0f) A[v].y = __fadd_rn(A[v].y, mean(c.y));
+                    if (c.z != 0.0f) A[v].z = __fadd_rn(A[v].z, mean(c.z));
+                    if (c.w != 0.0f) A[v].w = __fadd_rn(A[v].w, mean(c.w));
+                    st_rw4(a_rw + base + p, A[v]);
+                }
+            }
+            __syncwarp();                             // the warp's sums are read: its part of s_u is free again
+        } else {
+            const int64_t end = min(base + (int64_t)kSub, d);
+            for (int64_t j = base + threadIdx.x; j < end; j += kBlock) {
+                const float c = acc[j - base];
+                if (c != 0.0f) a_rw[j] = __fadd_rn(a_rw[j], mean(c));
+            }
+            __syncthreads();                          // the scalar pass below reads a from memory
+        }
+        if (!guess) return;                           // block-uniform: aggregation only
+    }
+    if (vec_tile) {
         // Few coordinates lie at or above the floor (a percent or two), so the per-coordinate
         // work is kept out of the dense loop: a thread only tests each of its four float4
         // groups as a whole (one vote per group), flagged groups are moved to a small list in
         // shared memory in index order, and the warp then works on that list densely - keys,
         // histogram, ranks and the writes of the tile's (position, value) list.
-        __shared__ float4 s_u[kBlock / 32][kWarpSpan / 4];
-        __shared__ uint16_t s_p[kBlock / 32][kWarpSpan / 4];
-        const int64_t wb = base + warp * kWarpSpan;
         const float fkf = __uint_as_float(fk);
-        float4 A[4], Bv[4];
-#pragma unroll
-        for (int v = 0; v < 4; ++v) {
-            const int64_t j = wb + v * 128 + lane * 4;
-            A[v] = ld_ro4(a + j);
-            if (HAS_B) Bv[v] = APPLY ? ld_cg4(b + j) : ld_ro4(b + j);
-        }
         uint32_t FB[4];
 #pragma unroll
         for (int v = 0; v < 4; ++v) {
@@ -443,7 +700,8 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
         for (int64_t j0 = base; j0 < end; j0 += kBlock) {
             const int64_t j = j0 + threadIdx.x;
             const bool valid = j < end;
-            const float u = !valid ? 0.0f : !HAS_B ? a[j] : __fsub_rn(a[j], APPLY ? __ldcg(b + j) : b[j]);
+            const float aj = !valid ? 0.0f : AGG ? __ldcg(a_rw + j) : a[j];
+            const float u = !valid ? 0.0f : !HAS_B ? aj : __fsub_rn(aj, APPLY ? __ldcg(b + j) : b[j]);
             const uint32_t key = key_of(u);
             const bool ge = valid && key >= fk;
             const uint32_t wg = __ballot_sync(kFull, ge);
@@ -673,48 +931,6 @@ k_topk_spec_ring(const float *__restrict__ a_all, float *b_all,
         if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
-// Did the guess hold?  It did if the k-th largest key lies in one of the regular fine bins
-// above the floor; then key bits 30..11 of the threshold follow from the histogram of those
-// coordinates.  Otherwise the row's level-1 histogram is cleared for the full pass.
-// grid = (rows), one block.
-__global__ void __launch_bounds__(kBlock)
-k_topk_pick_spec(uint32_t *__restrict__ hist_all, Sel *__restrict__ sel_all, uint32_t k,
-                 const uint32_t *__restrict__ floor_bucket,
-                 uint32_t *__restrict__ hit)
-{
-    __shared__ uint32_t tot[kBlock];
-    __shared__ uint32_t found;
-    const int row = blockIdx.x;
-    Sel *sel = sel_all + row;
-    uint32_t *hist = hist_all + (int64_t)row * kHistStride;
-    const uint32_t fl = floor_bucket[row];
-    if (threadIdx.x == 0) found = 0u;
-    const int per = kBins1 / kBlock, lo = threadIdx.x * per;
-    uint32_t mine = 0;
-    if (fl < (uint32_t)kBins1)
-        for (int t = 0; t < per; ++t) mine += hist[lo + t];
-    tot[threadIdx.x] = mine;
-    __syncthreads();
-    uint32_t above = 0;
-    for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
-    if (fl < (uint32_t)kBins1) {
-        for (int t = per - 1; t >= 0; --t) {
-            const uint32_t c = hist[lo + t];
-            if (above < k && above + c >= k && lo + t < kBins1 - 1) {    // the last bin is open-ended: no threshold from it
-                sel->pre = (fl << 20) + ((uint32_t)(lo + t) << 11);
-                sel->b1 = sel->pre >> 20; sel->k1 = k - above; sel->c1 = c;
-                found = 1u;
-            }
-            above += c;
-        }
-    }
-    __syncthreads();
-    const uint32_t ok = found;
-    if (threadIdx.x == 0) hit[row] = ok;
-    if (!ok)
-        for (int t = threadIdx.x; t < kBins1; t += kBlock) hist[t] = 0u;
-}
-
 // In the list passes below a warp owns kWarpTiles consecutive tiles and a block
 // kListTiles; lane L reads entries L, L + 32, ... of a tile's list (coalesced).  The passes
 // are bound by memory latency, so the first kPre chunks of every tile of the warp are loaded
@@ -758,15 +974,18 @@ __device__ __forceinline__ WarpLists warp_lists(const float *stash_all, const ui
 }
 
 // f(value) for every entry of the warp's lists (every coordinate of its dense tiles).
+// The first kPre chunks of a list are fetched without waiting for its length (a tile's list
+// has room for kStashCap >= 32 kPre entries, so the reads stay inside it; what lies beyond
+// the length is not used): the pass then costs one memory latency per tile instead of two.
 template <bool HAS_B, typename F>
-__device__ __forceinline__ void for_each_listed(const WarpLists &w, const float *a, const float *b, F f)
+__device__ __forceinline__ void for_each_listed(const WarpLists &w, const float *a, const float *b, F &f)
 {
     const uint32_t lane = threadIdx.x & 31;
     float v[kWarpTiles][kPre];
 #pragma unroll
     for (int m = 0; m < kWarpTiles; ++m)
 #pragma unroll
-        for (int i = 0; i < kPre; ++i) v[m][i] = lane + 32 * i < w.cnt[m] ? w.val[m][lane + 32 * i] : 0.0f;
+        for (int i = 0; i < kPre; ++i) v[m][i] = w.val[m][lane + 32 * i];      // beyond the list: unused (see for_each_listed)
 #pragma unroll
     for (int m = 0; m < kWarpTiles; ++m) {
 #pragma unroll
@@ -777,34 +996,65 @@ __device__ __forceinline__ void for_each_listed(const WarpLists &w, const float 
     }
 }
 
-struct HistLow11 {                    // keys that share bits 30..11 with the threshold, by bits 10..0
+constexpr int kCandPerTile = 4;       // candidates of a tile that are kept with the tile (more: the tile is re-read)
+
+// Per listed value: keys that share bits 30..11 with the threshold ("candidates") go to the
+// histogram of bits 10..0 and, as far as there is room, into the tile's candidate slots; keys
+// with higher bits 30..11 are certainly kept and only counted.
+struct SplitTile {
     uint32_t *h, pre11;
-    __device__ __forceinline__ void operator()(float v) const
+    uint32_t *slots;                  // shared: candidates seen in this warp's tile so far
+    uint16_t *cand;                   // global: the tile's kCandPerTile candidate slots (key bits 10..0)
+    uint32_t above;                   // this lane's count of certainly kept values
+    __device__ __forceinline__ void operator()(float v)
     {
-        const uint32_t key = key_of(v);
-        if ((key >> 11) == pre11) atomicAdd(&h[key & (kBins2 - 1)], 1u);
+        const uint32_t key = key_of(v), hi = key >> 11;
+        if (hi == pre11) {
+            atomicAdd(&h[key & (kBins2 - 1)], 1u);
+            const uint32_t at = atomicAdd(slots, 1u);
+            if (at < (uint32_t)kCandPerTile) cand[at] = (uint16_t)(key & (kBins2 - 1));
+        } else if (hi > pre11) {
+            ++above;
+        }
     }
 };
 
-// After a successful guess: the histogram of key bits 10..0 over the listed values that share
-// the threshold's bits 30..11; the pick that follows gives the exact threshold.
+// After a successful guess, one pass over the lists: the histogram of key bits 10..0 over the
+// listed values that share the threshold's bits 30..11 (the pick inside k_scan_lists gives the
+// exact threshold T from it), and per tile what the scan needs to place the tile's kept
+// coordinates without reading the list again: the number of values certainly above T
+// (cnt_gt), the number of candidates (cnt_eq) and the candidates' low key bits (cand; a tile
+// with more than kCandPerTile candidates is counted again from its list by the scan).
 // grid = (nbt, rows).
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
-             const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all, int64_t nt4k,
-             int64_t d, int64_t stride)
+             const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ hist_all,
+             uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all, uint16_t *__restrict__ cand_all,
+             int64_t nt4k, int64_t d, int64_t stride)
 {
     __shared__ uint32_t h[kBins2];
+    __shared__ uint32_t s_slots[kBlock / 32];
     const int row = blockIdx.y;
     if (!hit[row] || (int64_t)blockIdx.x * kListTiles >= nt4k) return;
     for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
+    if (threadIdx.x < kBlock / 32) s_slots[threadIdx.x] = 0u;
     __syncthreads();
-    for_each_listed<HAS_B>(warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d),
-                           a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr,
-                           HistLow11{h, sel_all[row].pre >> 11});
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
+    const int64_t g = (int64_t)row * nt4k + (w.tile[0] < nt4k ? w.tile[0] : 0);
+    SplitTile f{h, sel_all[row].pre >> 11, &s_slots[warp], cand_all + g * kCandPerTile, 0u};
+    for_each_listed<HAS_B>(w, a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr, f);
+    __syncwarp();
+    uint32_t above = f.above;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) above += __shfl_xor_sync(kFull, above, o);
+    if (lane == 0 && w.tile[0] < nt4k) {
+        cnt_gt_all[g] = above;
+        cnt_eq_all[g] = s_slots[warp];
+    }
     __syncthreads();
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
     for (int t = threadIdx.x; t < kBins2; t += kBlock)
@@ -821,7 +1071,7 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
              const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              const uint32_t *__restrict__ bm_cand_all, uint32_t *__restrict__ hist_all,
-             int64_t wp, int64_t nbt, int64_t stride)
+             int64_t wp, int64_t nbt, int64_t stride, RowTail tail)
 {
     __shared__ uint32_t h[kBins3];
     const int row = blockIdx.y;
@@ -848,109 +1098,62 @@ k_topk_hist3(const float *__restrict__ a_all, const float *__restrict__ b_all,
     uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1 + kBins2;
     for (int t = threadIdx.x; t < kBins3; t += kBlock)
         if (h[t]) atomicAdd(&hist[t], h[t]);
+    if (tail.tick && last_block_of_row(tail.tick + row, gridDim.x))
+        pick_row(hist_all + (int64_t)row * kHistStride, const_cast<Sel *>(sel_all) + row, 2, 0u, tail.floor_bucket + row);
 }
 
 // ------------------------------------------------------------------------------------
-// With the threshold key T known.  Rows with lists: per tile, the number of keys above T and
-// the number equal to T (the ties); the scans below turn them into payload offsets.  Other
-// rows: bm_in |= candidates with key > T; bm_cand := candidates with key == T; if all ties
-// are needed they are merged at once, otherwise the per-tile tie counts feed the ordered
-// pick below.  grid = (nbt, rows).
+// With the threshold key T known (rows whose guess failed; the rows selected from lists get
+// their per-tile counts in k_topk_split and k_scan_lists): bm_in |= candidates with key > T;
+// bm_cand := candidates with key == T; if all ties are needed they are merged at once,
+// otherwise the per-tile tie counts feed the ordered pick below.  grid = (nbt, rows).
 // ------------------------------------------------------------------------------------
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_resolve(const float *__restrict__ a_all, const float *__restrict__ b_all,
                const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
-               const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
-               const uint32_t *__restrict__ stash_cnt_all, uint32_t *__restrict__ cnt_gt_all,
-               uint32_t *__restrict__ cnt_eq_all,
                uint32_t *__restrict__ bm_in_all, uint32_t *__restrict__ bm_cand_all,
-               uint32_t *__restrict__ cnt_tie_all, int64_t d, int64_t wp, int64_t nbt, int64_t nt4k, int64_t stride)
+               uint32_t *__restrict__ cnt_tie_all, int64_t wp, int64_t nbt, int64_t stride, unsigned int *tick)
 {
     const int row = blockIdx.y;
+    if (hit[row]) return;
     uint32_t *bm_in = bm_in_all + (int64_t)row * wp, *bm_cand = bm_cand_all + (int64_t)row * wp;
     const Sel s = sel_all[row];
     const uint32_t T = (s.b1 << 20) | (s.b2 << 9) | s.b3;
     const bool all_ties = s.k3 == s.c3;
     uint32_t nt = 0;
-    if (hit[row]) {                                   // the tiles' lists hold the values
-        if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
-        const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
-        const float *a = a_all + (int64_t)row * stride;
-        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
-        const uint32_t lane = threadIdx.x & 31;
-        float v[kWarpTiles][kPre];
-#pragma unroll
-        for (int m = 0; m < kWarpTiles; ++m)
-#pragma unroll
-            for (int i = 0; i < kPre; ++i) v[m][i] = lane + 32 * i < w.cnt[m] ? w.val[m][lane + 32 * i] : 0.0f;
-#pragma unroll
-        for (int m = 0; m < kWarpTiles; ++m) {
-            uint32_t gt = 0, eq = 0;
-            for (uint32_t e = lane; e < w.dense[m]; e += 32) {
-                const uint32_t key = key_of(diff1<HAS_B>(a, b, w.tile[m] * kSub + e));
-                gt += key > T;
-                eq += key == T;
-            }
-#pragma unroll
-            for (int i = 0; i < kPre; ++i)
-                if (lane + 32 * i < w.cnt[m]) { gt += key_of(v[m][i]) > T; eq += key_of(v[m][i]) == T; }
-            for (uint32_t e = lane + 32 * kPre; e < w.cnt[m]; e += 32) {
-                const uint32_t key = key_of(w.val[m][e]);
-                gt += key > T;
-                eq += key == T;
-            }
-#pragma unroll
-            for (int o = 16; o >= 1; o >>= 1) {
-                gt += __shfl_xor_sync(kFull, gt, o);
-                eq += __shfl_xor_sync(kFull, eq, o);
-            }
-            if (w.tile[m] < nt4k && lane == 0) {
-                cnt_gt_all[(int64_t)row * nt4k + w.tile[m]] = gt;
-                cnt_eq_all[(int64_t)row * nt4k + w.tile[m]] = eq;
-            }
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
+    const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
+    for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
+        uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
+        while (word) {
+            const int bit = __ffs(word) - 1;
+            word &= word - 1;
+            const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
+            if (key > T) keep |= 1u << bit;
+            else if (key == T) tie |= 1u << bit;
         }
-        return;
-    } else {
-        const float *a = a_all + (int64_t)row * stride;
-        const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
-        const int64_t w0 = (int64_t)blockIdx.x * kTileWords;
-        for (int t = threadIdx.x; t < kTileWords && w0 + t < wp; t += kBlock) {
-            uint32_t word = bm_cand[w0 + t], keep = bm_in[w0 + t], tie = 0;
-            while (word) {
-                const int bit = __ffs(word) - 1;
-                word &= word - 1;
-                const uint32_t key = key_of(diff1<HAS_B>(a, b, (w0 + t) * 32 + bit));
-                if (key > T) keep |= 1u << bit;
-                else if (key == T) tie |= 1u << bit;
-            }
-            if (all_ties) keep |= tie;
-            bm_in[w0 + t] = keep;
-            bm_cand[w0 + t] = tie;
-            nt += __popc(tie);
-        }
+        if (all_ties) keep |= tie;
+        bm_in[w0 + t] = keep;
+        bm_cand[w0 + t] = tie;
+        nt += __popc(tie);
     }
     uint32_t total;
     block_excl_scan(nt, total);
     if (threadIdx.x == 0) cnt_tie_all[(int64_t)row * nbt + blockIdx.x] = total;
+    // the exclusive scan of the row's tie counts, by the block that finishes the row last
+    if (tick && last_block_of_row(tick + row, gridDim.x)) scan_row(cnt_tie_all + (int64_t)row * nbt, nbt, nullptr, true);
 }
 
 // Exclusive scan of the per-tile counts of the rows whose guess failed, in place
 // (skip_hit: rows with lists are left alone).  grid = (rows).
 __global__ void __launch_bounds__(kBlock)
-k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__restrict__ hit)
+k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__restrict__ hit,
+             uint32_t *__restrict__ totals = nullptr, bool in_place = true)
 {
     if (hit[blockIdx.x]) return;
-    uint32_t *cnt = cnt_all + (int64_t)blockIdx.x * nbt;
-    uint32_t carry = 0;
-    for (int64_t c = 0; c < nbt; c += kBlock) {
-        const int64_t t = c + threadIdx.x;
-        const uint32_t v = t < nbt ? cnt[t] : 0u;
-        uint32_t total;
-        const uint32_t ex = block_excl_scan(v, total);
-        if (t < nbt) cnt[t] = carry + ex;
-        carry += total;
-    }
+    scan_row(cnt_all + (int64_t)blockIdx.x * nbt, nbt, totals ? totals + blockIdx.x : nullptr, in_place);
 }
 
 // Rows with lists: from the per-tile counts of keys above / equal to the threshold to, per
@@ -964,26 +1167,100 @@ constexpr int kScanPer = 16;
 constexpr int kScanChunk = kBlock * kScanPer;
 __device__ __forceinline__ int scan_slot(int i) { return i + i / kScanPer; }
 
+template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
-k_scan_lists(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
+             Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
+             const uint32_t *__restrict__ hist_all, uint32_t *__restrict__ floor_bucket,
+             const float *__restrict__ stash_all, const uint32_t *__restrict__ stash_cnt_all,
+             const uint16_t *__restrict__ cand_all,
              uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all,
-             uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt)
+             uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt, int64_t d, int64_t stride)
 {
     __shared__ uint32_t s_eq[kScanChunk + kBlock], s_gt[kScanChunk + kBlock];
+    __shared__ uint32_t s_T, s_k3, s_c3;
     const int row = blockIdx.x;
     if (!hit[row]) return;
-    const Sel s = sel_all[row];
-    const bool all_ties = s.k3 == s.c3;
+    // The exact threshold first: the bucket of key bits 10..0 that holds the k1-th largest of
+    // the candidates (the histogram k_topk_split made), as k_topk_pick does for the classic rows.
+    {
+        uint32_t *tot = s_eq;                          // kBlock words, free until the scan starts
+        Sel *sel = sel_all + row;
+        const uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
+        const uint32_t want = sel->k1;
+        const int per = kBins2 / kBlock, lo = threadIdx.x * per;
+        uint32_t own[kBins2 / kBlock];
+        uint32_t mine = 0;
+#pragma unroll
+        for (int t = 0; t < per; ++t) { own[t] = hist[lo + t]; mine += own[t]; }
+        tot[threadIdx.x] = mine;
+        __syncthreads();
+        uint32_t above = 0;
+        for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+#pragma unroll
+        for (int t = per - 1; t >= 0; --t) {
+            const uint32_t c = own[t];
+            if (above < want && above + c >= want) {   // exactly one thread and bucket
+                const uint32_t T = sel->pre | (uint32_t)(lo + t);
+                sel->b1 = T >> 20; sel->b2 = (T >> 9) & (kBins2 - 1); sel->b3 = T & (kBins3 - 1);
+                sel->k3 = want - above; sel->c3 = c;
+                // guess for the next selection of this row: a little below this threshold
+                floor_bucket[row] = (T >> 20) > kGuessMargin ? (T >> 20) - kGuessMargin : 1u;
+                s_T = T; s_k3 = want - above; s_c3 = c;
+            }
+            above += c;
+        }
+        __syncthreads();
+    }
+    const uint32_t T = s_T, k3 = s_k3, Tlow = T & (kBins2 - 1);
+    const bool all_ties = k3 == s_c3;
     uint32_t *gt = cnt_gt_all + (int64_t)row * nt4k, *eq = cnt_eq_all + (int64_t)row * nt4k;
+    const uint2 *cand = reinterpret_cast<const uint2 *>(cand_all) + (int64_t)row * nt4k;
     uint32_t *fin = cnt_fin_all + (int64_t)row * nbt;
+    const float *a = a_all + (int64_t)row * stride;
+    const float *b = HAS_B ? b_all + (int64_t)row * stride : nullptr;
     uint32_t carry_eq = 0, carry_keep = 0;             // block-uniform
     for (int64_t c0 = 0; c0 < nt4k; c0 += kScanChunk) {
+        // all loads of the chunk first (independent, in flight together), then the counting
+        uint32_t G[kScanPer], NC[kScanPer];
+        uint2 C4[kScanPer];
+#pragma unroll
+        for (int m = 0; m < kScanPer; ++m) {
+            const int64_t t = c0 + m * kBlock + threadIdx.x;
+            const bool in = t < nt4k;
+            G[m] = in ? gt[t] : 0u;
+            NC[m] = in ? eq[t] : 0u;
+            C4[m] = in ? cand[t] : make_uint2(0u, 0u);
+        }
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
             const int i = m * kBlock + threadIdx.x;
             const int64_t t = c0 + i;
-            s_eq[scan_slot(i)] = t < nt4k ? eq[t] : 0u;
-            s_gt[scan_slot(i)] = t < nt4k ? gt[t] : 0u;
+            // keys above / equal to T in tile t: the certainly kept values plus the candidates
+            uint32_t g = G[m], e = 0u;
+            const uint32_t lows[4] = {C4[m].x & 0xffffu, C4[m].x >> 16, C4[m].y & 0xffffu, C4[m].y >> 16};
+#pragma unroll
+            for (int c = 0; c < kCandPerTile; ++c) {
+                const bool have = (uint32_t)c < NC[m];
+                g += have && lows[c] > Tlow;
+                e += have && lows[c] == Tlow;
+            }
+            if (NC[m] > (uint32_t)kCandPerTile) {
+                // more candidates than the tile's slots hold (ties in bulk, or a selection
+                // concentrated here): counted again from the tile's list, or from the data
+                g = 0u; e = 0u;
+                const int64_t tg = (int64_t)row * nt4k + t;
+                const uint32_t raw = stash_cnt_all[tg];
+                if (raw <= (uint32_t)kStashCap) {
+                    const float *val = stash_all + tg * kStashCap;
+                    for (uint32_t u = 0; u < raw; ++u) { const uint32_t key = key_of(val[u]); g += key > T; e += key == T; }
+                } else {
+                    const int64_t lo = t * kSub, hi = min(lo + (int64_t)kSub, d);
+                    for (int64_t j = lo; j < hi; ++j) { const uint32_t key = key_of(diff1<HAS_B>(a, b, j)); g += key > T; e += key == T; }
+                }
+            }
+            s_eq[scan_slot(i)] = e;
+            s_gt[scan_slot(i)] = g;
         }
         __syncthreads();
         const int mine = threadIdx.x * (kScanPer + 1);  // first slot of this thread's 16 tiles
@@ -996,7 +1273,7 @@ k_scan_lists(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
             const uint32_t e = s_eq[mine + m];
-            const uint32_t take = all_ties ? e : (tie_rank >= s.k3 ? 0u : min(e, s.k3 - tie_rank));
+            const uint32_t take = all_ties ? e : (tie_rank >= k3 ? 0u : min(e, k3 - tie_rank));
             s_eq[mine + m] = tie_rank;
             tie_rank += e;
             const uint32_t keep = s_gt[mine + m] + take;
@@ -1048,7 +1325,7 @@ __global__ void __launch_bounds__(kBlock)
 k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
             uint32_t *__restrict__ bm_in_all,
             const uint32_t *__restrict__ bm_cand_all, const uint32_t *__restrict__ tie_off_all,
-            uint32_t *__restrict__ cnt_fin_all, int64_t wp, int64_t nbt)
+            uint32_t *__restrict__ cnt_fin_all, int64_t wp, int64_t nbt, unsigned int *tick)
 {
     const int row = blockIdx.y;
     if (hit[row]) return;                             // rows with lists have no bitmaps
@@ -1080,6 +1357,7 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
     block_excl_scan(__popc(keep[0]) + __popc(keep[1]) + __popc(keep[2]) + __popc(keep[3]), total);
     if (threadIdx.x == 0) cnt_fin_all[(int64_t)row * nbt + bx] = total;
     }
+    if (tick && last_block_of_row(tick + row, gridDim.x)) scan_row(cnt_fin_all + (int64_t)row * nbt, nbt, nullptr, true);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1097,9 +1375,11 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
                 const float *__restrict__ stash_all, const uint16_t *__restrict__ stash_pos_all,
                 const uint32_t *__restrict__ stash_cnt_all, const uint32_t *__restrict__ cnt_gt_all,
                 const uint32_t *__restrict__ cnt_eq_all, uint32_t *__restrict__ idx_all,
-                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d, int64_t stride)
+                float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d, int64_t stride,
+                int kind)
 {
     const int row = blockIdx.y;
+    if (!(kind & (hit[row] ? kRowsListed : kRowsClassic))) return;
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
     if (hit[row]) {
@@ -1121,9 +1401,8 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
             tie_rank[m] = cnt_eq_all[g];
 #pragma unroll
             for (int i = 0; i < kPre; ++i) {
-                const bool valid = lane + 32 * i < w.cnt[m];
-                v[m][i] = valid ? w.val[m][lane + 32 * i] : 0.0f;
-                ps[m][i] = valid ? w.pos[m][lane + 32 * i] : 0u;
+                v[m][i] = w.val[m][lane + 32 * i];       // fetched whatever the length (see for_each_listed)
+                ps[m][i] = w.pos[m][lane + 32 * i];
             }
         }
 #pragma unroll
@@ -1194,32 +1473,34 @@ k_topk_gather(const float *__restrict__ a_all, float *__restrict__ b_all,
               uint32_t *__restrict__ pending)
 {
     const int row = blockIdx.y;
-    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
     // deferred state update: a row selected from lists (values already in the payload) keeps
     // its update for the next selection's dense pass
     const bool deferred = pending && have_val[row];
-    if (pending && t == 0) pending[row] = deferred ? 1u : 0u;
-    if (t >= k || deferred) return;
-    const int64_t j = idx_all[(int64_t)row * k + t];
-    if (j >= d) return;                       // caller-supplied sets are checked separately
+    if (pending && blockIdx.x == 0 && threadIdx.x == 0) pending[row] = deferred ? 1u : 0u;
+    if (deferred) return;
     const float *a = a_all + (int64_t)row * stride;
-    if (have_val && have_val[row]) {          // the payload values were written with the indices
-        if (HAS_B && UPDATE_B) {
-            float *b = b_all + (int64_t)row * stride;
-            b[j] = __fadd_rn(b[j], val_all[(int64_t)row * k + t]);
+    // (a grid smaller than the payload loops: where most rows defer, few blocks are launched)
+    for (int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x; t < k; t += (int64_t)gridDim.x * kBlock) {
+        const int64_t j = idx_all[(int64_t)row * k + t];
+        if (j >= d) continue;                 // caller-supplied sets are checked separately
+        if (have_val && have_val[row]) {      // the payload values were written with the indices
+            if (HAS_B && UPDATE_B) {
+                float *b = b_all + (int64_t)row * stride;
+                b[j] = __fadd_rn(b[j], val_all[(int64_t)row * k + t]);
+            }
+            continue;
         }
-        return;
+        float u;
+        if (HAS_B) {
+            float *b = b_all + (int64_t)row * stride;
+            const float bj = b[j];
+            u = __fsub_rn(a[j], bj);
+            if (UPDATE_B) b[j] = __fadd_rn(bj, u);
+        } else {
+            u = a[j];
+        }
+        val_all[(int64_t)row * k + t] = u;
     }
-    float u;
-    if (HAS_B) {
-        float *b = b_all + (int64_t)row * stride;
-        const float bj = b[j];
-        u = __fsub_rn(a[j], bj);
-        if (UPDATE_B) b[j] = __fadd_rn(bj, u);
-    } else {
-        u = a[j];
-    }
-    val_all[(int64_t)row * k + t] = u;
 }
 
 // Applies the payloads whose state update is still pending: b_j += u_j at the kept
@@ -1376,7 +1657,10 @@ static void free_ws(TopkWorkspace *w)
     cudaFree(w->cnt_tie); cudaFree(w->cnt_fin);
     cudaFree(w->floor_bucket); cudaFree(w->hit); cudaFree(w->stash);
     cudaFree(w->stash_pos); cudaFree(w->stash_cnt); cudaFree(w->cnt_gt); cudaFree(w->cnt_eq);
-    cudaFree(w->pending);
+    cudaFree(w->pending); cudaFree(w->cand); cudaFree(w->tick);
+    if (w->side) cudaStreamDestroy(w->side);
+    if (w->ev_fork) cudaEventDestroy(w->ev_fork);
+    if (w->ev_join) cudaEventDestroy(w->ev_join);
     if (w->own_payload) { cudaFree(w->idx); cudaFree(w->val); }
     delete w;
 }
@@ -1416,6 +1700,11 @@ int topk_workspace_create(TopkWorkspace **out, int64_t d, int64_t k, int rows, u
         get((void **)&w->cnt_tie, (size_t)rows * w->nbt * 4);
         get((void **)&w->cnt_fin, (size_t)rows * w->nbt * 4);
         get((void **)&w->pending, (size_t)rows * 4);
+        get((void **)&w->cand, (size_t)rows * w->nt4k * 4 * sizeof(uint16_t));
+        get((void **)&w->tick, (size_t)rows * 5 * sizeof(unsigned int));
+        if (ok && (cudaStreamCreateWithFlags(&w->side, cudaStreamNonBlocking) != cudaSuccess ||
+                   cudaEventCreateWithFlags(&w->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                   cudaEventCreateWithFlags(&w->ev_join, cudaEventDisableTiming) != cudaSuccess)) ok = false;
     }
     if (w->own_payload) {
         get((void **)&w->idx, (size_t)rows * k * 4);
@@ -1455,8 +1744,8 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
     *val = w->val + (int64_t)row * w->k;
 }
 
-constexpr int kSelectLaunches = 16;
-int topk_launches_per_step(int) { return 2 * kSelectLaunches + 1; }
+constexpr int kSelectLaunches = 12;      // dense pass, pick, six for the classic chain, three for the listed chain, gather
+int topk_launches_per_step(int) { return 2 * kSelectLaunches; }    // two selections; the aggregation kernel is counted by the caller
 
 // Whole tiles per row that the dense pass takes through the prefetch ring (0: none).
 static int64_t ring_tiles(const TopkWorkspace *w, bool vec_ok)
@@ -1476,7 +1765,7 @@ int topk_dense_launches(const TopkWorkspace *w, bool vec_ok)
 
 template <bool HAS_B>
 static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
-                        cudaStream_t st)
+                        cudaStream_t st, const Agg *agg = nullptr, float *a_rw = nullptr)
 {
     const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
     const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
@@ -1488,7 +1777,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // tiles enough to fill the device several times over with its three blocks of eight tiles
     // per SM (measured: 16 x 6250 tiles 0.50 -> 0.47 ms, 1 x 6250 tiles 0.039 -> 0.047 ms);
     // the ragged last tile, or everything else, through the plain kernel
-    const int64_t full_tiles = ring_tiles(w, vec_ok);
+    const int64_t full_tiles = agg ? 0 : ring_tiles(w, vec_ok);      // the fused aggregation lives in the plain kernel
     // deferred state update: the dense pass first applies the previous selection's payload
     const bool defer = HAS_B && update_b && w->defer;
     const Pending pd = {w->pending, w->idx, w->val, w->cnt_gt, w->k};
@@ -1502,26 +1791,35 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     }
     if (full_tiles < w->nt4k) {
         const dim3 rest((unsigned)(w->nt4k - full_tiles), (unsigned)w->rows);
-        auto kern = defer ? k_topk_spec<HAS_B, HAS_B> : k_topk_spec<HAS_B, false>;
+        auto kern = agg ? k_topk_spec<HAS_B, false, HAS_B> : defer ? k_topk_spec<HAS_B, HAS_B, false> : k_topk_spec<HAS_B, false, false>;
         kern<<<rest, kBlock, 0, st>>>(a, b, w->floor_bucket, w->hist, w->stash, w->stash_pos, w->stash_cnt, w->d, vec_ok,
-                                     w->stride, full_tiles, w->nt4k, pd);
+                                     w->stride, full_tiles, w->nt4k, pd, agg ? *agg : Agg{}, a_rw);
     }
     k_topk_pick_spec<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, (uint32_t)w->k, w->floor_bucket, w->hit);
-    k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)w->k, w->hit, w->floor_bucket);
-    k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok, w->stride);
-    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->nt4k, w->d, w->stride);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
+    // From here two chains run side by side (under stream capture: two branches of the graph).
+    // Rows whose guess failed (none, in the steady state: six launches that find nothing to do;
+    // every pick and scan is done by the block that finishes its row last) take the classic
+    // passes on the side stream ...
     const dim3 fallback_sparse(std::min(sparse.x, fallback.x), (unsigned)w->rows);
-    k_topk_hist3<HAS_B><<<fallback_sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_cand, w->hist, w->wp, w->nbt, w->stride);
-    k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
-    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->bm_in, w->bm_cand, w->cnt_tie, w->d, w->wp, w->nbt, w->nt4k, w->stride);
-    k_scan_lists<<<w->rows, kBlock, 0, st>>>(w->sel, w->hit, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt);
-    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
-    k_topk_ties<<<fallback_sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt);
-    k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit);
-    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride);
-    const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+    cudaStream_t sd = w->side;
+    cudaEventRecord(w->ev_fork, st);
+    cudaStreamWaitEvent(sd, w->ev_fork, 0);
+    const uint32_t k32 = (uint32_t)w->k;
+    auto tail = [&](int pass) { return RowTail{w->tick + (size_t)pass * w->rows, w->sel, w->floor_bucket, k32}; };
+    k_topk_hist1<HAS_B><<<fallback, kBlock, 0, sd>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride, tail(0));
+    k_topk_mark<HAS_B><<<fallback, kBlock, 0, sd>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok, w->stride, tail(1));
+    k_topk_hist3<HAS_B><<<fallback_sparse, kBlock, 0, sd>>>(a, b, w->sel, w->hit, w->bm_cand, w->hist, w->wp, w->nbt, w->stride, tail(2));
+    k_topk_resolve<HAS_B><<<sparse, kBlock, 0, sd>>>(a, b, w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->wp, w->nbt, w->stride, w->tick + (size_t)3 * w->rows);
+    k_topk_ties<<<fallback_sparse, kBlock, 0, sd>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt, w->tick + (size_t)4 * w->rows);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, sd>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic);
+    cudaEventRecord(w->ev_join, sd);
+    // ... and the rows selected from the dense pass's lists take three launches on this one
+    k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->cnt_gt, w->cnt_eq, w->cand, w->nt4k, w->d, w->stride);
+    k_scan_lists<HAS_B><<<w->rows, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->hist, w->floor_bucket, w->stash, w->stash_cnt, w->cand, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt, w->d, w->stride);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsListed);
+    cudaStreamWaitEvent(st, w->ev_join, 0);
+    dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+    if (defer) entries.x = std::min(entries.x, 96u);   // rows selected from lists defer: nothing to do for them
     if (HAS_B && update_b)
         k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride,
                                                                defer ? w->pending : nullptr);
@@ -1529,11 +1827,139 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
         k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);
 }
 
+// ------------------------------------------------------------------------------------
+// Coordinate-sharded selection.  Several workspaces, one per coordinate range of the same
+// rows, select the k largest of the WHOLE rows between them: the classic three levels, every
+// histogram summed over the ranges before its pick (integer sums: any order gives the same
+// threshold on every range), then the ties given out in coordinate order, i.e. in the order
+// of the ranges: range r takes those of the k3 ties that the ranges before it left.
+// The sums and counts travel through an exchange buffer of ranges x rows x kBins1 words:
+// a stage writes this range's slot, the caller gathers the slots of all ranges in place,
+// the next stage reads them all.
+// ------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kBlock)
+k_range_hist_out(const uint32_t *__restrict__ hist_all, int level_off, int bins, uint32_t *__restrict__ slot)
+{
+    const int row = blockIdx.y, t = blockIdx.x * kBlock + threadIdx.x;
+    if (t < bins) slot[(int64_t)row * kBins1 + t] = hist_all[(int64_t)row * kHistStride + level_off + t];
+}
+
+__global__ void __launch_bounds__(kBlock)
+k_range_hist_sum(const uint32_t *__restrict__ x_all, int ranges, int rows, int level_off, int bins,
+                 uint32_t *__restrict__ hist_all)
+{
+    const int row = blockIdx.y, t = blockIdx.x * kBlock + threadIdx.x;
+    if (t >= bins) return;
+    uint32_t sum = 0u;
+    for (int r = 0; r < ranges; ++r) sum += x_all[((int64_t)r * rows + row) * kBins1 + t];
+    hist_all[(int64_t)row * kHistStride + level_off + t] = sum;
+}
+
+// The ties this range may keep: k3 minus the ties of the ranges before it, at most its own.
+// A row that keeps all ties (k3 == c3) is left alone.  One thread per row.
+__global__ void k_range_ties_share(Sel *__restrict__ sel_all, const uint32_t *__restrict__ x_all, int range,
+                                   int rows)
+{
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    Sel *s = sel_all + row;
+    if (s->k3 == s->c3) return;
+    uint32_t before = 0u;
+    for (int r = 0; r < range; ++r) before += x_all[((int64_t)r * rows + row) * kBins1];
+    const uint32_t own = x_all[((int64_t)range * rows + row) * kBins1];
+    const uint32_t share = before >= s->k3 ? 0u : min(own, s->k3 - before);
+    s->k3 = share;
+    s->c3 = 0xffffffffu;              // != k3: the ordered pick of the ties runs
+}
+
+// Payload entries beyond the range's own count are marked with the coordinate 0xffffffff
+// (no vector has it: d < 2^32), which every later pass over a payload skips.
+__global__ void __launch_bounds__(kBlock)
+k_range_pad(uint32_t *__restrict__ idx_all, float *__restrict__ val_all, const uint32_t *__restrict__ count, int64_t k)
+{
+    const int row = blockIdx.y;
+    const int64_t t = (int64_t)blockIdx.x * kBlock + threadIdx.x;
+    if (t < k && t >= (int64_t)count[row]) {
+        idx_all[(int64_t)row * k + t] = 0xffffffffu;
+        val_all[(int64_t)row * k + t] = 0.0f;
+    }
+}
+
+template <bool HAS_B>
+static void range_stage_impl(TopkWorkspace *w, int stage, const float *a, float *b, bool vec_ok, int64_t k_all,
+                             uint32_t *x, int range, int ranges, cudaStream_t st)
+{
+    const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
+    const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
+    const dim3 fallback(std::min(dense.x, std::max(148u, 148u * 4u / (unsigned)w->rows)), (unsigned)w->rows);
+    const dim3 fallback_sparse(std::min(sparse.x, fallback.x), (unsigned)w->rows);
+    const dim3 bins((kBins1 + kBlock - 1) / kBlock, (unsigned)w->rows);
+    uint32_t *mine = x + (int64_t)range * w->rows * kBins1;
+    auto out = [&](int off, int nb) { k_range_hist_out<<<bins, kBlock, 0, st>>>(w->hist, off, nb, mine); };
+    auto sum = [&](int off, int nb) { k_range_hist_sum<<<bins, kBlock, 0, st>>>(x, ranges, w->rows, off, nb, w->hist); };
+    switch (stage) {
+    case 0:       // level 1 of this range
+        cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
+        cudaMemsetAsync(w->hit, 0, (size_t)w->rows * 4, st);         // every row takes the classic passes
+        k_topk_hist1<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->hist, w->hit, w->d, vec_ok, w->stride, RowTail{});
+        out(0, kBins1);
+        break;
+    case 1:       // level-1 bucket of the whole rows; level 2 of this range
+        sum(0, kBins1);
+        k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 0, (uint32_t)k_all, w->hit, w->floor_bucket);
+        k_topk_mark<HAS_B><<<fallback, kBlock, 0, st>>>(a, b, w->sel, w->bm_in, w->bm_cand, w->hist, w->hit, w->d, w->wp, vec_ok, w->stride, RowTail{});
+        out(kBins1, kBins2);
+        break;
+    case 2:
+        sum(kBins1, kBins2);
+        k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 1, 0, w->hit, w->floor_bucket);
+        k_topk_hist3<HAS_B><<<fallback_sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_cand, w->hist, w->wp, w->nbt, w->stride, RowTail{});
+        out(kBins1 + kBins2, kBins3);
+        break;
+    case 3:       // the exact threshold; this range's ties
+        sum(kBins1 + kBins2, kBins3);
+        k_topk_pick<<<w->rows, kBlock, 0, st>>>(w->hist, w->sel, 2, 0, w->hit, w->floor_bucket);
+        k_topk_resolve<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->wp, w->nbt, w->stride, nullptr);
+        // the row's number of ties in this range -> word 0 of the row's part of the slot
+        cudaMemsetAsync(mine, 0, (size_t)w->rows * kBins1 * 4, st);
+        k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit, w->cnt_eq, false);
+        cudaMemcpy2DAsync(mine, (size_t)kBins1 * 4, w->cnt_eq, 4, 4, (size_t)w->rows, cudaMemcpyDeviceToDevice, st);
+        break;
+    default: {    // the ties in the order of the ranges; ordered compaction; values and state update
+        k_range_ties_share<<<(w->rows + 63) / 64, 64, 0, st>>>(w->sel, x, range, w->rows);
+        k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
+        k_topk_ties<<<fallback_sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt, nullptr);
+        k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit, w->cnt_eq);      // cnt_eq[row] = entries this range keeps
+        k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic);
+        const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
+        k_range_pad<<<entries, kBlock, 0, st>>>(w->idx, w->val, w->cnt_eq, w->k);
+        k_topk_gather<HAS_B, HAS_B><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);
+        break;
+    }
+    }
+}
+
+void topk_range_stage(TopkWorkspace *w, int stage, const float *a, float *b, bool vec_ok, int64_t k_all,
+                      uint32_t *exchange, int range, int ranges, cudaStream_t st)
+{
+    if (b) range_stage_impl<true>(w, stage, a, b, vec_ok, k_all, exchange, range, ranges, st);
+    else range_stage_impl<false>(w, stage, a, nullptr, vec_ok, k_all, exchange, range, ranges, st);
+}
+
+int64_t topk_range_exchange_words(const TopkWorkspace *w) { return (int64_t)w->rows * kBins1; }
+
 void topk_select(TopkWorkspace *w, const float *a, float *b, bool update_b, bool vec_ok,
                  cudaStream_t st)
 {
     if (b) select_impl<true>(w, a, b, update_b, vec_ok, st);
     else select_impl<false>(w, a, nullptr, false, vec_ok, st);
+}
+
+void topk_select_aggregated(TopkWorkspace *ws, TopkWorkspace *ww, float *ghat_s, float *gtil, int n, bool vec_ok,
+                            cudaStream_t st)
+{
+    const Agg agg = {ww->idx, ww->val, ww->cnt_gt, ww->hit, ww->k, n, (n & (n - 1)) == 0 ? 1 : 0};
+    select_impl<true>(ws, ghat_s, gtil, true, vec_ok, st, &agg, ghat_s);
 }
 
 // Payload of a segment into the payload of the whole vector: entries [at, at + k_seg) of every

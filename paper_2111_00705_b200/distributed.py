@@ -153,7 +153,7 @@ def gather_range_sums(sums, group=None):
 
 
 class RangeShardedCDAdam:
-    """Algorithm 1 with scaled sign, coordinate-sharded across the processes of a
+    """Algorithm 1 with scaled sign (or top-k: ``compressor=binding.TOPK, k=...``), coordinate-sharded across the processes of a
     ``torch.distributed`` group: process r owns coordinates range_partition(d, world, r) of every
     vector.  ``step(grads_local)`` takes the n x (hi - lo) gradients of the owned coordinates;
     ``params()`` is the owned slice of x_{t+1}.  Two all-gathers of a few hundred bytes per
@@ -168,6 +168,13 @@ class RangeShardedCDAdam:
 
     def step(self, grads_local):
         r = self.range
+        if r.compressor == binding.TOPK:       # ten stages, a gather of the histograms / tie counts after eight
+            for stage in range(r.TOPK_STAGES):
+                r.range_topk(stage, grads_local if stage <= 4 else None)
+                buf = r.range_topk_buffer(stage)
+                if buf is not None:
+                    gather_range_sums(buf, self.group)
+            return
         r.range_workers(grads_local)
         gather_range_sums(r.range_buffers()["worker_sums"], self.group)
         r.range_server()

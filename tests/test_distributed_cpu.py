@@ -141,3 +141,26 @@ def test_l1_parts_are_gathered_slot_by_slot_and_added_in_rank_order(world, tmp_p
     for got in res:
         assert torch.equal(got["sums"], want)           # slot r holds rank r's parts, bit for bit
         assert torch.equal(got["total"], res[0]["total"])   # the same additions everywhere
+
+
+def _hist_main(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    # the top-k exchange buffer: [ranks, rows * 2048] words, own slot filled (histogram counts)
+    buf = torch.full((world, 2 * 2048), -1, dtype=torch.int32)
+    buf[rank] = torch.arange(2 * 2048, dtype=torch.int32) * (rank + 1)
+    dd.gather_range_sums(buf)
+    torch.save(buf, os.path.join(out_dir, "h%d.pt" % rank))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_topk_histogram_slots_are_gathered_in_place(tmp_path):
+    world = 3
+    port = 25000 + (os.getpid() * 5) % 1500
+    mp.spawn(_hist_main, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    want = torch.stack([torch.arange(2 * 2048, dtype=torch.int32) * (r + 1) for r in range(world)])
+    for r in range(world):
+        assert torch.equal(torch.load(os.path.join(str(tmp_path), "h%d.pt" % r)), want)
+    # summed over the ranges (what the next stage does) every process gets the same histogram
+    assert torch.equal(want.sum(0), torch.arange(2 * 2048, dtype=torch.int32) * 6)

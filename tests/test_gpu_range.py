@@ -137,7 +137,7 @@ def test_range_context_refuses_what_it_cannot_do():
     lib = cd.lib()
     for lo, hi, r, R in ((5, 5, 0, 1), (-1, 5, 0, 1), (0, 1001, 0, 1), (0, 10, 2, 2), (0, 10, 0, 0)):
         assert not lib.cdadam_create_range(1000, 2, lo, hi, r, R, cd.SIGN, 0, 0.9, 0.999, 1e-3, 1e-8)
-    assert not lib.cdadam_create_range(1000, 2, 0, 10, 0, 1, cd.TOPK, 5, 0.9, 0.999, 1e-3, 1e-8)
+    assert not lib.cdadam_create_range(1000, 2, 0, 10, 0, 1, cd.IDENTITY, 0, 0.9, 0.999, 1e-3, 1e-8)
 
 
 def test_range_sharded_optimizer_over_a_one_rank_group():
@@ -168,3 +168,109 @@ def test_range_sharded_optimizer_over_a_one_rank_group():
         opt.close(); o.close()
     finally:
         dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------- top-k
+
+def make_topk_ranges(w, cuts, x0):
+    return [cd.CDAdamRange(w.d, w.n, cuts[r], cuts[r + 1], r, len(cuts) - 1, beta1=w.beta1, beta2=w.beta2, lr=w.lr,
+                           eps=w.eps, x0=x0[cuts[r]:cuts[r + 1]].contiguous().cuda(), compressor=cd.TOPK, k=w.k)
+            for r in range(len(cuts) - 1)]
+
+
+def emulated_topk_step(ranges, grads):
+    local = [grads[:, c.lo:c.hi].contiguous().reshape(-1) for c in ranges]
+    for stage in range(cd.CDAdamRange.TOPK_STAGES):
+        for c, g in zip(ranges, local):
+            c.range_topk(stage, g if stage <= 4 else None)
+        bufs = [c.range_topk_buffer(stage) for c in ranges]
+        if bufs[0] is None:
+            assert stage in (4, 9)
+            continue
+        for r, b in enumerate(bufs):                    # the all-gather: slot r comes from range r
+            for other in bufs:
+                if other is not b:
+                    other[r].copy_(b[r])
+
+
+def gathered_payload(ranges, who):
+    """The message of `who` put together from the ranges: coordinates of the whole vector."""
+    idx, val = [], []
+    for c in ranges:
+        i, v = c.last_payload(who)
+        i = i.cpu().numpy().view(np.uint32); v = v.cpu().numpy()
+        keep = i != 0xffffffff
+        assert not keep[np.argmin(keep):].any() or keep.all()      # the marked entries come last
+        assert np.all(np.diff(i[keep].astype(np.int64)) > 0) and (i[keep] < c.d).all()
+        idx.append(i[keep].astype(np.int64) + c.lo); val.append(v[keep])
+    return np.concatenate(idx), np.concatenate(val)
+
+
+def run_topk_case(w, cuts, grads_of, steps):
+    x0 = w.x0("cpu")
+    ranges = make_topk_ranges(w, cuts, x0)
+    o = orc.Oracle(w.d, w.n, orc.TOPK, k=w.k, x0=x0.numpy(), beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps)
+    for t in range(1, steps + 1):
+        grads = grads_of(t)
+        emulated_topk_step(ranges, torch.from_numpy(grads).cuda().reshape(w.n, w.d))
+        o.step(grads)
+        torch.cuda.synchronize()
+        for who in list(range(w.n)) + [cd.SERVER]:
+            oi, ov = o.payload(who)
+            gi, gv = gathered_payload(ranges, who)
+            assert np.array_equal(gi, oi.astype(np.int64)), (t, who)
+            assert np.array_equal(gv.view(np.uint32), ov.view(np.uint32)), (t, who)
+        for c in ranges:
+            assert c.step_count() == t
+            for name in orc.STATE_NAMES:
+                got = c.get_state(name).cpu().numpy()
+                want = o.state(name)[..., c.lo:c.hi]
+                assert np.array_equal(got, want), (t, name, c.lo)
+    for c in ranges:
+        c.device_status()
+        c.close()
+    o.close()
+
+
+@pytest.mark.parametrize("cuts", [(0, 131072, 256000), (0, 4096, 100001, 256000), (0, 50000, 50001, 120000, 200003, 256000)])
+def test_topk_coordinate_ranges_equal_the_oracle(cuts):
+    """Top-k of the whole vector selected by 2, 3 and 5 ranges between them (the C3 recipe at
+    d = 256,000, n = 16, k = 2,560): aligned and odd cuts, a range of one coordinate."""
+    w = synth.workload("C3", scale=0.01, steps=3)
+    assert w.d == 256000
+    run_topk_case(w, cuts, lambda t: w.grads(t, "cpu").numpy(), 3)
+
+
+def test_topk_coordinate_ranges_share_the_ties_in_coordinate_order():
+    """Tie-dominated rows: few distinct magnitudes, so the k-th largest is shared by many
+    coordinates in every range and the lower coordinates must win across the cuts; also all
+    values equal, k = 1 and k = d."""
+    rng = np.random.default_rng(17)
+    d, n = 30000, 3
+    cuts = (0, 7000, 7001, 20480, 30000)
+
+    def tied(t):
+        return (rng.integers(-3, 4, size=(n, d)) * 0.5).astype(np.float32)
+
+    for k in (1, 2500, 29999, d):
+        w = synth.Workload("TIES", d, n, synth.TOPK, 3, k=k)
+        run_topk_case(w, cuts, tied, 3)
+    w = synth.Workload("FLAT", d, n, synth.TOPK, 2, k=777)
+    run_topk_case(w, cuts, lambda t: np.full((n, d), 1.5 * t, np.float32), 2)
+
+
+def test_topk_range_context_refuses_wrong_stages():
+    c = cd.CDAdamRange(10000, 2, 1000, 6000, 0, 2, compressor=cd.TOPK, k=50)
+    g = torch.zeros(2 * 5000, device="cuda")
+    with pytest.raises(cd.CdadamError) as e:
+        c.range_topk(1, g)
+    assert e.value.code == cd.ERR_STATE
+    with pytest.raises(cd.CdadamError):
+        c.range_workers(g)                              # the scaled-sign stages
+    with pytest.raises(cd.CdadamError):
+        c.step(g)
+    c.range_topk(0, g)
+    assert c.range_topk_buffer(0).shape == (2, 2 * 2048) and c.range_topk_buffer(5).shape == (2, 2048)
+    assert c.range_topk_buffer(4) is None
+    c.close()
+    assert not cd.lib().cdadam_create_range(1000, 2, 0, 10, 0, 1, cd.TOPK, 1001, 0.9, 0.999, 1e-3, 1e-8)
