@@ -211,8 +211,12 @@ def run_distributed(args, w, dev, rank, world):
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         os.environ.setdefault("MASTER_PORT", str(29000 + os.getpid() % 2000))
         dist.init_process_group("nccl", rank=0, world_size=1, device_id=dev)
-    server_rank = 0 if args.layout == "server" else None
     args.warmup = max(args.warmup, 3)
+    if args.layout == "range":
+        run_range(args, w, dev, rank, world)
+        dist.destroy_process_group()
+        return
+    server_rank = 0 if args.layout == "server" else None
     opt = dd.DistributedCDAdam(w.d, w.n, None, server_rank, beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps,
                                offsets=w.offsets, x0=w.x0(dev), device=dev, compressor=w.compressor, k=w.k)
     first, per = dd.partition(w.n, world, rank, server_rank)
@@ -246,6 +250,77 @@ def run_distributed(args, w, dev, rank, world):
             "gpu_launches": opt.shard.launches_per_step() * args.steps, "clocks": clocks}))
     opt.close()
     dist.destroy_process_group()
+
+
+def run_range(args, w, dev, rank, world):
+    """The coordinate-sharded deployment: every process owns d / N coordinates of all n workers
+    and of the server; the l1 parts (scaled sign) or the histograms and tie counts (top-k) are
+    all-gathered.  Strong scaling.  With --of-ranges R on ONE process the context is range 0 of
+    R: the time of one rank's share, its gathers being one-rank collectives - a projection of
+    the N = R step without the latency of R-rank collectives, said so in the line."""
+    import torch
+    import torch.distributed as dist
+    from paper_2111_00705_b200 import binding as cd
+    from paper_2111_00705_b200 import distributed as dd
+    ranges = args.of_ranges if (world == 1 and args.of_ranges > 1) else world
+    lo, hi = dd.range_partition(w.d, ranges, rank)
+    if ranges != world:
+        opt = dd.RangeShardedCDAdam.__new__(dd.RangeShardedCDAdam)
+        opt.group, opt.world, opt.rank, opt.lo, opt.hi = None, 1, 0, lo, hi
+        opt.range = cd.CDAdamRange(w.d, w.n, lo, hi, 0, ranges, beta1=w.beta1, beta2=w.beta2, lr=w.lr, eps=w.eps,
+                                   offsets=w.offsets, x0=w.x0(dev)[lo:hi].contiguous(), device=dev,
+                                   compressor=w.compressor, k=w.k)
+    else:
+        opt = dd.RangeShardedCDAdam(w.d, w.n, offsets=w.offsets, x0=w.x0(dev)[lo:hi].contiguous(), beta1=w.beta1,
+                                    beta2=w.beta2, lr=w.lr, eps=w.eps, device=dev, compressor=w.compressor, k=w.k)
+    grads = [w.grads(t + 1, dev).reshape(w.n, w.d)[:, lo:hi].contiguous().reshape(-1) for t in range(2)]
+    stream = torch.cuda.current_stream()
+
+    def step(t):
+        if ranges == world:
+            opt.step(grads[t % 2])
+            return
+        r = opt.range                                  # one range of several: its gathers stay on this process
+        if r.compressor == cd.TOPK:
+            for stage in range(r.TOPK_STAGES):
+                r.range_topk(stage, grads[t % 2] if stage <= 4 else None)
+                buf = r.range_topk_buffer(stage)
+                if buf is not None:
+                    dist.all_gather_into_tensor(buf[0], buf[0].clone())
+        else:
+            r.range_workers(grads[t % 2])
+            b = r.range_buffers()["worker_sums"]; dist.all_gather_into_tensor(b[0].view(-1), b[0].reshape(-1).clone())
+            r.range_server()
+            b = r.range_buffers()["server_sums"]; dist.all_gather_into_tensor(b[0].view(-1), b[0].reshape(-1).clone())
+            r.range_update()
+
+    for t in range(args.warmup):
+        step(t)
+    dist.barrier(); torch.cuda.synchronize()
+    sampler = ClockSampler(dev.index) if rank == 0 else None
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(stream)
+    for t in range(args.steps):
+        step(t)
+    b.record(stream)
+    dist.barrier(); torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    total_ms = max_over_ranks_ms(a.elapsed_time(b), dev)
+    opt.range.device_status()
+    value = args.steps / (total_ms * 1e-3)
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+            "scaling": "strong", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": describe(w), "layout": "range", "ranges": ranges,
+                       "coordinates_per_rank": hi - lo,
+                       "projection": None if ranges == world else
+                       "one process timed as range 0 of %d (its share of the work, one-rank gathers): "
+                       "not a %d-GPU measurement" % (ranges, ranges)},
+            "params_per_s": value * w.d,
+            "gpu_launches": opt.range.launches_per_step() * args.steps, "clocks": clocks}))
+    opt.close()
 
 
 def l2_small(w):
@@ -450,11 +525,15 @@ def main():
                     help="markov = Algorithm 1 (default); ef = classical error feedback, naive = naive "
                          "compression (the comparison schemes of Section 4; their bytes differ, so the "
                          "roofline figures of such a run are not the headline's)")
-    ap.add_argument("--layout", default="replicas", choices=["replicas", "sharded", "server"],
+    ap.add_argument("--of-ranges", type=int, default=0,
+                    help="--layout range on one process: time range 0 of this many ranges (a projection)")
+    ap.add_argument("--layout", default="replicas", choices=["replicas", "sharded", "server", "range"],
                     help="replicas (default): every rank runs the whole n-worker problem on its own.  "
                          "sharded: the distributed deployment, n/N workers per rank, worker messages "
                          "all-gathered over NCCL, server stage computed on every rank (scaled sign only; "
-                         "strong scaling).  server: rank 0 is the server and holds no worker (N >= 2)")
+                         "strong scaling).  server: rank 0 is the server and holds no worker (N >= 2).  "
+                         "range: the coordinate-sharded deployment, d/N coordinates of all workers per rank, "
+                         "only the l1 parts / top-k histograms gathered")
     ap.add_argument("--tile", type=int, default=0,
                     help="force the kernels' tile size (profiler captures of scaled-down cases)")
     ap.add_argument("--scale", type=float, default=1.0,

@@ -80,7 +80,7 @@ enum {
  * Create a context (inputs of Algorithm 1: beta1, beta2, nu = eps, step size lr, C).
  *   d          model dimension, 1 <= d < 2^32
  *   n          number of simulated workers, 1 <= n <= 65535
- *   compressor CDADAM_SIGN, CDADAM_TOPK or CDADAM_IDENTITY
+ *   compressor CDADAM_SIGN, CDADAM_TOPK, CDADAM_RANDK or CDADAM_IDENTITY
  *   k          entries kept by top-k / rand-k at the workers and at the server,
  *              1 <= k <= d; ignored for the other compressors
  * All state is allocated here, on the current device, and zero-initialised (Algorithm 1
@@ -103,7 +103,12 @@ void cdadam_destroy(cdadam_ctx *ctx);
  *   stream  cudaStream_t; must not be under stream capture (CDADAM_ERR_STATE, nothing
  *           queued): launch arguments alternate between steps, so a step replayed from a
  *           caller's graph would be wrong
- * Allocates no device memory.  Where the step is launch-bound (scaled sign, every pass a
+ * Allocates no device memory for the method's data: all vectors and scratch were allocated
+ * by cdadam_create.  Two kinds of call do create CUDA objects, once each: the second step on a
+ * given gradient buffer of a configuration that is replayed from a graph (see below)
+ * instantiates that graph (up to four per context; milliseconds, and the driver may allocate
+ * for it), and cdadam_step_bf16 / cdadam_step_host allocate their staging buffer at their
+ * first call.  Where the step is launch-bound (scaled sign, every pass a
  * single wave of blocks, about n*d <= 2.4e6) the scales are finished inside the passes
  * (3 launches instead of 5) and, from the second step on the same gradient buffer, the
  * launches are replayed from a CUDA graph owned by the context; so are the some thirty

@@ -558,6 +558,8 @@ static cdadam_ctx *create_impl(int64_t d, int n, int first, int nloc, int compre
         }
     } while (0);
     if (rc != CDADAM_OK || cudaDeviceSynchronize() != cudaSuccess) { cdadam_destroy(c); return nullptr; }
+    // the stream on which a step is recorded for replay (not inside cdadam_step)
+    if (cudaStreamCreateWithFlags(&c->cap_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); c->cap_stream = nullptr; }
     topk_workspace_set_error_flag(c->tk_w, c->error_flag);
     topk_workspace_set_error_flag(c->tk_s, c->error_flag);
     // Algorithm 1 with top-k: ghat^(i) += c^(i) at the kept coordinates is left to the next

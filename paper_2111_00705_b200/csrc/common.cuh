@@ -153,7 +153,7 @@ __device__ __forceinline__ float ld_cg_f32(const float *p) { return __ldcg(p); }
 __device__ __forceinline__ float4 ld_cg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
 
 // ------------------------------------------------------------------------------------
-// Bulk asynchronous copies (TMA, one-dimensional, no multicast) global -> shared, completed
+// Plain bulk asynchronous copies (TMA, one-dimensional, one destination block) global -> shared, completed
 // on an mbarrier.  Addresses and sizes must be multiples of 16 bytes.  Every wait is
 // bounded: a barrier that does not complete makes the caller report an error and leave.
 // ------------------------------------------------------------------------------------

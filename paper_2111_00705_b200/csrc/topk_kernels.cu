@@ -16,12 +16,19 @@
 // keeps them per 4096-coordinate tile as a short list (position in the tile, value) in index
 // order.  The histogram fixes key bits 30..11 of the threshold; one pass over the lists
 // (bits 10..0) fixes the rest: two levels instead of three.  Every later pass of such a row
-// walks these lists, one warp per tile, with coalesced reads; selection, ties and the ordered
-// compaction follow from per-tile counts and two scans, without bitmaps.  A tile with more coordinates above the floor than its list holds
+// walks these lists, one warp per tile, with coalesced reads: k_topk_split (low-bits histogram
+// and per-tile candidate records), k_scan_lists (exact threshold, per-tile counts, tie ranks
+// and payload offsets, one block per row) and k_topk_emit_idx (ordered compaction with the
+// values), without bitmaps.  A tile with more coordinates above the floor than its list holds
 // (a selection concentrated in one tensor) is read again from the data by those passes.  If
 // fewer than k coordinates lie above the floor, or the threshold lies above the fine bins,
-// the classic two dense passes and the bitmap passes run instead.  The same file holds the sparse
-// server aggregation and the rand-k path, which shares the payload kernels.
+// the classic two dense passes and the bitmap passes run instead, as a second chain of
+// launches beside the first.  The state update b += u at the kept coordinates is part of the
+// compaction, or, for rows selected from lists of a workspace that defers it, of the next
+// selection's dense pass (one streaming pass instead of k random read-modify-writes per row).
+// The server's aggregation of the workers' messages runs inside the dense pass of the server's
+// selection.  The same file holds the separate sparse aggregation kernel, the rand-k path,
+// which shares the payload kernels, and the staged selection over coordinate ranges.
 #include "topk.h"
 
 #include <algorithm>
@@ -93,10 +100,11 @@ __device__ __forceinline__ float diff1(const float *a, const float *b, int64_t j
     return HAS_B ? __fsub_rn(a[j], b[j]) : a[j];
 }
 
-// exclusive prefix sum over the 256 threads of a block; all threads must call
-__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
+// exclusive prefix sum over the NT threads of a block; all threads must call
+template <int NT>
+__device__ __forceinline__ uint32_t block_excl_scan_n(uint32_t v, uint32_t &total)
 {
-    __shared__ uint32_t ws[kBlock / 32];
+    __shared__ uint32_t ws[NT / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t inc = v;
 #pragma unroll
@@ -109,7 +117,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
     __syncthreads();
     uint32_t before = 0, all = 0;
 #pragma unroll
-    for (int w = 0; w < kBlock / 32; ++w) {
+    for (int w = 0; w < NT / 32; ++w) {
         const uint32_t s = ws[w];
         if (w < warp) before += s;
         all += s;
@@ -117,6 +125,7 @@ __device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total)
     total = all;
     return before + inc - v;
 }
+__device__ __forceinline__ uint32_t block_excl_scan(uint32_t v, uint32_t &total) { return block_excl_scan_n<kBlock>(v, total); }
 
 // ------------------------------------------------------------------------------------
 // Pick the bucket that holds the `want`-th largest entry of a row's histogram: the bucket b
@@ -729,7 +738,7 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
 // ------------------------------------------------------------------------------------
 // The same pass over whole tiles with a prefetch ring.  A block owns kSpecTiles consecutive
 // tiles of a row; the a and b sub-tiles arrive in a two-stage shared-memory ring by bulk
-// asynchronous copies (TMA, no multicast) issued by one thread, so the next tile is in
+// asynchronous copies (plain TMA bulk copies) issued by one thread, so the next tile is in
 // flight while the block works on the current one.  Arithmetic, histogram and lists are those
 // of k_topk_spec; the flagged groups are kept as positions only and read back from the stage.
 // Every wait on a copy is bounded; one that runs out sets *error_flag (if given), lets the
@@ -1160,15 +1169,19 @@ k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__rest
 // tile, the rank of its first tie among the row's ties (cnt_eq) and the payload offset of its
 // first kept coordinate (cnt_gt); a tile keeps its keys above T and those of its ties whose
 // rank is below k3.  Every eighth tile's offset is also the offset of its 32768-coordinate
-// span (cnt_fin), which the server aggregation uses.  The counts pass through shared memory
-// in chunks of 4096 tiles (coalesced loads and stores); inside a chunk a thread owns 16
-// consecutive tiles (padded rows, no bank conflicts).  grid = (rows).
-constexpr int kScanPer = 16;
-constexpr int kScanChunk = kBlock * kScanPer;
+// span (cnt_fin), which the server aggregation uses.  The counts come from k_topk_split's
+// per-tile records (certainly kept values, candidates and their low key bits) once this kernel
+// has picked the exact threshold from the low-bits histogram.  They pass through shared memory
+// in chunks of 4096 tiles (coalesced loads and stores); inside a chunk a thread owns 4
+// consecutive tiles (padded rows, no bank conflicts).  grid = (rows), 1024 threads: the row's
+// scan is one block's serial work, so the block is as wide as it gets.
+constexpr int kScanBlock = 1024;      // one block per row does the whole scan: as wide as a block gets
+constexpr int kScanPer = 4;
+constexpr int kScanChunk = kScanBlock * kScanPer;
 __device__ __forceinline__ int scan_slot(int i) { return i + i / kScanPer; }
 
 template <bool HAS_B>
-__global__ void __launch_bounds__(kBlock)
+__global__ void __launch_bounds__(kScanBlock)
 k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
              Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
              const uint32_t *__restrict__ hist_all, uint32_t *__restrict__ floor_bucket,
@@ -1177,26 +1190,25 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
              uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all,
              uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt, int64_t d, int64_t stride)
 {
-    __shared__ uint32_t s_eq[kScanChunk + kBlock], s_gt[kScanChunk + kBlock];
+    __shared__ uint32_t s_eq[kScanChunk + kScanBlock], s_gt[kScanChunk + kScanBlock];
     __shared__ uint32_t s_T, s_k3, s_c3;
     const int row = blockIdx.x;
     if (!hit[row]) return;
     // The exact threshold first: the bucket of key bits 10..0 that holds the k1-th largest of
     // the candidates (the histogram k_topk_split made), as k_topk_pick does for the classic rows.
     {
-        uint32_t *tot = s_eq;                          // kBlock words, free until the scan starts
         Sel *sel = sel_all + row;
         const uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
         const uint32_t want = sel->k1;
-        const int per = kBins2 / kBlock, lo = threadIdx.x * per;
-        uint32_t own[kBins2 / kBlock];
+        constexpr int per = kBins2 / kScanBlock;
+        const int lo = threadIdx.x * per;
+        uint32_t own[per];
         uint32_t mine = 0;
 #pragma unroll
         for (int t = 0; t < per; ++t) { own[t] = hist[lo + t]; mine += own[t]; }
-        tot[threadIdx.x] = mine;
-        __syncthreads();
-        uint32_t above = 0;
-        for (int t = threadIdx.x + 1; t < kBlock; ++t) above += tot[t];
+        uint32_t all;
+        const uint32_t before = block_excl_scan_n<kScanBlock>(mine, all);
+        uint32_t above = all - before - mine;          // entries in bins owned by later threads
 #pragma unroll
         for (int t = per - 1; t >= 0; --t) {
             const uint32_t c = own[t];
@@ -1226,7 +1238,7 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
         uint2 C4[kScanPer];
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
-            const int64_t t = c0 + m * kBlock + threadIdx.x;
+            const int64_t t = c0 + m * kScanBlock + threadIdx.x;
             const bool in = t < nt4k;
             G[m] = in ? gt[t] : 0u;
             NC[m] = in ? eq[t] : 0u;
@@ -1234,7 +1246,7 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
         }
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
-            const int i = m * kBlock + threadIdx.x;
+            const int i = m * kScanBlock + threadIdx.x;
             const int64_t t = c0 + i;
             // keys above / equal to T in tile t: the certainly kept values plus the candidates
             uint32_t g = G[m], e = 0u;
@@ -1263,12 +1275,12 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
             s_gt[scan_slot(i)] = g;
         }
         __syncthreads();
-        const int mine = threadIdx.x * (kScanPer + 1);  // first slot of this thread's 16 tiles
+        const int mine = threadIdx.x * (kScanPer + 1);  // first slot of this thread's tiles
         uint32_t sum_eq = 0;
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) sum_eq += s_eq[mine + m];
         uint32_t total_eq, total_keep;
-        uint32_t tie_rank = carry_eq + block_excl_scan(sum_eq, total_eq);
+        uint32_t tie_rank = carry_eq + block_excl_scan_n<kScanBlock>(sum_eq, total_eq);
         uint32_t sum_keep = 0;
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
@@ -1280,7 +1292,7 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
             s_gt[mine + m] = keep;
             sum_keep += keep;
         }
-        uint32_t off = carry_keep + block_excl_scan(sum_keep, total_keep);
+        uint32_t off = carry_keep + block_excl_scan_n<kScanBlock>(sum_keep, total_keep);
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
             const uint32_t keep = s_gt[mine + m];
@@ -1290,7 +1302,7 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
         __syncthreads();
 #pragma unroll
         for (int m = 0; m < kScanPer; ++m) {
-            const int i = m * kBlock + threadIdx.x;
+            const int i = m * kScanBlock + threadIdx.x;
             const int64_t t = c0 + i;
             if (t < nt4k) {
                 const uint32_t o = s_gt[scan_slot(i)];
@@ -1367,6 +1379,18 @@ k_topk_ties(const Sel *__restrict__ sel_all, const uint32_t *__restrict__ hit,
 // is written with the index.  Other rows: from the selection bitmap; a thread owns 4
 // consecutive bitmap words, ranks come from popcount scans, values follow in k_topk_gather.
 // ------------------------------------------------------------------------------------
+// What the compaction does besides writing the payload.  b_rw != NULL: b_j += u_j at the kept
+// coordinates (rows x stride floats, the same array the selection subtracted), unless the row
+// defers it (pending != NULL and the row was selected from lists: pending[row] = 1 and the
+// next dense pass applies the payload).  classic_values: rows whose guess failed get their
+// values (u_j = a_j - b_j, read here) and their update in this kernel too; without it only
+// their coordinates are written and k_topk_gather follows.
+struct EmitUpdate {
+    float *b_rw;
+    uint32_t *pending;
+    int classic_values;
+};
+
 template <bool HAS_B>
 __global__ void __launch_bounds__(kBlock)
 k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all,
@@ -1376,12 +1400,16 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
                 const uint32_t *__restrict__ stash_cnt_all, const uint32_t *__restrict__ cnt_gt_all,
                 const uint32_t *__restrict__ cnt_eq_all, uint32_t *__restrict__ idx_all,
                 float *__restrict__ val_all, int64_t wp, int64_t nbt, int64_t k, int64_t nt4k, int64_t d, int64_t stride,
-                int kind)
+                int kind, EmitUpdate upd)
 {
     const int row = blockIdx.y;
     if (!(kind & (hit[row] ? kRowsListed : kRowsClassic))) return;
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
+    float *b_rw = upd.b_rw ? upd.b_rw + (int64_t)row * stride : nullptr;
+    // a row selected from lists may leave its state update to the next selection's dense pass
+    const bool deferred = upd.pending != nullptr && hit[row] != 0u;
+    if (upd.pending && blockIdx.x == 0 && threadIdx.x == 0) upd.pending[row] = deferred ? 1u : 0u;
     if (hit[row]) {
         if ((int64_t)blockIdx.x * kListTiles >= nt4k) return;
         const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
@@ -1420,6 +1448,7 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
                 if (keep && at < k) {
                     idx[at] = base + pos_e;
                     val[at] = val_e;
+                    if (b_rw && !deferred) b_rw[base + pos_e] = __fadd_rn(b_rw[base + pos_e], val_e);   // b += u (Algorithm 1)
                 }
                 out[m] += __popc(km);
                 tie_rank[m] += __popc(eqm);
@@ -1454,7 +1483,22 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
         while (word) {
             const int bit = __ffs(word) - 1;
             word &= word - 1;
-            if (rank < k) idx[rank] = (uint32_t)((w0 + m) * 32 + bit);
+            const int64_t j = (w0 + m) * 32 + bit;
+            if (rank < k) {
+                idx[rank] = (uint32_t)j;
+                if (upd.classic_values) {             // the value u_j and the state update with it
+                    const float aj = a_all[(int64_t)row * stride + j];
+                    if (HAS_B) {
+                        // (read through the writable pointer where there is one: this kernel writes b)
+                        const float bj = b_rw ? b_rw[j] : b_all[(int64_t)row * stride + j];
+                        const float u = __fsub_rn(aj, bj);
+                        val[rank] = u;
+                        if (b_rw) b_rw[j] = __fadd_rn(bj, u);
+                    } else {
+                        val[rank] = aj;
+                    }
+                }
+            }
             ++rank;
         }
     }
@@ -1744,7 +1788,7 @@ void topk_payload(TopkWorkspace *w, int row, const uint32_t **idx, const float *
     *val = w->val + (int64_t)row * w->k;
 }
 
-constexpr int kSelectLaunches = 12;      // dense pass, pick, six for the classic chain, three for the listed chain, gather
+constexpr int kSelectLaunches = 11;      // dense pass, pick, six for the classic chain, three for the listed chain
 int topk_launches_per_step(int) { return 2 * kSelectLaunches; }    // two selections; the aggregation kernel is counted by the caller
 
 // Whole tiles per row that the dense pass takes through the prefetch ring (0: none).
@@ -1801,6 +1845,8 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // every pick and scan is done by the block that finishes its row last) take the classic
     // passes on the side stream ...
     const dim3 fallback_sparse(std::min(sparse.x, fallback.x), (unsigned)w->rows);
+    // values, state update (or its deferral) happen inside the ordered compaction
+    const EmitUpdate upd = {HAS_B && update_b ? b : nullptr, defer ? w->pending : nullptr, 1};
     cudaStream_t sd = w->side;
     cudaEventRecord(w->ev_fork, st);
     cudaStreamWaitEvent(sd, w->ev_fork, 0);
@@ -1811,20 +1857,13 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     k_topk_hist3<HAS_B><<<fallback_sparse, kBlock, 0, sd>>>(a, b, w->sel, w->hit, w->bm_cand, w->hist, w->wp, w->nbt, w->stride, tail(2));
     k_topk_resolve<HAS_B><<<sparse, kBlock, 0, sd>>>(a, b, w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->wp, w->nbt, w->stride, w->tick + (size_t)3 * w->rows);
     k_topk_ties<<<fallback_sparse, kBlock, 0, sd>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt, w->tick + (size_t)4 * w->rows);
-    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, sd>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, sd>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic, upd);
     cudaEventRecord(w->ev_join, sd);
     // ... and the rows selected from the dense pass's lists take three launches on this one
     k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->cnt_gt, w->cnt_eq, w->cand, w->nt4k, w->d, w->stride);
-    k_scan_lists<HAS_B><<<w->rows, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->hist, w->floor_bucket, w->stash, w->stash_cnt, w->cand, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt, w->d, w->stride);
-    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsListed);
+    k_scan_lists<HAS_B><<<w->rows, kScanBlock, 0, st>>>(a, b, w->sel, w->hit, w->hist, w->floor_bucket, w->stash, w->stash_cnt, w->cand, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt, w->d, w->stride);
+    k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsListed, upd);
     cudaStreamWaitEvent(st, w->ev_join, 0);
-    dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
-    if (defer) entries.x = std::min(entries.x, 96u);   // rows selected from lists defer: nothing to do for them
-    if (HAS_B && update_b)
-        k_topk_gather<HAS_B, true><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride,
-                                                               defer ? w->pending : nullptr);
-    else
-        k_topk_gather<HAS_B, false><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);
 }
 
 // ------------------------------------------------------------------------------------
@@ -1930,7 +1969,7 @@ static void range_stage_impl(TopkWorkspace *w, int stage, const float *a, float 
         k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
         k_topk_ties<<<fallback_sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt, nullptr);
         k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit, w->cnt_eq);      // cnt_eq[row] = entries this range keeps
-        k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic);
+        k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic, EmitUpdate{nullptr, nullptr, 0});
         const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
         k_range_pad<<<entries, kBlock, 0, st>>>(w->idx, w->val, w->cnt_eq, w->k);
         k_topk_gather<HAS_B, HAS_B><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);
