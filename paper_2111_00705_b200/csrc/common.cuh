@@ -145,6 +145,25 @@ __device__ __forceinline__ void st_rw4(float *p, float4 v)
     __stcs(reinterpret_cast<float4 *>(p), v);
 }
 __device__ __forceinline__ uint32_t ld_ro_u32(const uint32_t *p) { return __ldg(p); }
+// 256-bit accesses (eight consecutive floats of one thread, 32-byte aligned): a warp then
+// covers 1 KiB of a vector with whole 32-byte sectors per thread.
+__device__ __forceinline__ void ld_ro8(const float *p, float (&v)[8])
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ void ld_rw8(const float *p, float (&v)[8])
+{
+    asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_rw8(float *p, const float (&v)[8])
+{
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(v[0]), "f"(v[1]), "f"(v[2]),
+                 "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]) : "memory");
+}
 // Coherent (L2) loads for what the kernel queued just before wrote: under programmatic
 // dependent launch this grid is already resident while that kernel runs, so such data is not
 // read-only for this grid's lifetime and must not go through the non-coherent path.

@@ -520,12 +520,12 @@ __device__ __forceinline__ uint64_t transpose8x8(uint64_t x)
 }
 
 template <int VPT, int MODE>
-__global__ void __launch_bounds__(kBlock)
+__global__ void __launch_bounds__(kBlock, 4)
 k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wscale,
               float *__restrict__ ghat_s, const float *__restrict__ gtil,
               uint32_t *__restrict__ sbits, dd *__restrict__ spart, Tables tb, int n,
               int64_t wp, int vec_ok, int n_pow2, float *__restrict__ sscale,
-              unsigned int *__restrict__ done)
+              unsigned int *__restrict__ done, int vec8_ok)
 {
     constexpr bool EF = MODE != 0;
     __shared__ __align__(16) uint32_t wsm[kBlock / 32][kNC][4][VPT];   // [warp][worker][g][v]
@@ -544,6 +544,74 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
     grid_dep_launch();
     grid_dep_wait();                          // worker sign words and scales come from the kernels before
 
+    if (vec8_ok && first == last && base + tb.tile <= tb.d) {
+        // Eight consecutive coordinates per thread (256-bit accesses; d % 8 == 0).  A lane's
+        // coordinates are one byte of a sign word: byte (lane & 3) of word (lane >> 2) of the
+        // warp's eight.  The lane gathers that byte from the words of workers 0..7 (PRMT),
+        // one 8x8 bit transpose turns the eight bytes into the eight coordinates' sender
+        // patterns, and the pattern table gives each coordinate's sum; further workers are
+        // added one by one.  The new sign bits are packed as a byte per lane and joined
+        // across the four lanes of a word by two shuffles (no ballots, no interleave).
+        constexpr int kSpan8 = 256, kIter8 = kSpan8 * (kBlock / 32);
+        const int nt = min(n, kTabWorkers);
+        if (threadIdx.x < nt) ssm[threadIdx.x] = ld_cg_f32(wscale + (int64_t)threadIdx.x * tb.q + first);
+        __syncthreads();
+        {
+            float t = 0.0f;
+            for (int i = 0; i < nt; ++i) t = __fadd_rn(t, signed_scale((threadIdx.x >> i) & 1u, ssm[i]));
+            tab[threadIdx.x] = t;                         // kBlock == 256 patterns (bits above nt are never set)
+        }
+        __syncthreads();
+        const uint32_t bsel = lane & 3u;
+        const uint32_t sel01 = bsel | ((bsel + 4u) << 4);     // PRMT: byte bsel of a, byte bsel of b
+        dd acc = {0.0, 0.0};
+        for (int it = 0; it < tb.tile / kIter8; ++it) {
+            const int64_t wb = base + (int64_t)it * kIter8 + warp * kSpan8;
+            const int64_t j = wb + lane * 8;
+            float H[8], Gt[8];
+#pragma unroll
+            for (int c = 0; c < 8; ++c) H[c] = Gt[c] = 0.0f;
+            if (!EF) ld_rw8(ghat_s + j, H);               // error feedback overwrites this buffer
+            if (MODE != 2) ld_ro8(gtil + j, Gt);
+            const uint32_t *wrow = wbits + (wb >> 5) + (lane >> 2);
+            uint32_t W[kTabWorkers];
+#pragma unroll
+            for (int i = 0; i < kTabWorkers; ++i) W[i] = i < nt ? ld_cg_u32(wrow + (int64_t)i * wp) : 0u;
+            const uint32_t lo = __byte_perm(__byte_perm(W[0], W[1], sel01), __byte_perm(W[2], W[3], sel01), 0x5410u);
+            const uint32_t hi = __byte_perm(__byte_perm(W[4], W[5], sel01), __byte_perm(W[6], W[7], sel01), 0x5410u);
+            const uint64_t pat = transpose8x8(((uint64_t)hi << 32) | lo);
+            const uint32_t plo = (uint32_t)pat, phi = (uint32_t)(pat >> 32);
+            float a[8];
+            a[0] = tab[plo & 0xFFu];         a[1] = tab[(plo >> 8) & 0xFFu];
+            a[2] = tab[(plo >> 16) & 0xFFu]; a[3] = tab[plo >> 24];
+            a[4] = tab[phi & 0xFFu];         a[5] = tab[(phi >> 8) & 0xFFu];
+            a[6] = tab[(phi >> 16) & 0xFFu]; a[7] = tab[phi >> 24];
+            for (int i = nt; i < n; ++i) {                // workers in increasing order
+                const float s = ld_cg_f32(wscale + (int64_t)i * tb.q + first);
+                const uint32_t byte = ld_cg_u32(wrow + (int64_t)i * wp) >> (8u * bsel);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) a[c] = __fadd_rn(a[c], signed_scale((byte >> c) & 1u, s));
+            }
+            float S[8];
+            uint32_t bits = 0u;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                const float mean = n_pow2 ? __fmul_rn(a[c], rn) : __fdiv_rn(a[c], fn);
+                const float w = server_step<EF>(mean, H[c], Gt[c], S[c]);
+                dd_acc(acc, fabsf(w));
+                bits |= (w >= 0.0f ? 1u : 0u) << c;
+            }
+            st_rw8(ghat_s + j, S);
+            uint32_t word = bits << (8u * bsel);
+            word |= __shfl_xor_sync(kFull, word, 1);
+            word |= __shfl_xor_sync(kFull, word, 2);
+            if (bsel == 0u) sbits[(wb >> 5) + (lane >> 2)] = word;
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) part[0] = acc;
+        if (sscale) finish_segment(spart, sscale, done, first, tb.off, tb.tile_first, tb.pbase, tb.tile);
+        return;
+    }
     if (vec_ok && first == last && base + tb.tile <= tb.d) {
         constexpr int kSpan = 128 * VPT;                  // coordinates per warp per iteration
         constexpr int kIter = kSpan * (kBlock / 32);      // per block per iteration
@@ -921,8 +989,10 @@ void launch_server_sign(const uint32_t *wbits, const float *wscale, float *ghat_
 {
     const int pow2 = (n & (n - 1)) == 0;
     auto kern = mode == 2 ? k_server_sign<2, 2> : mode == 1 ? k_server_sign<2, 1> : k_server_sign<2, 0>;
+    // 256-bit accesses need d % 8 == 0 (the vectors are the context's own: 256-byte aligned)
+    const int vec8 = vec_ok && tb.d % 8 == 0 && (((uintptr_t)ghat_s | (uintptr_t)gtil) & 31u) == 0;
     launch_after(kern, dim3((unsigned)tb.ntiles), dim3(kBlock), 0, st, wbits, wscale, ghat_s, gtil, sbits, spart, tb, n, wp,
-                 (int)vec_ok, pow2, sscale, done);
+                 (int)vec_ok, pow2, sscale, done, vec8);
 }
 
 void launch_update_sign(const uint32_t *sbits, const float *sscale, const float *ghat_s, float *gtil,
