@@ -91,6 +91,18 @@ __device__ __forceinline__ float4 grad_ld4(const bf16_t *g)
     return make_float4(__uint_as_float(raw.x << 16), __uint_as_float(raw.x & 0xffff0000u),
                        __uint_as_float(raw.y << 16), __uint_as_float(raw.y & 0xffff0000u));
 }
+// eight consecutive gradients (32-byte / 16-byte aligned)
+__device__ __forceinline__ void grad_ld8(const float *g, float (&v)[8]) { ld_ro8(g, v); }
+__device__ __forceinline__ void grad_ld8(const bf16_t *g, float (&v)[8])
+{
+    uint4 raw;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(raw.x), "=r"(raw.y), "=r"(raw.z), "=r"(raw.w) : "l"(g));
+    v[0] = __uint_as_float(raw.x << 16); v[1] = __uint_as_float(raw.x & 0xffff0000u);
+    v[2] = __uint_as_float(raw.y << 16); v[3] = __uint_as_float(raw.y & 0xffff0000u);
+    v[4] = __uint_as_float(raw.z << 16); v[5] = __uint_as_float(raw.z & 0xffff0000u);
+    v[6] = __uint_as_float(raw.w << 16); v[7] = __uint_as_float(raw.w & 0xffff0000u);
+}
 // four consecutive gradients from a shared-memory copy of a sub-tile
 __device__ __forceinline__ float4 grad_lds4(const float *g) { return *reinterpret_cast<const float4 *>(g); }
 __device__ __forceinline__ float4 grad_lds4(const bf16_t *g)
@@ -252,7 +264,7 @@ __global__ void __launch_bounds__(kBlock, 4)
 k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
               uint32_t *__restrict__ wbits, const float *__restrict__ scale_old,
               dd *__restrict__ wpart, Tables tb, int64_t wp, int vec_ok,
-              float *__restrict__ scale_new, unsigned int *__restrict__ done)
+              float *__restrict__ scale_new, unsigned int *__restrict__ done, int vec8_ok)
 {
     grid_dep_launch();
     const int i = blockIdx.y;
@@ -267,6 +279,47 @@ k_worker_sign(const G *__restrict__ grads, float *__restrict__ ghat_w,
     if (!(vec_ok && first == last && base + tb.tile <= tb.d)) {
         worker_tile_scalar<EF, G>(g, gh, bw, so, wpart + (int64_t)i * tb.nparts + tb.pbase[T], tb.off, base,
                            min(base + (int64_t)tb.tile, tb.d), first, last);
+    } else if (vec8_ok) {
+        // Eight consecutive coordinates per thread (256-bit accesses; rows 32-byte aligned): a
+        // lane's coordinates are byte (lane & 3) of word (lane >> 2) of the warp's eight sign
+        // words, both of the previous payload that is applied first and of the new one, which
+        // is packed as a byte per lane and joined over the word's four lanes by two shuffles.
+        const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+        const float s = so[first];
+        const uint32_t bsel = lane & 3u;
+        dd acc = {0.0, 0.0};
+        // two 2048-coordinate sub-tiles per round: both rounds of loads are in flight together
+        for (int it = 0; it < tb.tile / (8 * kBlock); it += 2) {
+            float Gv[2][8], H[2][8];
+            uint32_t old[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t wb = base + (int64_t)(it + h) * (8 * kBlock) + warp * 256;
+                grad_ld8(g + wb + lane * 8, Gv[h]);
+                ld_rw8(gh + wb + lane * 8, H[h]);
+                old[h] = bw[(wb >> 5) + (lane >> 2)] >> (8u * bsel);
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int64_t wb = base + (int64_t)(it + h) * (8 * kBlock) + warp * 256;
+                uint32_t bits = 0u;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    float hn;
+                    const float u = worker_step<EF>(Gv[h][c], H[h][c], signed_scale((old[h] >> c) & 1u, s), hn);
+                    H[h][c] = hn;
+                    dd_acc(acc, fabsf(u));
+                    bits |= (u >= 0.0f ? 1u : 0u) << c;
+                }
+                st_rw8(gh + wb + lane * 8, H[h]);
+                uint32_t word = bits << (8u * bsel);
+                word |= __shfl_xor_sync(kFull, word, 1);
+                word |= __shfl_xor_sync(kFull, word, 2);
+                if (bsel == 0u) bw[(wb >> 5) + (lane >> 2)] = word;
+            }
+        }
+        acc = block_sum<kBlock>(acc);
+        if (threadIdx.x == 0) wpart[(int64_t)i * tb.nparts + tb.pbase[T]] = acc;
     } else {
         const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
         const float s = so[first];
@@ -744,9 +797,18 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
         if (valid) {
             const int r = find_segment(tb.off, first, last, j);
             float a = 0.0f;
-            for (int i = 0; i < n; ++i) {
-                const uint32_t bit = (ld_cg_u32(wbits + (int64_t)i * wp + (j >> 5)) >> (j & 31)) & 1u;
-                a = __fadd_rn(a, signed_scale(bit, ld_cg_f32(wscale + (int64_t)i * tb.q + r)));
+            for (int i0 = 0; i0 < n; i0 += 8) {        // eight workers' loads in flight, then their additions in order
+                uint32_t wd[8];
+                float sc[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = min(i0 + u, n - 1);
+                    wd[u] = ld_cg_u32(wbits + (int64_t)i * wp + (j >> 5));
+                    sc[u] = ld_cg_f32(wscale + (int64_t)i * tb.q + r);
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u)
+                    if (i0 + u < n) a = __fadd_rn(a, signed_scale((wd[u] >> (j & 31)) & 1u, sc[u]));
             }
             float hn;
             w = server_step<EF>(__fdiv_rn(a, fn), EF ? 0.0f : ghat_s[j], MODE == 2 ? 0.0f : gtil[j], hn);
@@ -934,12 +996,15 @@ static void launch_worker_sign_t(const G *grads, float *ghat_w, uint32_t *wbits,
         cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmemBytes);
         kern<<<grid, kBlock, kRingSmemBytes, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, error_flag,
                                                    scale_new, done, wait_limit);
-    } else if (ef) {
-        k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
-                                                        scale_new, done);
     } else {
-        k_worker_sign<false, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
-                                                         scale_new, done);
+        // 256-bit accesses: every row 32-byte aligned (state rows by d % 8; gradient rows by the
+        // base address and d times the element size)
+        const int vec8 = vec_ok && tb.d % 8 == 0 && ((uintptr_t)ghat_w & 31u) == 0 &&
+                         ((uintptr_t)grads & (sizeof(G) == 4 ? 31u : 15u)) == 0;
+        if (ef) k_worker_sign<true, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
+                                                                scale_new, done, vec8);
+        else k_worker_sign<false, G><<<grid, kBlock, 0, st>>>(grads, ghat_w, wbits, scale_old, wpart, tb, wp, vec_ok,
+                                                              scale_new, done, vec8);
     }
 }
 

@@ -382,8 +382,9 @@ __device__ __forceinline__ uint32_t fine_bin(uint32_t key, uint32_t fk) { return
 // above the floor; then key bits 30..11 of the threshold follow from the histogram of those
 // coordinates.  Otherwise the row's level-1 histogram is cleared for the full pass.  Run by
 // one whole block for the row.  (Folding this into the dense pass - the block that finishes a
-// row last takes it over - was measured: the memory fence every block then needs before its
-// ticket drains the block's outstanding writes and cost the bandwidth-bound pass 0.2 ms.)
+// row last takes it over - was measured twice: the memory fence before a block's ticket, in
+// every thread or in the ticket-taking thread alone after a barrier, waits for the block's
+// outstanding writes and cost the bandwidth-bound pass 0.2 ms either way.)
 __device__ __forceinline__ void pick_spec_row(uint32_t *hist, Sel *sel, uint32_t k, uint32_t fl, uint32_t *hit_row)
 {
     __shared__ uint32_t tot[kBlock];
