@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
     # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "7f8da041b7e2dc41", "bytes_per_launch": 4 * (1.797478e+09 + 8.56346624e+08),
+    "C4": {"hash": "6133ecb9258b1fb9", "bytes_per_launch": 4 * (1.797276e+09 + 8.56718592e+08),
            "note": "extrapolated from an ncu capture of the same kernel on the workload scaled by 0.25 "
                    "(same tile and kernel variant), multiplied by 4: traffic is proportional to n*d"},
 }
