@@ -12,7 +12,7 @@ Two layouts:
 * ``server_rank=None`` (default): every process holds n / world workers.  One all-gather
   gives every process all n worker messages and each computes the server stage itself; the
   results are identical everywhere (same operations, same order), so the server's broadcast
-  is not needed.  One collective per iteration instead of two sends.
+  is not needed.  One grouped collective per iteration instead of two sends.
 * ``server_rank=r``: the paper's layout.  Process r is the server and holds no worker; the
   other world - 1 processes hold n / (world - 1) workers each.  The worker messages go to r,
   r runs the server stage, and the server message is broadcast; every process (the server
@@ -47,6 +47,19 @@ def partition(n, world, rank, server_rank=None):
     return pos * per, per
 
 
+def _all_gather_together(pairs, group=None):
+    """In-place all-gathers of several (whole buffer, own rows) pairs.  On NCCL they are queued
+    as one grouped call (one launch moves the sign words and the scales of a message, which
+    live in two arrays); other backends get one call per pair."""
+    if dist.get_backend(group) == "nccl" and hasattr(dist, "_coalescing_manager"):
+        with dist._coalescing_manager(group=group):
+            for whole, own in pairs:
+                dist.all_gather_into_tensor(whole, own, group=group)
+        return
+    for whole, own in pairs:
+        dist.all_gather_into_tensor(whole, own, group=group)
+
+
 def exchange_worker_messages(bits, scales, n, group=None, server_rank=None):
     """Deliver the worker messages.  `bits` (n x words, int32) and `scales` (n x q, float32)
     are the full message buffers of this process with its own rows filled in; on return the
@@ -56,8 +69,7 @@ def exchange_worker_messages(bits, scales, n, group=None, server_rank=None):
     rank = dist.get_rank(group)
     first, per = partition(n, world, rank, server_rank)
     if server_rank is None:
-        dist.all_gather_into_tensor(bits, bits[first:first + per], group=group)
-        dist.all_gather_into_tensor(scales, scales[first:first + per], group=group)
+        _all_gather_together([(bits, bits[first:first + per]), (scales, scales[first:first + per])], group)
         return
     ops = []
     if rank == server_rank:
