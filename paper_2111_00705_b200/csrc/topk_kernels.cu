@@ -1407,6 +1407,7 @@ struct EmitUpdate {
     float *b_rw;
     uint32_t *pending;
     int classic_values;
+    uint32_t *hist_clear;             // rows x kHistStride, or NULL: the row's histograms, cleared for the next selection
 };
 
 template <bool HAS_B>
@@ -1422,6 +1423,11 @@ k_topk_emit_idx(const float *__restrict__ a_all, const float *__restrict__ b_all
 {
     const int row = blockIdx.y;
     if (!(kind & (hit[row] ? kRowsListed : kRowsClassic))) return;
+    // Nothing reads the row's histograms after the scans before this kernel: the row's first
+    // block leaves them zero for the next selection (which then needs no memset of its own in
+    // front of its dense pass).
+    if (upd.hist_clear && blockIdx.x == 0)
+        for (int t = threadIdx.x; t < kHistStride; t += kBlock) upd.hist_clear[(int64_t)row * kHistStride + t] = 0u;
     uint32_t *idx = idx_all + (int64_t)row * k;
     float *val = val_all + (int64_t)row * k;
     float *b_rw = upd.b_rw ? upd.b_rw + (int64_t)row * stride : nullptr;
@@ -1831,7 +1837,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
 {
     const dim3 dense((unsigned)((w->d + kSub - 1) / kSub), (unsigned)w->rows);
     const dim3 sparse((unsigned)w->nbt, (unsigned)w->rows);
-    cudaMemsetAsync(w->hist, 0, (size_t)w->rows * kHistStride * 4, st);
+    // (the histograms are zero: from the allocation, then from the previous selection's compaction)
     // one dense pass with the guessed floor; the two classic passes (small looping grids)
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, std::max(148u, 148u * 4u / (unsigned)w->rows)), (unsigned)w->rows);
@@ -1864,7 +1870,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // passes on the side stream ...
     const dim3 fallback_sparse(std::min(sparse.x, fallback.x), (unsigned)w->rows);
     // values, state update (or its deferral) happen inside the ordered compaction
-    const EmitUpdate upd = {HAS_B && update_b ? b : nullptr, defer ? w->pending : nullptr, 1};
+    const EmitUpdate upd = {HAS_B && update_b ? b : nullptr, defer ? w->pending : nullptr, 1, w->hist};
     cudaStream_t sd = w->side;
     cudaEventRecord(w->ev_fork, st);
     cudaStreamWaitEvent(sd, w->ev_fork, 0);
@@ -1989,7 +1995,7 @@ static void range_stage_impl(TopkWorkspace *w, int stage, const float *a, float 
         k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_tie, w->nbt, w->hit);
         k_topk_ties<<<fallback_sparse, kBlock, 0, st>>>(w->sel, w->hit, w->bm_in, w->bm_cand, w->cnt_tie, w->cnt_fin, w->wp, w->nbt, nullptr);
         k_scan_tiles<<<w->rows, kBlock, 0, st>>>(w->cnt_fin, w->nbt, w->hit, w->cnt_eq);      // cnt_eq[row] = entries this range keeps
-        k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic, EmitUpdate{nullptr, nullptr, 0});
+        k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsClassic, EmitUpdate{nullptr, nullptr, 0, nullptr});
         const dim3 entries((unsigned)((w->k + kBlock - 1) / kBlock), (unsigned)w->rows);
         k_range_pad<<<entries, kBlock, 0, st>>>(w->idx, w->val, w->cnt_eq, w->k);
         k_topk_gather<HAS_B, HAS_B><<<entries, kBlock, 0, st>>>(a, b, w->idx, w->val, w->hit, w->d, w->k, w->stride, nullptr);

@@ -474,6 +474,28 @@ def test_topk_prefetch_ring_with_failed_guesses_and_dense_tiles():
     g.close(); o.close()
 
 
+@pytest.mark.parametrize("n", [4, 5, 9, 16])
+def test_topk_prefetch_ring_rows_that_hit_beside_rows_that_miss(n):
+    """Scale jumps make the guesses of all rows fail; a jump in some workers only leaves rows
+    selected from the dense pass's lists and rows on the classic chain side by side in the
+    same launches (the two chains run as two branches of the step)."""
+    rng = np.random.default_rng(100 + n)
+    d, k = 12 * 4096 + 1000, 1500
+    w = synth.Workload("GROUPS", d, n, synth.TOPK, 9, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d))
+    g.set_tile(16384)
+    some = np.arange(n) % 3 == 1
+    for t, scale in enumerate((1.0, 1.0, 0.02, 0.02, 1.0, 1.0, 1.0, 50.0, 50.0)):
+        grads = (rng.standard_normal((n, d)) * scale).astype(np.float32)
+        if t in (5, 6):
+            grads[some] *= 0.01                             # only these rows miss (and miss again coming back)
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.device_status()
+    g.close(); o.close()
+
+
 @pytest.mark.parametrize("case", ["ragged", "aligned_large", "one_segment"])
 def test_topk_per_segment_matches_oracle(case):
     """Top-k applied to every segment on its own (per tensor): concatenated payloads bit-exact,
