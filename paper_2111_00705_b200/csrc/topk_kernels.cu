@@ -1036,7 +1036,7 @@ constexpr int kCandPerTile = 4;       // candidates of a tile that are kept with
 // histogram of bits 10..0 and, as far as there is room, into the tile's candidate slots; keys
 // with higher bits 30..11 are certainly kept and only counted.
 struct SplitTile {
-    uint32_t *h, pre11;
+    uint32_t *h, pre11;               // h: the row's histogram of key bits 10..0 (global)
     uint32_t *slots;                  // shared: candidates seen in this warp's tile so far
     uint16_t *cand;                   // global: the tile's kCandPerTile candidate slots (key bits 10..0)
     uint32_t above;                   // this lane's count of certainly kept values
@@ -1044,9 +1044,14 @@ struct SplitTile {
     {
         const uint32_t key = key_of(v), hi = key >> 11;
         if (hi == pre11) {
-            atomicAdd(&h[key & (kBins2 - 1)], 1u);
+            // Candidates are few (one fine bin of the dense pass's histogram), so they go to
+            // the row's histogram in global memory directly; the lanes that are here together
+            // with the same bin send one addition between them (tie-heavy rows).
+            const uint32_t bin = key & (kBins2 - 1);
+            const uint32_t same = __match_any_sync(__activemask(), bin);
+            if ((__ffs(same) - 1) == (int)(threadIdx.x & 31)) atomicAdd(&h[bin], (uint32_t)__popc(same));
             const uint32_t at = atomicAdd(slots, 1u);
-            if (at < (uint32_t)kCandPerTile) cand[at] = (uint16_t)(key & (kBins2 - 1));
+            if (at < (uint32_t)kCandPerTile) cand[at] = (uint16_t)bin;
         } else if (hi > pre11) {
             ++above;
         }
@@ -1069,17 +1074,16 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
              uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all, uint16_t *__restrict__ cand_all,
              int64_t nt4k, int64_t d, int64_t stride)
 {
-    __shared__ uint32_t h[kBins2];
     __shared__ uint32_t s_slots[kBlock / 32];
     const int row = blockIdx.y;
     if (!hit[row] || (int64_t)blockIdx.x * kListTiles >= nt4k) return;
-    for (int t = threadIdx.x; t < kBins2; t += kBlock) h[t] = 0;
-    if (threadIdx.x < kBlock / 32) s_slots[threadIdx.x] = 0u;
-    __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) s_slots[warp] = 0u;
+    __syncwarp();
     const WarpLists w = warp_lists(stash_all, stash_pos_all, stash_cnt_all, row, nt4k, d);
     const int64_t g = (int64_t)row * nt4k + (w.tile[0] < nt4k ? w.tile[0] : 0);
-    SplitTile f{h, sel_all[row].pre >> 11, &s_slots[warp], cand_all + g * kCandPerTile, 0u};
+    SplitTile f{hist_all + (int64_t)row * kHistStride + kBins1, sel_all[row].pre >> 11, &s_slots[warp],
+                cand_all + g * kCandPerTile, 0u};
     for_each_listed<HAS_B>(w, a_all + (int64_t)row * stride, HAS_B ? b_all + (int64_t)row * stride : nullptr, f);
     __syncwarp();
     uint32_t above = f.above;
@@ -1089,10 +1093,6 @@ k_topk_split(const float *__restrict__ a_all, const float *__restrict__ b_all,
         cnt_gt_all[g] = above;
         cnt_eq_all[g] = s_slots[warp];
     }
-    __syncthreads();
-    uint32_t *hist = hist_all + (int64_t)row * kHistStride + kBins1;
-    for (int t = threadIdx.x; t < kBins2; t += kBlock)
-        if (h[t]) atomicAdd(&hist[t], h[t]);
 }
 
 // ------------------------------------------------------------------------------------
