@@ -1197,12 +1197,14 @@ k_scan_tiles(uint32_t *__restrict__ cnt_all, int64_t nbt, const uint32_t *__rest
 // span (cnt_fin), which the server aggregation uses.  The counts come from k_topk_split's
 // per-tile records (certainly kept values, candidates and their low key bits) once this kernel
 // has picked the exact threshold from the low-bits histogram.  They pass through shared memory
-// in chunks of 4096 tiles (coalesced loads and stores); inside a chunk a thread owns 4
-// consecutive tiles (padded rows, no bank conflicts).  grid = (rows), 1024 threads: the row's
-// scan is one block's serial work, so the block is as wide as it gets.
+// in chunks of 8192 tiles (coalesced loads and stores; a row of up to 33.5 M coordinates is one
+// chunk: one round of loads and two block scans); inside a chunk a thread owns 8 consecutive
+// tiles (padded rows, no bank conflicts).  grid = (rows), 1024 threads: the row's scan is one
+// block's serial work, so the block is as wide as it gets.  Dynamic shared memory: kScanSmemBytes.
 constexpr int kScanBlock = 1024;      // one block per row does the whole scan: as wide as a block gets
-constexpr int kScanPer = 4;
+constexpr int kScanPer = 8;
 constexpr int kScanChunk = kScanBlock * kScanPer;
+constexpr int kScanSmemBytes = 2 * (kScanChunk + kScanBlock) * (int)sizeof(uint32_t);
 __device__ __forceinline__ int scan_slot(int i) { return i + i / kScanPer; }
 
 template <bool HAS_B>
@@ -1215,7 +1217,8 @@ k_scan_lists(const float *__restrict__ a_all, const float *__restrict__ b_all,
              uint32_t *__restrict__ cnt_gt_all, uint32_t *__restrict__ cnt_eq_all,
              uint32_t *__restrict__ cnt_fin_all, int64_t nt4k, int64_t nbt, int64_t d, int64_t stride)
 {
-    __shared__ uint32_t s_eq[kScanChunk + kScanBlock], s_gt[kScanChunk + kScanBlock];
+    extern __shared__ uint32_t scan_smem[];
+    uint32_t *s_eq = scan_smem, *s_gt = scan_smem + kScanChunk + kScanBlock;
     __shared__ uint32_t s_T, s_k3, s_c3;
     const int row = blockIdx.x;
     if (!hit[row]) return;
@@ -1894,7 +1897,8 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // (queued the ordinary way: with programmatic dependent launch from the pick to the
     // compaction the worker stage of 16 x 25.6 M measured 0.675 ms against 0.664)
     k_topk_split<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->sel, w->hit, w->stash, w->stash_pos, w->stash_cnt, w->hist, w->cnt_gt, w->cnt_eq, w->cand, w->nt4k, w->d, w->stride);
-    k_scan_lists<HAS_B><<<w->rows, kScanBlock, 0, st>>>(a, b, w->sel, w->hit, w->hist, w->floor_bucket, w->stash, w->stash_cnt, w->cand, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt, w->d, w->stride);
+    cudaFuncSetAttribute(k_scan_lists<HAS_B>, cudaFuncAttributeMaxDynamicSharedMemorySize, kScanSmemBytes);
+    k_scan_lists<HAS_B><<<w->rows, kScanBlock, kScanSmemBytes, st>>>(a, b, w->sel, w->hit, w->hist, w->floor_bucket, w->stash, w->stash_cnt, w->cand, w->cnt_gt, w->cnt_eq, w->cnt_fin, w->nt4k, w->nbt, w->d, w->stride);
     k_topk_emit_idx<HAS_B><<<sparse, kBlock, 0, st>>>(a, b, w->bm_in, w->cnt_fin, w->hit, w->sel, w->stash, w->stash_pos, w->stash_cnt, w->cnt_gt, w->cnt_eq, w->idx, w->val, w->wp, w->nbt, w->k, w->nt4k, w->d, w->stride, kRowsListed, upd);
     cudaStreamWaitEvent(st, w->ev_join, 0);
 }
