@@ -601,11 +601,24 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
             // entries among its coordinates (one worker sends a coordinate at most once, so the
             // lanes never meet inside a worker; __syncwarp orders one worker's additions before
             // the next one's).  No barrier, no atomics.
+            // (lane i holds the range of worker i; the loop takes it by shuffle)
+            uint32_t my_lo = 0u, my_hi = 0u;
+            if (lane < ag.n) {
+                my_lo = s_first[lane][warp];
+                my_hi = min((uint32_t)s_first[lane][warp + 1], (uint32_t)kAggStageCap);
+            }
             for (int i = 0; i < ag.n; ++i) {
-                const uint32_t lo = s_first[i][warp], hi = min((uint32_t)s_first[i][warp + 1], (uint32_t)kAggStageCap);
-                for (uint32_t e = lo + lane; e < hi; e += 32) {
+                const uint32_t lo = __shfl_sync(kFull, my_lo, i), hi = __shfl_sync(kFull, my_hi, i);
+                const uint32_t e = lo + lane;
+                if (e < hi) {
                     const uint32_t q = s_epos[i][e];
                     if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i][e]);
+                }
+                if (hi > lo + 32u) {                   // warp-uniform: more than 32 of a worker's entries in one warp's span
+                    for (uint32_t e2 = e + 32u; e2 < hi; e2 += 32u) {
+                        const uint32_t q = s_epos[i][e2];
+                        if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i][e2]);
+                    }
                 }
                 __syncwarp();
             }
