@@ -647,9 +647,16 @@ k_server_sign(const uint32_t *__restrict__ wbits, const float *__restrict__ wsca
             }
             float S[8];
             uint32_t bits = 0u;
+            if (n_pow2) {                                 // (decided once, outside the per-coordinate code)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) a[c] = __fmul_rn(a[c], rn);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) a[c] = __fdiv_rn(a[c], fn);
+            }
 #pragma unroll
             for (int c = 0; c < 8; ++c) {
-                const float mean = n_pow2 ? __fmul_rn(a[c], rn) : __fdiv_rn(a[c], fn);
+                const float mean = a[c];
                 const float w = server_step<EF>(mean, H[c], Gt[c], S[c]);
                 dd_acc(acc, fabsf(w));
                 bits |= (w >= 0.0f ? 1u : 0u) << c;

@@ -640,18 +640,24 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
         auto mean = [&](float v) { return ag.n_pow2 ? __fmul_rn(v, rn) : __fdiv_rn(v, fn); };
         if (vec_tile) load_tile(true, false);         // (after the aggregation: the other blocks of the SM hide the wait)
         if (vec_tile) {
+            // (the choice between the multiplication and the division is made once, outside the
+            // per-coordinate code; untouched coordinates keep their bits: no addition of a zero)
+            auto add_means = [&](auto mean_of) {
 #pragma unroll
-            for (int v = 0; v < 4; ++v) {
-                const int p = warp * kWarpSpan + v * 128 + lane * 4;
-                const float4 c = *reinterpret_cast<const float4 *>(acc + p);
-                if (c.x != 0.0f || c.y != 0.0f || c.z != 0.0f || c.w != 0.0f) {   // adding an exact zero changes nothing
-                    if (c.x != 0.0f) A[v].x = __fadd_rn(A[v].x, mean(c.x));
-                    if (c.y != 0.0f) A[v].y = __fadd_rn(A[v].y, mean(c.y));
-                    if (c.z != 0.0f) A[v].z = __fadd_rn(A[v].z, mean(c.z));
-                    if (c.w != 0.0f) A[v].w = __fadd_rn(A[v].w, mean(c.w));
-                    st_rw4(a_rw + base + p, A[v]);
+                for (int v = 0; v < 4; ++v) {
+                    const int p = warp * kWarpSpan + v * 128 + lane * 4;
+                    const float4 c = *reinterpret_cast<const float4 *>(acc + p);
+                    if (c.x != 0.0f || c.y != 0.0f || c.z != 0.0f || c.w != 0.0f) {
+                        const float sx = __fadd_rn(A[v].x, mean_of(c.x)), sy = __fadd_rn(A[v].y, mean_of(c.y));
+                        const float sz = __fadd_rn(A[v].z, mean_of(c.z)), sw = __fadd_rn(A[v].w, mean_of(c.w));
+                        A[v].x = c.x != 0.0f ? sx : A[v].x; A[v].y = c.y != 0.0f ? sy : A[v].y;
+                        A[v].z = c.z != 0.0f ? sz : A[v].z; A[v].w = c.w != 0.0f ? sw : A[v].w;
+                        st_rw4(a_rw + base + p, A[v]);
+                    }
                 }
-            }
+            };
+            if (ag.n_pow2) add_means([&](float v) { return __fmul_rn(v, rn); });
+            else add_means([&](float v) { return __fdiv_rn(v, fn); });
             __syncwarp();                             // the warp's sums are read: its part of s_u is free again
             load_tile(false, true);
         } else {
