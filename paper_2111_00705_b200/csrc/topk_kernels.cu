@@ -601,25 +601,36 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
             // entries among its coordinates (one worker sends a coordinate at most once, so the
             // lanes never meet inside a worker; __syncwarp orders one worker's additions before
             // the next one's).  No barrier, no atomics.
-            // (lane i holds the range of worker i; the loop takes it by shuffle)
+            // (lane i holds the range of worker i; the loop takes it by shuffle.)  Two workers
+            // per turn, sixteen lanes each, fetch their entries together and add one after the
+            // other; a range of more than sixteen entries sends the pair through the plain loop.
             uint32_t my_lo = 0u, my_hi = 0u;
             if (lane < ag.n) {
                 my_lo = s_first[lane][warp];
                 my_hi = min((uint32_t)s_first[lane][warp + 1], (uint32_t)kAggStageCap);
             }
-            for (int i = 0; i < ag.n; ++i) {
-                const uint32_t lo = __shfl_sync(kFull, my_lo, i), hi = __shfl_sync(kFull, my_hi, i);
-                const uint32_t e = lo + lane;
-                if (e < hi) {
-                    const uint32_t q = s_epos[i][e];
-                    if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i][e]);
-                }
-                if (hi > lo + 32u) {                   // warp-uniform: more than 32 of a worker's entries in one warp's span
-                    for (uint32_t e2 = e + 32u; e2 < hi; e2 += 32u) {
-                        const uint32_t q = s_epos[i][e2];
-                        if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i][e2]);
+            const int half = lane >> 4, slot = lane & 15;
+            for (int i0 = 0; i0 < ag.n; i0 += 2) {
+                const int wk = i0 + half;              // (<= 16: lanes 16.. of the last odd turn find an empty range)
+                const uint32_t lo = __shfl_sync(kFull, my_lo, wk), hi = __shfl_sync(kFull, my_hi, wk);
+                if (__any_sync(kFull, hi > lo + 16u)) {
+                    for (int t = 0; t < 2; ++t) {
+                        const uint32_t lo2 = __shfl_sync(kFull, lo, 16 * t), hi2 = __shfl_sync(kFull, hi, 16 * t);
+                        for (uint32_t e = lo2 + lane; e < hi2; e += 32) {
+                            const uint32_t q = s_epos[i0 + t][e];
+                            if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i0 + t][e]);
+                        }
+                        __syncwarp();
                     }
+                    continue;
                 }
+                const uint32_t e = lo + slot;
+                const uint32_t q = e < hi ? (uint32_t)s_epos[wk & (kAggStageWorkers - 1)][e] : 0xffffu;
+                const bool on = q < (uint32_t)kSub;
+                const float val = on ? s_eval[wk & (kAggStageWorkers - 1)][e] : 0.0f;
+                if (on && half == 0) acc[q] = __fadd_rn(acc[q], val);        // the lower worker adds first
+                __syncwarp();
+                if (on && half == 1) acc[q] = __fadd_rn(acc[q], val);
                 __syncwarp();
             }
             if (!vec_tile) __syncthreads();           // the scalar path below reads other warps' sums
