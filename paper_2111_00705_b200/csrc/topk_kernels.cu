@@ -800,7 +800,7 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
 // copies in flight land and leaves the block.  grid = (ceil(full tiles / kSpecTiles), rows);
 // rows 16-byte aligned, stride % 4 == 0.
 // ------------------------------------------------------------------------------------
-constexpr int kSpecTiles = 8;
+constexpr int kSpecTiles = 7;        // (16 x 6250 tiles: 5 -> 0.911, 6 -> 0.902, 7 -> 0.901, 8 -> 0.906, 10 -> 0.901, 12 -> 0.904, 16 -> 0.912 ms per step)
 constexpr int kSpecStages = 2;
 
 template <bool HAS_B, bool APPLY>
@@ -1882,7 +1882,7 @@ static void select_impl(TopkWorkspace *w, const float *a, float *b, bool update_
     // do work only for rows whose guess failed
     const dim3 fallback(std::min(dense.x, std::max(148u, 148u * 4u / (unsigned)w->rows)), (unsigned)w->rows);
     // whole tiles through the prefetch ring where rows are 16-byte aligned and there are
-    // tiles enough to fill the device several times over with its three blocks of eight tiles
+    // tiles enough to fill the device several times over with its three blocks of seven tiles
     // per SM (measured: 16 x 6250 tiles 0.50 -> 0.47 ms, 1 x 6250 tiles 0.039 -> 0.047 ms);
     // the ragged last tile, or everything else, through the plain kernel
     const int64_t full_tiles = agg ? 0 : ring_tiles(w, vec_ok);      // the fused aggregation lives in the plain kernel
