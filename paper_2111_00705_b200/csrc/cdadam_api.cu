@@ -60,6 +60,11 @@ int choose_tile(int64_t d, int q, bool server_side)
     if (d >= ((int64_t)1 << 23) && (int64_t)(q - 1) * (2 * kSub) * slack <= d && !server_side) tile = 2 * kSub;
     if (d >= ((int64_t)1 << 24) && (int64_t)(q - 1) * (2 * kSub) * slack <= d) tile = 2 * kSub;
     if (d >= ((int64_t)1 << 25) && (int64_t)(q - 1) * (4 * kSub) * slack <= d) tile = 4 * kSub;
+    // The worker pass with its prefetch ring gains from long tiles (a block's ring starts empty
+    // and its partial sum costs a block reduction): on 8 x 110 M coordinates 16384 -> 1.60 ms,
+    // 20480 -> 1.56, 32768 -> 1.57, 65536 -> 1.61 per pass under a power cap, the step 2.62 ->
+    // 2.54 ms; 4 x 1.5 G: 11.3 -> 10.6 ms per pass.  The server pass is best at 16384.
+    if (!server_side && d >= ((int64_t)1 << 26) && (int64_t)(q - 1) * (8 * kSub) * slack <= d) tile = 8 * kSub;
     return tile;
 }
 
