@@ -43,8 +43,8 @@ FALLBACK_HBM_GBS = 6650.0
 # keyed by workload, with the hash of the kernel sources at capture time.  A changed source
 # makes the figure stale and bench reports null.
 NCU_TRAFFIC = {
-    # k_worker_sign_ring: 2.654 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
-    "C4": {"hash": "6133ecb9258b1fb9", "bytes_per_launch": 4 * (1.797276e+09 + 8.56718592e+08),
+    # k_worker_sign_ring: 2.673 GB measured on C4 scaled by 0.25 (same tile), x4 by the units
+    "C4": {"hash": "43a020d7013fe046", "bytes_per_launch": 4 * (1.814689e+09 + 8.5882368e+08),
            "note": "extrapolated from an ncu capture of the same kernel on the workload scaled by 0.25 "
                    "(same tile and kernel variant), multiplied by 4: traffic is proportional to n*d"},
 }
