@@ -479,8 +479,8 @@ struct Pending {
 // issued first and four blocks (and 0.174 with six blocks, which spill).
 // With up to kAggStageWorkers workers and kAggStageCap entries each in the tile, the entries
 // are staged in shared memory and every warp adds, worker by worker, those among its own 512
-// coordinates; otherwise the block adds worker by worker with a barrier after each.  A row without a guess
-// still gets the aggregation.
+// coordinates; otherwise the block adds worker by worker with a barrier after each.  A row
+// without a guess still gets the aggregation.
 template <bool HAS_B, bool APPLY, bool AGG>
 __global__ void __launch_bounds__(kBlock, AGG ? 5 : 1)
 k_topk_spec(const float *__restrict__ a_all, float *b_all,
@@ -600,10 +600,10 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
             // sums of its 512 coordinates: it walks the workers in order and adds each worker's
             // entries among its coordinates (one worker sends a coordinate at most once, so the
             // lanes never meet inside a worker; __syncwarp orders one worker's additions before
-            // the next one's).  No barrier, no atomics.
-            // (lane i holds the range of worker i; the loop takes it by shuffle.)  Two workers
-            // per turn, sixteen lanes each, fetch their entries together and add one after the
-            // other; a range of more than sixteen entries sends the pair through the plain loop.
+            // the next one's).  No block barrier, no atomics.  Lane i holds the range of worker i
+            // and the loop takes it by shuffle; two workers per turn, sixteen lanes each, fetch
+            // their entries together and add one after the other; a range of more than sixteen
+            // entries sends the pair through the plain loop.
             uint32_t my_lo = 0u, my_hi = 0u;
             if (lane < ag.n) {
                 my_lo = s_first[lane][warp];
