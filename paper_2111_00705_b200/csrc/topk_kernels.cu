@@ -441,6 +441,7 @@ struct Agg {
     int n, n_pow2;
 };
 constexpr int kAggStageWorkers = 16;  // workers whose tile entries are staged in shared memory at once
+constexpr int kAggMaxWorkers = 64;    // workers that the staged path takes, batch after batch
 constexpr int kAggStageCap = 64;      // entries per worker and tile that the staged path holds
 
 __device__ __forceinline__ int64_t lower_bound_idx(const uint32_t *p, int64_t count, int64_t key)
@@ -477,9 +478,10 @@ struct Pending {
 // added, so that the kernel fits five blocks on an SM (46 registers), which hide those waits:
 // measured 0.166 ms for the server stage of 25.6 M coordinates against 0.175 with the loads
 // issued first and four blocks (and 0.174 with six blocks, which spill).
-// With up to kAggStageWorkers workers and kAggStageCap entries each in the tile, the entries
-// are staged in shared memory and every warp adds, worker by worker, those among its own 512
-// coordinates; otherwise the block adds worker by worker with a barrier after each.  A row
+// With up to kAggMaxWorkers workers and kAggStageCap entries each in the tile, the entries
+// are staged in shared memory, kAggStageWorkers workers at a time, and every warp adds, worker
+// by worker, those among its own 512 coordinates; otherwise the block adds worker by worker
+// with a barrier after each.  A row
 // without a guess still gets the aggregation.
 template <bool HAS_B, bool APPLY, bool AGG>
 __global__ void __launch_bounds__(kBlock, AGG ? 5 : 1)
@@ -544,22 +546,23 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
             if (ag.hit[i]) return t + side < nt4k ? ag.tile_off[(int64_t)i * nt4k + t + side] : (uint32_t)ag.k;
             return (uint32_t)lower_bound_idx(ag.idx + (int64_t)i * ag.k, ag.k, base + (int64_t)side * kSub);
         };
-        // Staged path (up to 16 workers, all with tile offsets, up to kAggStageCap entries each in
-        // this tile): sixteen threads copy the entries of one worker to shared memory, four each
-        // (entry u = 16 r + thread), and note where the entries pass from one warp's coordinates
-        // to the next one's.
+        // Staged path (up to kAggMaxWorkers workers, all with tile offsets, up to kAggStageCap
+        // entries each in this tile), in batches of kAggStageWorkers workers: sixteen threads
+        // copy the entries of one worker to shared memory, four each (entry u = 16 r + thread),
+        // and note where the entries pass from one warp's coordinates to the next one's.
         const int wi = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-        bool staged = ag.n <= kAggStageWorkers;
-        {
-            uint32_t cnt = 0u, beg = 0u;
-            if (staged && wi < ag.n) {
-                const uint32_t has = ag.hit[wi];
-                beg = ag.tile_off[(int64_t)wi * nt4k + t];
-                const uint32_t end = t + 1 < nt4k ? ag.tile_off[(int64_t)wi * nt4k + t + 1] : (uint32_t)ag.k;
-                cnt = end - beg;
-                staged = has != 0u && end >= beg && cnt <= (uint32_t)kAggStageCap;
-                if (!staged) cnt = 0u;
-            }
+        bool staged = ag.n <= kAggMaxWorkers;
+        // entries [beg, beg + cnt) of worker i's payload lie in this tile (cnt = 0 if i >= n)
+        auto entries_of = [&](int i, uint32_t &beg, uint32_t &cnt) -> bool {
+            beg = 0u; cnt = 0u;
+            if (i >= ag.n) return true;
+            const uint32_t has = ag.hit[i];
+            beg = ag.tile_off[(int64_t)i * nt4k + t];
+            const uint32_t end = t + 1 < nt4k ? ag.tile_off[(int64_t)i * nt4k + t + 1] : (uint32_t)ag.k;
+            cnt = end - beg;
+            return has != 0u && end >= beg && cnt <= (uint32_t)kAggStageCap;
+        };
+        auto stage = [&](int i, uint32_t beg, uint32_t cnt) {
             uint32_t pos[4];
             float val[4];
 #pragma unroll
@@ -568,8 +571,8 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
                 pos[r] = 0xffffffffu;
                 val[r] = 0.0f;
                 if (u < cnt) {
-                    pos[r] = ag.idx[(int64_t)wi * ag.k + beg + u] - (uint32_t)base;
-                    val[r] = ag.val[(int64_t)wi * ag.k + beg + u];
+                    pos[r] = ag.idx[(int64_t)i * ag.k + beg + u] - (uint32_t)base;
+                    val[r] = ag.val[(int64_t)i * ag.k + beg + u];
                 }
             }
             // warp of the coordinate of entry u (8 = past the tile or no entry), and of entry u - 1
@@ -582,43 +585,41 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
                 int wprev = __shfl_up_sync(kFull, wq, 1, 16);
                 if (l16 == 0) wprev = prev_last;
                 prev_last = __shfl_sync(kFull, wq, 15, 16);
-                if (wi < ag.n) {
-                    if (u < cnt) {
-                        s_epos[wi][u] = (uint16_t)min(pos[r], 0xffffu);
-                        s_eval[wi][u] = val[r];
-                    }
-                    // entries beyond cnt have wq = 8: the first of them opens the warps that are left
-                    if (u <= cnt)
-                        for (int w8 = wprev + 1; w8 <= wq; ++w8) s_first[wi][w8] = (uint8_t)u;
+                if (u < cnt) {
+                    s_epos[wi][u] = (uint16_t)min(pos[r], 0xffffu);
+                    s_eval[wi][u] = val[r];
                 }
+                // entries beyond cnt have wq = 8: the first of them opens the warps that are left
+                if (u <= cnt)
+                    for (int w8 = wprev + 1; w8 <= wq; ++w8) s_first[wi][w8] = (uint8_t)u;
             }
-            if (wi < ag.n && cnt == (uint32_t)kAggStageCap && l16 == 15)      // a full list: nothing opened the rest
+            if (cnt == (uint32_t)kAggStageCap && l16 == 15)      // a full list: nothing opened the rest
                 for (int w8 = prev_last + 1; w8 <= kBlock / 32; ++w8) s_first[wi][w8] = (uint8_t)kAggStageCap;
-        }
-        if (!__syncthreads_or(!staged)) {             // (the barrier also orders the zeroing and the staging)
-            // The sum of a coordinate runs over the workers in increasing order.  A warp owns the
-            // sums of its 512 coordinates: it walks the workers in order and adds each worker's
-            // entries among its coordinates (one worker sends a coordinate at most once, so the
-            // lanes never meet inside a worker; __syncwarp orders one worker's additions before
-            // the next one's).  No block barrier, no atomics.  Lane i holds the range of worker i
-            // and the loop takes it by shuffle; two workers per turn, sixteen lanes each, fetch
-            // their entries together and add one after the other; a range of more than sixteen
-            // entries sends the pair through the plain loop.
+        };
+        // The sum of a coordinate runs over the workers in increasing order.  A warp owns the
+        // sums of its 512 coordinates: it walks the staged workers in order and adds each
+        // worker's entries among its coordinates (one worker sends a coordinate at most once, so
+        // the lanes never meet inside a worker; __syncwarp orders one worker's additions before
+        // the next one's).  No block barrier, no atomics.  Lane i holds the range of staged
+        // worker i and the loop takes it by shuffle; two workers per turn, sixteen lanes each,
+        // fetch their entries together and add one after the other; a range of more than
+        // sixteen entries sends the pair through the plain loop.
+        auto add_staged = [&](int count) {             // count staged workers (an absent one has an empty range)
             uint32_t my_lo = 0u, my_hi = 0u;
-            if (lane < ag.n) {
+            if (lane < count) {
                 my_lo = s_first[lane][warp];
                 my_hi = min((uint32_t)s_first[lane][warp + 1], (uint32_t)kAggStageCap);
             }
             const int half = lane >> 4, slot = lane & 15;
-            for (int i0 = 0; i0 < ag.n; i0 += 2) {
+            for (int i0 = 0; i0 < count; i0 += 2) {
                 const int wk = i0 + half;              // (<= 16: lanes 16.. of the last odd turn find an empty range)
                 const uint32_t lo = __shfl_sync(kFull, my_lo, wk), hi = __shfl_sync(kFull, my_hi, wk);
                 if (__any_sync(kFull, hi > lo + 16u)) {
-                    for (int t = 0; t < 2; ++t) {
-                        const uint32_t lo2 = __shfl_sync(kFull, lo, 16 * t), hi2 = __shfl_sync(kFull, hi, 16 * t);
+                    for (int t2 = 0; t2 < 2; ++t2) {
+                        const uint32_t lo2 = __shfl_sync(kFull, lo, 16 * t2), hi2 = __shfl_sync(kFull, hi, 16 * t2);
                         for (uint32_t e = lo2 + lane; e < hi2; e += 32) {
-                            const uint32_t q = s_epos[i0 + t][e];
-                            if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[i0 + t][e]);
+                            const uint32_t q = s_epos[(i0 + t2) & (kAggStageWorkers - 1)][e];
+                            if (q < (uint32_t)kSub) acc[q] = __fadd_rn(acc[q], s_eval[(i0 + t2) & (kAggStageWorkers - 1)][e]);
                         }
                         __syncwarp();
                     }
@@ -632,6 +633,27 @@ k_topk_spec(const float *__restrict__ a_all, float *b_all,
                 __syncwarp();
                 if (on && half == 1) acc[q] = __fadd_rn(acc[q], val);
                 __syncwarp();
+            }
+        };
+        // every batch must qualify before anything is added (the general path starts from zero sums)
+        uint32_t beg0 = 0u, cnt0 = 0u;
+        if (staged) {
+            staged = entries_of(wi, beg0, cnt0);
+            for (int w0 = kAggStageWorkers; w0 < ag.n; w0 += kAggStageWorkers) {
+                uint32_t bx, cx;
+                if (!entries_of(w0 + wi, bx, cx)) staged = false;
+            }
+        }
+        stage(wi, beg0, staged ? cnt0 : 0u);          // (by all threads: it shuffles)
+        if (!__syncthreads_or(!staged)) {             // (the barrier also orders the zeroing and the staging)
+            add_staged(min(ag.n, kAggStageWorkers));
+            for (int w0 = kAggStageWorkers; w0 < ag.n; w0 += kAggStageWorkers) {     // more than sixteen workers: batch after batch
+                __syncthreads();                      // the batch before has been read by all warps
+                uint32_t bx, cx;
+                entries_of(w0 + wi, bx, cx);
+                stage(w0 + wi, bx, cx);
+                __syncthreads();
+                add_staged(min(ag.n - w0, kAggStageWorkers));
             }
             if (!vec_tile) __syncthreads();           // the scalar path below reads other warps' sums
         } else {

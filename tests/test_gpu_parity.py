@@ -496,6 +496,25 @@ def test_topk_prefetch_ring_rows_that_hit_beside_rows_that_miss(n):
     g.close(); o.close()
 
 
+@pytest.mark.parametrize("n", [17, 24, 32, 33, 64, 65])
+def test_topk_aggregation_of_many_workers(n):
+    """The server's dense pass adds the workers' messages in batches of sixteen workers (up to
+    64; beyond that worker by worker): sums in worker order whatever the batch a worker is in.
+    A quarter of the coordinates is sent by every worker, so most sums have many terms."""
+    rng = np.random.default_rng(n)
+    d, k = 6 * 4096 + 123, 900
+    w = synth.Workload("MANYW", d, n, synth.TOPK, 5, k=k)
+    g, o = make_pair(w, x0=torch.zeros(d))
+    common = rng.choice(d, 300, replace=False)
+    for t in range(5):
+        grads = rng.standard_normal((n, d)).astype(np.float32)
+        grads[:, common] *= 50.0
+        g.step(torch.from_numpy(grads).cuda()); o.step(grads)
+        check_payloads(g, o, w)
+    check_state(g, o, FINAL_TOL, exact=True)
+    g.close(); o.close()
+
+
 @pytest.mark.parametrize("case", ["ragged", "aligned_large", "one_segment"])
 def test_topk_per_segment_matches_oracle(case):
     """Top-k applied to every segment on its own (per tensor): concatenated payloads bit-exact,
