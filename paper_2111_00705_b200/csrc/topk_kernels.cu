@@ -1025,7 +1025,7 @@ k_topk_spec_ring(const float *__restrict__ a_all, float *b_all,
 constexpr int kTilesPerBlock = kTileWords * 32 / kSub;      // tiles per 32768-coordinate span
 constexpr int kWarpTiles = 1;
 constexpr int kListTiles = kWarpTiles * (kBlock / 32);
-constexpr int kPre = 4;
+constexpr int kPre = 3;        // (lists of C3 hold about 80 entries: 2 -> 0.9023, 3 -> 0.8988, 4 -> 0.9008, 5 -> 0.9045 ms per step)
 
 // A tile with more than kStashCap coordinates at or above the floor (the selection is
 // concentrated there) has no complete list: the passes walk its coordinates in a and b
